@@ -1,0 +1,334 @@
+#!/usr/bin/env python
+"""Benchmark of the stairs validation pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2|cfg3|cfg4]
+
+One step = one stairs_validate call (stair rows, embedding, every layer, LM head, argmax,
+accept) on the validation-microbench model (24 layers, d_model 1024, vocab 32128, bf16) with a
+2048-token prefix already in the KV cache and k = 8 drafted tokens (9 rows).  Prints ONE JSON
+line.  With --gpus N > 1 (under torchrun) every rank runs an independent replica: requests do
+not interact, so there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2407_19947_b200 import workloads as wl  # noqa: E402
+
+METRIC = "stairs_validate_us_per_call"
+UNIT = "us/call"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+def pick_workload(name: str):
+    idx = {"cfg2": 2, "cfg3": 3, "cfg4": 4}[name]
+    w = wl.workload(idx)
+    if idx == 2:
+        prefix, k = 2048, 8
+    elif idx == 3:
+        prefix, k = 512, 4
+    else:
+        prefix, k = 1024, 8
+    return w, prefix, k
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.rows, self.proc = index, [], None
+
+    def run(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            for line in self.proc.stdout:
+                self.rows.append([c.strip() for c in line.split(",")])
+        except Exception:
+            pass
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+        self.join(timeout=2)
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = set()
+        for r in self.rows:
+            for i, n in enumerate(names):
+                if len(r) > 4 + i and r[4 + i].lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def algorithmic_bytes(shape, prefix: int, k: int) -> int:
+    """Bytes one validate call must move: every weight matrix once plus the visible K/V once."""
+    return shape.weight_bytes_per_call() + shape.kv_bytes_per_token() * (prefix + k + 1)
+
+
+def oracle_row_seconds(w, tsrc, prompt, draft, rows):
+    """Times the CPU oracle (as it stands) on the given stair rows; returns seconds per row."""
+    from oracle import stairs_oracle as so
+    tgt = so.OracleModel(w.target, tsrc, keep=True)
+    all_rows = so.stairs_rows(prompt, draft)
+    t0 = time.perf_counter()
+    toks = [so.argmax_lowest(so.forward_logits(tgt, all_rows[r])) for r in rows]
+    return (time.perf_counter() - t0) / len(rows), toks
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p["num_threads"] for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def run_reference(args, rank, world):
+    """The oracle timed on the host cores.  Each step is one stair row (an independent no-cache
+    fp32 forward) at a prefix shortened so that the whole run stays within a few minutes; the
+    reported us/call scales the mean row time linearly in tokens to the full prefix and
+    multiplies by the k+1 rows of a call."""
+    if rank != 0:
+        return
+    from oracle import stairs_oracle as so
+    w, prefix, k = pick_workload(args.workload)
+    tsrc, _ = wl.make_sources(w, backend="numpy")
+    tgt = so.OracleModel(w.target, tsrc, keep=True)
+    prompt = list(wl.prompt_tokens(w, n=prefix + 1))
+    draft = list(wl.uniform_tokens(k, w.target.vocab, 77))
+    so.forward_logits(tgt, prompt[:16])                      # widens the weights once
+    t0 = time.perf_counter()
+    so.forward_logits(tgt, prompt[:64])
+    t64 = time.perf_counter() - t0
+    budget = args.ref_seconds / max(args.steps + args.warmup, 1)
+    p_s = int(max(16, min(prefix + 1, 64 * budget / max(t64, 1e-4))))
+    times = []
+    for i in range(args.warmup + args.steps):
+        r = i % (k + 1)
+        row = prompt[:p_s] + draft[:r]
+        t0 = time.perf_counter()
+        so.argmax_lowest(so.forward_logits(tgt, row))
+        if i >= args.warmup:
+            times.append((time.perf_counter() - t0) * (prefix + 1 + r) / len(row))
+    row_s = float(np.mean(times))
+    value = row_s * (k + 1) * 1e6
+    sample = (f"{args.steps} stair rows at prefix {p_s} of {prefix + 1}, one no-cache fp32 forward each, "
+              f"scaled linearly in tokens to the full prefix and to {k + 1} rows per call")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(np.mean(times)) * 1e3,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{w.name}: prefix {prefix}, k {k}, {k + 1} stair rows, 1 request"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def run_ours(args, rank, local_rank, world):
+    import torch
+    from paper_2407_19947_b200 import build, stairs
+    if rank == 0:
+        build.build()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+        dist.barrier()
+    w, prefix, k = pick_workload(args.workload)
+    shape = w.target
+    tsrc, dsrc = wl.make_sources(w, backend="torch-cuda")
+    torch.cuda.set_device(local_rank)
+    max_seq = prefix + 256 if shape.pos == wl.POS_ROPE else min(prefix + 256, shape.max_pos)
+    eng = stairs.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=max_seq, k_max=k, kv_page_tokens=64,
+                        device_index=local_rank)
+    prompt = wl.prompt_tokens(w, n=prefix + 1)     # prefix tokens in the cache + the last committed token
+    eng.prefill(0, prompt)
+    eng.sync()
+    # forced draft (first a tokens equal the target's own continuation, then a mismatch)
+    cont, _ = eng.generate(0, prompt, 0, k + 1)
+    eng.prefill(0, prompt)
+    a_list = wl.forced_accept_lengths(k, 64, 1234)
+    drafts = np.stack([wl.forced_draft(np.array(cont), a, shape.vocab, 50 + i) for i, a in enumerate(a_list)])
+    d_dev = torch.from_numpy(drafts).to(eng.device)
+    tt = torch.zeros((1, k + 1), dtype=torch.int32, device=eng.device)
+    al = torch.zeros((1,), dtype=torch.int32, device=eng.device)
+    stream = eng.stream
+
+    def step(i):
+        eng.validate([0], [k], d_dev[i % len(a_list)], commit=False, out=(tt, al))
+
+    # accept lengths must come out as forced (checks the path end to end before timing it)
+    for i in range(min(8, len(a_list))):
+        step(i)
+        eng.sync()
+        assert int(al.cpu()[0]) == a_list[i], (int(al.cpu()[0]), a_list[i])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = eng.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = eng.launch_count() - launches0
+    clocks = sampler.stop()
+
+    # per-launch events around the weight-streaming GEMMs, over the same steps
+    eng.profile(True)
+    gemm_ms, gemm_n, call_ms = 0.0, 0, 0.0
+    for i in range(args.steps):
+        step(i)
+        g, n, c = eng.profile_read()
+        gemm_ms += g
+        gemm_n += n
+        call_ms += c
+    eng.profile(False)
+
+    # end to end through the host-buffer entry point (drafts in, tokens and accept length out)
+    pin_d = torch.from_numpy(drafts).pin_memory()
+    for i in range(3):
+        eng.validate_host([0], [k], pin_d[i].numpy()[None])
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        eng.validate_host([0], [k], pin_d[i % len(a_list)].numpy()[None])
+    e2e_s = time.perf_counter() - t0
+
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms, e2e_s * 1e3], device=eng.device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+    else:
+        e2e_ms = e2e_s * 1e3
+    if rank != 0:
+        return
+    total_calls = args.steps * world
+    us_per_call = ms * 1e3 / total_calls
+    peaks, peak_kind = measured_peaks()
+    peak = float(peaks["hbm_gbs"])
+    wbytes = shape.weight_bytes_per_call()
+    abytes = algorithmic_bytes(shape, prefix, k)
+    gemm_s_per_call = gemm_ms * 1e-3 / args.steps
+    achieved = wbytes / gemm_s_per_call / 1e9 if gemm_s_per_call > 0 else None
+    line = {
+        "metric": METRIC, "value": us_per_call, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{w.name}: prefix {prefix}, k {k}, {k + 1} stair rows, 1 request per GPU, commit=0",
+                   "l2": "inputs larger than L2 (weights %.2f GB per call)" % (wbytes / 1e9),
+                   "replicas": world},
+        "clocks": clocks,
+        "gpu_launches": int(launches),
+        "e2e": {"value": e2e_ms * 1e3 / total_calls, "unit": UNIT,
+                "h2d_bytes_per_step": int(k * 4 + 3 * 4), "d2h_bytes_per_step": int((k + 1) * 4 + 4)},
+        "roofline": {"bound": "hbm", "kernel": "weight-streaming GEMMs (QKV, O, MLP, LM head)",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak if achieved else None,
+                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS if achieved else None,
+                     "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "launches_per_call": gemm_n / max(args.steps, 1),
+                     "timing": "per-launch CUDA events in a second pass over the same steps"},
+        "call": {"algorithmic_bytes": abytes, "hbm_gbs_whole_call": abytes / (us_per_call * 1e-6) / 1e9,
+                 "frac_of_measured_peak": abytes / (us_per_call * 1e-6) / 1e9 / peak,
+                 "frac_of_nominal_8TBs": abytes / (us_per_call * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
+                 "profiled_call_us": call_ms * 1e3 / max(args.steps, 1)},
+    }
+    # generation: tokens/s with stairs against k=0 greedy on the same kernels (short run)
+    try:
+        gen_prompt = prompt[: min(len(prompt), 512)]
+        n_new = 48
+        out0, st0 = eng.generate(0, gen_prompt, 0, n_new)
+        outk, stk = eng.generate(0, gen_prompt, min(4, k), n_new)
+        line["generation"] = {
+            "prompt": len(gen_prompt), "new_tokens": n_new, "k": min(4, k),
+            "greedy_tokens_per_s": n_new / ((st0["total_ms"] - st0["prefill_ms"]) * 1e-3),
+            "stairs_tokens_per_s": n_new / ((stk["total_ms"] - stk["prefill_ms"]) * 1e-3),
+            "acceptance": stk["accepted"] / max(stk["drafted"], 1), "identical_output": out0 == outk}
+        line["generation"]["speedup_vs_k0"] = (line["generation"]["stairs_tokens_per_s"]
+                                               / line["generation"]["greedy_tokens_per_s"])
+    except Exception as ex:  # reported, never hidden
+        line["generation"] = {"error": str(ex)}
+    # the oracle beside it, on this host's cores, on a bounded sample
+    if world == 1 and not args.no_cpu_baseline:
+        cb_prefix = min(prefix, args.cpu_prefix)
+        osrc = tsrc
+        cb_prompt = list(prompt[: cb_prefix + 1])
+        row_s, _ = oracle_row_seconds(w, osrc, cb_prompt, list(drafts[0]), [0])
+        n_rows = int(max(1, min(k + 1, 15.0 // max(row_s, 1e-3))))
+        if n_rows > 1:
+            row_s, _ = oracle_row_seconds(w, osrc, cb_prompt, list(drafts[0]), list(range(n_rows)))
+        line["cpu_baseline"] = {"value": row_s * (k + 1) * 1e6, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                "sample": f"{n_rows} of the {k + 1} stair rows at prefix {cb_prefix} "
+                                          f"(no-cache fp32 forwards), scaled to {k + 1} rows"}
+    print(json.dumps(line))
+    eng.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-prefix", type=int, default=2048, help="prefix length of the CPU-baseline sample")
+    ap.add_argument("--ref-seconds", type=float, default=120.0, help="--impl reference: time budget of the run")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    args.warmup = max(args.warmup, 3)
+    run_ours(args, rank, local_rank, world)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,673 @@
+// Host engine and C-ABI of the stairs library: context, workspace layout, KV page
+// allocator, the per-pass kernel sequence, draft / validate / generate.
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <type_traits>
+#include <vector>
+
+#include "../../include/stairs.h"
+#include "common.cuh"
+#include "gemm_simt.cuh"
+#include "kernels_basic.cuh"
+
+using namespace stairs;
+
+namespace {
+
+thread_local std::string g_init_error;
+
+struct DevModel {
+  stairs_model m{};
+  bool present = false;
+  stairs_weights w{};
+  std::vector<stairs_layer_w> layers;
+  char* kpool = nullptr;  // [n_layers][pool_tokens][Hkv*hd] elements of the weight dtype
+  char* vpool = nullptr;
+  size_t kv_layer_bytes = 0;
+};
+
+struct Layout {
+  size_t status, seq, n_seq, page_table, tok, pos, req, val_req, val_k, val_off, keys, x, h, qkv, q,
+      o, ff, logits, draft_buf, tt_buf, al_buf, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
+  int max_rows, logit_rows, max_pages, n_pages;
+  size_t kv_t_layer, kv_d_layer;
+};
+
+}  // namespace
+
+struct stairs_ctx {
+  stairs_config cfg{};
+  DevModel target, draft;
+  Layout lay{};
+  cudaStream_t stream = nullptr;
+  char* ws = nullptr;
+  std::string err;
+  int64_t launches = 0;
+  // host mirrors
+  std::vector<int> free_pages;
+  std::vector<std::vector<int>> pages;  // per slot
+  std::vector<int> n_seq_ub;            // upper bound of the device-side sequence length
+  std::vector<char> active;
+  // profiling
+  bool profile = false;
+  std::vector<cudaEvent_t> ev;
+  int ev_used = 0;
+  cudaEvent_t call_begin = nullptr, call_end = nullptr;
+  bool in_validate = false;
+};
+
+namespace {
+
+int fail(stairs_ctx* c, int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (c) c->err = buf; else g_init_error = buf;
+  return code;
+}
+
+#define CK(call)                                                                              \
+  do {                                                                                        \
+    cudaError_t e_ = (call);                                                                  \
+    if (e_ != cudaSuccess)                                                                    \
+      return fail(ctx, STAIRS_ECUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_),  \
+                  __FILE__, __LINE__);                                                        \
+  } while (0)
+
+size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+int esize(const stairs_model& m) { return m.wdtype == 0 ? 4 : 2; }
+
+const char* check_model(const stairs_model& m) {
+  if (m.n_layers < 0 || m.d_model <= 0 || m.n_heads <= 0 || m.n_kv_heads <= 0 || m.head_dim <= 0 ||
+      m.d_ff <= 0 || m.vocab <= 0)
+    return "model dimensions must be positive";
+  if (m.n_heads % m.n_kv_heads) return "n_heads must be a multiple of n_kv_heads";
+  if (m.head_dim % 8 || m.head_dim > 256) return "head_dim must be a multiple of 8 and <= 256";
+  if (m.d_model % 8 || m.d_ff % 8) return "d_model and d_ff must be multiples of 8";
+  if (m.norm < 0 || m.norm > 1 || m.act < 0 || m.act > 1 || m.pos < 0 || m.pos > 1) return "norm/act/pos out of range";
+  if (m.wdtype < 0 || m.wdtype > 1) return "wdtype must be 0 (fp32) or 1 (bf16)";
+  if (m.pos == 0 && m.max_pos <= 0) return "max_pos must be positive with learned positions";
+  return nullptr;
+}
+
+bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
+  *why = nullptr;
+  if (c.struct_size != sizeof(stairs_config)) { *why = "struct_size does not match this library"; return false; }
+  if ((*why = check_model(c.target))) return false;
+  const bool has_draft = c.draft.n_layers > 0;
+  if (has_draft) {
+    if ((*why = check_model(c.draft))) return false;
+    if (c.draft.d_model != c.target.d_model || c.draft.vocab != c.target.vocab ||
+        c.draft.wdtype != c.target.wdtype || c.draft.norm != c.target.norm ||
+        c.draft.act != c.target.act || c.draft.pos != c.target.pos) {
+      *why = "draft must share d_model, vocab, wdtype and the norm/act/pos family with the target";
+      return false;
+    }
+  }
+  if (c.max_requests <= 0 || c.max_seq_len < 4 || c.k_max < 0 || c.k_max > 63) {
+    *why = "max_requests > 0, max_seq_len >= 4 and 0 <= k_max <= 63 required"; return false;
+  }
+  const int pt = c.kv_page_tokens;
+  if (pt != 16 && pt != 32 && pt != 64 && pt != 128) { *why = "kv_page_tokens must be 16, 32, 64 or 128"; return false; }
+  if (c.target.pos == 0 && c.max_seq_len > c.target.max_pos) { *why = "max_seq_len exceeds max_pos of the learned positions"; return false; }
+  if (c.kv_pages < 0 || c.prefill_chunk < 0) { *why = "kv_pages and prefill_chunk must not be negative"; return false; }
+  const int chunk = c.prefill_chunk > 0 ? c.prefill_chunk : 256;
+  L->max_rows = std::max(std::max(chunk, c.max_requests * (c.k_max + 1)), 2);
+  L->logit_rows = std::max(c.max_requests * (c.k_max + 1), 1);
+  L->max_pages = (c.max_seq_len + pt - 1) / pt;
+  L->n_pages = c.kv_pages > 0 ? c.kv_pages : L->max_pages * c.max_requests;
+  const stairs_model& t = c.target;
+  const stairs_model& d = c.draft;
+  auto mx = [&](int a, int b) { return has_draft ? std::max(a, b) : a; };
+  const size_t es = esize(t);
+  const size_t dm = t.d_model;
+  const size_t nq = mx(t.n_heads * t.head_dim, d.n_heads * d.head_dim);
+  const size_t nqkv = mx((t.n_heads + 2 * t.n_kv_heads) * t.head_dim, (d.n_heads + 2 * d.n_kv_heads) * d.head_dim);
+  const size_t ff = mx(t.d_ff, d.d_ff);
+  const size_t R = L->max_rows;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  L->status = take(STATUS_WORDS * 4);
+  L->seq = take((size_t)c.max_requests * c.max_seq_len * 4);
+  L->n_seq = take((size_t)c.max_requests * 4);
+  L->page_table = take((size_t)c.max_requests * L->max_pages * 4);
+  L->tok = take(R * 4); L->pos = take(R * 4); L->req = take(R * 4);
+  L->val_req = take((size_t)c.max_requests * 4);
+  L->val_k = take((size_t)c.max_requests * 4);
+  L->val_off = take((size_t)c.max_requests * 4);
+  L->keys = take(R * 8);
+  L->x = take(R * dm * 4);
+  L->h = take(R * dm * es);
+  L->qkv = take(R * nqkv * 4);
+  L->q = take(R * nq * es);
+  L->o = take(R * nq * es);
+  L->ff = take(R * ff * es);
+  L->logits = take((size_t)L->logit_rows * t.vocab * 4);
+  L->draft_buf = take((size_t)c.max_requests * std::max(c.k_max, 1) * 4);
+  L->tt_buf = take((size_t)c.max_requests * (c.k_max + 1) * 4);
+  L->al_buf = take((size_t)c.max_requests * 4);
+  const size_t pool_tokens = (size_t)L->n_pages * pt;
+  L->kv_t_layer = pool_tokens * t.n_kv_heads * t.head_dim * es;
+  L->kv_t_k = take(L->kv_t_layer * t.n_layers);
+  L->kv_t_v = take(L->kv_t_layer * t.n_layers);
+  L->kv_d_layer = has_draft ? pool_tokens * d.n_kv_heads * d.head_dim * es : 0;
+  L->kv_d_k = take(L->kv_d_layer * (has_draft ? d.n_layers : 0));
+  L->kv_d_v = take(L->kv_d_layer * (has_draft ? d.n_layers : 0));
+  L->total = off;
+  return true;
+}
+
+// ---------------------------------------------------------------------------------------------
+// KV pages: a free list on the host; the device page table is patched with small copies.
+// Both models index positions the same way, so one page table serves both caches.
+// ---------------------------------------------------------------------------------------------
+int ensure_pages(stairs_ctx* ctx, int slot, int n_tokens) {
+  const int pt = ctx->cfg.kv_page_tokens;
+  const int need = (n_tokens + pt - 1) / pt;
+  auto& pg = ctx->pages[slot];
+  if ((int)pg.size() >= need) return STAIRS_OK;
+  if (need > ctx->lay.max_pages) return fail(ctx, STAIRS_ENOSPC, "request %d would exceed max_seq_len", slot);
+  const int first_new = (int)pg.size();
+  if ((int)ctx->free_pages.size() < need - first_new)
+    return fail(ctx, STAIRS_ENOSPC, "KV page pool exhausted (%d pages)", ctx->lay.n_pages);
+  while ((int)pg.size() < need) { pg.push_back(ctx->free_pages.back()); ctx->free_pages.pop_back(); }
+  int* dst = reinterpret_cast<int*>(ctx->ws + ctx->lay.page_table) + (size_t)slot * ctx->lay.max_pages + first_new;
+  CK(cudaMemcpyAsync(dst, pg.data() + first_new, (size_t)(need - first_new) * 4, cudaMemcpyHostToDevice, ctx->stream));
+  return STAIRS_OK;
+}
+
+void release_pages(stairs_ctx* ctx, int slot) {
+  for (int p : ctx->pages[slot]) ctx->free_pages.push_back(p);
+  ctx->pages[slot].clear();
+  ctx->active[slot] = 0;
+  ctx->n_seq_ub[slot] = 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// One forward pass over T rows (tok/pos/req already built on the device).
+// ---------------------------------------------------------------------------------------------
+struct GemmTimer {
+  stairs_ctx* c;
+  bool on;
+  explicit GemmTimer(stairs_ctx* ctx)
+      : c(ctx), on(ctx->profile && ctx->in_validate && ctx->ev_used + 2 <= (int)ctx->ev.size()) {
+    if (on) cudaEventRecord(c->ev[c->ev_used++], c->stream);
+  }
+  ~GemmTimer() { if (on) cudaEventRecord(c->ev[c->ev_used++], c->stream); }
+};
+
+template <typename WT>
+int forward_rows(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, int n_logit_rows, float* logits_out) {
+  const stairs_model& m = M.m;
+  const Layout& L = ctx->lay;
+  cudaStream_t st = ctx->stream;
+  char* ws = ctx->ws;
+  const int d = m.d_model, hq = m.n_heads, hkv = m.n_kv_heads, hd = m.head_dim, F = m.d_ff;
+  const int nq = hq * hd, nkv = hkv * hd, nqkv = nq + 2 * nkv;
+  const int* tok = reinterpret_cast<int*>(ws + L.tok);
+  const int* pos = reinterpret_cast<int*>(ws + L.pos);
+  const int* req = reinterpret_cast<int*>(ws + L.req);
+  const int* page_table = reinterpret_cast<int*>(ws + L.page_table);
+  float* x = reinterpret_cast<float*>(ws + L.x);
+  WT* h = reinterpret_cast<WT*>(ws + L.h);
+  float* qkv = reinterpret_cast<float*>(ws + L.qkv);
+  WT* q = reinterpret_cast<WT*>(ws + L.q);
+  WT* o = reinterpret_cast<WT*>(ws + L.o);
+  WT* ff = reinterpret_cast<WT*>(ws + L.ff);
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(ws + L.keys);
+  const int pt = ctx->cfg.kv_page_tokens;
+
+  k_embed<WT><<<T, 256, 0, st>>>((const WT*)M.w.tok_emb, (const WT*)M.w.pos_emb, tok, pos, x, d);
+  ctx->launches++;
+  for (int l = 0; l < m.n_layers; ++l) {
+    const stairs_layer_w& w = M.layers[l];
+    WT* kc = reinterpret_cast<WT*>(M.kpool + (size_t)l * M.kv_layer_bytes);
+    WT* vc = reinterpret_cast<WT*>(M.vpool + (size_t)l * M.kv_layer_bytes);
+    k_norm<WT><<<T, 256, 0, st>>>(x, (const float*)w.norm1_w, (const float*)w.norm1_b, h, d, m.norm, m.norm_eps);
+    {
+      GemmTimer tm(ctx);
+      launch_gemm_rows<WT, false>(st, (const WT*)w.wq, nullptr, h, T, nq, d, EPI_STORE_F32, qkv, nullptr, nqkv);
+      launch_gemm_rows<WT, false>(st, (const WT*)w.wk, nullptr, h, T, nkv, d, EPI_STORE_F32, qkv + nq, nullptr, nqkv);
+      launch_gemm_rows<WT, false>(st, (const WT*)w.wv, nullptr, h, T, nkv, d, EPI_STORE_F32, qkv + nq + nkv, nullptr, nqkv);
+    }
+    k_rope_append<WT><<<T, 256, 0, st>>>(qkv, pos, req, page_table, q, kc, vc, hq, hkv, hd, m.pos, m.rope_theta, pt, L.max_pages);
+    k_attn_plain<WT, 8><<<dim3(hq, T), 128, (size_t)5 * hd * sizeof(float), st>>>(
+        q, kc, vc, page_table, req, pos, o, hq, hkv, hd, pt, L.max_pages, 1.0f / sqrtf((float)hd));
+    {
+      GemmTimer tm(ctx);
+      launch_gemm_rows<WT, false>(st, (const WT*)w.wo, nullptr, o, T, d, nq, EPI_ADD_F32, x, nullptr, d);
+    }
+    k_norm<WT><<<T, 256, 0, st>>>(x, (const float*)w.norm2_w, (const float*)w.norm2_b, h, d, m.norm, m.norm_eps);
+    {
+      GemmTimer tm(ctx);
+      if (m.act == 1)
+        launch_gemm_rows<WT, true>(st, (const WT*)w.w_gate_or_fc1, (const WT*)w.w_up, h, T, F, d, EPI_SWIGLU, nullptr, ff, F);
+      else
+        launch_gemm_rows<WT, false>(st, (const WT*)w.w_gate_or_fc1, nullptr, h, T, F, d, EPI_GELU, nullptr, ff, F);
+      launch_gemm_rows<WT, false>(st, (const WT*)w.w_down_or_fc2, nullptr, ff, T, d, F, EPI_ADD_F32, x, nullptr, d);
+    }
+    ctx->launches += 10;
+  }
+  if (n_logit_rows > 0) {
+    float* lg = logits_out ? logits_out : reinterpret_cast<float*>(ws + L.logits);
+    k_norm<WT><<<n_logit_rows, 256, 0, st>>>(x + (size_t)logit_first_row * d, (const float*)M.w.final_norm_w,
+                                             (const float*)M.w.final_norm_b, h, d, m.norm, m.norm_eps);
+    {
+      GemmTimer tm(ctx);
+      launch_gemm_rows<WT, false>(st, (const WT*)M.w.lm_head, nullptr, h, n_logit_rows, m.vocab, d, EPI_STORE_F32, lg, nullptr, m.vocab);
+    }
+    const int slices = std::max(1, std::min(64, m.vocab / 2048));
+    k_argmax<<<dim3(slices, n_logit_rows), 256, 0, st>>>(lg, m.vocab, m.vocab, keys + logit_first_row);
+    ctx->launches += 3;
+  }
+  CK(cudaGetLastError());
+  return STAIRS_OK;
+}
+
+int forward(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, int n_logit_rows, float* logits_out) {
+  if (M.m.wdtype == 0) return forward_rows<float>(ctx, M, T, logit_first_row, n_logit_rows, logits_out);
+  return forward_rows<bf16>(ctx, M, T, logit_first_row, n_logit_rows, logits_out);
+}
+
+RowParams base_rows(stairs_ctx* ctx) {
+  RowParams p{};
+  char* ws = ctx->ws;
+  const Layout& L = ctx->lay;
+  p.val_req = reinterpret_cast<int*>(ws + L.val_req);
+  p.val_k = reinterpret_cast<int*>(ws + L.val_k);
+  p.val_off = reinterpret_cast<int*>(ws + L.val_off);
+  p.k_max = ctx->cfg.k_max;
+  p.seq = reinterpret_cast<int*>(ws + L.seq);
+  p.n_seq = reinterpret_cast<int*>(ws + L.n_seq);
+  p.max_seq_len = ctx->cfg.max_seq_len;
+  p.vocab = ctx->cfg.target.vocab;
+  p.tok = reinterpret_cast<int*>(ws + L.tok);
+  p.pos = reinterpret_cast<int*>(ws + L.pos);
+  p.req = reinterpret_cast<int*>(ws + L.req);
+  p.keys = reinterpret_cast<unsigned long long*>(ws + L.keys);
+  p.n_keys = L.max_rows;
+  return p;
+}
+
+int launch_rows(stairs_ctx* ctx, const RowParams& p, int threads_needed) {
+  const int n = std::max(threads_needed, p.n_keys);
+  k_rows<<<(n + 255) / 256, 256, 0, ctx->stream>>>(p);
+  ctx->launches++;
+  CK(cudaGetLastError());
+  return STAIRS_OK;
+}
+
+int check_slot(stairs_ctx* ctx, int req, bool must_be_active) {
+  if (!ctx) return STAIRS_EINVAL;
+  if (req < 0 || req >= ctx->cfg.max_requests) return fail(ctx, STAIRS_EINVAL, "request slot %d out of range", req);
+  if (must_be_active && !ctx->active[req]) return fail(ctx, STAIRS_ESTATE, "request %d has not been prefilled", req);
+  return STAIRS_OK;
+}
+
+int prefill_model(stairs_ctx* ctx, DevModel& M, int slot, int n_ctx) {
+  const int chunk = ctx->cfg.prefill_chunk > 0 ? ctx->cfg.prefill_chunk : 256;
+  for (int c0 = 0; c0 < n_ctx; c0 += chunk) {
+    const int n = std::min(chunk, n_ctx - c0);
+    RowParams p = base_rows(ctx);
+    p.mode = ROWS_PREFILL; p.slot = slot; p.first = c0; p.n_rows = n;
+    int rc = launch_rows(ctx, p, n);
+    if (rc) return rc;
+    rc = forward(ctx, M, n, 0, 0, nullptr);
+    if (rc) return rc;
+  }
+  return STAIRS_OK;
+}
+
+}  // namespace
+
+// =============================================================================================
+// C-ABI
+// =============================================================================================
+extern "C" {
+
+size_t stairs_workspace_bytes(const stairs_config* cfg) {
+  if (!cfg) return 0;
+  Layout L{};
+  const char* why = nullptr;
+  if (!compute_layout(*cfg, &L, &why)) { g_init_error = why ? why : "bad configuration"; return 0; }
+  return L.total;
+}
+
+int stairs_init(const stairs_config* cfg, const stairs_weights* target, const stairs_weights* draft, stairs_ctx** out) {
+  if (!cfg || !target || !out) return fail(nullptr, STAIRS_EINVAL, "cfg, target and out must not be NULL");
+  *out = nullptr;
+  Layout L{};
+  const char* why = nullptr;
+  if (!compute_layout(*cfg, &L, &why)) return fail(nullptr, STAIRS_EINVAL, "%s", why ? why : "bad configuration");
+  const bool has_draft = cfg->draft.n_layers > 0;
+  if (has_draft && !draft) return fail(nullptr, STAIRS_EINVAL, "draft weights missing");
+  if (!cfg->workspace || (reinterpret_cast<uintptr_t>(cfg->workspace) & 255))
+    return fail(nullptr, STAIRS_EINVAL, "workspace must be a 256-byte aligned device pointer");
+  if (cfg->workspace_bytes < L.total)
+    return fail(nullptr, STAIRS_ENOSPC, "workspace too small: %zu < %zu bytes", cfg->workspace_bytes, L.total);
+  auto check_w = [&](const stairs_model& m, const stairs_weights* w) -> const char* {
+    if (!w->tok_emb || !w->final_norm_w || !w->lm_head || (m.n_layers > 0 && !w->layers)) return "global weight pointer missing";
+    if (m.pos == 0 && !w->pos_emb) return "pos_emb missing";
+    if (m.norm == 0 && !w->final_norm_b) return "final_norm_b missing";
+    for (int l = 0; l < m.n_layers; ++l) {
+      const stairs_layer_w& y = w->layers[l];
+      if (!y.norm1_w || !y.wq || !y.wk || !y.wv || !y.wo || !y.norm2_w || !y.w_gate_or_fc1 || !y.w_down_or_fc2)
+        return "layer weight pointer missing";
+      if (m.act == 1 && !y.w_up) return "w_up missing for SwiGLU";
+      if (m.norm == 0 && (!y.norm1_b || !y.norm2_b)) return "LayerNorm bias missing";
+    }
+    return nullptr;
+  };
+  if ((why = check_w(cfg->target, target))) return fail(nullptr, STAIRS_EINVAL, "target: %s", why);
+  if (has_draft && (why = check_w(cfg->draft, draft))) return fail(nullptr, STAIRS_EINVAL, "draft: %s", why);
+
+  cudaError_t e = cudaSetDevice(cfg->device);
+  if (e != cudaSuccess) return fail(nullptr, STAIRS_ECUDA, "cudaSetDevice(%d): %s", cfg->device, cudaGetErrorString(e));
+  stairs_ctx* ctx = new (std::nothrow) stairs_ctx();
+  if (!ctx) return fail(nullptr, STAIRS_ENOSPC, "out of host memory");
+  ctx->cfg = *cfg;
+  ctx->lay = L;
+  ctx->stream = reinterpret_cast<cudaStream_t>(cfg->stream);
+  ctx->ws = reinterpret_cast<char*>(cfg->workspace);
+  auto fill = [&](DevModel& M, const stairs_model& m, const stairs_weights* w) {
+    M.m = m; M.present = true; M.w = *w;
+    M.layers.assign(w->layers, w->layers + m.n_layers);
+    M.w.layers = M.layers.data();
+  };
+  fill(ctx->target, cfg->target, target);
+  ctx->target.kpool = ctx->ws + L.kv_t_k; ctx->target.vpool = ctx->ws + L.kv_t_v; ctx->target.kv_layer_bytes = L.kv_t_layer;
+  if (has_draft) {
+    fill(ctx->draft, cfg->draft, draft);
+    ctx->draft.kpool = ctx->ws + L.kv_d_k; ctx->draft.vpool = ctx->ws + L.kv_d_v; ctx->draft.kv_layer_bytes = L.kv_d_layer;
+  }
+  ctx->pages.resize(cfg->max_requests);
+  ctx->n_seq_ub.assign(cfg->max_requests, 0);
+  ctx->active.assign(cfg->max_requests, 0);
+  for (int p = L.n_pages - 1; p >= 0; --p) ctx->free_pages.push_back(p);
+  // clear status words, sequences, lengths and page tables (KV pages need no clearing: a
+  // position is always written before it becomes visible)
+  e = cudaMemsetAsync(ctx->ws, 0, L.tok, ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+  if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_begin);
+  if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_end);
+  if (e != cudaSuccess) {
+    int rc = fail(nullptr, STAIRS_ECUDA, "context set-up failed: %s", cudaGetErrorString(e));
+    delete ctx;
+    return rc;
+  }
+  *out = ctx;
+  return STAIRS_OK;
+}
+
+int stairs_prefill(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_prompt) {
+  int rc = check_slot(ctx, req, false);
+  if (rc) return rc;
+  if (!prompt_host || n_prompt < 2) return fail(ctx, STAIRS_EINVAL, "prompt must hold at least 2 tokens");
+  if (n_prompt + 1 > ctx->cfg.max_seq_len)
+    return fail(ctx, STAIRS_ENOSPC, "prompt of %d tokens does not fit max_seq_len %d", n_prompt, ctx->cfg.max_seq_len);
+  for (int i = 0; i < n_prompt; ++i)
+    if (prompt_host[i] < 0 || prompt_host[i] >= ctx->cfg.target.vocab)
+      return fail(ctx, STAIRS_EINVAL, "prompt token %d out of range at %d", prompt_host[i], i);
+  release_pages(ctx, req);
+  rc = ensure_pages(ctx, req, n_prompt);
+  if (rc) return rc;
+  int* seq = reinterpret_cast<int*>(ctx->ws + ctx->lay.seq) + (size_t)req * ctx->cfg.max_seq_len;
+  int* nseq = reinterpret_cast<int*>(ctx->ws + ctx->lay.n_seq) + req;
+  CK(cudaMemcpyAsync(seq, prompt_host, (size_t)n_prompt * 4, cudaMemcpyHostToDevice, ctx->stream));
+  CK(cudaMemcpyAsync(nseq, &n_prompt, 4, cudaMemcpyHostToDevice, ctx->stream));
+  ctx->active[req] = 1;
+  ctx->n_seq_ub[req] = n_prompt;
+  rc = prefill_model(ctx, ctx->target, req, n_prompt - 1);
+  if (rc) return rc;
+  if (ctx->draft.present) rc = prefill_model(ctx, ctx->draft, req, n_prompt - 1);
+  return rc;
+}
+
+int stairs_draft(stairs_ctx* ctx, int req, int k, int32_t* draft_dev) {
+  int rc = check_slot(ctx, req, true);
+  if (rc) return rc;
+  if (!ctx->draft.present) return fail(ctx, STAIRS_ESTATE, "no draft model configured");
+  if (k < 0 || k > ctx->cfg.k_max || (k > 0 && !draft_dev)) return fail(ctx, STAIRS_EINVAL, "draft length %d outside 0..k_max", k);
+  if (k == 0) return STAIRS_OK;
+  if (ctx->n_seq_ub[req] + k > ctx->cfg.max_seq_len)
+    return fail(ctx, STAIRS_ENOSPC, "request %d: sequence would exceed max_seq_len", req);
+  rc = ensure_pages(ctx, req, ctx->n_seq_ub[req] + k);
+  if (rc) return rc;
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(ctx->ws + ctx->lay.keys);
+  for (int j = 0; j < k; ++j) {
+    RowParams p = base_rows(ctx);
+    p.slot = req; p.draft = draft_dev; p.first = j;
+    p.mode = j == 0 ? ROWS_DRAFT_FIRST : ROWS_DRAFT_NEXT;
+    const int T = j == 0 ? 2 : 1;
+    if ((rc = launch_rows(ctx, p, T))) return rc;
+    if ((rc = forward(ctx, ctx->draft, T, T - 1, 1, nullptr))) return rc;
+    k_take_token<<<1, 32, 0, ctx->stream>>>(keys, T - 1, draft_dev, j);
+    ctx->launches++;
+  }
+  CK(cudaGetLastError());
+  return STAIRS_OK;
+}
+
+int stairs_validate(stairs_ctx* ctx, int n_req, const int32_t* req_ids_host, const int32_t* k_host,
+                    const int32_t* draft_dev, int32_t* target_tokens_dev, int32_t* accept_len_dev,
+                    float* logits_dev_or_null, int commit) {
+  if (!ctx) return STAIRS_EINVAL;
+  if (n_req <= 0 || n_req > ctx->cfg.max_requests || !req_ids_host || !k_host || !target_tokens_dev || !accept_len_dev)
+    return fail(ctx, STAIRS_EINVAL, "bad validate arguments");
+  std::vector<int> off(n_req);
+  int T = 0;
+  for (int i = 0; i < n_req; ++i) {
+    int rc = check_slot(ctx, req_ids_host[i], true);
+    if (rc) return rc;
+    for (int j = 0; j < i; ++j)
+      if (req_ids_host[j] == req_ids_host[i]) return fail(ctx, STAIRS_EINVAL, "request %d listed twice", req_ids_host[i]);
+    if (k_host[i] < 0 || k_host[i] > ctx->cfg.k_max) return fail(ctx, STAIRS_EINVAL, "k[%d]=%d outside 0..k_max", i, k_host[i]);
+    if (k_host[i] > 0 && !draft_dev) return fail(ctx, STAIRS_EINVAL, "draft_dev is NULL");
+    off[i] = T;
+    T += k_host[i] + 1;
+  }
+  for (int i = 0; i < n_req; ++i) {
+    const int slot = req_ids_host[i];
+    const int need = ctx->n_seq_ub[slot] + k_host[i] + 1;  // sequence length after a full accept
+    if (need > ctx->cfg.max_seq_len) return fail(ctx, STAIRS_ENOSPC, "request %d: sequence would exceed max_seq_len", slot);
+    int rc = ensure_pages(ctx, slot, need);
+    if (rc) return rc;
+  }
+  char* ws = ctx->ws;
+  const Layout& L = ctx->lay;
+  CK(cudaMemcpyAsync(ws + L.val_req, req_ids_host, (size_t)n_req * 4, cudaMemcpyHostToDevice, ctx->stream));
+  CK(cudaMemcpyAsync(ws + L.val_k, k_host, (size_t)n_req * 4, cudaMemcpyHostToDevice, ctx->stream));
+  CK(cudaMemcpyAsync(ws + L.val_off, off.data(), (size_t)n_req * 4, cudaMemcpyHostToDevice, ctx->stream));
+  if (ctx->profile) { ctx->ev_used = 0; cudaEventRecord(ctx->call_begin, ctx->stream); }
+  ctx->in_validate = true;
+  RowParams p = base_rows(ctx);
+  p.mode = ROWS_VALIDATE; p.n_req = n_req; p.draft = draft_dev;
+  int rc = launch_rows(ctx, p, n_req * (ctx->cfg.k_max + 1));
+  if (!rc) rc = forward(ctx, ctx->target, T, 0, T, logits_dev_or_null);
+  ctx->in_validate = false;
+  if (rc) return rc;
+  AcceptParams a{};
+  a.n_req = n_req; a.val_req = p.val_req; a.val_k = p.val_k; a.val_off = p.val_off;
+  a.draft = draft_dev; a.k_max = ctx->cfg.k_max;
+  a.keys = reinterpret_cast<unsigned long long*>(ws + L.keys);
+  a.target_tokens = target_tokens_dev; a.accept_len = accept_len_dev; a.commit = commit;
+  a.seq = reinterpret_cast<int*>(ws + L.seq); a.n_seq = reinterpret_cast<int*>(ws + L.n_seq);
+  a.max_seq_len = ctx->cfg.max_seq_len;
+  k_accept<<<(n_req + 63) / 64, 64, 0, ctx->stream>>>(a);
+  ctx->launches++;
+  CK(cudaGetLastError());
+  if (ctx->profile) cudaEventRecord(ctx->call_end, ctx->stream);
+  if (commit)
+    for (int i = 0; i < n_req; ++i) ctx->n_seq_ub[req_ids_host[i]] += k_host[i] + 1;
+  return STAIRS_OK;
+}
+
+int stairs_validate_host(stairs_ctx* ctx, int n_req, const int32_t* req_ids_host, const int32_t* k_host,
+                         const int32_t* draft_host, int32_t* target_tokens_host, int32_t* accept_len_host, int commit) {
+  if (!ctx) return STAIRS_EINVAL;
+  if (n_req <= 0 || n_req > ctx->cfg.max_requests || !target_tokens_host || !accept_len_host)
+    return fail(ctx, STAIRS_EINVAL, "bad validate arguments");
+  char* ws = ctx->ws;
+  const Layout& L = ctx->lay;
+  const int km = ctx->cfg.k_max;
+  int* d_dev = reinterpret_cast<int*>(ws + L.draft_buf);
+  int* tt_dev = reinterpret_cast<int*>(ws + L.tt_buf);
+  int* al_dev = reinterpret_cast<int*>(ws + L.al_buf);
+  if (km > 0 && draft_host)
+    CK(cudaMemcpyAsync(d_dev, draft_host, (size_t)n_req * km * 4, cudaMemcpyHostToDevice, ctx->stream));
+  int rc = stairs_validate(ctx, n_req, req_ids_host, k_host, draft_host ? d_dev : nullptr, tt_dev, al_dev, nullptr, commit);
+  if (rc) return rc;
+  CK(cudaMemcpyAsync(target_tokens_host, tt_dev, (size_t)n_req * (km + 1) * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  CK(cudaMemcpyAsync(accept_len_host, al_dev, (size_t)n_req * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  rc = stairs_sync(ctx);
+  if (rc) return rc;
+  if (commit)  // the host now knows the exact new lengths
+    for (int i = 0; i < n_req; ++i) ctx->n_seq_ub[req_ids_host[i]] += accept_len_host[i] - k_host[i];
+  return STAIRS_OK;
+}
+
+int stairs_generate(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_prompt, int k, int max_new,
+                    int32_t eos, int32_t* out_host, int32_t* n_out, stairs_stats* stats) {
+  int rc = check_slot(ctx, req, false);
+  if (rc) return rc;
+  if (!out_host || !n_out || max_new < 0) return fail(ctx, STAIRS_EINVAL, "bad generate arguments");
+  if (k < 0 || k > ctx->cfg.k_max) return fail(ctx, STAIRS_EINVAL, "k=%d outside 0..k_max", k);
+  if (k > 0 && !ctx->draft.present) return fail(ctx, STAIRS_ESTATE, "k > 0 needs a draft model");
+  if (n_prompt + max_new > ctx->cfg.max_seq_len) return fail(ctx, STAIRS_ENOSPC, "prompt + max_new exceeds max_seq_len");
+  stairs_stats s{};
+  cudaEvent_t e0, e1, e2, e3;
+  CK(cudaEventCreate(&e0)); CK(cudaEventCreate(&e1)); CK(cudaEventCreate(&e2)); CK(cudaEventCreate(&e3));
+  auto cleanup = [&]() { cudaEventDestroy(e0); cudaEventDestroy(e1); cudaEventDestroy(e2); cudaEventDestroy(e3); };
+  cudaEventRecord(e0, ctx->stream);
+  rc = stairs_prefill(ctx, req, prompt_host, n_prompt);
+  cudaEventRecord(e1, ctx->stream);
+  if (!rc) rc = stairs_sync(ctx);
+  if (rc) { cleanup(); return rc; }
+  float ms = 0.f;
+  cudaEventElapsedTime(&ms, e0, e1);
+  s.prefill_ms = ms;
+  const int km = ctx->cfg.k_max;
+  int* d_dev = reinterpret_cast<int*>(ctx->ws + ctx->lay.draft_buf);
+  int* tt_dev = reinterpret_cast<int*>(ctx->ws + ctx->lay.tt_buf);
+  int* al_dev = reinterpret_cast<int*>(ctx->ws + ctx->lay.al_buf);
+  std::vector<int> tt(km + 1);
+  std::vector<int> draft_h(std::max(km, 1));
+  int produced = 0;
+  bool stop = false;
+  while (produced < max_new && !stop) {
+    const int k_eff = std::min(k, max_new - produced - 1);
+    int al = 0;
+    cudaEventRecord(e1, ctx->stream);
+    if (k_eff > 0 && (rc = stairs_draft(ctx, req, k_eff, d_dev))) break;
+    cudaEventRecord(e2, ctx->stream);
+    if ((rc = stairs_validate(ctx, 1, &req, &k_eff, d_dev, tt_dev, al_dev, nullptr, 1))) break;
+    cudaEventRecord(e3, ctx->stream);
+    if (k_eff > 0) cudaMemcpyAsync(draft_h.data(), d_dev, (size_t)k_eff * 4, cudaMemcpyDeviceToHost, ctx->stream);
+    cudaMemcpyAsync(tt.data(), tt_dev, (size_t)(k_eff + 1) * 4, cudaMemcpyDeviceToHost, ctx->stream);
+    cudaMemcpyAsync(&al, al_dev, 4, cudaMemcpyDeviceToHost, ctx->stream);
+    if ((rc = stairs_sync(ctx))) break;
+    ctx->n_seq_ub[req] += al - k_eff;
+    cudaEventElapsedTime(&ms, e1, e2); s.draft_ms += ms;
+    cudaEventElapsedTime(&ms, e2, e3); s.validate_ms += ms;
+    s.iterations++; s.drafted += k_eff; s.accepted += al;
+    for (int r = 0; r <= al && !stop; ++r) {
+      const int t = r < al ? draft_h[r] : tt[al];
+      if (produced < max_new) out_host[produced] = t;
+      produced++; s.emitted++;
+      if (eos >= 0 && t == eos) stop = true;
+    }
+  }
+  if (!rc) {
+    cudaEventRecord(e3, ctx->stream);
+    rc = stairs_sync(ctx);
+    cudaEventElapsedTime(&ms, e0, e3);
+    s.total_ms = ms;
+  }
+  cleanup();
+  if (rc) return rc;
+  *n_out = std::min(produced, max_new);
+  if (stats) *stats = s;
+  return STAIRS_OK;
+}
+
+int stairs_sequence(stairs_ctx* ctx, int req, int32_t* seq_host, int capacity, int32_t* n_seq) {
+  int rc = check_slot(ctx, req, true);
+  if (rc) return rc;
+  if (!n_seq) return fail(ctx, STAIRS_EINVAL, "n_seq is NULL");
+  int n = 0;
+  CK(cudaMemcpyAsync(&n, reinterpret_cast<int*>(ctx->ws + ctx->lay.n_seq) + req, 4, cudaMemcpyDeviceToHost, ctx->stream));
+  if ((rc = stairs_sync(ctx))) return rc;
+  *n_seq = n;
+  ctx->n_seq_ub[req] = n;
+  if (seq_host && capacity > 0) {
+    const int* seq = reinterpret_cast<int*>(ctx->ws + ctx->lay.seq) + (size_t)req * ctx->cfg.max_seq_len;
+    CK(cudaMemcpyAsync(seq_host, seq, (size_t)std::min(n, capacity) * 4, cudaMemcpyDeviceToHost, ctx->stream));
+    rc = stairs_sync(ctx);
+  }
+  return rc;
+}
+
+int stairs_sync(stairs_ctx* ctx) {
+  if (!ctx) return STAIRS_EINVAL;
+  CK(cudaStreamSynchronize(ctx->stream));
+  return STAIRS_OK;
+}
+
+int64_t stairs_launch_count(const stairs_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int stairs_profile(stairs_ctx* ctx, int enable) {
+  if (!ctx) return STAIRS_EINVAL;
+  if (enable && ctx->ev.empty()) {
+    ctx->ev.resize(4096);
+    for (auto& e : ctx->ev) CK(cudaEventCreate(&e));
+  }
+  ctx->profile = enable != 0;
+  ctx->ev_used = 0;
+  return STAIRS_OK;
+}
+
+int stairs_profile_read(stairs_ctx* ctx, float* gemm_ms, int32_t* gemm_launches, float* call_ms) {
+  if (!ctx) return STAIRS_EINVAL;
+  if (!ctx->profile) return fail(ctx, STAIRS_ESTATE, "profiling is off");
+  int rc = stairs_sync(ctx);
+  if (rc) return rc;
+  float total = 0.f;
+  for (int i = 0; i + 1 < ctx->ev_used; i += 2) {
+    float ms = 0.f;
+    CK(cudaEventElapsedTime(&ms, ctx->ev[i], ctx->ev[i + 1]));
+    total += ms;
+  }
+  if (gemm_ms) *gemm_ms = total;
+  if (gemm_launches) *gemm_launches = ctx->ev_used / 2;
+  if (call_ms) { float ms = 0.f; CK(cudaEventElapsedTime(&ms, ctx->call_begin, ctx->call_end)); *call_ms = ms; }
+  return STAIRS_OK;
+}
+
+int stairs_reset(stairs_ctx* ctx, int req) {
+  int rc = check_slot(ctx, req, false);
+  if (rc) return rc;
+  release_pages(ctx, req);
+  int zero = 0;
+  CK(cudaMemcpyAsync(reinterpret_cast<int*>(ctx->ws + ctx->lay.n_seq) + req, &zero, 4, cudaMemcpyHostToDevice, ctx->stream));
+  return STAIRS_OK;
+}
+
+int stairs_destroy(stairs_ctx* ctx) {
+  if (!ctx) return STAIRS_EINVAL;
+  cudaStreamSynchronize(ctx->stream);
+  for (auto& e : ctx->ev) cudaEventDestroy(e);
+  if (ctx->call_begin) cudaEventDestroy(ctx->call_begin);
+  if (ctx->call_end) cudaEventDestroy(ctx->call_end);
+  delete ctx;
+  return STAIRS_OK;
+}
+
+const char* stairs_last_error(const stairs_ctx* ctx) { return ctx ? ctx->err.c_str() : g_init_error.c_str(); }
+
+}  // extern "C"

@@ -252,7 +252,8 @@ class WeightSource:
         if not src.shape.has_tensor(name):
             return None
         if src.backend == "torch-cuda":
-            t = self.torch_tensor(layer, name, "cuda").cpu()
+            cached = [v for k, v in src._cache.items() if k.startswith(f"{layer}:{name}:")]
+            t = (cached[0] if cached else self.torch_tensor(layer, name, "cuda")).cpu()
             if t.dtype == torch.bfloat16:
                 return t.view(torch.int16).numpy().view(np.uint16)
             return t.numpy()
