@@ -4,14 +4,17 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <new>
 #include <string>
+#include <tuple>
 #include <type_traits>
 #include <vector>
 
 #include "../../include/stairs.h"
 #include "common.cuh"
 #include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
 #include "kernels_basic.cuh"
 
 using namespace stairs;
@@ -20,7 +23,18 @@ namespace {
 
 thread_local std::string g_init_error;
 
+struct LayerMaps { CUtensorMap wq, wk, wv, wo, w1, w3, w2; };
+
+constexpr int TC_GRID_MAX = 160;        // scratch is sized for at most this many CTAs
+constexpr int TC_COUNTERS = 1 << 16;    // tiles per GEMM the split bookkeeping can hold
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
 struct DevModel {
+  std::vector<LayerMaps> maps;   // tensor maps of the bf16 weight matrices (tensor-core path)
+  CUtensorMap head_map{};
   stairs_model m{};
   bool present = false;
   stairs_weights w{};
@@ -32,8 +46,8 @@ struct DevModel {
 
 struct Layout {
   size_t status, seq, n_seq, page_table, tok, pos, req, val_req, val_k, val_off, keys, x, h, qkv, q,
-      o, ff, logits, draft_buf, tt_buf, al_buf, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
-  int max_rows, logit_rows, max_pages, n_pages;
+      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
+  int max_rows, logit_rows, max_pages, n_pages, t_box_max;
   size_t kv_t_layer, kv_d_layer;
 };
 
@@ -58,6 +72,14 @@ struct stairs_ctx {
   int ev_used = 0;
   cudaEvent_t call_begin = nullptr, call_end = nullptr;
   bool in_validate = false;
+  // tensor-core path
+  bool use_tc = false;
+  int sm_count = 0;
+  EncodeTiledFn encode = nullptr;
+  std::map<std::tuple<const void*, int, int>, CUtensorMap> act_maps;
+  unsigned int* status_host = nullptr;  // pinned, device-visible status words
+  unsigned int* status_dev = nullptr;
+  unsigned long long wait_limit = 0;
 };
 
 namespace {
@@ -118,7 +140,8 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
   if (c.target.pos == 0 && c.max_seq_len > c.target.max_pos) { *why = "max_seq_len exceeds max_pos of the learned positions"; return false; }
   if (c.kv_pages < 0 || c.prefill_chunk < 0) { *why = "kv_pages and prefill_chunk must not be negative"; return false; }
   const int chunk = c.prefill_chunk > 0 ? c.prefill_chunk : 256;
-  L->max_rows = std::max(std::max(chunk, c.max_requests * (c.k_max + 1)), 2);
+  L->max_rows = (std::max(std::max(chunk, c.max_requests * (c.k_max + 1)), 2) + 15) / 16 * 16;
+  L->t_box_max = std::min(256, L->max_rows);
   L->logit_rows = std::max(c.max_requests * (c.k_max + 1), 1);
   L->max_pages = (c.max_seq_len + pt - 1) / pt;
   L->n_pages = c.kv_pages > 0 ? c.kv_pages : L->max_pages * c.max_requests;
@@ -152,6 +175,8 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
   L->draft_buf = take((size_t)c.max_requests * std::max(c.k_max, 1) * 4);
   L->tt_buf = take((size_t)c.max_requests * (c.k_max + 1) * 4);
   L->al_buf = take((size_t)c.max_requests * 4);
+  L->gemm_partial = take(t.wdtype == 1 ? (size_t)TC_GRID_MAX * 2 * L->t_box_max * tc::BM * 4 : 0);
+  L->gemm_counters = take(t.wdtype == 1 ? (size_t)TC_COUNTERS * 4 : 0);
   const size_t pool_tokens = (size_t)L->n_pages * pt;
   L->kv_t_layer = pool_tokens * t.n_kv_heads * t.head_dim * es;
   L->kv_t_k = take(L->kv_t_layer * t.n_layers);
@@ -190,6 +215,112 @@ void release_pages(stairs_ctx* ctx, int slot) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Tensor-core GEMM plumbing: tensor maps and job set-up.
+// ---------------------------------------------------------------------------------------------
+// 2-D map of a row-major bf16 matrix [rows, K]; box = 64 k-elements x box_rows rows, 128-byte swizzle.
+bool encode_map(stairs_ctx* ctx, CUtensorMap* out, const void* ptr, long long rows, long long K, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {(cuuint32_t)tc::BK, (cuuint32_t)box_rows};
+  cuuint32_t es[2] = {1, 1};
+  CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int build_weight_maps(stairs_ctx* ctx, DevModel& M) {
+  const stairs_model& m = M.m;
+  const int nq = m.n_heads * m.head_dim, nkv = m.n_kv_heads * m.head_dim;
+  M.maps.resize(m.n_layers);
+  bool ok = true;
+  for (int l = 0; l < m.n_layers && ok; ++l) {
+    const stairs_layer_w& w = M.layers[l];
+    LayerMaps& t = M.maps[l];
+    ok = ok && encode_map(ctx, &t.wq, w.wq, nq, m.d_model, tc::BM);
+    ok = ok && encode_map(ctx, &t.wk, w.wk, nkv, m.d_model, tc::BM);
+    ok = ok && encode_map(ctx, &t.wv, w.wv, nkv, m.d_model, tc::BM);
+    ok = ok && encode_map(ctx, &t.wo, w.wo, m.d_model, nq, tc::BM);
+    if (m.act == 1) {
+      ok = ok && encode_map(ctx, &t.w1, w.w_gate_or_fc1, m.d_ff, m.d_model, 64);
+      ok = ok && encode_map(ctx, &t.w3, w.w_up, m.d_ff, m.d_model, 64);
+    } else {
+      ok = ok && encode_map(ctx, &t.w1, w.w_gate_or_fc1, m.d_ff, m.d_model, tc::BM);
+    }
+    ok = ok && encode_map(ctx, &t.w2, w.w_down_or_fc2, m.d_model, m.d_ff, tc::BM);
+  }
+  ok = ok && encode_map(ctx, &M.head_map, M.w.lm_head, m.vocab, m.d_model, tc::BM);
+  if (!ok) return fail(ctx, STAIRS_ECUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
+  return STAIRS_OK;
+}
+
+struct TcArgs {
+  const CUtensorMap* w[3] = {nullptr, nullptr, nullptr};
+  int rows[3] = {0, 0, 0};   // output features of each source
+  int n_src = 1;
+  bool dual = false;         // w[0] = gate, w[1] = up; rows[0] = d_ff
+  const void* x = nullptr;   // activations [*, K] bf16
+  int K = 0, T = 0;
+  int epi = tc::TC_STORE_F32;
+  float* out_f32 = nullptr; int ldo = 0;
+  bf16* out_act = nullptr;
+  unsigned long long* keys = nullptr;
+};
+
+int launch_gemm_tc(stairs_ctx* ctx, const TcArgs& a) {
+  tc::GemmJob job;
+  memset(&job, 0, sizeof job);
+  const Layout& L = ctx->lay;
+  job.t_tiles = (a.T + 255) / 256;
+  job.t_box = ((a.T + job.t_tiles - 1) / job.t_tiles + 15) / 16 * 16;
+  job.kblocks = (a.K + tc::BK - 1) / tc::BK;
+  job.dual = a.dual ? 1 : 0;
+  job.n_src = a.n_src;
+  int col = 0, tiles = 0;
+  if (a.dual) {
+    job.w_map[0] = *a.w[0]; job.w_map[1] = *a.w[1]; job.w_map[2] = *a.w[0];
+    job.N = a.rows[0];
+    tiles = (a.rows[0] + 63) / 64;
+    job.src_tiles[0] = tiles;
+  } else {
+    for (int s = 0; s < 3; ++s) {
+      job.w_map[s] = *a.w[s < a.n_src ? s : 0];
+      if (s < a.n_src) {
+        job.src_tiles[s] = (a.rows[s] + tc::BM - 1) / tc::BM;
+        job.src_col[s] = col;
+        col += a.rows[s];
+        tiles += job.src_tiles[s];
+      }
+    }
+    job.N = col;
+  }
+  job.n_tiles = tiles;
+  job.T = a.T;
+  if (job.t_box > L.t_box_max || (long long)tiles * job.t_tiles > TC_COUNTERS)
+    return fail(ctx, STAIRS_EUNSUPPORTED, "GEMM shape outside the tensor-core path's scratch");
+  auto key = std::make_tuple(a.x, a.K, job.t_box);
+  auto it = ctx->act_maps.find(key);
+  if (it == ctx->act_maps.end()) {
+    CUtensorMap mp;
+    if (!encode_map(ctx, &mp, a.x, L.max_rows, a.K, job.t_box))
+      return fail(ctx, STAIRS_ECUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+    it = ctx->act_maps.emplace(key, mp).first;
+  }
+  job.x_map = it->second;
+  job.stages = tc::pick_stages(job.t_box);
+  job.epi = a.epi;
+  job.out_f32 = a.out_f32; job.ldo = a.ldo; job.out_act = a.out_act; job.keys = a.keys;
+  job.partial = reinterpret_cast<float*>(ctx->ws + L.gemm_partial);
+  job.counters = reinterpret_cast<int*>(ctx->ws + L.gemm_counters);
+  job.status = ctx->status_dev;
+  job.wait_limit = ctx->wait_limit;
+  const long long total = (long long)tiles * job.t_tiles * job.kblocks;
+  const int grid = (int)std::min<long long>(std::min(ctx->sm_count, TC_GRID_MAX), total);
+  tc::k_gemm_tc<<<grid, tc::THREADS, tc::smem_bytes(job.t_box, job.stages), ctx->stream>>>(job);
+  return STAIRS_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // One forward pass over T rows (tok/pos/req already built on the device).
 // ---------------------------------------------------------------------------------------------
 struct GemmTimer {
@@ -223,48 +354,98 @@ int forward_rows(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, int n
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(ws + L.keys);
   const int pt = ctx->cfg.kv_page_tokens;
 
+  constexpr bool kBf16 = std::is_same<WT, bf16>::value;
+  const bool use_tc = kBf16 && ctx->use_tc;
+  int rc = STAIRS_OK;
   k_embed<WT><<<T, 256, 0, st>>>((const WT*)M.w.tok_emb, (const WT*)M.w.pos_emb, tok, pos, x, d);
   ctx->launches++;
-  for (int l = 0; l < m.n_layers; ++l) {
+  for (int l = 0; l < m.n_layers && !rc; ++l) {
     const stairs_layer_w& w = M.layers[l];
     WT* kc = reinterpret_cast<WT*>(M.kpool + (size_t)l * M.kv_layer_bytes);
     WT* vc = reinterpret_cast<WT*>(M.vpool + (size_t)l * M.kv_layer_bytes);
     k_norm<WT><<<T, 256, 0, st>>>(x, (const float*)w.norm1_w, (const float*)w.norm1_b, h, d, m.norm, m.norm_eps);
     {
       GemmTimer tm(ctx);
-      launch_gemm_rows<WT, false>(st, (const WT*)w.wq, nullptr, h, T, nq, d, EPI_STORE_F32, qkv, nullptr, nqkv);
-      launch_gemm_rows<WT, false>(st, (const WT*)w.wk, nullptr, h, T, nkv, d, EPI_STORE_F32, qkv + nq, nullptr, nqkv);
-      launch_gemm_rows<WT, false>(st, (const WT*)w.wv, nullptr, h, T, nkv, d, EPI_STORE_F32, qkv + nq + nkv, nullptr, nqkv);
+      if (use_tc) {
+        TcArgs a;
+        a.w[0] = &M.maps[l].wq; a.w[1] = &M.maps[l].wk; a.w[2] = &M.maps[l].wv;
+        a.rows[0] = nq; a.rows[1] = nkv; a.rows[2] = nkv; a.n_src = 3;
+        a.x = h; a.K = d; a.T = T; a.epi = tc::TC_STORE_F32; a.out_f32 = qkv; a.ldo = nqkv;
+        rc = launch_gemm_tc(ctx, a);
+        ctx->launches += 1;
+      } else {
+        launch_gemm_rows<WT, false>(st, (const WT*)w.wq, nullptr, h, T, nq, d, EPI_STORE_F32, qkv, nullptr, nqkv);
+        launch_gemm_rows<WT, false>(st, (const WT*)w.wk, nullptr, h, T, nkv, d, EPI_STORE_F32, qkv + nq, nullptr, nqkv);
+        launch_gemm_rows<WT, false>(st, (const WT*)w.wv, nullptr, h, T, nkv, d, EPI_STORE_F32, qkv + nq + nkv, nullptr, nqkv);
+        ctx->launches += 3;
+      }
     }
+    if (rc) break;
     k_rope_append<WT><<<T, 256, 0, st>>>(qkv, pos, req, page_table, q, kc, vc, hq, hkv, hd, m.pos, m.rope_theta, pt, L.max_pages);
     k_attn_plain<WT, 8><<<dim3(hq, T), 128, (size_t)5 * hd * sizeof(float), st>>>(
         q, kc, vc, page_table, req, pos, o, hq, hkv, hd, pt, L.max_pages, 1.0f / sqrtf((float)hd));
     {
       GemmTimer tm(ctx);
-      launch_gemm_rows<WT, false>(st, (const WT*)w.wo, nullptr, o, T, d, nq, EPI_ADD_F32, x, nullptr, d);
+      if (use_tc) {
+        TcArgs a;
+        a.w[0] = &M.maps[l].wo; a.rows[0] = d; a.x = o; a.K = nq; a.T = T;
+        a.epi = tc::TC_ADD_F32; a.out_f32 = x; a.ldo = d;
+        rc = launch_gemm_tc(ctx, a);
+      } else {
+        launch_gemm_rows<WT, false>(st, (const WT*)w.wo, nullptr, o, T, d, nq, EPI_ADD_F32, x, nullptr, d);
+      }
     }
+    if (rc) break;
     k_norm<WT><<<T, 256, 0, st>>>(x, (const float*)w.norm2_w, (const float*)w.norm2_b, h, d, m.norm, m.norm_eps);
     {
       GemmTimer tm(ctx);
-      if (m.act == 1)
-        launch_gemm_rows<WT, true>(st, (const WT*)w.w_gate_or_fc1, (const WT*)w.w_up, h, T, F, d, EPI_SWIGLU, nullptr, ff, F);
-      else
-        launch_gemm_rows<WT, false>(st, (const WT*)w.w_gate_or_fc1, nullptr, h, T, F, d, EPI_GELU, nullptr, ff, F);
-      launch_gemm_rows<WT, false>(st, (const WT*)w.w_down_or_fc2, nullptr, ff, T, d, F, EPI_ADD_F32, x, nullptr, d);
+      if (use_tc) {
+        TcArgs a;
+        a.w[0] = &M.maps[l].w1; a.rows[0] = F; a.x = h; a.K = d; a.T = T;
+        a.out_act = reinterpret_cast<bf16*>(ff); a.ldo = F;
+        if (m.act == 1) { a.w[1] = &M.maps[l].w3; a.dual = true; a.epi = tc::TC_SWIGLU; }
+        else a.epi = tc::TC_GELU;
+        rc = launch_gemm_tc(ctx, a);
+        if (!rc) {
+          TcArgs b;
+          b.w[0] = &M.maps[l].w2; b.rows[0] = d; b.x = ff; b.K = F; b.T = T;
+          b.epi = tc::TC_ADD_F32; b.out_f32 = x; b.ldo = d;
+          rc = launch_gemm_tc(ctx, b);
+        }
+      } else {
+        if (m.act == 1)
+          launch_gemm_rows<WT, true>(st, (const WT*)w.w_gate_or_fc1, (const WT*)w.w_up, h, T, F, d, EPI_SWIGLU, nullptr, ff, F);
+        else
+          launch_gemm_rows<WT, false>(st, (const WT*)w.w_gate_or_fc1, nullptr, h, T, F, d, EPI_GELU, nullptr, ff, F);
+        launch_gemm_rows<WT, false>(st, (const WT*)w.w_down_or_fc2, nullptr, ff, T, d, F, EPI_ADD_F32, x, nullptr, d);
+      }
     }
-    ctx->launches += 10;
+    ctx->launches += 7;
   }
+  if (rc) return rc;
   if (n_logit_rows > 0) {
-    float* lg = logits_out ? logits_out : reinterpret_cast<float*>(ws + L.logits);
     k_norm<WT><<<n_logit_rows, 256, 0, st>>>(x + (size_t)logit_first_row * d, (const float*)M.w.final_norm_w,
                                              (const float*)M.w.final_norm_b, h, d, m.norm, m.norm_eps);
-    {
+    ctx->launches += 1;
+    if (use_tc) {
+      // LM head with the vocabulary argmax fused into the epilogue; logits are stored only on request
       GemmTimer tm(ctx);
-      launch_gemm_rows<WT, false>(st, (const WT*)M.w.lm_head, nullptr, h, n_logit_rows, m.vocab, d, EPI_STORE_F32, lg, nullptr, m.vocab);
+      TcArgs a;
+      a.w[0] = &M.head_map; a.rows[0] = m.vocab; a.x = h; a.K = d; a.T = n_logit_rows;
+      a.epi = tc::TC_LMHEAD; a.out_f32 = logits_out; a.ldo = m.vocab; a.keys = keys + logit_first_row;
+      rc = launch_gemm_tc(ctx, a);
+      ctx->launches += 1;
+      if (rc) return rc;
+    } else {
+      float* lg = logits_out ? logits_out : reinterpret_cast<float*>(ws + L.logits);
+      {
+        GemmTimer tm(ctx);
+        launch_gemm_rows<WT, false>(st, (const WT*)M.w.lm_head, nullptr, h, n_logit_rows, m.vocab, d, EPI_STORE_F32, lg, nullptr, m.vocab);
+      }
+      const int slices = std::max(1, std::min(64, m.vocab / 2048));
+      k_argmax<<<dim3(slices, n_logit_rows), 256, 0, st>>>(lg, m.vocab, m.vocab, keys + logit_first_row);
+      ctx->launches += 2;
     }
-    const int slices = std::max(1, std::min(64, m.vocab / 2048));
-    k_argmax<<<dim3(slices, n_logit_rows), 256, 0, st>>>(lg, m.vocab, m.vocab, keys + logit_first_row);
-    ctx->launches += 3;
   }
   CK(cudaGetLastError());
   return STAIRS_OK;
@@ -393,6 +574,8 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
   // clear status words, sequences, lengths and page tables (KV pages need no clearing: a
   // position is always written before it becomes visible)
   e = cudaMemsetAsync(ctx->ws, 0, L.tok, ctx->stream);
+  if (e == cudaSuccess && L.kv_t_k > L.gemm_counters)  // split-tile counters start at zero and return to zero
+    e = cudaMemsetAsync(ctx->ws + L.gemm_counters, 0, L.kv_t_k - L.gemm_counters, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
   if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_begin);
   if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_end);
@@ -400,6 +583,48 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
     int rc = fail(nullptr, STAIRS_ECUDA, "context set-up failed: %s", cudaGetErrorString(e));
     delete ctx;
     return rc;
+  }
+  // tensor-core path: bf16 weights on a device with tcgen05 (compute capability 10.x)
+  {
+    int major = 0;
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, cfg->device);
+    cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
+    ctx->wait_limit = cfg->wait_limit_cycles ? cfg->wait_limit_cycles : 2000000000ull;
+    e = cudaHostAlloc(reinterpret_cast<void**>(&ctx->status_host), STATUS_WORDS * 4, cudaHostAllocMapped);
+    if (e == cudaSuccess) {
+      memset(ctx->status_host, 0, STATUS_WORDS * 4);
+      e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&ctx->status_dev), ctx->status_host, 0);
+    }
+    if (e != cudaSuccess) {
+      int rc = fail(nullptr, STAIRS_ECUDA, "status word set-up failed: %s", cudaGetErrorString(e));
+      delete ctx;
+      return rc;
+    }
+    if (cfg->target.wdtype == 1 && cfg->gemm_impl == 0) {
+      if (major != 10) {
+        int rc = fail(nullptr, STAIRS_EUNSUPPORTED, "bf16 models need an sm_100 device (found compute capability %d.x)", major);
+        stairs_destroy(ctx);
+        return rc;
+      }
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+      if (e != cudaSuccess || !fn || qres != cudaDriverEntryPointSuccess) {
+        int rc = fail(nullptr, STAIRS_ECUDA, "cuTensorMapEncodeTiled is not available from the driver");
+        stairs_destroy(ctx);
+        return rc;
+      }
+      ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+      e = cudaFuncSetAttribute(tc::k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_LIMIT);
+      int rc = e == cudaSuccess ? build_weight_maps(ctx, ctx->target) : fail(ctx, STAIRS_ECUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+      if (!rc && has_draft) rc = build_weight_maps(ctx, ctx->draft);
+      if (rc) {
+        g_init_error = ctx->err;
+        stairs_destroy(ctx);
+        return rc;
+      }
+      ctx->use_tc = true;
+    }
   }
   *out = ctx;
   return STAIRS_OK;
@@ -616,6 +841,11 @@ int stairs_sequence(stairs_ctx* ctx, int req, int32_t* seq_host, int capacity, i
 int stairs_sync(stairs_ctx* ctx) {
   if (!ctx) return STAIRS_EINVAL;
   CK(cudaStreamSynchronize(ctx->stream));
+  if (ctx->status_host && ctx->status_host[STATUS_ERROR]) {
+    const unsigned int code = ctx->status_host[STATUS_ERROR];
+    ctx->status_host[STATUS_ERROR] = 0;
+    return fail(ctx, (int)code, "a device-side bounded wait expired (code %u); results of the last calls are invalid", code);
+  }
   return STAIRS_OK;
 }
 
@@ -664,6 +894,7 @@ int stairs_destroy(stairs_ctx* ctx) {
   for (auto& e : ctx->ev) cudaEventDestroy(e);
   if (ctx->call_begin) cudaEventDestroy(ctx->call_begin);
   if (ctx->call_end) cudaEventDestroy(ctx->call_end);
+  if (ctx->status_host) cudaFreeHost(ctx->status_host);
   delete ctx;
   return STAIRS_OK;
 }
