@@ -171,6 +171,11 @@ int stairs_generate(stairs_ctx *ctx, int req, const int32_t *prompt_host, int n_
  * capacity tokens of the sequence) to the host.  Waits. */
 int stairs_sequence(stairs_ctx *ctx, int req, int32_t *seq_host, int capacity, int32_t *n_seq);
 
+/* Rolls request `req` back to its first n_tokens committed tokens (2 <= n_tokens <= current
+ * length; the host must know the current length, e.g. from stairs_sequence).  Cache entries
+ * past the new end are simply overwritten by later calls.  Enqueued on the stream. */
+int stairs_truncate(stairs_ctx *ctx, int req, int n_tokens);
+
 /* Waits for the stream and reports a device-side failure recorded since the last call
  * (ETIMEOUT if a bounded wait expired). */
 int stairs_sync(stairs_ctx *ctx);

@@ -838,6 +838,15 @@ int stairs_sequence(stairs_ctx* ctx, int req, int32_t* seq_host, int capacity, i
   return rc;
 }
 
+int stairs_truncate(stairs_ctx* ctx, int req, int n_tokens) {
+  int rc = check_slot(ctx, req, true);
+  if (rc) return rc;
+  if (n_tokens < 2 || n_tokens > ctx->n_seq_ub[req]) return fail(ctx, STAIRS_EINVAL, "truncate length %d outside 2..%d", n_tokens, ctx->n_seq_ub[req]);
+  CK(cudaMemcpyAsync(reinterpret_cast<int*>(ctx->ws + ctx->lay.n_seq) + req, &n_tokens, 4, cudaMemcpyHostToDevice, ctx->stream));
+  ctx->n_seq_ub[req] = n_tokens;
+  return STAIRS_OK;
+}
+
 int stairs_sync(stairs_ctx* ctx) {
   if (!ctx) return STAIRS_EINVAL;
   CK(cudaStreamSynchronize(ctx->stream));

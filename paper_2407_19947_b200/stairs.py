@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libstairs_b200.so")
 STATUS = {0: "OK", 1: "EINVAL", 2: "ENOSPC", 3: "ESTATE", 4: "ECUDA", 5: "ETIMEOUT", 6: "EUNSUPPORTED"}
 
 EXPORTS = ["stairs_workspace_bytes", "stairs_init", "stairs_prefill", "stairs_draft", "stairs_validate",
-           "stairs_validate_host", "stairs_generate", "stairs_sequence", "stairs_sync",
+           "stairs_validate_host", "stairs_generate", "stairs_sequence", "stairs_truncate", "stairs_sync",
            "stairs_launch_count", "stairs_profile", "stairs_profile_read", "stairs_reset",
            "stairs_destroy", "stairs_last_error"]
 
@@ -82,6 +82,7 @@ def load_library(path: Optional[str] = None):
     lib.stairs_generate.argtypes = [vp, C.c_int, i32p, C.c_int, C.c_int, C.c_int, C.c_int32, i32p, i32p,
                                     C.POINTER(CStats)]
     lib.stairs_sequence.argtypes = [vp, C.c_int, i32p, C.c_int, i32p]
+    lib.stairs_truncate.argtypes = [vp, C.c_int, C.c_int]
     lib.stairs_sync.argtypes = [vp]
     lib.stairs_launch_count.restype = C.c_int64
     lib.stairs_launch_count.argtypes = [vp]
@@ -256,6 +257,9 @@ class Stairs:
         n = C.c_int32(0)
         self._ck(self.lib.stairs_sequence(self.h, req, _ptr(buf), cap, C.byref(n)))
         return [int(x) for x in buf[: n.value]]
+
+    def truncate(self, req: int, n_tokens: int):
+        self._ck(self.lib.stairs_truncate(self.h, req, n_tokens))
 
     def sync(self):
         self._ck(self.lib.stairs_sync(self.h))

@@ -31,7 +31,7 @@ def small_a(layers=3, d=256, heads=4, f=512, v=2048, wdtype=wl.WDTYPE_BF16):
     return wl.family_a(layers, d, heads, f, v, 512, wdtype)
 
 
-def sources(shape, draft_layers=1, std=0.05, jitter=0.1, seed=7):
+def sources(shape, draft_layers=1, std=0.03, jitter=0.1, seed=7):
     tsrc = wl.WeightSource(shape, seed, "numpy", norm_jitter=jitter, std=std)
     dshape = shape.replace(n_layers=draft_layers)
     dsrc = wl.WeightSource(dshape, seed, "numpy", norm_jitter=jitter, std=std,
@@ -155,7 +155,7 @@ def test_gpu_stairs_equals_gpu_greedy_token_for_token(early_exit):
     tsrc, dsrc = sources(shape, draft_layers=2)
     if not early_exit:
         dshape = shape.replace(n_layers=2)
-        dsrc = wl.WeightSource(dshape, 99, "numpy", norm_jitter=0.1, std=0.05, share_globals_with=tsrc)
+        dsrc = wl.WeightSource(dshape, 99, "numpy", norm_jitter=0.1, std=0.03, share_globals_with=tsrc)
     eng = st.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=160, k_max=6, kv_page_tokens=16)
     prompt = list(wl.zipf_tokens(50, shape.vocab, 8))
     ref, _ = eng.generate(0, prompt, 0, 64)
