@@ -199,6 +199,39 @@ int stairs_destroy(stairs_ctx *ctx);
  * a failed stairs_init / stairs_workspace_bytes on this thread. */
 const char *stairs_last_error(const stairs_ctx *ctx);
 
+/* Greedy token per row and accept length per request, computed from logits the caller
+ * already holds - for callers that must not allocate device memory at all.  (The paper has
+ * no counterpart to this entry point; it exists for the callers described here.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a memory pool that
+ * owns the whole device, in a latency-critical section where an allocation would
+ * synchronise the device, or in a plug-in that is only handed finished buffers.  Such a
+ * caller cannot create a context either, because a context needs a workspace.  This call
+ * takes only inputs and outputs; its one piece of scratch (one packed 64-bit argmax key per
+ * row) lives in a fixed array inside the library, 8 KB, which every GPU that loads the
+ * library holds until the process exits.  It calls no cudaMalloc/cudaFree and no allocating
+ * library routine.
+ *
+ *   logits_dev        fp32 [n_rows, ld], row r of request i at row off(i)+r, where off(i) is
+ *                     the sum of k_host[j]+1 over j < i; n_rows = sum of k_host[i]+1
+ *   draft_dev         int32 [n_req, k_max]
+ *   target_tokens_dev int32 [n_req, k_max+1]   (out) argmax of each row, lowest id on ties
+ *   accept_len_dev    int32 [n_req]            (out) first r with draft[r] != target[r], else k
+ *
+ * Limits: n_rows <= STAIRS_STATIC_MAX_ROWS, 1 <= n_req <= STAIRS_STATIC_MAX_REQ,
+ * 0 <= k_host[i] <= k_max <= 63; anything larger returns STAIRS_ENOSPC or STAIRS_EINVAL with
+ * a text in stairs_last_error(NULL).  Work is enqueued on `stream` (NULL = default stream)
+ * of the current device.  The first call on a device looks up the array's device address
+ * (cudaGetSymbolAddress); make that first call before starting any stream capture.  All
+ * calls share the array and it keeps the previous call's keys: each call clears the part it
+ * uses before use, and two calls that overlap on the GPU (different streams, no ordering
+ * between them) race on it - order them. */
+#define STAIRS_STATIC_MAX_ROWS 1024
+#define STAIRS_STATIC_MAX_REQ 64
+int stairs_accept_static(const float *logits_dev, int vocab, int ld, int n_req, const int32_t *k_host,
+                         const int32_t *draft_dev, int k_max, int32_t *target_tokens_dev,
+                         int32_t *accept_len_dev, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -911,3 +911,84 @@ int stairs_destroy(stairs_ctx* ctx) {
 const char* stairs_last_error(const stairs_ctx* ctx) { return ctx ? ctx->err.c_str() : g_init_error.c_str(); }
 
 }  // extern "C"
+
+// =============================================================================================
+// Allocation-free argmax + accept on caller-provided logits (see stairs_accept_static in the
+// header).  The only scratch, one packed argmax key per row, is this fixed device array; the
+// host side must not use the symbol itself as a pointer, so its device address is looked up
+// once per device with cudaGetSymbolAddress.
+// =============================================================================================
+namespace {
+
+static __device__ __align__(256) unsigned long long g_static_keys[STAIRS_STATIC_MAX_ROWS];
+
+struct StaticAcceptParams {
+  int n_req, k_max;
+  int k[STAIRS_STATIC_MAX_REQ];
+  int off[STAIRS_STATIC_MAX_REQ];
+  const int* draft;
+  int* target_tokens;
+  int* accept_len;
+};
+
+// Same walk as k_accept without the commit step; reads the keys from the fixed array directly.
+__global__ void k_accept_static(const __grid_constant__ StaticAcceptParams p) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= p.n_req) return;
+  const int k = p.k[i], off = p.off[i];
+  int a = -1;
+  for (int r = 0; r <= k; ++r) {
+    const int tr = argmax_key_index(g_static_keys[off + r]);
+    p.target_tokens[i * (p.k_max + 1) + r] = tr;
+    if (a < 0 && r < k && p.draft[i * p.k_max + r] != tr) a = r;
+  }
+  p.accept_len[i] = a < 0 ? k : a;
+}
+
+constexpr int kMaxDevices = 64;
+unsigned long long* g_static_keys_addr[kMaxDevices] = {};
+
+}  // namespace
+
+extern "C" int stairs_accept_static(const float* logits_dev, int vocab, int ld, int n_req, const int32_t* k_host,
+                                    const int32_t* draft_dev, int k_max, int32_t* target_tokens_dev,
+                                    int32_t* accept_len_dev, void* stream) {
+  stairs_ctx* ctx = nullptr;  // errors go to the thread-local text read by stairs_last_error(NULL)
+  if (!logits_dev || !k_host || !target_tokens_dev || !accept_len_dev || vocab <= 0 || ld < vocab)
+    return fail(nullptr, STAIRS_EINVAL, "stairs_accept_static: NULL buffer, vocab <= 0 or ld < vocab");
+  if (n_req < 1 || n_req > STAIRS_STATIC_MAX_REQ)
+    return fail(nullptr, STAIRS_ENOSPC, "stairs_accept_static: n_req=%d outside 1..%d", n_req, STAIRS_STATIC_MAX_REQ);
+  if (k_max < 0 || k_max > 63) return fail(nullptr, STAIRS_EINVAL, "stairs_accept_static: k_max=%d outside 0..63", k_max);
+  StaticAcceptParams p{};
+  int rows = 0;
+  for (int i = 0; i < n_req; ++i) {
+    if (k_host[i] < 0 || k_host[i] > k_max)
+      return fail(nullptr, STAIRS_EINVAL, "stairs_accept_static: k[%d]=%d outside 0..k_max=%d", i, k_host[i], k_max);
+    if (k_host[i] > 0 && !draft_dev) return fail(nullptr, STAIRS_EINVAL, "stairs_accept_static: draft_dev is NULL");
+    p.k[i] = k_host[i];
+    p.off[i] = rows;
+    rows += k_host[i] + 1;
+  }
+  if (rows > STAIRS_STATIC_MAX_ROWS)
+    return fail(nullptr, STAIRS_ENOSPC, "stairs_accept_static: %d rows exceed the fixed scratch of %d rows", rows,
+                STAIRS_STATIC_MAX_ROWS);
+  int dev = 0;
+  CK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return fail(nullptr, STAIRS_EUNSUPPORTED, "stairs_accept_static: device ordinal %d", dev);
+  if (!g_static_keys_addr[dev]) {  // once per device, with that device current
+    unsigned long long* ptr = nullptr;
+    CK(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_keys));
+    g_static_keys_addr[dev] = ptr;
+  }
+  unsigned long long* keys = g_static_keys_addr[dev];
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  // the array still holds the previous call's keys: the atomic max below needs zeros
+  CK(cudaMemsetAsync(keys, 0, (size_t)rows * sizeof(unsigned long long), st));
+  const int slices = std::max(1, std::min(64, vocab / 2048));
+  k_argmax<<<dim3(slices, rows), 256, 0, st>>>(logits_dev, vocab, ld, keys);
+  p.n_req = n_req; p.k_max = k_max; p.draft = draft_dev;
+  p.target_tokens = target_tokens_dev; p.accept_len = accept_len_dev;
+  k_accept_static<<<(n_req + 63) / 64, 64, 0, st>>>(p);
+  CK(cudaGetLastError());
+  return STAIRS_OK;
+}

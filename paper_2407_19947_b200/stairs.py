@@ -20,7 +20,9 @@ STATUS = {0: "OK", 1: "EINVAL", 2: "ENOSPC", 3: "ESTATE", 4: "ECUDA", 5: "ETIMEO
 EXPORTS = ["stairs_workspace_bytes", "stairs_init", "stairs_prefill", "stairs_draft", "stairs_validate",
            "stairs_validate_host", "stairs_generate", "stairs_sequence", "stairs_truncate", "stairs_sync",
            "stairs_launch_count", "stairs_profile", "stairs_profile_read", "stairs_reset",
-           "stairs_destroy", "stairs_last_error"]
+           "stairs_destroy", "stairs_last_error", "stairs_accept_static"]
+
+STATIC_MAX_ROWS, STATIC_MAX_REQ = 1024, 64
 
 
 class StairsError(RuntimeError):
@@ -90,6 +92,7 @@ def load_library(path: Optional[str] = None):
     lib.stairs_profile_read.argtypes = [vp, C.POINTER(C.c_float), i32p, C.POINTER(C.c_float)]
     lib.stairs_reset.argtypes = [vp, C.c_int]
     lib.stairs_destroy.argtypes = [vp]
+    lib.stairs_accept_static.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, vp, C.c_int, vp, vp, vp]
     lib.stairs_last_error.restype = C.c_char_p
     lib.stairs_last_error.argtypes = [vp]
     for name in EXPORTS:
@@ -278,3 +281,24 @@ class Stairs:
 
     def reset(self, req: int):
         self._ck(self.lib.stairs_reset(self.h, req))
+
+
+def accept_static(logits_dev, k: Sequence[int], draft_dev, k_max: int, *, vocab: Optional[int] = None, stream=None):
+    """stairs_accept_static: greedy token per row and accept length per request from logits that
+    are already on the device, without a context and without any allocation inside the library
+    (for callers that may not allocate device memory; the output tensors below are allocated
+    here, by the caller's own torch allocator).  logits_dev: fp32 [rows, ld] torch tensor;
+    draft_dev: int32 [n_req, k_max].  Returns (target_tokens [n_req, k_max+1], accept_len [n_req])."""
+    import torch
+    lib = load_library()
+    kk = _i32(k)
+    n = len(kk)
+    tt = torch.zeros((n, k_max + 1), dtype=torch.int32, device=logits_dev.device)
+    al = torch.zeros((n,), dtype=torch.int32, device=logits_dev.device)
+    st = stream if stream is not None else torch.cuda.current_stream()
+    rc = lib.stairs_accept_static(logits_dev.data_ptr(), vocab or logits_dev.shape[1], logits_dev.stride(0), n, _ptr(kk),
+                                  draft_dev.data_ptr() if draft_dev is not None else None, k_max,
+                                  tt.data_ptr(), al.data_ptr(), st.cuda_stream)
+    if rc:
+        raise StairsError(rc, lib.stairs_last_error(None).decode())
+    return tt, al
