@@ -96,8 +96,10 @@ typedef struct stairs_config {
                              max_seq_len                                             */
   int32_t prefill_chunk;  /* rows per prefill pass; 0 = 256                          */
   int32_t device;         /* CUDA device ordinal                                     */
-  int32_t gemm_impl;      /* 0 = best available for the shape, 1 = force the plain
-                             SIMT kernels (reference path for cross-checks)          */
+  int32_t gemm_impl;      /* 0 = best available (bf16: one persistent kernel per pass
+                             of <= 64 rows, tensor-core GEMMs otherwise), 1 = force
+                             the plain SIMT kernels (reference path for cross-checks),
+                             2 = tensor-core GEMMs, one launch per GEMM               */
   void *stream;           /* cudaStream_t, borrowed; NULL = default stream           */
   void *workspace;        /* device memory, 256-byte aligned                         */
   size_t workspace_bytes;
@@ -189,6 +191,11 @@ int64_t stairs_launch_count(const stairs_ctx *ctx);
  * most recent stairs_validate. */
 int stairs_profile(stairs_ctx *ctx, int enable);
 int stairs_profile_read(stairs_ctx *ctx, float *gemm_ms, int32_t *gemm_launches, float *call_ms);
+
+/* Inspection hook for tests: device address and size of one activation buffer inside the
+ * workspace after a pass (which: 0 residual x fp32 [rows, d], 1 normed h, 2 qkv fp32,
+ * 3 attention output o, 4 MLP activation ff, 5 argmax keys u64). */
+int stairs_debug_buffer(stairs_ctx *ctx, int which, void **ptr_dev, size_t *bytes);
 
 /* Frees the slot's KV pages and forgets its sequence. */
 int stairs_reset(stairs_ctx *ctx, int req);

@@ -16,6 +16,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "kernels_basic.cuh"
+#include "megakernel.cuh"
 
 using namespace stairs;
 
@@ -32,7 +33,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+constexpr int MK_MAX_ROWS = 64;          // rows per call the persistent kernel handles
+constexpr int MK_TBOX_SLOTS = MK_MAX_ROWS / 16;
+
 struct DevModel {
+  bool prog_built[MK_TBOX_SLOTS] = {false, false, false, false};
+  char* prog_base = nullptr;     // device: per t_box slot, phases followed by tensor maps
+  size_t prog_slot_bytes = 0, prog_maps_off = 0;
+  int n_phases = 0;
   std::vector<LayerMaps> maps;   // tensor maps of the bf16 weight matrices (tensor-core path)
   CUtensorMap head_map{};
   stairs_model m{};
@@ -46,8 +54,9 @@ struct DevModel {
 
 struct Layout {
   size_t status, seq, n_seq, page_table, tok, pos, req, val_req, val_k, val_off, keys, x, h, qkv, q,
-      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
-  int max_rows, logit_rows, max_pages, n_pages, t_box_max;
+      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_bar, attn_part, prog_t, prog_d, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
+  int max_rows, logit_rows, max_pages, n_pages, t_box_max, attn_units;
+  size_t prog_slot_t, prog_slot_d, prog_maps_off_t, prog_maps_off_d;
   size_t kv_t_layer, kv_d_layer;
 };
 
@@ -80,6 +89,8 @@ struct stairs_ctx {
   unsigned int* status_host = nullptr;  // pinned, device-visible status words
   unsigned int* status_dev = nullptr;
   unsigned long long wait_limit = 0;
+  bool use_mk = false;
+  unsigned long long bar_base = 0;   // grid-barrier arrivals consumed by earlier launches
 };
 
 namespace {
@@ -157,6 +168,7 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   L->status = take(STATUS_WORDS * 4);
+  L->mk_bar = take(64);
   L->seq = take((size_t)c.max_requests * c.max_seq_len * 4);
   L->n_seq = take((size_t)c.max_requests * 4);
   L->page_table = take((size_t)c.max_requests * L->max_pages * 4);
@@ -177,6 +189,24 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
   L->al_buf = take((size_t)c.max_requests * 4);
   L->gemm_partial = take(t.wdtype == 1 ? (size_t)TC_GRID_MAX * 2 * L->t_box_max * tc::BM * 4 : 0);
   L->gemm_counters = take(t.wdtype == 1 ? (size_t)TC_COUNTERS * 4 : 0);
+  {
+    // persistent-kernel scratch: attention unit states and the per-(model, row box) programs
+    const int hkv = mx(t.n_kv_heads, d.n_kv_heads), hdm = mx(t.head_dim, d.head_dim);
+    const int gq = mx(t.n_heads / t.n_kv_heads, has_draft ? d.n_heads / d.n_kv_heads : 1);
+    const int rows_req = std::min(c.k_max + 1, MK_MAX_ROWS);
+    const int n_qblk = (rows_req * gq + mk::ATT_QBLK - 1) / mk::ATT_QBLK;
+    L->attn_units = c.max_requests * (2 * TC_GRID_MAX + 2 * hkv) * std::max(n_qblk, 1);
+    L->attn_part = take(t.wdtype == 1 ? (size_t)L->attn_units * mk::ATT_QBLK * (hdm + 2) * 4 : 0);
+    auto prog = [&](const stairs_model& m, size_t* maps_off) {
+      const size_t ph = align_up((size_t)(8 * std::max(m.n_layers, 1) + 4) * sizeof(mk::Phase), 128);
+      *maps_off = ph;
+      return ph + (size_t)(7 * std::max(m.n_layers, 1) + 4) * sizeof(CUtensorMap);
+    };
+    L->prog_slot_t = t.wdtype == 1 ? prog(t, &L->prog_maps_off_t) : 0;
+    L->prog_slot_d = (t.wdtype == 1 && has_draft) ? prog(d, &L->prog_maps_off_d) : 0;
+    L->prog_t = take(L->prog_slot_t * MK_TBOX_SLOTS);
+    L->prog_d = take(L->prog_slot_d * MK_TBOX_SLOTS);
+  }
   const size_t pool_tokens = (size_t)L->n_pages * pt;
   L->kv_t_layer = pool_tokens * t.n_kv_heads * t.head_dim * es;
   L->kv_t_k = take(L->kv_t_layer * t.n_layers);
@@ -317,6 +347,144 @@ int launch_gemm_tc(stairs_ctx* ctx, const TcArgs& a) {
   const long long total = (long long)tiles * job.t_tiles * job.kblocks;
   const int grid = (int)std::min<long long>(std::min(ctx->sm_count, TC_GRID_MAX), total);
   tc::k_gemm_tc<<<grid, tc::THREADS, tc::smem_bytes(job.t_box, job.stages), ctx->stream>>>(job);
+  return STAIRS_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Persistent forward kernel: per (model, row box) program and launch.
+// ---------------------------------------------------------------------------------------------
+int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
+  const stairs_model& m = M.m;
+  const Layout& L = ctx->lay;
+  const int slot = t_box / 16 - 1;
+  const int d = m.d_model, nq = m.n_heads * m.head_dim, nkv = m.n_kv_heads * m.head_dim, nqkv = nq + 2 * nkv, F = m.d_ff;
+  char* ws = ctx->ws;
+  std::vector<CUtensorMap> maps((size_t)7 * m.n_layers + 4);
+  for (int l = 0; l < m.n_layers; ++l) {
+    const LayerMaps& t = M.maps[l];
+    CUtensorMap* b = &maps[(size_t)7 * l];
+    b[0] = t.wq; b[1] = t.wk; b[2] = t.wv; b[3] = t.wo; b[4] = t.w1; b[5] = t.w3; b[6] = t.w2;
+  }
+  const int i_head = 7 * m.n_layers, i_h = i_head + 1, i_o = i_head + 2, i_ff = i_head + 3;
+  maps[i_head] = M.head_map;
+  bool ok = encode_map(ctx, &maps[i_h], ws + L.h, L.max_rows, d, t_box) &&
+            encode_map(ctx, &maps[i_o], ws + L.o, L.max_rows, nq, t_box) &&
+            encode_map(ctx, &maps[i_ff], ws + L.ff, L.max_rows, F, t_box);
+  if (!ok) return fail(ctx, STAIRS_ECUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+  std::vector<mk::Phase> ph;
+  auto gemm = [&](int layer, int w0, int w1, int w2, int n_src, const int* rows, bool dual, int xmap, int K, int epi, void* out, int ldo) {
+    mk::Phase p;
+    memset(&p, 0, sizeof p);
+    p.kind = mk::PH_GEMM; p.layer = layer;
+    p.w_map[0] = w0; p.w_map[1] = w1; p.w_map[2] = w2; p.x_map = xmap;
+    p.n_src = n_src; p.dual = dual ? 1 : 0;
+    p.kblocks = (K + tc::BK - 1) / tc::BK;
+    int col = 0, tiles = 0;
+    if (dual) { p.N = rows[0]; tiles = (rows[0] + 63) / 64; p.src_tiles[0] = tiles; }
+    else {
+      for (int s2 = 0; s2 < n_src; ++s2) {
+        p.src_tiles[s2] = (rows[s2] + tc::BM - 1) / tc::BM; p.src_col[s2] = col; col += rows[s2]; tiles += p.src_tiles[s2];
+      }
+      p.N = col;
+    }
+    p.n_tiles = tiles; p.epi = epi; p.out = out; p.ldo = ldo;
+    ph.push_back(p);
+  };
+  auto simple = [&](int kind, int layer, const void* g, const void* b, void* kc, void* vc) {
+    mk::Phase p;
+    memset(&p, 0, sizeof p);
+    p.kind = kind; p.layer = layer; p.g = (const float*)g; p.b = (const float*)b; p.kc = kc; p.vc = vc;
+    ph.push_back(p);
+  };
+  for (int l = 0; l < m.n_layers; ++l) {
+    const stairs_layer_w& w = M.layers[l];
+    const int b = 7 * l;
+    simple(l == 0 ? mk::PH_EMBED : mk::PH_NORM, l, w.norm1_w, w.norm1_b, nullptr, nullptr);
+    const int r3[3] = {nq, nkv, nkv};
+    gemm(l, b + 0, b + 1, b + 2, 3, r3, false, i_h, d, tc::TC_STORE_F32, ws + L.qkv, nqkv);
+    simple(mk::PH_ATTN, l, nullptr, nullptr, M.kpool + (size_t)l * M.kv_layer_bytes, M.vpool + (size_t)l * M.kv_layer_bytes);
+    simple(mk::PH_COMBINE, l, nullptr, nullptr, nullptr, nullptr);
+    const int rd[1] = {d};
+    gemm(l, b + 3, b + 3, b + 3, 1, rd, false, i_o, nq, tc::TC_ADD_F32, ws + L.x, d);
+    simple(mk::PH_NORM, l, w.norm2_w, w.norm2_b, nullptr, nullptr);
+    const int rf[1] = {F};
+    if (m.act == 1) gemm(l, b + 4, b + 5, b + 4, 1, rf, true, i_h, d, tc::TC_SWIGLU, ws + L.ff, F);
+    else gemm(l, b + 4, b + 4, b + 4, 1, rf, false, i_h, d, tc::TC_GELU, ws + L.ff, F);
+    gemm(l, b + 6, b + 6, b + 6, 1, rd, false, i_ff, F, tc::TC_ADD_F32, ws + L.x, d);
+  }
+  simple(mk::PH_FINAL_NORM, -1, M.w.final_norm_w, M.w.final_norm_b, nullptr, nullptr);
+  {
+    const int rv[1] = {m.vocab};
+    gemm(-1, i_head, i_head, i_head, 1, rv, false, i_h, d, tc::TC_LMHEAD, nullptr, m.vocab);
+    ph.back().logit_rows = 1;
+  }
+  simple(mk::PH_ACCEPT, -1, nullptr, nullptr, nullptr, nullptr);
+  for (const mk::Phase& p : ph)
+    if (p.kind == mk::PH_GEMM && p.n_tiles > TC_COUNTERS) return fail(ctx, STAIRS_EUNSUPPORTED, "too many tiles for the split bookkeeping");
+  M.n_phases = (int)ph.size();
+  char* base = M.prog_base + (size_t)slot * M.prog_slot_bytes;
+  if (ph.size() * sizeof(mk::Phase) > M.prog_maps_off || M.prog_maps_off + maps.size() * sizeof(CUtensorMap) > M.prog_slot_bytes)
+    return fail(ctx, STAIRS_ENOSPC, "program area too small");
+  CK(cudaMemcpyAsync(base, ph.data(), ph.size() * sizeof(mk::Phase), cudaMemcpyHostToDevice, ctx->stream));
+  CK(cudaMemcpyAsync(base + M.prog_maps_off, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, ctx->stream));
+  CK(cudaStreamSynchronize(ctx->stream));   // the host vectors go away
+  M.prog_built[slot] = true;
+  return STAIRS_OK;
+}
+
+struct MkCall {
+  int mode = mk::CALL_VALIDATE, n_req = 0, slot = 0, draft_step = 0;
+  const int* draft = nullptr;
+  int* target_tokens = nullptr; int* accept_len = nullptr; int commit = 0; int* draft_out = nullptr;
+  float* logits = nullptr;
+};
+
+bool mk_eligible(const stairs_ctx* ctx, const DevModel& M, int T) {
+  return ctx->use_mk && M.m.n_layers >= 1 && T >= 1 && T <= MK_MAX_ROWS;
+}
+
+int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, int n_logit_rows, const MkCall& c) {
+  const stairs_model& m = M.m;
+  const Layout& L = ctx->lay;
+  char* ws = ctx->ws;
+  const int t_box = (T + 15) / 16 * 16;
+  const int slot = t_box / 16 - 1;
+  if (!M.prog_built[slot]) {
+    int rc = build_program(ctx, M, t_box);
+    if (rc) return rc;
+  }
+  mk::Params P;
+  memset(&P, 0, sizeof P);
+  char* base = M.prog_base + (size_t)slot * M.prog_slot_bytes;
+  P.phases = reinterpret_cast<const mk::Phase*>(base); P.n_phases = M.n_phases;
+  P.maps = reinterpret_cast<const CUtensorMap*>(base + M.prog_maps_off);
+  P.T = T; P.t_box = t_box; P.stages = mk::pick_stages(t_box, m.head_dim);
+  P.logit_first_row = logit_first_row; P.n_logit_rows = n_logit_rows;
+  P.d = m.d_model; P.Hq = m.n_heads; P.Hkv = m.n_kv_heads; P.hd = m.head_dim; P.F = m.d_ff; P.vocab = m.vocab;
+  P.norm_kind = m.norm; P.rope = m.pos; P.rope_theta = m.rope_theta; P.eps = m.norm_eps;
+  P.tok_emb = (const bf16*)M.w.tok_emb; P.pos_emb = (const bf16*)M.w.pos_emb;
+  P.mode = c.mode; P.n_req = c.n_req; P.slot = c.slot; P.draft_step = c.draft_step;
+  P.val_req = reinterpret_cast<int*>(ws + L.val_req); P.val_k = reinterpret_cast<int*>(ws + L.val_k);
+  P.val_off = reinterpret_cast<int*>(ws + L.val_off);
+  P.draft = c.draft; P.k_max = ctx->cfg.k_max;
+  P.seq = reinterpret_cast<int*>(ws + L.seq); P.n_seq = reinterpret_cast<int*>(ws + L.n_seq); P.max_seq_len = ctx->cfg.max_seq_len;
+  P.tok = reinterpret_cast<int*>(ws + L.tok); P.pos = reinterpret_cast<int*>(ws + L.pos); P.req = reinterpret_cast<int*>(ws + L.req);
+  P.page_table = reinterpret_cast<int*>(ws + L.page_table); P.page_tokens = ctx->cfg.kv_page_tokens; P.max_pages = L.max_pages;
+  P.x = reinterpret_cast<float*>(ws + L.x); P.h = reinterpret_cast<bf16*>(ws + L.h); P.qkv = reinterpret_cast<float*>(ws + L.qkv);
+  P.o = reinterpret_cast<bf16*>(ws + L.o); P.ff = reinterpret_cast<bf16*>(ws + L.ff);
+  P.keys = reinterpret_cast<unsigned long long*>(ws + L.keys); P.n_keys = L.max_rows;
+  P.logits = c.logits;
+  P.target_tokens = c.target_tokens; P.accept_len = c.accept_len; P.commit = c.commit; P.draft_out = c.draft_out;
+  P.partial = reinterpret_cast<float*>(ws + L.gemm_partial); P.counters = reinterpret_cast<int*>(ws + L.gemm_counters);
+  P.attn_part = reinterpret_cast<float*>(ws + L.attn_part); P.attn_part_units = L.attn_units;
+  P.bar = reinterpret_cast<unsigned long long*>(ws + L.mk_bar); P.bar_base = ctx->bar_base;
+  P.status = ctx->status_dev; P.wait_limit = ctx->wait_limit;
+  const int grid = std::min(ctx->sm_count, TC_GRID_MAX);
+  void* args[] = {&P};
+  CK(cudaLaunchCooperativeKernel((const void*)mk::k_forward, dim3(grid), dim3(tc::THREADS), args,
+                                 mk::smem_bytes(t_box, P.stages, m.head_dim), ctx->stream));
+  ctx->bar_base += (unsigned long long)M.n_phases * grid;
+  ctx->launches++;
   return STAIRS_OK;
 }
 
@@ -600,7 +768,7 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
       delete ctx;
       return rc;
     }
-    if (cfg->target.wdtype == 1 && cfg->gemm_impl == 0) {
+    if (cfg->target.wdtype == 1 && cfg->gemm_impl != 1) {
       if (major != 10) {
         int rc = fail(nullptr, STAIRS_EUNSUPPORTED, "bf16 models need an sm_100 device (found compute capability %d.x)", major);
         stairs_destroy(ctx);
@@ -624,6 +792,21 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
         return rc;
       }
       ctx->use_tc = true;
+      // persistent whole-pass kernel (gemm_impl 0 only; 2 keeps one launch per GEMM)
+      int coop = 0;
+      cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, cfg->device);
+      const int hdm = has_draft ? std::max(cfg->target.head_dim, cfg->draft.head_dim) : cfg->target.head_dim;
+      const long long worst_chunks = ((long long)cfg->max_seq_len + mk::ATT_CHUNK - 1) / mk::ATT_CHUNK;
+      const int hkvm = has_draft ? std::max(cfg->target.n_kv_heads, cfg->draft.n_kv_heads) : cfg->target.n_kv_heads;
+      const bool fits = mk::pick_stages(MK_MAX_ROWS, hdm) >= 3 && worst_chunks * hkvm / 64 <= 2 * std::min(ctx->sm_count, TC_GRID_MAX);
+      if (coop && fits && cfg->gemm_impl == 0) {
+        e = cudaFuncSetAttribute(mk::k_forward, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_LIMIT);
+        if (e == cudaSuccess) {
+          ctx->use_mk = true;
+          ctx->target.prog_base = ctx->ws + L.prog_t; ctx->target.prog_slot_bytes = L.prog_slot_t; ctx->target.prog_maps_off = L.prog_maps_off_t;
+          ctx->draft.prog_base = ctx->ws + L.prog_d; ctx->draft.prog_slot_bytes = L.prog_slot_d; ctx->draft.prog_maps_off = L.prog_maps_off_d;
+        }
+      }
     }
   }
   *out = ctx;
@@ -670,6 +853,13 @@ int stairs_draft(stairs_ctx* ctx, int req, int k, int32_t* draft_dev) {
     p.slot = req; p.draft = draft_dev; p.first = j;
     p.mode = j == 0 ? ROWS_DRAFT_FIRST : ROWS_DRAFT_NEXT;
     const int T = j == 0 ? 2 : 1;
+    if (mk_eligible(ctx, ctx->draft, T)) {
+      MkCall c;
+      c.mode = j == 0 ? mk::CALL_DRAFT_FIRST : mk::CALL_DRAFT_NEXT;
+      c.slot = req; c.draft_step = j; c.draft = draft_dev; c.draft_out = draft_dev;
+      if ((rc = launch_forward_mk(ctx, ctx->draft, T, T - 1, 1, c))) return rc;
+      continue;
+    }
     if ((rc = launch_rows(ctx, p, T))) return rc;
     if ((rc = forward(ctx, ctx->draft, T, T - 1, 1, nullptr))) return rc;
     k_take_token<<<1, 32, 0, ctx->stream>>>(keys, T - 1, draft_dev, j);
@@ -710,6 +900,17 @@ int stairs_validate(stairs_ctx* ctx, int n_req, const int32_t* req_ids_host, con
   CK(cudaMemcpyAsync(ws + L.val_k, k_host, (size_t)n_req * 4, cudaMemcpyHostToDevice, ctx->stream));
   CK(cudaMemcpyAsync(ws + L.val_off, off.data(), (size_t)n_req * 4, cudaMemcpyHostToDevice, ctx->stream));
   if (ctx->profile) { ctx->ev_used = 0; cudaEventRecord(ctx->call_begin, ctx->stream); }
+  if (mk_eligible(ctx, ctx->target, T)) {
+    MkCall c;
+    c.mode = mk::CALL_VALIDATE; c.n_req = n_req; c.draft = draft_dev;
+    c.target_tokens = target_tokens_dev; c.accept_len = accept_len_dev; c.commit = commit; c.logits = logits_dev_or_null;
+    int rc = launch_forward_mk(ctx, ctx->target, T, 0, T, c);
+    if (rc) return rc;
+    if (ctx->profile) cudaEventRecord(ctx->call_end, ctx->stream);
+    if (commit)
+      for (int i = 0; i < n_req; ++i) ctx->n_seq_ub[req_ids_host[i]] += k_host[i] + 1;
+    return STAIRS_OK;
+  }
   ctx->in_validate = true;
   RowParams p = base_rows(ctx);
   p.mode = ROWS_VALIDATE; p.n_req = n_req; p.draft = draft_dev;
@@ -853,6 +1054,10 @@ int stairs_sync(stairs_ctx* ctx) {
   if (ctx->status_host && ctx->status_host[STATUS_ERROR]) {
     const unsigned int code = ctx->status_host[STATUS_ERROR];
     ctx->status_host[STATUS_ERROR] = 0;
+    cudaMemsetAsync(ctx->ws + ctx->lay.mk_bar, 0, 64, ctx->stream);   // barrier count and abort word
+    cudaMemsetAsync(ctx->ws + ctx->lay.gemm_counters, 0, (size_t)TC_COUNTERS * 4, ctx->stream);
+    cudaStreamSynchronize(ctx->stream);
+    ctx->bar_base = 0;
     return fail(ctx, (int)code, "a device-side bounded wait expired (code %u); results of the last calls are invalid", code);
   }
   return STAIRS_OK;
@@ -885,6 +1090,23 @@ int stairs_profile_read(stairs_ctx* ctx, float* gemm_ms, int32_t* gemm_launches,
   if (gemm_ms) *gemm_ms = total;
   if (gemm_launches) *gemm_launches = ctx->ev_used / 2;
   if (call_ms) { float ms = 0.f; CK(cudaEventElapsedTime(&ms, ctx->call_begin, ctx->call_end)); *call_ms = ms; }
+  return STAIRS_OK;
+}
+
+int stairs_debug_buffer(stairs_ctx* ctx, int which, void** ptr_dev, size_t* bytes) {
+  if (!ctx || !ptr_dev || !bytes) return STAIRS_EINVAL;
+  const Layout& L = ctx->lay;
+  const size_t off[7] = {L.x, L.h, L.qkv, L.q, L.o, L.ff, L.logits};
+  const size_t keys_end = L.x;
+  switch (which) {
+    case 0: *ptr_dev = ctx->ws + off[0]; *bytes = off[1] - off[0]; break;
+    case 1: *ptr_dev = ctx->ws + off[1]; *bytes = off[2] - off[1]; break;
+    case 2: *ptr_dev = ctx->ws + off[2]; *bytes = off[3] - off[2]; break;
+    case 3: *ptr_dev = ctx->ws + off[4]; *bytes = off[5] - off[4]; break;
+    case 4: *ptr_dev = ctx->ws + off[5]; *bytes = off[6] - off[5]; break;
+    case 5: *ptr_dev = ctx->ws + L.keys; *bytes = keys_end - L.keys; break;
+    default: return fail(ctx, STAIRS_EINVAL, "unknown buffer %d", which);
+  }
   return STAIRS_OK;
 }
 

@@ -281,7 +281,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_gemm_tc(const __grid_constant__ 
       const long long tile_first = (long long)tile * job.kblocks, tile_end = tile_first + job.kblocks;
       const long long seg_end = tile_end < kb_end ? tile_end : kb_end;
       const bool whole = (kk0 == 0) && (seg_end == tile_end);
-      ok = mbar_wait(acc_full + buf, acc_phase[buf], abort_flag, job.wait_limit);
+      mbar_wait(acc_full + buf, acc_phase[buf], abort_flag, job.wait_limit);
+      // one verdict for all 128 epilogue threads: a divergent exit would strand the others at
+      // the named barriers below
+      epi_bar_sync();
+      if (et == 0) *last_flag = *abort_flag ? 0 : 1;
+      epi_bar_sync();
+      ok = *last_flag != 0;
+      epi_bar_sync();
       if (!ok) break;
       acc_phase[buf] ^= 1;
       tc_fence_after();

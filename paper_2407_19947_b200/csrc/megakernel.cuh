@@ -1,0 +1,876 @@
+// One persistent kernel for a whole forward pass over T <= 64 rows (a stairs validation call, an
+// assistant step, plain greedy decoding): stair rows, embedding, every layer, LM head, argmax,
+// accept - one cooperative launch, one CTA per SM, grid-wide barriers between dependent phases.
+//
+// Why: at these row counts a layer streams its weights in a few microseconds, so per-kernel
+// launch gaps and pipeline fill/drain would dominate.  Here the TMA producer warp of every CTA
+// walks a static schedule of weight tiles for the WHOLE pass and keeps the shared-memory ring
+// full across phase boundaries: weight tiles (which depend on nothing) are fetched as soon as a
+// slot frees up, while the small activation tile of a stage is fetched only once the grid
+// barrier that publishes it has completed.  HBM therefore keeps streaming through barriers,
+// norms and attention.
+//
+// Roles per CTA (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner,
+// warps 2-5 = "compute group": GEMM epilogues and every non-GEMM phase (rows+embedding, norms,
+// attention, combine, accept).  GEMM work is split exactly as in k_gemm_tc (contiguous k-block
+// ranges per CTA, split tiles finished by the last arriver in k order).
+//
+// Attention (staircase mask over the paged cache): a unit is (request, kv head, range of
+// 64-position chunks, block of <= 48 queries); all rows x grouped heads of the request share the
+// K/V chunk, which is staged in shared memory by bulk async copies (one per cache row, so pages
+// need not be contiguous) completing on an mbarrier.  Scores: lane = position; softmax state
+// per query with warp shuffles; P.V: lane = slice of head_dim.  New positions' K (rotated) and V
+// are computed in the unit that owns their chunk, patched into the staged tile and written to
+// the cache.  Unit boundaries depend only on absolute positions and on the request's own
+// committed length, never on the other rows or requests in the call.
+//
+// All waits (mbarriers, grid barrier) are clock-bounded: on expiry the CTA raises an abort flag
+// (shared memory) and a global abort word that every other CTA's waits poll, so the whole grid
+// drains, frees TMEM and exits with STAIRS_ETIMEOUT in the status word.
+#pragma once
+#include "gemm_tc.cuh"
+#include "kernels_basic.cuh"
+
+namespace stairs {
+namespace mk {
+
+using namespace tc;
+
+enum PhaseKind { PH_EMBED = 0, PH_NORM = 1, PH_GEMM = 2, PH_ATTN = 3, PH_COMBINE = 4, PH_FINAL_NORM = 5, PH_ACCEPT = 6 };
+
+struct Phase {
+  int kind, layer;
+  // PH_GEMM
+  int w_map[3], x_map;
+  int src_tiles[3], src_col[3];
+  int n_src, dual, n_tiles, kblocks, N, epi, ldo;
+  int logit_rows;            // 1: valid rows = n_logit_rows (LM head), else T
+  void* out;                 // fp32 or bf16 output
+  // PH_NORM / PH_EMBED / PH_FINAL_NORM
+  const float* g; const float* b;
+  // PH_ATTN
+  void* kc; void* vc;
+};
+
+enum CallMode { CALL_VALIDATE = 0, CALL_DRAFT_FIRST = 1, CALL_DRAFT_NEXT = 2 };
+
+struct Params {
+  const Phase* phases; int n_phases;
+  const CUtensorMap* maps;
+  int T, t_box, stages;
+  int logit_first_row, n_logit_rows;
+  // model
+  int d, Hq, Hkv, hd, F, vocab, norm_kind, rope; float rope_theta, eps;
+  const bf16* tok_emb; const bf16* pos_emb;
+  // call
+  int mode; int n_req; int slot; int draft_step;
+  const int* val_req; const int* val_k; const int* val_off;
+  const int* draft; int k_max;
+  int* seq; int* n_seq; int max_seq_len;
+  int* tok; int* pos; int* req;
+  const int* page_table; int page_tokens, max_pages;
+  float* x; bf16* h; float* qkv; bf16* o; bf16* ff;
+  unsigned long long* keys; int n_keys;
+  float* logits;            // optional dump
+  int* target_tokens; int* accept_len; int commit; int* draft_out;
+  // scratch
+  float* partial; int* counters;
+  float* attn_part;         // [units][QBLK][hd + 2]
+  int attn_part_units;
+  unsigned long long* bar;  // [0] arrivals (monotonic), [1] abort word
+  unsigned long long bar_base;
+  unsigned int* status; unsigned long long wait_limit;
+};
+
+constexpr int ATT_CHUNK = 64;
+constexpr int ATT_QBLK = 48;
+
+struct AttnSmem {   // carved after the GEMM ring
+  static __host__ __device__ size_t k_pitch(int hd) { return (size_t)hd * 2 + 16; }
+  static __host__ __device__ size_t bytes(int hd) {
+    return (size_t)ATT_QBLK * hd * 4 + (size_t)ATT_QBLK * (hd + 2) * 4 + 2 * ATT_CHUNK * k_pitch(hd) + 64;
+  }
+};
+
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_release_add_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void tma_load_2d_ptr(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar, uint64_t policy) {
+  tma_load_2d(dst, map, c0, c1, bar, policy);
+}
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+// k-block range of this CTA in a GEMM phase: the phase is cut over min(G, total) CTAs so that no
+// participating range is empty (the split-tile bookkeeping counts one segment per CTA touching a tile).
+struct KRange { long long begin, end; int ge; };
+__device__ __forceinline__ KRange phase_range(long long total, int cta, int G) {
+  KRange r;
+  r.ge = (int)(total < (long long)G ? total : (long long)G);
+  if (cta >= r.ge) { r.begin = r.end = 0; return r; }
+  r.begin = range_begin(total, cta, r.ge); r.end = range_begin(total, cta + 1, r.ge);
+  return r;
+}
+
+// Shared per-CTA control block.
+struct Ctl {
+  uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2], att_bar;
+  uint32_t tmem_slot;
+  volatile int abort_flag;
+  volatile int last_flag;
+  volatile int bcast;
+};
+
+// Uniform verdict for the 128 compute threads after any of them may have timed out in a wait:
+// a divergent exit would strand the others at a named barrier.
+__device__ __forceinline__ bool group_ok(Ctl* ctl, int et) {
+  epi_bar_sync();
+  if (et == 0) ctl->bcast = ctl->abort_flag ? 0 : 1;
+  epi_bar_sync();
+  return ctl->bcast != 0;
+}
+
+struct Waiter {
+  volatile int* abort_flag; const unsigned long long* gabort; unsigned long long limit;
+  __device__ __forceinline__ bool poll_abort(long long t0) const {
+    if (*abort_flag) return true;
+    if ((unsigned long long)(clock64() - t0) > limit) { *abort_flag = 1; return true; }
+    return false;
+  }
+  // mbarrier wait (bounded)
+  __device__ __forceinline__ bool wait(uint64_t* bar, uint32_t parity) const {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    int spins = 0;
+    while (true) {
+      if (mbar_try(bar, parity)) return true;
+      if (poll_abort(t0)) return false;
+      if ((++spins & 255) == 0 && ld_acquire_u64(gabort)) { *abort_flag = 1; return false; }
+    }
+  }
+  // grid barrier wait: arrivals >= target
+  __device__ __forceinline__ bool wait_grid(const unsigned long long* counter, unsigned long long target) const {
+    const long long t0 = clock64();
+    int spins = 0;
+    while (ld_acquire_u64(counter) < target) {
+      if (poll_abort(t0)) return false;
+      if ((++spins & 63) == 0 && ld_acquire_u64(gabort)) { *abort_flag = 1; return false; }
+    }
+    return true;
+  }
+};
+
+// ---------------------------------------------------------------------------------------------
+// Row helpers
+// ---------------------------------------------------------------------------------------------
+struct RowInfo { int tok, pos, slot; };
+
+__device__ __forceinline__ RowInfo row_info(const Params& P, int t) {
+  RowInfo r;
+  auto clampv = [&](int v) { return v < 0 ? 0 : (v >= P.vocab ? P.vocab - 1 : v); };
+  if (P.mode == CALL_VALIDATE) {
+    int i = 0;
+    while (i + 1 < P.n_req && P.val_off[i + 1] <= t) ++i;
+    const int rr = t - P.val_off[i];
+    r.slot = P.val_req[i];
+    const int base = P.n_seq[r.slot] - 1;
+    r.pos = base + rr;
+    r.tok = clampv(rr == 0 ? P.seq[(size_t)r.slot * P.max_seq_len + base] : P.draft[i * P.k_max + rr - 1]);
+  } else if (P.mode == CALL_DRAFT_FIRST) {
+    r.slot = P.slot;
+    const int n = P.n_seq[P.slot];
+    r.pos = n - 2 + t;
+    r.tok = clampv(P.seq[(size_t)P.slot * P.max_seq_len + r.pos]);
+  } else {
+    r.slot = P.slot;
+    r.pos = P.n_seq[P.slot] - 1 + P.draft_step;
+    r.tok = clampv(P.draft[P.draft_step - 1]);
+  }
+  return r;
+}
+
+// sum over the 128 compute threads (4 warps); red = 4 floats
+__device__ __forceinline__ float group_sum(float v, float* red, int et) {
+  v = warp_sum(v);
+  epi_bar_sync();
+  if ((et & 31) == 0) red[et >> 5] = v;
+  epi_bar_sync();
+  return red[0] + red[1] + red[2] + red[3];
+}
+
+// h[row] = norm(x[row]) (bf16), by the 128 compute threads
+__device__ void norm_row(const Params& P, const float* xr, const float* g, const float* b, bf16* hr, float* red, int et) {
+  const int d = P.d;
+  float mean = 0.f;
+  if (P.norm_kind == 0) {
+    float s = 0.f;
+    for (int i = et; i < d; i += 128) s += xr[i];
+    mean = group_sum(s, red, et) / (float)d;
+  }
+  float ss = 0.f;
+  for (int i = et; i < d; i += 128) { const float c = xr[i] - mean; ss += c * c; }
+  const float var = group_sum(ss, red, et) / (float)d;
+  const float rstd = 1.0f / sqrtf(var + P.eps);
+  for (int i = et; i < d; i += 128) {
+    float v = (xr[i] - mean) * rstd * g[i];
+    if (b) v += b[i];
+    hr[i] = __float2bfloat16_rn(v);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Attention units
+// ---------------------------------------------------------------------------------------------
+struct AttnReq { int slot, base, R, off, n_chunks, cpu, n_ranges, n_qblk, units; };
+
+__device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
+  AttnReq a;
+  if (P.mode == CALL_VALIDATE) {
+    a.slot = P.val_req[i]; a.R = P.val_k[i] + 1; a.off = P.val_off[i];
+    a.base = P.n_seq[a.slot] - 1;
+  } else if (P.mode == CALL_DRAFT_FIRST) {
+    a.slot = P.slot; a.R = 2; a.off = 0; a.base = P.n_seq[P.slot] - 2;
+  } else {
+    a.slot = P.slot; a.R = 1; a.off = 0; a.base = P.n_seq[P.slot] - 1 + P.draft_step;
+  }
+  a.n_chunks = (a.base + a.R + ATT_CHUNK - 1) / ATT_CHUNK;
+  // chunks per unit: from the first row's position only (so it is the same for any draft length)
+  const int c0 = (a.base + ATT_CHUNK) / ATT_CHUNK;
+  int cpu = 1;
+  while (cpu < 64 && (c0 * P.Hkv) / cpu > 2 * G) cpu <<= 1;
+  a.cpu = cpu;
+  a.n_ranges = (a.n_chunks + cpu - 1) / cpu;
+  a.n_qblk = (a.R * (P.Hq / P.Hkv) + ATT_QBLK - 1) / ATT_QBLK;
+  a.units = P.Hkv * a.n_ranges * a.n_qblk;
+  return a;
+}
+
+__device__ __forceinline__ float rope_inv_freq(int i, int hd, float theta) {
+  return (float)exp2(-(double)(2 * i) / (double)hd * log2((double)theta));
+}
+
+// One attention unit, executed by the 128 compute threads.
+__device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot,
+                          uint8_t* att_smem, Ctl* ctl, uint32_t& att_parity, const Waiter& W, int et, bool& ok) {
+  const int hd = P.hd, G = P.Hq / P.Hkv, nkv = P.Hkv * hd, nq = P.Hq * hd, nqkv = nq + 2 * nkv;
+  const int lane = et & 31, w = et >> 5;
+  const int Q = a.R * G;
+  const int q0 = qblk * ATT_QBLK, nQ = min(ATT_QBLK, Q - q0);
+  float* qs = reinterpret_cast<float*>(att_smem);                       // [QBLK][hd] rotated, pre-scaled
+  float* state = qs + (size_t)ATT_QBLK * hd;                            // [QBLK][hd + 2]
+  const size_t pitch = AttnSmem::k_pitch(hd);
+  uint8_t* ks = reinterpret_cast<uint8_t*>(state + (size_t)ATT_QBLK * (hd + 2));
+  uint8_t* vs = ks + ATT_CHUNK * pitch;
+  bf16* kc = reinterpret_cast<bf16*>(ph.kc);
+  bf16* vc = reinterpret_cast<bf16*>(ph.vc);
+  const int* pt = P.page_table + (size_t)a.slot * P.max_pages;
+  const float scale = 1.0f / sqrtf((float)hd);
+  const int half = hd / 2;
+
+  // queries of this block: query index q -> row r = q / G, head g = q % G
+  for (int idx = et; idx < nQ * half; idx += 128) {
+    const int ql = idx / half, i = idx % half, q = q0 + ql;
+    const int r = q / G, head = kvh * G + (q % G);
+    const float* src = P.qkv + (size_t)(a.off + r) * nqkv + (size_t)head * hd;
+    float x0 = src[i], x1 = src[i + half];
+    if (P.rope) {
+      const float ang = (float)(a.base + r) * rope_inv_freq(i, hd, P.rope_theta);
+      float s, c;
+      sincosf(ang, &s, &c);
+      const float r0 = x0 * c - x1 * s, r1 = x1 * c + x0 * s;
+      x0 = r0; x1 = r1;
+    }
+    qs[(size_t)ql * hd + i] = x0 * scale;
+    qs[(size_t)ql * hd + i + half] = x1 * scale;
+  }
+  for (int idx = et; idx < nQ * (hd + 2); idx += 128) {
+    const int c = idx % (hd + 2);
+    state[idx] = (c == hd) ? -INFINITY : 0.f;   // [.. acc .., m, l]
+  }
+  epi_bar_sync();
+
+  const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
+  for (int c = c_begin; c < c_end && ok; ++c) {
+    const int p0 = c * ATT_CHUNK;
+    const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
+    // stage the chunk: one bulk async copy per cached row (K and V); rows of new positions are
+    // produced below instead
+    if (et == 0) {
+      int cached = min(n_pos, max(0, a.base - p0));
+      mbar_expect_tx(&ctl->att_bar, (uint32_t)(cached * 2 * hd * 2));
+    }
+    epi_bar_sync();
+    for (int j = et; j < n_pos; j += 128) {
+      const int p = p0 + j;
+      if (p < a.base) {
+        const size_t slot = (size_t)pt[p / P.page_tokens] * P.page_tokens + (p % P.page_tokens);
+        bulk_copy_g2s(ks + j * pitch, kc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
+        bulk_copy_g2s(vs + j * pitch, vc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
+      }
+    }
+    // new positions in this chunk: rotate k, round to bf16, patch the tile, write the cache
+    {
+      const int r_lo = max(0, p0 - a.base), r_hi = min(a.R, p0 + n_pos - a.base);
+      for (int idx = et; idx < (r_hi - r_lo) * half; idx += 128) {
+        const int r = r_lo + idx / half, i = idx % half, p = a.base + r, j = p - p0;
+        const float* row = P.qkv + (size_t)(a.off + r) * nqkv;
+        const float* ksrc = row + nq + (size_t)kvh * hd;
+        const float* vsrc = row + nq + nkv + (size_t)kvh * hd;
+        float x0 = ksrc[i], x1 = ksrc[i + half];
+        if (P.rope) {
+          const float ang = (float)p * rope_inv_freq(i, hd, P.rope_theta);
+          float s, cc;
+          sincosf(ang, &s, &cc);
+          const float r0 = x0 * cc - x1 * s, r1 = x1 * cc + x0 * s;
+          x0 = r0; x1 = r1;
+        }
+        const bf16 k0 = __float2bfloat16_rn(x0), k1 = __float2bfloat16_rn(x1);
+        const bf16 v0 = __float2bfloat16_rn(vsrc[i]), v1 = __float2bfloat16_rn(vsrc[i + half]);
+        bf16* kd = reinterpret_cast<bf16*>(ks + j * pitch);
+        bf16* vd = reinterpret_cast<bf16*>(vs + j * pitch);
+        kd[i] = k0; kd[i + half] = k1; vd[i] = v0; vd[i + half] = v1;
+        if (qblk == 0) {
+          const size_t slot = (size_t)pt[p / P.page_tokens] * P.page_tokens + (p % P.page_tokens);
+          bf16* kg = kc + slot * nkv + (size_t)kvh * hd;
+          bf16* vg = vc + slot * nkv + (size_t)kvh * hd;
+          kg[i] = k0; kg[i + half] = k1; vg[i] = v0; vg[i + half] = v1;
+        }
+      }
+    }
+    W.wait(&ctl->att_bar, att_parity);
+    att_parity ^= 1;
+    ok = group_ok(ctl, et);
+    if (!ok) break;
+
+    // each warp takes queries w, w+4, ... of the block
+    for (int ql = w; ql < nQ; ql += 4) {
+      const int q = q0 + ql, r = q / G;
+      const int last = a.base + r;                 // last visible position of this query
+      const float* qv = qs + (size_t)ql * hd;
+      float s0 = -INFINITY, s1 = -INFINITY;
+      // scores: lane handles positions p0+lane and p0+lane+32
+      {
+        const int j0 = lane, j1 = lane + 32;
+        const bool v0 = (j0 < n_pos) && (p0 + j0 <= last), v1 = (j1 < n_pos) && (p0 + j1 <= last);
+        float d0 = 0.f, d1 = 0.f;
+        const uint8_t* k0p = ks + (size_t)(v0 ? j0 : 0) * pitch;
+        const uint8_t* k1p = ks + (size_t)(v1 ? j1 : 0) * pitch;
+        for (int d8 = 0; d8 < hd; d8 += 8) {
+          float ka[8], kb[8];
+          Vec16<bf16>::unpack(*reinterpret_cast<const uint4*>(k0p + d8 * 2), ka);
+          Vec16<bf16>::unpack(*reinterpret_cast<const uint4*>(k1p + d8 * 2), kb);
+          const float4 qa = *reinterpret_cast<const float4*>(qv + d8), qb = *reinterpret_cast<const float4*>(qv + d8 + 4);
+          d0 = fmaf(qa.x, ka[0], d0); d0 = fmaf(qa.y, ka[1], d0); d0 = fmaf(qa.z, ka[2], d0); d0 = fmaf(qa.w, ka[3], d0);
+          d0 = fmaf(qb.x, ka[4], d0); d0 = fmaf(qb.y, ka[5], d0); d0 = fmaf(qb.z, ka[6], d0); d0 = fmaf(qb.w, ka[7], d0);
+          d1 = fmaf(qa.x, kb[0], d1); d1 = fmaf(qa.y, kb[1], d1); d1 = fmaf(qa.z, kb[2], d1); d1 = fmaf(qa.w, kb[3], d1);
+          d1 = fmaf(qb.x, kb[4], d1); d1 = fmaf(qb.y, kb[5], d1); d1 = fmaf(qb.z, kb[6], d1); d1 = fmaf(qb.w, kb[7], d1);
+        }
+        if (v0) s0 = d0;
+        if (v1) s1 = d1;
+      }
+      float* st = state + (size_t)ql * (hd + 2);
+      const float m_old = st[hd], l_old = st[hd + 1];
+      const float m_new = fmaxf(m_old, warp_max(fmaxf(s0, s1)));
+      if (m_new == -INFINITY) continue;            // nothing visible in this chunk (warp-uniform)
+      const float e0 = (s0 == -INFINITY) ? 0.f : expf(s0 - m_new), e1 = (s1 == -INFINITY) ? 0.f : expf(s1 - m_new);
+      const float corr = expf(m_old - m_new);
+      const float l_new = l_old * corr + warp_sum(e0 + e1);
+      // P.V: lane owns elements lane*? of head_dim in strides of 32 (pairs), up to 8 per lane
+      float acc[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { const int dd = lane + 32 * i; acc[i] = dd < hd ? st[dd] * corr : 0.f; }
+      const int jmax = min(n_pos, last - p0 + 1);
+      for (int j = 0; j < jmax; ++j) {
+        const float pj = __shfl_sync(0xffffffffu, j < 32 ? e0 : e1, j & 31);
+        const bf16* vr = reinterpret_cast<const bf16*>(vs + (size_t)j * pitch);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { const int dd = lane + 32 * i; if (dd < hd) acc[i] = fmaf(pj, __bfloat162float(vr[dd]), acc[i]); }
+      }
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { const int dd = lane + 32 * i; if (dd < hd) st[dd] = acc[i]; }
+      if (lane == 0) { st[hd] = m_new; st[hd + 1] = l_new; }
+      __syncwarp();
+    }
+    epi_bar_sync();   // tile may be overwritten by the next chunk
+  }
+  // park the unit's state for the combine phase
+  float* dst = P.attn_part + (size_t)part_slot * ATT_QBLK * (hd + 2);
+  for (int idx = et; idx < nQ * (hd + 2); idx += 128) dst[idx] = state[idx];
+  epi_bar_sync();
+}
+
+// ---------------------------------------------------------------------------------------------
+// The kernel
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ Params P) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int stages = P.stages;
+  const int b_stage_bytes = P.t_box * BK * 2;
+  const int stage_bytes = A_STAGE_BYTES + b_stage_bytes;
+  uint8_t* tail = smem + (size_t)stages * stage_bytes;
+  float* xch = reinterpret_cast<float*>(tail);
+  Ctl* ctl = reinterpret_cast<Ctl*>(tail + XCH_BYTES);
+  uint8_t* att_smem = tail + XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = gridDim.x, cta = blockIdx.x;
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < 2 * P.t_box) tmem_cols <<= 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(ctl->full + s, 1); mbar_init(ctl->empty + s, 1); }
+    mbar_init(ctl->acc_full + 0, 1); mbar_init(ctl->acc_full + 1, 1);
+    mbar_init(ctl->acc_empty + 0, 4); mbar_init(ctl->acc_empty + 1, 4);
+    mbar_init(&ctl->att_bar, 1);
+    ctl->abort_flag = 0; ctl->last_flag = 0; ctl->bcast = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(&ctl->tmem_slot, tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_slot;
+  const Waiter W{&ctl->abort_flag, P.bar + 1, P.wait_limit};
+  const unsigned long long* bar_count = P.bar;
+  // producer bookkeeping for the abort path
+  int issued = 0, p_stage = 0;
+  uint32_t p_phase = 0;
+
+  if (warp == 0) {
+    // ================================================================== TMA producer
+    if (lane == 0) {
+      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      // cursor A (weights) runs ahead of cursor B (activations)
+      int a_ph = 0, b_ph = 0;
+      long long a_kb = 0, a_end = -1, b_kb = 0, b_end = -1;
+      int a_stage = 0, b_stage = 0;
+      uint32_t a_par = 0;
+      long long a_count = 0, b_count = 0;
+      int ready_ph = -1;   // phases <= ready_ph have their inputs published
+      auto seek = [&](int& ph, long long& kb, long long& end) {   // advance to the next GEMM phase with work
+        while (ph < P.n_phases) {
+          const Phase& p = P.phases[ph];
+          if (p.kind == PH_GEMM) {
+            const long long total = (long long)p.n_tiles * p.kblocks;
+            if (end < 0) { const KRange kr = phase_range(total, cta, G); kb = kr.begin; end = kr.end; }
+            if (kb < end) return true;
+          }
+          ++ph; end = -1;
+        }
+        return false;
+      };
+      bool a_ok = seek(a_ph, a_kb, a_end), b_ok = seek(b_ph, b_kb, b_end);
+      long long t_idle = clock64();
+      while (b_ok) {
+        bool progress = false;
+        if (a_ok && mbar_test(ctl->empty + a_stage, a_par ^ 1)) {
+          const Phase& p = P.phases[a_ph];
+          const int n_tile = (int)(a_kb / p.kblocks), kk = (int)(a_kb % p.kblocks);
+          uint8_t* a_dst = smem + (size_t)a_stage * stage_bytes;
+          mbar_expect_tx(ctl->full + a_stage, (uint32_t)stage_bytes);
+          if (p.dual) {
+            tma_load_2d(a_dst, P.maps + p.w_map[0], kk * BK, n_tile * 64, ctl->full + a_stage, pol_w);
+            tma_load_2d(a_dst + A_STAGE_BYTES / 2, P.maps + p.w_map[1], kk * BK, n_tile * 64, ctl->full + a_stage, pol_w);
+          } else {
+            int s = 0, local = n_tile;
+            while (s + 1 < p.n_src && local >= p.src_tiles[s]) { local -= p.src_tiles[s]; ++s; }
+            tma_load_2d(a_dst, P.maps + p.w_map[s], kk * BK, local * BM, ctl->full + a_stage, pol_w);
+          }
+          ++issued; ++a_count;
+          if (++a_stage == stages) { a_stage = 0; a_par ^= 1; }
+          p_stage = a_stage; p_phase = a_par;
+          ++a_kb;
+          a_ok = seek(a_ph, a_kb, a_end);
+          progress = true;
+        }
+        if (b_count < a_count) {
+          if (b_ph > ready_ph) {
+            // inputs of phase b_ph are published once every CTA has finished phase b_ph - 1
+            if (ld_acquire_u64(bar_count) >= P.bar_base + (unsigned long long)b_ph * G) { ready_ph = b_ph; fence_proxy_async(); }
+          }
+          if (b_ph <= ready_ph) {
+            const Phase& p = P.phases[b_ph];
+            const int kk = (int)(b_kb % p.kblocks);
+            uint8_t* b_dst = smem + (size_t)b_stage * stage_bytes + A_STAGE_BYTES;
+            tma_load_2d(b_dst, P.maps + p.x_map, kk * BK, 0, ctl->full + b_stage, pol_x);
+            ++b_count;
+            if (++b_stage == stages) b_stage = 0;
+            ++b_kb;
+            b_ok = seek(b_ph, b_kb, b_end);
+            progress = true;
+          }
+        }
+        if (progress) t_idle = clock64();
+        else if (W.poll_abort(t_idle) || ld_acquire_u64(P.bar + 1)) { ctl->abort_flag = 1; break; }
+      }
+    }
+  } else if (warp == 1) {
+    // ================================================================== MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_bf16(P.t_box);
+      int stage = 0; uint32_t phase = 0;
+      int buf = 0; uint32_t acc_phase[2] = {0, 0};
+      bool ok = true;
+      for (int ph = 0; ph < P.n_phases && ok; ++ph) {
+        const Phase& p = P.phases[ph];
+        if (p.kind != PH_GEMM) continue;
+        const long long total = (long long)p.n_tiles * p.kblocks;
+        const KRange kr = phase_range(total, cta, G);
+        const long long kb_begin = kr.begin, kb_end = kr.end;
+        for (long long kb = kb_begin; kb < kb_end && ok; ++kb) {
+          const int kk = (int)(kb % p.kblocks);
+          const bool seg_first = (kb == kb_begin) || kk == 0;
+          const bool seg_last = (kb + 1 == kb_end) || kk == p.kblocks - 1;
+          if (seg_first) {
+            ok = W.wait(ctl->acc_empty + buf, acc_phase[buf] ^ 1);
+            if (!ok) break;
+            tc_fence_after();
+          }
+          ok = W.wait(ctl->full + stage, phase);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + (size_t)stage * stage_bytes);
+          const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + A_STAGE_BYTES);
+          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * P.t_box);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_bf16(d_tmem, a_desc + (uint64_t)(k * UMMA_K * 2 / 16), b_desc + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
+                      (seg_first && k == 0) ? 0u : 1u);
+          umma_commit(ctl->empty + stage);
+          if (seg_last) { umma_commit(ctl->acc_full + buf); acc_phase[buf] ^= 1; buf ^= 1; }
+          if (++stage == stages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else {
+    // ================================================================== compute group (warps 2..5)
+    const int quad = warp & 3;
+    const int m = quad * 32 + lane;
+    const int et = threadIdx.x - 64;
+    float* red = xch;   // 4 floats of scratch for group sums (xch is free outside SwiGLU epilogues)
+    int buf = 0; uint32_t acc_phase[2] = {0, 0};
+    uint32_t att_parity = 0;
+    bool ok = true;
+    bool waited = true;   // true when every earlier phase is known complete grid-wide
+
+    for (int ph = 0; ph < P.n_phases && ok; ++ph) {
+      const Phase& p = P.phases[ph];
+      if (p.kind != PH_GEMM && !waited) {
+        // inputs come from other CTAs: wait until all of them finished phase ph - 1
+        if (et == 0) {
+          const bool g = W.wait_grid(bar_count, P.bar_base + (unsigned long long)ph * G);
+          ctl->bcast = g ? 1 : 0;
+        }
+        epi_bar_sync();
+        ok = ctl->bcast != 0;
+        epi_bar_sync();
+        if (!ok) break;
+      }
+
+      if (p.kind == PH_EMBED) {
+        if (cta == 0)
+          for (int i = et; i < P.n_keys; i += 128) P.keys[i] = 0ull;
+        for (int t = cta; t < P.T; t += G) {
+          const RowInfo r = row_info(P, t);
+          if (et == 0) { P.tok[t] = r.tok; P.pos[t] = r.pos; P.req[t] = r.slot; }
+          float* xr = P.x + (size_t)t * P.d;
+          const bf16* e = P.tok_emb + (size_t)r.tok * P.d;
+          const bf16* pe = P.pos_emb ? P.pos_emb + (size_t)r.pos * P.d : nullptr;
+          for (int i = et; i < P.d; i += 128) {
+            float v = __bfloat162float(e[i]);
+            if (pe) v += __bfloat162float(pe[i]);
+            xr[i] = v;
+          }
+          epi_bar_sync();
+          norm_row(P, xr, p.g, p.b, P.h + (size_t)t * P.d, red, et);
+        }
+      } else if (p.kind == PH_NORM) {
+        for (int t = cta; t < P.T; t += G)
+          norm_row(P, P.x + (size_t)t * P.d, p.g, p.b, P.h + (size_t)t * P.d, red, et);
+      } else if (p.kind == PH_FINAL_NORM) {
+        for (int t = cta; t < P.n_logit_rows; t += G)
+          norm_row(P, P.x + (size_t)(P.logit_first_row + t) * P.d, p.g, p.b, P.h + (size_t)t * P.d, red, et);
+      } else if (p.kind == PH_ATTN) {
+        const int n_req = P.mode == CALL_VALIDATE ? P.n_req : 1;
+        int u0 = 0;
+        for (int i = 0; i < n_req && ok; ++i) {
+          const AttnReq a = attn_req(P, i, G);
+          // units of this request: index = ((kvh * n_ranges) + range) * n_qblk + qblk
+          int first = (cta - u0 % G + G) % G;
+          for (int u = first; u < a.units && ok; u += G) {
+            const int qblk = u % a.n_qblk, rest = u / a.n_qblk;
+            const int range = rest % a.n_ranges, kvh = rest / a.n_ranges;
+            const int slot = u0 + u;
+            if (slot < P.attn_part_units)
+              attn_unit(P, p, a, kvh, range, qblk, slot, att_smem, ctl, att_parity, W, et, ok);
+          }
+          u0 += a.units;
+        }
+      } else if (p.kind == PH_COMBINE) {
+        // merge the units of every (request, kv head, query) in position order -> o (bf16)
+        const int n_req = P.mode == CALL_VALIDATE ? P.n_req : 1;
+        const int hd = P.hd, Gq = P.Hq / P.Hkv;
+        int u0 = 0, item0 = 0;
+        for (int i = 0; i < n_req; ++i) {
+          const AttnReq a = attn_req(P, i, G);
+          const int Q = a.R * Gq;
+          const int items = P.Hkv * Q;   // one warp per (kvh, q)
+          for (int it = (cta * 4 + (et >> 5)) - item0 % (G * 4); it < items; it += G * 4) {
+            if (it < 0) continue;
+            const int kvh = it / Q, q = it % Q, qblk = q / ATT_QBLK, ql = q % ATT_QBLK;
+            const int r = q / Gq, head = kvh * Gq + (q % Gq);
+            float M = -INFINITY;
+            for (int rg = 0; rg < a.n_ranges; ++rg) {
+              const int slot = u0 + (kvh * a.n_ranges + rg) * a.n_qblk + qblk;
+              M = fmaxf(M, __ldcg(P.attn_part + ((size_t)slot * ATT_QBLK + ql) * (hd + 2) + hd));
+            }
+            float L = 0.f, acc[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+            for (int rg = 0; rg < a.n_ranges; ++rg) {
+              const int slot = u0 + (kvh * a.n_ranges + rg) * a.n_qblk + qblk;
+              const float* st = P.attn_part + ((size_t)slot * ATT_QBLK + ql) * (hd + 2);
+              const float mu = __ldcg(st + hd);
+              if (mu == -INFINITY) continue;
+              const float wgt = expf(mu - M);
+              L += __ldcg(st + hd + 1) * wgt;
+#pragma unroll
+              for (int j = 0; j < 8; ++j) { const int dd = (et & 31) + 32 * j; if (dd < hd) acc[j] += __ldcg(st + dd) * wgt; }
+            }
+            bf16* orow = P.o + (size_t)(a.off + r) * P.Hq * hd + (size_t)head * hd;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { const int dd = (et & 31) + 32 * j; if (dd < hd) orow[dd] = __float2bfloat16_rn(acc[j] / L); }
+          }
+          u0 += a.units; item0 += items;
+        }
+      } else if (p.kind == PH_ACCEPT) {
+        if (cta == 0) {
+          if (P.mode == CALL_VALIDATE) {
+            for (int i = et; i < P.n_req; i += 128) {
+              const int k = P.val_k[i], off = P.val_off[i], slot = P.val_req[i];
+              int a = -1;
+              for (int r = 0; r <= k; ++r) {
+                const int tr = argmax_key_index(__ldcg(P.keys + off + r));
+                P.target_tokens[i * (P.k_max + 1) + r] = tr;
+                if (a < 0 && r < k && P.draft[i * P.k_max + r] != tr) a = r;
+              }
+              if (a < 0) a = k;
+              P.accept_len[i] = a;
+              if (P.commit) {
+                int* s = P.seq + (size_t)slot * P.max_seq_len;
+                int wpos = P.n_seq[slot];
+                for (int r = 0; r < a && wpos < P.max_seq_len; ++r) s[wpos++] = P.draft[i * P.k_max + r];
+                if (wpos < P.max_seq_len) s[wpos++] = argmax_key_index(__ldcg(P.keys + off + a));
+                P.n_seq[slot] = wpos;
+              }
+            }
+          } else if (et == 0) {
+            P.draft_out[P.draft_step] = argmax_key_index(__ldcg(P.keys + P.logit_first_row));
+          }
+        }
+      } else {
+        // ---------------------------------------------------------------- GEMM epilogue
+        const long long total = (long long)p.n_tiles * p.kblocks;
+        const KRange kr = phase_range(total, cta, G);
+        const long long kb_begin = kr.begin, kb_end = kr.end;
+        const int Ge = kr.ge;
+        const int Tvalid = p.logit_rows ? P.n_logit_rows : P.T;
+        float* out_f32 = (p.epi == TC_LMHEAD) ? P.logits : reinterpret_cast<float*>(p.out);
+        bf16* out_act = reinterpret_cast<bf16*>(p.out);
+        unsigned long long* keys = P.keys + P.logit_first_row;
+        long long kb = kb_begin;
+        while (kb < kb_end && ok) {
+          const int tile = (int)(kb / p.kblocks), kk0 = (int)(kb % p.kblocks);
+          const long long tile_first = (long long)tile * p.kblocks, tile_end = tile_first + p.kblocks;
+          const long long seg_end = tile_end < kb_end ? tile_end : kb_end;
+          const bool whole = (kk0 == 0) && (seg_end == tile_end);
+          W.wait(ctl->acc_full + buf, acc_phase[buf]);
+          ok = group_ok(ctl, et);
+          if (!ok) break;
+          acc_phase[buf] ^= 1;
+          tc_fence_after();
+          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * P.t_box);
+          int n_out, n_valid;
+          if (p.dual) { n_out = tile * 64 + (m & 63); n_valid = n_out < p.N; }
+          else {
+            int s = 0, local = tile;
+            while (s + 1 < p.n_src && local >= p.src_tiles[s]) { local -= p.src_tiles[s]; ++s; }
+            const int in_src = local * BM + m;
+            const int src_n = (s + 1 < p.n_src ? p.src_col[s + 1] : p.N) - p.src_col[s];
+            n_out = p.src_col[s] + in_src; n_valid = in_src < src_n;
+          }
+          auto finish = [&](int c0, float* v) {
+            if (p.epi == TC_SWIGLU) {
+              if (m >= 64) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) xch[(m - 64) * 16 + j] = v[j];
+              }
+              epi_bar_sync();
+              if (m < 64 && n_valid) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                  const int t = c0 + j;
+                  if (t < Tvalid) out_act[(size_t)t * p.ldo + n_out] = __float2bfloat16_rn(silu_f(v[j]) * xch[m * 16 + j]);
+                }
+              }
+              epi_bar_sync();
+              return;
+            }
+            if (p.epi == TC_LMHEAD) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const int t = c0 + j;
+                if (t >= Tvalid) break;
+                if (out_f32 && n_valid) out_f32[(size_t)t * p.ldo + n_out] = v[j];
+                unsigned long long key = n_valid ? argmax_key(v[j], (uint32_t)n_out) : 0ull;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                  const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+                  key = other > key ? other : key;
+                }
+                if (lane == 0 && key) atomicMax(keys + t, key);
+              }
+              return;
+            }
+            if (!n_valid) return;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int t = c0 + j;
+              if (t >= Tvalid) break;
+              const size_t o = (size_t)t * p.ldo + n_out;
+              if (p.epi == TC_STORE_F32) out_f32[o] = v[j];
+              else if (p.epi == TC_ADD_F32) out_f32[o] += v[j];
+              else out_act[o] = __float2bfloat16_rn(gelu_erf(v[j]));
+            }
+          };
+          if (whole) {
+            for (int c0 = 0; c0 < P.t_box; c0 += 16) {
+              float v[16];
+              tmem_ld16(taddr + (uint32_t)c0, v);
+              finish(c0, v);
+            }
+            tc_fence_before();
+            if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
+          } else {
+            const int slot = 2 * cta + (kb == kb_begin ? 0 : 1);
+            float* mine = P.partial + (size_t)slot * P.t_box * BM;
+            for (int c0 = 0; c0 < P.t_box; c0 += 16) {
+              float v[16];
+              tmem_ld16(taddr + (uint32_t)c0, v);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) mine[(size_t)(c0 + j) * BM + m] = v[j];
+            }
+            tc_fence_before();
+            if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
+            __threadfence();
+            epi_bar_sync();
+            int first_c = (int)((tile_first * Ge) / total);
+            while (range_begin(total, first_c + 1, Ge) <= tile_first) ++first_c;
+            while (first_c > 0 && range_begin(total, first_c, Ge) > tile_first) --first_c;
+            int last_c = first_c;
+            while (last_c + 1 < Ge && range_begin(total, last_c + 1, Ge) < tile_end) ++last_c;
+            const int nseg = last_c - first_c + 1;
+            if (et == 0) {
+              const int old = atomicAdd(P.counters + tile, 1);
+              ctl->last_flag = (old == nseg - 1) ? 1 : 0;
+              if (old == nseg - 1) P.counters[tile] = 0;
+            }
+            epi_bar_sync();
+            const bool last = ctl->last_flag != 0;
+            epi_bar_sync();
+            if (last) {
+              __threadfence();
+              for (int c0 = 0; c0 < P.t_box; c0 += 16) {
+                float v[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = 0.f;
+                for (int c = first_c; c <= last_c; ++c) {
+                  const long long cb = range_begin(total, c, Ge);
+                  const int sl = 2 * c + (cb >= tile_first ? 0 : 1);
+                  const float* part = P.partial + (size_t)sl * P.t_box * BM;
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) v[j] += __ldcg(part + (size_t)(c0 + j) * BM + m);
+                }
+                finish(c0, v);
+              }
+            }
+          }
+          buf ^= 1;
+          kb = seg_end;
+        }
+      }
+      if (!ok) break;
+      // Publish this CTA's part of the phase.  A CTA may arrive for phase ph only once every
+      // CTA has arrived for phase ph-1: otherwise CTAs without work in two consecutive GEMM
+      // phases would run ahead and their arrivals would be mistaken for the slower CTAs' ones
+      // (one monotonic counter serves all phases).  For a CTA that had GEMM work the wait is
+      // already satisfied - its own activation tiles were gated on the same count.
+      __threadfence();
+      fence_proxy_async();   // later TMA (async proxy) reads of these generic-proxy writes
+      if (ph > 0 && p.kind == PH_GEMM) {
+        if (et == 0) ctl->bcast = W.wait_grid(bar_count, P.bar_base + (unsigned long long)ph * G) ? 1 : 0;
+        epi_bar_sync();
+        ok = ctl->bcast != 0;
+        epi_bar_sync();
+        if (!ok) break;
+      } else {
+        epi_bar_sync();
+      }
+      if (et == 0) red_release_add_u64(P.bar, 1ull);
+      waited = false;
+    }
+  }
+
+  // ================================================================== teardown
+  tc_fence_before();
+  __syncthreads();
+  if (ctl->abort_flag) {
+    if (threadIdx.x == 0) {
+      atomicExch(P.bar + 1, 1ull);   // tell the other CTAs
+      *reinterpret_cast<volatile unsigned int*>(P.status + STATUS_ERROR) = 5u;  // STAIRS_ETIMEOUT
+      __threadfence_system();
+      const long long t0 = clock64();
+      int s = p_stage; uint32_t phs = p_phase;
+      for (int i = 0; i < stages && i < issued; ++i) {
+        if (--s < 0) { s = stages - 1; phs ^= 1; }
+        while (!mbar_try(ctl->full + s, phs)) {
+          if ((unsigned long long)(clock64() - t0) > P.wait_limit) break;
+        }
+      }
+    }
+    __syncthreads();
+  }
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, tmem_cols); }
+}
+
+inline size_t smem_bytes(int t_box, int stages, int hd) {
+  return 1024 + (size_t)stages * (A_STAGE_BYTES + (size_t)t_box * BK * 2) + XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127) +
+         AttnSmem::bytes(hd) + 64;
+}
+inline int pick_stages(int t_box, int hd) {
+  int s = MAX_STAGES;
+  while (s > 1 && smem_bytes(t_box, s, hd) > (size_t)SMEM_LIMIT) --s;
+  return s;
+}
+
+}  // namespace mk
+}  // namespace stairs

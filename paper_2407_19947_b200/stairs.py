@@ -20,7 +20,7 @@ STATUS = {0: "OK", 1: "EINVAL", 2: "ENOSPC", 3: "ESTATE", 4: "ECUDA", 5: "ETIMEO
 EXPORTS = ["stairs_workspace_bytes", "stairs_init", "stairs_prefill", "stairs_draft", "stairs_validate",
            "stairs_validate_host", "stairs_generate", "stairs_sequence", "stairs_truncate", "stairs_sync",
            "stairs_launch_count", "stairs_profile", "stairs_profile_read", "stairs_reset",
-           "stairs_destroy", "stairs_last_error", "stairs_accept_static"]
+           "stairs_destroy", "stairs_last_error", "stairs_accept_static", "stairs_debug_buffer"]
 
 STATIC_MAX_ROWS, STATIC_MAX_REQ = 1024, 64
 
@@ -91,6 +91,7 @@ def load_library(path: Optional[str] = None):
     lib.stairs_profile.argtypes = [vp, C.c_int]
     lib.stairs_profile_read.argtypes = [vp, C.POINTER(C.c_float), i32p, C.POINTER(C.c_float)]
     lib.stairs_reset.argtypes = [vp, C.c_int]
+    lib.stairs_debug_buffer.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(C.c_size_t)]
     lib.stairs_destroy.argtypes = [vp]
     lib.stairs_accept_static.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, vp, C.c_int, vp, vp, vp]
     lib.stairs_last_error.restype = C.c_char_p
@@ -278,6 +279,17 @@ class Stairs:
         g, n, c = C.c_float(0), C.c_int32(0), C.c_float(0)
         self._ck(self.lib.stairs_profile_read(self.h, C.byref(g), C.byref(n), C.byref(c)))
         return g.value, n.value, c.value
+
+    def debug_buffer(self, which: int, dtype, count: int):
+        """Copy of the first `count` elements of an internal activation buffer (tests only)."""
+        ptr, nbytes = C.c_void_p(), C.c_size_t()
+        self._ck(self.lib.stairs_debug_buffer(self.h, which, C.byref(ptr), C.byref(nbytes)))
+        t = self.torch
+        off = ptr.value - self.workspace.data_ptr()
+        esz = t.empty(0, dtype=dtype).element_size()
+        assert count * esz <= nbytes.value
+        self.sync()
+        return self.workspace[off: off + count * esz].view(dtype).clone()
 
     def reset(self, req: int):
         self._ck(self.lib.stairs_reset(self.h, req))
