@@ -54,7 +54,7 @@ struct DevModel {
 
 struct Layout {
   size_t status, seq, n_seq, page_table, tok, pos, req, val_req, val_k, val_off, keys, x, h, qkv, q,
-      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_bar, attn_part, prog_t, prog_d, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
+      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_bar, attn_part, prog_t, prog_d, mk_trace, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
   int max_rows, logit_rows, max_pages, n_pages, t_box_max, attn_units;
   size_t prog_slot_t, prog_slot_d, prog_maps_off_t, prog_maps_off_d;
   size_t kv_t_layer, kv_d_layer;
@@ -206,6 +206,7 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     L->prog_slot_d = (t.wdtype == 1 && has_draft) ? prog(d, &L->prog_maps_off_d) : 0;
     L->prog_t = take(L->prog_slot_t * MK_TBOX_SLOTS);
     L->prog_d = take(L->prog_slot_d * MK_TBOX_SLOTS);
+    L->mk_trace = take(t.wdtype == 1 ? (size_t)2 * (8 * std::max(t.n_layers, 1) + 4) * 3 * 8 : 0);
   }
   const size_t pool_tokens = (size_t)L->n_pages * pt;
   L->kv_t_layer = pool_tokens * t.n_kv_heads * t.head_dim * es;
@@ -479,6 +480,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.attn_part = reinterpret_cast<float*>(ws + L.attn_part); P.attn_part_units = L.attn_units;
   P.bar = reinterpret_cast<unsigned long long*>(ws + L.mk_bar); P.bar_base = ctx->bar_base;
   P.status = ctx->status_dev; P.wait_limit = ctx->wait_limit;
+  P.trace = (ctx->profile && &M == &ctx->target) ? reinterpret_cast<unsigned long long*>(ws + L.mk_trace) : nullptr;
   const int grid = std::min(ctx->sm_count, TC_GRID_MAX);
   void* args[] = {&P};
   CK(cudaLaunchCooperativeKernel((const void*)mk::k_forward, dim3(grid), dim3(tc::THREADS), args,
@@ -1105,6 +1107,7 @@ int stairs_debug_buffer(stairs_ctx* ctx, int which, void** ptr_dev, size_t* byte
     case 3: *ptr_dev = ctx->ws + off[4]; *bytes = off[5] - off[4]; break;
     case 4: *ptr_dev = ctx->ws + off[5]; *bytes = off[6] - off[5]; break;
     case 5: *ptr_dev = ctx->ws + L.keys; *bytes = keys_end - L.keys; break;
+    case 6: *ptr_dev = ctx->ws + L.mk_trace; *bytes = L.kv_t_k - L.mk_trace; break;
     default: return fail(ctx, STAIRS_EINVAL, "unknown buffer %d", which);
   }
   return STAIRS_OK;

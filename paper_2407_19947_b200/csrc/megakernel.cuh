@@ -80,6 +80,7 @@ struct Params {
   unsigned long long* bar;  // [0] arrivals (monotonic), [1] abort word
   unsigned long long bar_base;
   unsigned int* status; unsigned long long wait_limit;
+  unsigned long long* trace;   // optional: per phase {start, work done, arrived} ns timestamps of CTA 0 and of the last CTA
 };
 
 constexpr int ATT_CHUNK = 64;
@@ -99,6 +100,11 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 }
 __device__ __forceinline__ void red_release_add_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
@@ -459,68 +465,84 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     // ================================================================== TMA producer
     if (lane == 0) {
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
-      // cursor A (weights) runs ahead of cursor B (activations)
-      int a_ph = 0, b_ph = 0;
-      long long a_kb = 0, a_end = -1, b_kb = 0, b_end = -1;
+      // Cursor over this CTA's k-blocks of all GEMM phases, in program order.  Per-phase fields
+      // are hoisted into registers on phase entry; tile and k indices advance incrementally.
+      struct Cursor {
+        int ph, kk, n_tile, remaining, kblocks, dual, n_src, x_map;
+        int src_tiles[3], w_map[3];
+        const CUtensorMap* wm0; const CUtensorMap* wm1; int row;
+        bool valid;
+      };
+      auto locate = [&](Cursor& c) {   // source map and row coordinate of tile c.n_tile
+        if (c.dual) { c.wm0 = P.maps + c.w_map[0]; c.wm1 = P.maps + c.w_map[1]; c.row = c.n_tile * 64; }
+        else {
+          int s2 = 0, local = c.n_tile;
+          while (s2 + 1 < c.n_src && local >= c.src_tiles[s2]) { local -= c.src_tiles[s2]; ++s2; }
+          c.wm0 = P.maps + c.w_map[s2]; c.row = local * BM;
+        }
+      };
+      auto enter = [&](Cursor& c, int from) {   // first GEMM phase >= from in which this CTA has work
+        for (int ph = from; ph < P.n_phases; ++ph) {
+          const Phase& p = P.phases[ph];
+          if (p.kind != PH_GEMM) continue;
+          const KRange kr = phase_range((long long)p.n_tiles * p.kblocks, cta, G);
+          if (kr.begin >= kr.end) continue;
+          c.ph = ph; c.kblocks = p.kblocks; c.dual = p.dual; c.n_src = p.n_src; c.x_map = p.x_map;
+#pragma unroll
+          for (int q = 0; q < 3; ++q) { c.src_tiles[q] = p.src_tiles[q]; c.w_map[q] = p.w_map[q]; }
+          c.n_tile = (int)(kr.begin / p.kblocks); c.kk = (int)(kr.begin % p.kblocks);
+          c.remaining = (int)(kr.end - kr.begin);
+          locate(c);
+          c.valid = true;
+          return;
+        }
+        c.valid = false;
+      };
+      auto advance = [&](Cursor& c) {
+        if (--c.remaining == 0) { enter(c, c.ph + 1); return; }
+        if (++c.kk == c.kblocks) { c.kk = 0; ++c.n_tile; locate(c); }
+      };
+      Cursor A, B;
+      enter(A, 0); enter(B, 0);
       int a_stage = 0, b_stage = 0;
       uint32_t a_par = 0;
-      long long a_count = 0, b_count = 0;
+      unsigned int a_count = 0, b_count = 0, idle = 0;
       int ready_ph = -1;   // phases <= ready_ph have their inputs published
-      auto seek = [&](int& ph, long long& kb, long long& end) {   // advance to the next GEMM phase with work
-        while (ph < P.n_phases) {
-          const Phase& p = P.phases[ph];
-          if (p.kind == PH_GEMM) {
-            const long long total = (long long)p.n_tiles * p.kblocks;
-            if (end < 0) { const KRange kr = phase_range(total, cta, G); kb = kr.begin; end = kr.end; }
-            if (kb < end) return true;
-          }
-          ++ph; end = -1;
-        }
-        return false;
-      };
-      bool a_ok = seek(a_ph, a_kb, a_end), b_ok = seek(b_ph, b_kb, b_end);
       long long t_idle = clock64();
-      while (b_ok) {
+      while (B.valid) {
         bool progress = false;
-        if (a_ok && mbar_test(ctl->empty + a_stage, a_par ^ 1)) {
-          const Phase& p = P.phases[a_ph];
-          const int n_tile = (int)(a_kb / p.kblocks), kk = (int)(a_kb % p.kblocks);
+        if (A.valid && mbar_test(ctl->empty + a_stage, a_par ^ 1)) {
           uint8_t* a_dst = smem + (size_t)a_stage * stage_bytes;
           mbar_expect_tx(ctl->full + a_stage, (uint32_t)stage_bytes);
-          if (p.dual) {
-            tma_load_2d(a_dst, P.maps + p.w_map[0], kk * BK, n_tile * 64, ctl->full + a_stage, pol_w);
-            tma_load_2d(a_dst + A_STAGE_BYTES / 2, P.maps + p.w_map[1], kk * BK, n_tile * 64, ctl->full + a_stage, pol_w);
-          } else {
-            int s = 0, local = n_tile;
-            while (s + 1 < p.n_src && local >= p.src_tiles[s]) { local -= p.src_tiles[s]; ++s; }
-            tma_load_2d(a_dst, P.maps + p.w_map[s], kk * BK, local * BM, ctl->full + a_stage, pol_w);
-          }
+          tma_load_2d(a_dst, A.wm0, A.kk * BK, A.row, ctl->full + a_stage, pol_w);
+          if (A.dual) tma_load_2d(a_dst + A_STAGE_BYTES / 2, A.wm1, A.kk * BK, A.row, ctl->full + a_stage, pol_w);
           ++issued; ++a_count;
           if (++a_stage == stages) { a_stage = 0; a_par ^= 1; }
           p_stage = a_stage; p_phase = a_par;
-          ++a_kb;
-          a_ok = seek(a_ph, a_kb, a_end);
+          advance(A);
           progress = true;
         }
-        if (b_count < a_count) {
-          if (b_ph > ready_ph) {
-            // inputs of phase b_ph are published once every CTA has finished phase b_ph - 1
-            if (ld_acquire_u64(bar_count) >= P.bar_base + (unsigned long long)b_ph * G) { ready_ph = b_ph; fence_proxy_async(); }
+        if (b_count != a_count) {
+          // inputs of phase B.ph are published once every CTA has finished phase B.ph - 1; the
+          // poll is a global acquire load, so it is only made when no weight tile could be issued
+          if (B.ph > ready_ph && !progress) {
+            if (ld_acquire_u64(bar_count) >= P.bar_base + (unsigned long long)B.ph * G) { ready_ph = B.ph; fence_proxy_async(); }
           }
-          if (b_ph <= ready_ph) {
-            const Phase& p = P.phases[b_ph];
-            const int kk = (int)(b_kb % p.kblocks);
+          if (B.ph <= ready_ph) {
             uint8_t* b_dst = smem + (size_t)b_stage * stage_bytes + A_STAGE_BYTES;
-            tma_load_2d(b_dst, P.maps + p.x_map, kk * BK, 0, ctl->full + b_stage, pol_x);
+            tma_load_2d(b_dst, P.maps + B.x_map, B.kk * BK, 0, ctl->full + b_stage, pol_x);
             ++b_count;
             if (++b_stage == stages) b_stage = 0;
-            ++b_kb;
-            b_ok = seek(b_ph, b_kb, b_end);
+            advance(B);
             progress = true;
           }
         }
-        if (progress) t_idle = clock64();
-        else if (W.poll_abort(t_idle) || ld_acquire_u64(P.bar + 1)) { ctl->abort_flag = 1; break; }
+        if (progress) { idle = 0; t_idle = clock64(); }
+        else {
+          ++idle;
+          if (W.poll_abort(t_idle)) break;
+          if ((idle & 4095u) == 0 && ld_acquire_u64(P.bar + 1)) { ctl->abort_flag = 1; break; }
+        }
       }
     }
   } else if (warp == 1) {
@@ -533,13 +555,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       for (int ph = 0; ph < P.n_phases && ok; ++ph) {
         const Phase& p = P.phases[ph];
         if (p.kind != PH_GEMM) continue;
-        const long long total = (long long)p.n_tiles * p.kblocks;
-        const KRange kr = phase_range(total, cta, G);
-        const long long kb_begin = kr.begin, kb_end = kr.end;
-        for (long long kb = kb_begin; kb < kb_end && ok; ++kb) {
-          const int kk = (int)(kb % p.kblocks);
-          const bool seg_first = (kb == kb_begin) || kk == 0;
-          const bool seg_last = (kb + 1 == kb_end) || kk == p.kblocks - 1;
+        const int kblocks = p.kblocks;
+        const KRange kr = phase_range((long long)p.n_tiles * kblocks, cta, G);
+        int remaining = (int)(kr.end - kr.begin);
+        if (remaining <= 0) continue;
+        int kk = (int)(kr.begin % kblocks);
+        bool seg_first = true;
+        while (remaining > 0 && ok) {
+          const bool seg_last = (remaining == 1) || (kk == kblocks - 1);
           if (seg_first) {
             ok = W.wait(ctl->acc_empty + buf, acc_phase[buf] ^ 1);
             if (!ok) break;
@@ -557,6 +580,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                       (seg_first && k == 0) ? 0u : 1u);
           umma_commit(ctl->empty + stage);
           if (seg_last) { umma_commit(ctl->acc_full + buf); acc_phase[buf] ^= 1; buf ^= 1; }
+          seg_first = seg_last;
+          if (++kk == kblocks) kk = 0;
+          --remaining;
           if (++stage == stages) { stage = 0; phase ^= 1; }
         }
       }
@@ -586,6 +612,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         if (!ok) break;
       }
 
+      const bool tracing = P.trace && et == 0 && (cta == 0 || cta == G - 1);
+      unsigned long long* tr = tracing ? P.trace + ((size_t)(cta == 0 ? 0 : 1) * P.n_phases + ph) * 3 : nullptr;
+      if (tracing) tr[0] = globaltimer_ns();
       if (p.kind == PH_EMBED) {
         if (cta == 0)
           for (int i = et; i < P.n_keys; i += 128) P.keys[i] = 0ull;
@@ -819,6 +848,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         }
       }
       if (!ok) break;
+      if (tracing) tr[1] = globaltimer_ns();
       // Publish this CTA's part of the phase.  A CTA may arrive for phase ph only once every
       // CTA has arrived for phase ph-1: otherwise CTAs without work in two consecutive GEMM
       // phases would run ahead and their arrivals would be mistaken for the slower CTAs' ones
@@ -836,6 +866,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         epi_bar_sync();
       }
       if (et == 0) red_release_add_u64(P.bar, 1ull);
+      if (tracing) tr[2] = globaltimer_ns();
       waited = false;
     }
   }
