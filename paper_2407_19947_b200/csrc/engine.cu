@@ -37,6 +37,8 @@ constexpr int MK_MAX_ROWS = 64;          // rows per call the persistent kernel 
 constexpr int MK_TBOX_SLOTS = MK_MAX_ROWS / 16;
 
 struct DevModel {
+  float* rope_inv = nullptr;     // device: theta^(-2i/hd), i < hd/2
+  float* ln_aux = nullptr;       // device: LayerNorm u/c vectors (see build_program)
   bool prog_built[MK_TBOX_SLOTS] = {false, false, false, false};
   char* prog_base = nullptr;     // device: per t_box slot, phases followed by tensor maps
   size_t prog_slot_bytes = 0, prog_maps_off = 0;
@@ -54,8 +56,8 @@ struct DevModel {
 
 struct Layout {
   size_t status, seq, n_seq, page_table, tok, pos, req, val_req, val_k, val_off, keys, x, h, qkv, q,
-      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_bar, attn_part, prog_t, prog_d, mk_trace, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
-  int max_rows, logit_rows, max_pages, n_pages, t_box_max, attn_units;
+      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_bar, attn_part, prog_t, prog_d, mk_trace, mk_stats, attn_cnt, rope_t, rope_d, aux_t, aux_d, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
+  int max_rows, logit_rows, max_pages, n_pages, t_box_max, attn_units, stat_tiles, attn_cnt_n;
   size_t prog_slot_t, prog_slot_d, prog_maps_off_t, prog_maps_off_d;
   size_t kv_t_layer, kv_d_layer;
 };
@@ -207,6 +209,20 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     L->prog_t = take(L->prog_slot_t * MK_TBOX_SLOTS);
     L->prog_d = take(L->prog_slot_d * MK_TBOX_SLOTS);
     L->mk_trace = take(t.wdtype == 1 ? (size_t)2 * (8 * std::max(t.n_layers, 1) + 4) * 3 * 8 : 0);
+    L->stat_tiles = (t.d_model + tc::BM - 1) / tc::BM;
+    L->mk_stats = take(t.wdtype == 1 ? (size_t)MK_MAX_ROWS * L->stat_tiles * 16 : 0);
+    L->attn_cnt_n = c.max_requests * hkv * std::max(n_qblk, 1);
+    L->attn_cnt = take(t.wdtype == 1 ? (size_t)L->attn_cnt_n * 4 : 0);
+    L->rope_t = take(t.wdtype == 1 ? (size_t)t.head_dim * 2 : 0);
+    L->rope_d = take((t.wdtype == 1 && has_draft) ? (size_t)d.head_dim * 2 : 0);
+    // LayerNorm models: u = W.gain and c = W.bias per normalised GEMM (fp32)
+    auto aux = [&](const stairs_model& m) {
+      if (m.norm != 0) return (size_t)0;
+      const size_t nqkv2 = (size_t)(m.n_heads + 2 * m.n_kv_heads) * m.head_dim, f2 = (size_t)m.d_ff * (m.act == 1 ? 2 : 1);
+      return ((nqkv2 + f2) * m.n_layers + m.vocab) * 2 * 4;
+    };
+    L->aux_t = take(t.wdtype == 1 ? aux(t) : 0);
+    L->aux_d = take((t.wdtype == 1 && has_draft) ? aux(d) : 0);
   }
   const size_t pool_tokens = (size_t)L->n_pages * pt;
   L->kv_t_layer = pool_tokens * t.n_kv_heads * t.head_dim * es;
@@ -354,6 +370,55 @@ int launch_gemm_tc(stairs_ctx* ctx, const TcArgs& a) {
 // ---------------------------------------------------------------------------------------------
 // Persistent forward kernel: per (model, row box) program and launch.
 // ---------------------------------------------------------------------------------------------
+// u[n] = sum_k W[n,k] * g[k],  c[n] = sum_k W[n,k] * b[k]   (one warp per row, fp32)
+__global__ void k_ln_aux(const bf16* __restrict__ W, const float* __restrict__ g, const float* __restrict__ b,
+                         float* __restrict__ u, float* __restrict__ c, int N, int K) {
+  const int n = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (n >= N) return;
+  float su = 0.f, sc = 0.f;
+  for (int k = lane; k < K; k += 32) {
+    const float w = __bfloat162float(W[(size_t)n * K + k]);
+    su = fmaf(w, g[k], su);
+    sc = fmaf(w, b[k], sc);
+  }
+  su = warp_sum(su); sc = warp_sum(sc);
+  if (lane == 0) { u[n] = su; c[n] = sc; }
+}
+
+// One-time per model: rotary frequency table and, for LayerNorm models, the u/c vectors.
+int setup_mk_model(stairs_ctx* ctx, DevModel& M, size_t rope_off, size_t aux_off) {
+  const stairs_model& m = M.m;
+  M.rope_inv = reinterpret_cast<float*>(ctx->ws + rope_off);
+  std::vector<float> inv(std::max(m.head_dim / 2, 1));
+  for (int i = 0; i < m.head_dim / 2; ++i)
+    inv[i] = (float)exp2(-(double)(2 * i) / (double)m.head_dim * log2((double)m.rope_theta));
+  CK(cudaMemcpyAsync(M.rope_inv, inv.data(), (size_t)(m.head_dim / 2) * 4, cudaMemcpyHostToDevice, ctx->stream));
+  CK(cudaStreamSynchronize(ctx->stream));
+  if (m.norm != 0) return STAIRS_OK;
+  M.ln_aux = reinterpret_cast<float*>(ctx->ws + aux_off);
+  const int d = m.d_model, nq = m.n_heads * m.head_dim, nkv = m.n_kv_heads * m.head_dim, nqkv = nq + 2 * nkv, F = m.d_ff;
+  const size_t f_aux = (size_t)F * (m.act == 1 ? 2 : 1);
+  const size_t aux_layer = ((size_t)nqkv + f_aux) * 2;
+  auto run = [&](const void* W, const void* g, const void* b, float* u, float* c, int N) {
+    k_ln_aux<<<(N + 7) / 8, 256, 0, ctx->stream>>>((const bf16*)W, (const float*)g, (const float*)b, u, c, N, d);
+  };
+  for (int l = 0; l < m.n_layers; ++l) {
+    const stairs_layer_w& w = M.layers[l];
+    float* b2 = M.ln_aux + (size_t)l * aux_layer;
+    float* qu = b2; float* qc = b2 + nqkv; float* fu = b2 + 2 * (size_t)nqkv; float* fc = fu + f_aux;
+    run(w.wq, w.norm1_w, w.norm1_b, qu, qc, nq);
+    run(w.wk, w.norm1_w, w.norm1_b, qu + nq, qc + nq, nkv);
+    run(w.wv, w.norm1_w, w.norm1_b, qu + nq + nkv, qc + nq + nkv, nkv);
+    run(w.w_gate_or_fc1, w.norm2_w, w.norm2_b, fu, fc, F);
+    if (m.act == 1) run(w.w_up, w.norm2_w, w.norm2_b, fu + F, fc + F, F);
+  }
+  float* hu = M.ln_aux + (size_t)m.n_layers * aux_layer;
+  run(M.w.lm_head, M.w.final_norm_w, M.w.final_norm_b, hu, hu + m.vocab, m.vocab);
+  CK(cudaGetLastError());
+  CK(cudaStreamSynchronize(ctx->stream));
+  return STAIRS_OK;
+}
+
 int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
   const stairs_model& m = M.m;
   const Layout& L = ctx->lay;
@@ -373,7 +438,7 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
             encode_map(ctx, &maps[i_ff], ws + L.ff, L.max_rows, F, t_box);
   if (!ok) return fail(ctx, STAIRS_ECUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
   std::vector<mk::Phase> ph;
-  auto gemm = [&](int layer, int w0, int w1, int w2, int n_src, const int* rows, bool dual, int xmap, int K, int epi, void* out, int ldo) {
+  auto gemm = [&](int layer, int w0, int w1, int w2, int n_src, const int* rows, bool dual, int xmap, int K, int epi, void* out, int ldo) -> mk::Phase& {
     mk::Phase p;
     memset(&p, 0, sizeof p);
     p.kind = mk::PH_GEMM; p.layer = layer;
@@ -390,36 +455,59 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
     }
     p.n_tiles = tiles; p.epi = epi; p.out = out; p.ldo = ldo;
     ph.push_back(p);
+    return ph.back();
   };
-  auto simple = [&](int kind, int layer, const void* g, const void* b, void* kc, void* vc) {
+  auto simple = [&](int kind, int layer, const void* g, void* kc, void* vc) {
     mk::Phase p;
     memset(&p, 0, sizeof p);
-    p.kind = kind; p.layer = layer; p.g = (const float*)g; p.b = (const float*)b; p.kc = kc; p.vc = vc;
+    p.kind = kind; p.layer = layer; p.g = (const float*)g; p.kc = kc; p.vc = vc;
     ph.push_back(p);
   };
+  // LayerNorm auxiliary vectors, laid out per layer as [qkv u | qkv c | mlp u | mlp c], then [head u | head c]
+  const bool ln = m.norm == 0;
+  const size_t f_aux = (size_t)F * (m.act == 1 ? 2 : 1);
+  const size_t aux_layer = ((size_t)nqkv + f_aux) * 2;
+  auto aux_ptr = [&](int l, int which) -> const float* {   // which: 0 qkv u, 1 qkv c, 2 mlp u, 3 mlp c
+    if (!ln) return nullptr;
+    const float* b2 = M.ln_aux + (size_t)l * aux_layer;
+    if (which == 0) return b2;
+    if (which == 1) return b2 + nqkv;
+    if (which == 2) return b2 + 2 * (size_t)nqkv;
+    return b2 + 2 * (size_t)nqkv + f_aux;
+  };
+  simple(mk::PH_EMBED, 0, M.layers[0].norm1_w, nullptr, nullptr);
   for (int l = 0; l < m.n_layers; ++l) {
     const stairs_layer_w& w = M.layers[l];
     const int b = 7 * l;
-    simple(l == 0 ? mk::PH_EMBED : mk::PH_NORM, l, w.norm1_w, w.norm1_b, nullptr, nullptr);
     const int r3[3] = {nq, nkv, nkv};
-    gemm(l, b + 0, b + 1, b + 2, 3, r3, false, i_h, d, tc::TC_STORE_F32, ws + L.qkv, nqkv);
-    simple(mk::PH_ATTN, l, nullptr, nullptr, M.kpool + (size_t)l * M.kv_layer_bytes, M.vpool + (size_t)l * M.kv_layer_bytes);
-    simple(mk::PH_COMBINE, l, nullptr, nullptr, nullptr, nullptr);
+    {
+      mk::Phase& p = gemm(l, b + 0, b + 1, b + 2, 3, r3, false, i_h, d, tc::TC_STORE_F32, ws + L.qkv, nqkv);
+      p.norm_in = 1; p.u = aux_ptr(l, 0); p.c = aux_ptr(l, 1);
+    }
+    simple(mk::PH_ATTN, l, nullptr, M.kpool + (size_t)l * M.kv_layer_bytes, M.vpool + (size_t)l * M.kv_layer_bytes);
     const int rd[1] = {d};
-    gemm(l, b + 3, b + 3, b + 3, 1, rd, false, i_o, nq, tc::TC_ADD_F32, ws + L.x, d);
-    simple(mk::PH_NORM, l, w.norm2_w, w.norm2_b, nullptr, nullptr);
+    {
+      mk::Phase& p = gemm(l, b + 3, b + 3, b + 3, 1, rd, false, i_o, nq, tc::TC_ADD_F32, ws + L.x, d);
+      p.next_g = (const float*)w.norm2_w;
+    }
     const int rf[1] = {F};
-    if (m.act == 1) gemm(l, b + 4, b + 5, b + 4, 1, rf, true, i_h, d, tc::TC_SWIGLU, ws + L.ff, F);
-    else gemm(l, b + 4, b + 4, b + 4, 1, rf, false, i_h, d, tc::TC_GELU, ws + L.ff, F);
-    gemm(l, b + 6, b + 6, b + 6, 1, rd, false, i_ff, F, tc::TC_ADD_F32, ws + L.x, d);
+    {
+      mk::Phase& p = (m.act == 1) ? gemm(l, b + 4, b + 5, b + 4, 1, rf, true, i_h, d, tc::TC_SWIGLU, ws + L.ff, F)
+                                  : gemm(l, b + 4, b + 4, b + 4, 1, rf, false, i_h, d, tc::TC_GELU, ws + L.ff, F);
+      p.norm_in = 1; p.u = aux_ptr(l, 2); p.c = aux_ptr(l, 3);
+    }
+    {
+      mk::Phase& p = gemm(l, b + 6, b + 6, b + 6, 1, rd, false, i_ff, F, tc::TC_ADD_F32, ws + L.x, d);
+      p.next_g = (const float*)(l + 1 < m.n_layers ? M.layers[l + 1].norm1_w : M.w.final_norm_w);
+    }
   }
-  simple(mk::PH_FINAL_NORM, -1, M.w.final_norm_w, M.w.final_norm_b, nullptr, nullptr);
   {
     const int rv[1] = {m.vocab};
-    gemm(-1, i_head, i_head, i_head, 1, rv, false, i_h, d, tc::TC_LMHEAD, nullptr, m.vocab);
-    ph.back().logit_rows = 1;
+    mk::Phase& p = gemm(-1, i_head, i_head, i_head, 1, rv, false, i_h, d, tc::TC_LMHEAD, nullptr, m.vocab);
+    p.norm_in = 1;
+    if (ln) { p.u = M.ln_aux + (size_t)m.n_layers * aux_layer; p.c = p.u + m.vocab; }
   }
-  simple(mk::PH_ACCEPT, -1, nullptr, nullptr, nullptr, nullptr);
+  simple(mk::PH_ACCEPT, -1, nullptr, nullptr, nullptr);
   for (const mk::Phase& p : ph)
     if (p.kind == mk::PH_GEMM && p.n_tiles > TC_COUNTERS) return fail(ctx, STAIRS_EUNSUPPORTED, "too many tiles for the split bookkeeping");
   M.n_phases = (int)ph.size();
@@ -478,6 +566,8 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.target_tokens = c.target_tokens; P.accept_len = c.accept_len; P.commit = c.commit; P.draft_out = c.draft_out;
   P.partial = reinterpret_cast<float*>(ws + L.gemm_partial); P.counters = reinterpret_cast<int*>(ws + L.gemm_counters);
   P.attn_part = reinterpret_cast<float*>(ws + L.attn_part); P.attn_part_units = L.attn_units;
+  P.stats = reinterpret_cast<float4*>(ws + L.mk_stats); P.stat_tiles = L.stat_tiles;
+  P.rope_inv = M.rope_inv; P.attn_cnt = reinterpret_cast<int*>(ws + L.attn_cnt);
   P.bar = reinterpret_cast<unsigned long long*>(ws + L.mk_bar); P.bar_base = ctx->bar_base;
   P.status = ctx->status_dev; P.wait_limit = ctx->wait_limit;
   P.trace = (ctx->profile && &M == &ctx->target) ? reinterpret_cast<unsigned long long*>(ws + L.mk_trace) : nullptr;
@@ -807,6 +897,13 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
           ctx->use_mk = true;
           ctx->target.prog_base = ctx->ws + L.prog_t; ctx->target.prog_slot_bytes = L.prog_slot_t; ctx->target.prog_maps_off = L.prog_maps_off_t;
           ctx->draft.prog_base = ctx->ws + L.prog_d; ctx->draft.prog_slot_bytes = L.prog_slot_d; ctx->draft.prog_maps_off = L.prog_maps_off_d;
+          int rc2 = setup_mk_model(ctx, ctx->target, L.rope_t, L.aux_t);
+          if (!rc2 && has_draft) rc2 = setup_mk_model(ctx, ctx->draft, L.rope_d, L.aux_d);
+          if (rc2) {
+            g_init_error = ctx->err;
+            stairs_destroy(ctx);
+            return rc2;
+          }
         }
       }
     }
@@ -1058,6 +1155,7 @@ int stairs_sync(stairs_ctx* ctx) {
     ctx->status_host[STATUS_ERROR] = 0;
     cudaMemsetAsync(ctx->ws + ctx->lay.mk_bar, 0, 64, ctx->stream);   // barrier count and abort word
     cudaMemsetAsync(ctx->ws + ctx->lay.gemm_counters, 0, (size_t)TC_COUNTERS * 4, ctx->stream);
+    cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)ctx->lay.attn_cnt_n * 4, ctx->stream);
     cudaStreamSynchronize(ctx->stream);
     ctx->bar_base = 0;
     return fail(ctx, (int)code, "a device-side bounded wait expired (code %u); results of the last calls are invalid", code);

@@ -36,7 +36,7 @@ namespace mk {
 
 using namespace tc;
 
-enum PhaseKind { PH_EMBED = 0, PH_NORM = 1, PH_GEMM = 2, PH_ATTN = 3, PH_COMBINE = 4, PH_FINAL_NORM = 5, PH_ACCEPT = 6 };
+enum PhaseKind { PH_EMBED = 0, PH_GEMM = 2, PH_ATTN = 3, PH_ACCEPT = 6 };
 
 struct Phase {
   int kind, layer;
@@ -44,10 +44,16 @@ struct Phase {
   int w_map[3], x_map;
   int src_tiles[3], src_col[3];
   int n_src, dual, n_tiles, kblocks, N, epi, ldo;
-  int logit_rows;            // 1: valid rows = n_logit_rows (LM head), else T
   void* out;                 // fp32 or bf16 output
-  // PH_NORM / PH_EMBED / PH_FINAL_NORM
-  const float* g; const float* b;
+  // Normalisation folded into the GEMMs.  norm_in: the activation operand is bf16(x * gain) and
+  // the epilogue applies y = rstd_t * (acc - mean_t * u[n]) + c[n] with u = W.gain, c = W.bias
+  // (LayerNorm; both NULL for RMSNorm, where y = rstd_t * acc).  next_g: this residual GEMM's
+  // finisher also writes bf16(x * next_g) for the following GEMM and per-tile row statistics.
+  int norm_in;
+  const float* u; const float* c;
+  const float* next_g;
+  // PH_EMBED
+  const float* g;
   // PH_ATTN
   void* kc; void* vc;
 };
@@ -71,6 +77,10 @@ struct Params {
   const int* page_table; int page_tokens, max_pages;
   float* x; bf16* h; float* qkv; bf16* o; bf16* ff;
   unsigned long long* keys; int n_keys;
+  float4* stats;            // [64 rows][stat_tiles] (mean, M2, count, -) per 128-column tile of x
+  int stat_tiles;
+  const float* rope_inv;    // [hd/2] theta^(-2i/hd)
+  int* attn_cnt;            // split-KV arrival counters per (request, kv head, query block)
   float* logits;            // optional dump
   int* target_tokens; int* accept_len; int commit; int* draft_out;
   // scratch
@@ -142,6 +152,8 @@ struct Ctl {
   volatile int abort_flag;
   volatile int last_flag;
   volatile int bcast;
+  float rstd[64], mu[64];       // per-row statistics of the current norm_in GEMM phase
+  float red[4][16], red2[4][16];
 };
 
 // Uniform verdict for the 128 compute threads after any of them may have timed out in a wait:
@@ -221,24 +233,35 @@ __device__ __forceinline__ float group_sum(float v, float* red, int et) {
   return red[0] + red[1] + red[2] + red[3];
 }
 
-// h[row] = norm(x[row]) (bf16), by the 128 compute threads
-__device__ void norm_row(const Params& P, const float* xr, const float* g, const float* b, bf16* hr, float* red, int et) {
+// Row t of the residual stream from the embedding tables, the next GEMM's operand bf16(x * g)
+// and the row's statistics (one entry covering the whole row), by the 128 compute threads.
+__device__ void embed_row(const Params& P, int t, const RowInfo& r, const float* g, float* red, int et) {
   const int d = P.d;
-  float mean = 0.f;
-  if (P.norm_kind == 0) {
-    float s = 0.f;
-    for (int i = et; i < d; i += 128) s += xr[i];
-    mean = group_sum(s, red, et) / (float)d;
+  float* xr = P.x + (size_t)t * d;
+  bf16* hr = P.h + (size_t)t * d;
+  const bf16* e = P.tok_emb + (size_t)r.tok * d;
+  const bf16* pe = P.pos_emb ? P.pos_emb + (size_t)r.pos * d : nullptr;
+  float xv[64];   // d <= 8192
+  float s1 = 0.f;
+#pragma unroll
+  for (int i = 0; i < 64; ++i) {
+    const int col = et + 128 * i;
+    float v = 0.f;
+    if (col < d) {
+      v = __bfloat162float(e[col]);
+      if (pe) v += __bfloat162float(pe[col]);
+      xr[col] = v;
+      hr[col] = __float2bfloat16_rn(v * g[col]);
+    }
+    xv[i] = v; s1 += v;
   }
-  float ss = 0.f;
-  for (int i = et; i < d; i += 128) { const float c = xr[i] - mean; ss += c * c; }
-  const float var = group_sum(ss, red, et) / (float)d;
-  const float rstd = 1.0f / sqrtf(var + P.eps);
-  for (int i = et; i < d; i += 128) {
-    float v = (xr[i] - mean) * rstd * g[i];
-    if (b) v += b[i];
-    hr[i] = __float2bfloat16_rn(v);
-  }
+  const float mean = group_sum(s1, red, et) / (float)d;
+  float s2 = 0.f;
+#pragma unroll
+  for (int i = 0; i < 64; ++i) { const int col = et + 128 * i; if (col < d) { const float c = xv[i] - mean; s2 += c * c; } }
+  const float m2 = group_sum(s2, red, et);
+  for (int tile = et; tile < P.stat_tiles; tile += 128)
+    P.stats[(size_t)t * P.stat_tiles + tile] = tile == 0 ? make_float4(mean, m2, (float)d, 0.f) : make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -268,13 +291,10 @@ __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
   return a;
 }
 
-__device__ __forceinline__ float rope_inv_freq(int i, int hd, float theta) {
-  return (float)exp2(-(double)(2 * i) / (double)hd * log2((double)theta));
-}
 
 // One attention unit, executed by the 128 compute threads.
 __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot,
-                          uint8_t* att_smem, Ctl* ctl, uint32_t& att_parity, const Waiter& W, int et, bool& ok) {
+                          int first_slot, int cnt_idx, uint8_t* att_smem, Ctl* ctl, uint32_t& att_parity, const Waiter& W, int et, bool& ok) {
   const int hd = P.hd, G = P.Hq / P.Hkv, nkv = P.Hkv * hd, nq = P.Hq * hd, nqkv = nq + 2 * nkv;
   const int lane = et & 31, w = et >> 5;
   const int Q = a.R * G;
@@ -297,7 +317,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     const float* src = P.qkv + (size_t)(a.off + r) * nqkv + (size_t)head * hd;
     float x0 = src[i], x1 = src[i + half];
     if (P.rope) {
-      const float ang = (float)(a.base + r) * rope_inv_freq(i, hd, P.rope_theta);
+      const float ang = (float)(a.base + r) * P.rope_inv[i];
       float s, c;
       sincosf(ang, &s, &c);
       const float r0 = x0 * c - x1 * s, r1 = x1 * c + x0 * s;
@@ -341,7 +361,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
         const float* vsrc = row + nq + nkv + (size_t)kvh * hd;
         float x0 = ksrc[i], x1 = ksrc[i + half];
         if (P.rope) {
-          const float ang = (float)p * rope_inv_freq(i, hd, P.rope_theta);
+          const float ang = (float)p * P.rope_inv[i];
           float s, cc;
           sincosf(ang, &s, &cc);
           const float r0 = x0 * cc - x1 * s, r1 = x1 * cc + x0 * s;
@@ -417,9 +437,55 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     }
     epi_bar_sync();   // tile may be overwritten by the next chunk
   }
-  // park the unit's state for the combine phase
+  if (!ok) return;
+  const int Hq = P.Hq;
+  if (a.n_ranges == 1) {
+    // the unit saw every visible position: normalise and write the attention output directly
+    for (int idx = et; idx < nQ * hd; idx += 128) {
+      const int ql = idx / hd, dd = idx % hd, q = q0 + ql;
+      const float* st = state + (size_t)ql * (hd + 2);
+      P.o[(size_t)(a.off + q / G) * Hq * hd + (size_t)(kvh * G + q % G) * hd + dd] = __float2bfloat16_rn(st[dd] / st[hd + 1]);
+    }
+    epi_bar_sync();
+    return;
+  }
+  // several units share the positions: park this unit's state; whichever unit of this
+  // (request, kv head, query block) arrives last merges all of them in position order
   float* dst = P.attn_part + (size_t)part_slot * ATT_QBLK * (hd + 2);
   for (int idx = et; idx < nQ * (hd + 2); idx += 128) dst[idx] = state[idx];
+  __threadfence();
+  epi_bar_sync();
+  if (et == 0) {
+    const int old = atomicAdd(P.attn_cnt + cnt_idx, 1);
+    ctl->last_flag = (old == a.n_ranges - 1) ? 1 : 0;
+    if (old == a.n_ranges - 1) P.attn_cnt[cnt_idx] = 0;
+  }
+  epi_bar_sync();
+  const bool last = ctl->last_flag != 0;
+  epi_bar_sync();
+  if (!last) return;
+  __threadfence();
+  for (int ql = w; ql < nQ; ql += 4) {
+    const int q = q0 + ql;
+    float M = -INFINITY;
+    for (int rg = 0; rg < a.n_ranges; ++rg)
+      M = fmaxf(M, __ldcg(P.attn_part + ((size_t)(first_slot + rg * a.n_qblk) * ATT_QBLK + ql) * (hd + 2) + hd));
+    float L = 0.f, acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    for (int rg = 0; rg < a.n_ranges; ++rg) {
+      const float* st = P.attn_part + ((size_t)(first_slot + rg * a.n_qblk) * ATT_QBLK + ql) * (hd + 2);
+      const float mu = __ldcg(st + hd);
+      if (mu == -INFINITY) continue;
+      const float wgt = expf(mu - M);
+      L += __ldcg(st + hd + 1) * wgt;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { const int dd = lane + 32 * j; if (dd < hd) acc[j] += __ldcg(st + dd) * wgt; }
+    }
+    bf16* orow = P.o + (size_t)(a.off + q / G) * Hq * hd + (size_t)(kvh * G + q % G) * hd;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { const int dd = lane + 32 * j; if (dd < hd) orow[dd] = __float2bfloat16_rn(acc[j] / L); }
+  }
   epi_bar_sync();
 }
 
@@ -621,26 +687,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         for (int t = cta; t < P.T; t += G) {
           const RowInfo r = row_info(P, t);
           if (et == 0) { P.tok[t] = r.tok; P.pos[t] = r.pos; P.req[t] = r.slot; }
-          float* xr = P.x + (size_t)t * P.d;
-          const bf16* e = P.tok_emb + (size_t)r.tok * P.d;
-          const bf16* pe = P.pos_emb ? P.pos_emb + (size_t)r.pos * P.d : nullptr;
-          for (int i = et; i < P.d; i += 128) {
-            float v = __bfloat162float(e[i]);
-            if (pe) v += __bfloat162float(pe[i]);
-            xr[i] = v;
-          }
-          epi_bar_sync();
-          norm_row(P, xr, p.g, p.b, P.h + (size_t)t * P.d, red, et);
+          embed_row(P, t, r, p.g, red, et);
         }
-      } else if (p.kind == PH_NORM) {
-        for (int t = cta; t < P.T; t += G)
-          norm_row(P, P.x + (size_t)t * P.d, p.g, p.b, P.h + (size_t)t * P.d, red, et);
-      } else if (p.kind == PH_FINAL_NORM) {
-        for (int t = cta; t < P.n_logit_rows; t += G)
-          norm_row(P, P.x + (size_t)(P.logit_first_row + t) * P.d, p.g, p.b, P.h + (size_t)t * P.d, red, et);
       } else if (p.kind == PH_ATTN) {
         const int n_req = P.mode == CALL_VALIDATE ? P.n_req : 1;
-        int u0 = 0;
+        int u0 = 0, g0 = 0;
         for (int i = 0; i < n_req && ok; ++i) {
           const AttnReq a = attn_req(P, i, G);
           // units of this request: index = ((kvh * n_ranges) + range) * n_qblk + qblk
@@ -649,47 +700,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const int qblk = u % a.n_qblk, rest = u / a.n_qblk;
             const int range = rest % a.n_ranges, kvh = rest / a.n_ranges;
             const int slot = u0 + u;
+            const int first_slot = u0 + (kvh * a.n_ranges) * a.n_qblk + qblk;   // range 0 of this (kvh, qblk)
             if (slot < P.attn_part_units)
-              attn_unit(P, p, a, kvh, range, qblk, slot, att_smem, ctl, att_parity, W, et, ok);
+              attn_unit(P, p, a, kvh, range, qblk, slot, first_slot, g0 + kvh * a.n_qblk + qblk, att_smem, ctl, att_parity, W, et, ok);
           }
-          u0 += a.units;
-        }
-      } else if (p.kind == PH_COMBINE) {
-        // merge the units of every (request, kv head, query) in position order -> o (bf16)
-        const int n_req = P.mode == CALL_VALIDATE ? P.n_req : 1;
-        const int hd = P.hd, Gq = P.Hq / P.Hkv;
-        int u0 = 0, item0 = 0;
-        for (int i = 0; i < n_req; ++i) {
-          const AttnReq a = attn_req(P, i, G);
-          const int Q = a.R * Gq;
-          const int items = P.Hkv * Q;   // one warp per (kvh, q)
-          for (int it = (cta * 4 + (et >> 5)) - item0 % (G * 4); it < items; it += G * 4) {
-            if (it < 0) continue;
-            const int kvh = it / Q, q = it % Q, qblk = q / ATT_QBLK, ql = q % ATT_QBLK;
-            const int r = q / Gq, head = kvh * Gq + (q % Gq);
-            float M = -INFINITY;
-            for (int rg = 0; rg < a.n_ranges; ++rg) {
-              const int slot = u0 + (kvh * a.n_ranges + rg) * a.n_qblk + qblk;
-              M = fmaxf(M, __ldcg(P.attn_part + ((size_t)slot * ATT_QBLK + ql) * (hd + 2) + hd));
-            }
-            float L = 0.f, acc[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-            for (int rg = 0; rg < a.n_ranges; ++rg) {
-              const int slot = u0 + (kvh * a.n_ranges + rg) * a.n_qblk + qblk;
-              const float* st = P.attn_part + ((size_t)slot * ATT_QBLK + ql) * (hd + 2);
-              const float mu = __ldcg(st + hd);
-              if (mu == -INFINITY) continue;
-              const float wgt = expf(mu - M);
-              L += __ldcg(st + hd + 1) * wgt;
-#pragma unroll
-              for (int j = 0; j < 8; ++j) { const int dd = (et & 31) + 32 * j; if (dd < hd) acc[j] += __ldcg(st + dd) * wgt; }
-            }
-            bf16* orow = P.o + (size_t)(a.off + r) * P.Hq * hd + (size_t)head * hd;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) { const int dd = (et & 31) + 32 * j; if (dd < hd) orow[dd] = __float2bfloat16_rn(acc[j] / L); }
-          }
-          u0 += a.units; item0 += items;
+          u0 += a.units; g0 += P.Hkv * a.n_qblk;
         }
       } else if (p.kind == PH_ACCEPT) {
         if (cta == 0) {
@@ -722,10 +737,35 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         const KRange kr = phase_range(total, cta, G);
         const long long kb_begin = kr.begin, kb_end = kr.end;
         const int Ge = kr.ge;
-        const int Tvalid = p.logit_rows ? P.n_logit_rows : P.T;
+        const int Tvalid = P.T;
         float* out_f32 = (p.epi == TC_LMHEAD) ? P.logits : reinterpret_cast<float*>(p.out);
         bf16* out_act = reinterpret_cast<bf16*>(p.out);
-        unsigned long long* keys = P.keys + P.logit_first_row;
+        unsigned long long* keys = P.keys;
+        if (p.norm_in && kb_begin < kb_end) {
+          // row statistics of the operand: merge the per-tile entries (published by the phase
+          // that produced x) into mean and 1/std per row
+          if (et == 0) ctl->bcast = W.wait_grid(bar_count, P.bar_base + (unsigned long long)ph * G) ? 1 : 0;
+          epi_bar_sync();
+          ok = ctl->bcast != 0;
+          epi_bar_sync();
+          if (!ok) break;
+          if (et < Tvalid) {
+            float n = 0.f, mean = 0.f, m2 = 0.f;
+            for (int tl = 0; tl < P.stat_tiles; ++tl) {
+              const float4 sv = __ldcg(P.stats + (size_t)et * P.stat_tiles + tl);
+              if (sv.z > 0.f) {
+                const float delta = sv.x - mean, tot = n + sv.z;
+                mean += delta * sv.z / tot;
+                m2 += sv.y + delta * delta * n * sv.z / tot;
+                n = tot;
+              }
+            }
+            if (P.norm_kind == 0) { ctl->mu[et] = mean; ctl->rstd[et] = 1.0f / sqrtf(m2 / (float)P.d + P.eps); }
+            else { ctl->mu[et] = 0.f; ctl->rstd[et] = 1.0f / sqrtf((m2 + n * mean * mean) / (float)P.d + P.eps); }
+          }
+          epi_bar_sync();
+        }
+        const int tile_cols = BM;
         long long kb = kb_begin;
         while (kb < kb_end && ok) {
           const int tile = (int)(kb / p.kblocks), kk0 = (int)(kb % p.kblocks);
@@ -748,6 +788,16 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             n_out = p.src_col[s] + in_src; n_valid = in_src < src_n;
           }
           auto finish = [&](int c0, float* v) {
+            if (p.norm_in) {
+              // fold the normalisation in: y = rstd_t * (acc - mean_t * u[n]) + c[n]
+              const int ncol = (p.dual && m >= 64) ? p.N + n_out : n_out;
+              const float un = (p.u && n_valid) ? p.u[ncol] : 0.f, cn = (p.c && n_valid) ? p.c[ncol] : 0.f;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const int t = c0 + j;
+                if (t < Tvalid) v[j] = ctl->rstd[t] * (v[j] - ctl->mu[t] * un) + cn;
+              }
+            }
             if (p.epi == TC_SWIGLU) {
               if (m >= 64) {
 #pragma unroll
@@ -778,6 +828,42 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                 }
                 if (lane == 0 && key) atomicMax(keys + t, key);
               }
+              return;
+            }
+            if (p.epi == TC_ADD_F32 && p.next_g) {
+              // residual update; also the next GEMM's operand bf16(x * gain) and this tile's row
+              // statistics (mean and centred sum of squares over the tile's columns)
+              const float gn = n_valid ? p.next_g[n_out] : 0.f;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const int t = c0 + j;
+                float xn = 0.f;
+                if (n_valid && t < Tvalid) {
+                  const size_t o = (size_t)t * p.ldo + n_out;
+                  xn = out_f32[o] + v[j];
+                  out_f32[o] = xn;
+                  P.h[o] = __float2bfloat16_rn(xn * gn);
+                }
+                v[j] = xn;
+                const float s1 = warp_sum(xn);
+                if (lane == 0) ctl->red[quad][j] = s1;
+              }
+              epi_bar_sync();
+              const int cnt = min(tile_cols, p.N - tile * BM);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const float mean = (ctl->red[0][j] + ctl->red[1][j] + ctl->red[2][j] + ctl->red[3][j]) / (float)cnt;
+                const float dl = n_valid ? v[j] - mean : 0.f;
+                const float s2 = warp_sum(dl * dl);
+                if (lane == 0) ctl->red2[quad][j] = s2;
+              }
+              epi_bar_sync();
+              if (et < 16 && c0 + et < Tvalid) {
+                const float mean = (ctl->red[0][et] + ctl->red[1][et] + ctl->red[2][et] + ctl->red[3][et]) / (float)cnt;
+                const float m2 = ctl->red2[0][et] + ctl->red2[1][et] + ctl->red2[2][et] + ctl->red2[3][et];
+                P.stats[(size_t)(c0 + et) * P.stat_tiles + tile] = make_float4(mean, m2, (float)cnt, 0.f);
+              }
+              epi_bar_sync();
               return;
             }
             if (!n_valid) return;
