@@ -749,10 +749,12 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           ok = ctl->bcast != 0;
           epi_bar_sync();
           if (!ok) break;
-          if (et < Tvalid) {
+          // one warp per row, one lane per tile entry (all loads of a row in flight at once), then
+          // a shuffle tree merges (count, mean, M2) triples pairwise
+          for (int t = quad; t < Tvalid; t += 4) {
             float n = 0.f, mean = 0.f, m2 = 0.f;
-            for (int tl = 0; tl < P.stat_tiles; ++tl) {
-              const float4 sv = __ldcg(P.stats + (size_t)et * P.stat_tiles + tl);
+            for (int tl = lane; tl < P.stat_tiles; tl += 32) {
+              const float4 sv = __ldcg(P.stats + (size_t)t * P.stat_tiles + tl);
               if (sv.z > 0.f) {
                 const float delta = sv.x - mean, tot = n + sv.z;
                 mean += delta * sv.z / tot;
@@ -760,8 +762,23 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                 n = tot;
               }
             }
-            if (P.norm_kind == 0) { ctl->mu[et] = mean; ctl->rstd[et] = 1.0f / sqrtf(m2 / (float)P.d + P.eps); }
-            else { ctl->mu[et] = 0.f; ctl->rstd[et] = 1.0f / sqrtf((m2 + n * mean * mean) / (float)P.d + P.eps); }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+              const float n2 = __shfl_xor_sync(0xffffffffu, n, o), mean2 = __shfl_xor_sync(0xffffffffu, mean, o),
+                          m22 = __shfl_xor_sync(0xffffffffu, m2, o);
+              const float tot = n + n2;
+              if (tot > 0.f) {
+                // symmetric form so that both partners compute the same merged triple
+                const float delta = mean2 - mean;
+                const float mm = (n * mean + n2 * mean2) / tot;
+                m2 = m2 + m22 + delta * delta * n * n2 / tot;
+                mean = mm; n = tot;
+              }
+            }
+            if (lane == 0) {
+              if (P.norm_kind == 0) { ctl->mu[t] = mean; ctl->rstd[t] = 1.0f / sqrtf(m2 / (float)P.d + P.eps); }
+              else { ctl->mu[t] = 0.f; ctl->rstd[t] = 1.0f / sqrtf((m2 + n * mean * mean) / (float)P.d + P.eps); }
+            }
           }
           epi_bar_sync();
         }
@@ -834,8 +851,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               // residual update; also the next GEMM's operand bf16(x * gain) and this tile's row
               // statistics (mean and centred sum of squares over the tile's columns)
               const float gn = n_valid ? p.next_g[n_out] : 0.f;
+              const int jn = min(16, Tvalid - c0);   // rows of this chunk that exist (uniform)
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
+                if (j >= jn) break;
                 const int t = c0 + j;
                 float xn = 0.f;
                 if (n_valid && t < Tvalid) {
@@ -852,6 +871,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               const int cnt = min(tile_cols, p.N - tile * BM);
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
+                if (j >= jn) break;
                 const float mean = (ctl->red[0][j] + ctl->red[1][j] + ctl->red[2][j] + ctl->red[3][j]) / (float)cnt;
                 const float dl = n_valid ? v[j] - mean : 0.f;
                 const float s2 = warp_sum(dl * dl);
