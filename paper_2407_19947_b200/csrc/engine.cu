@@ -198,7 +198,7 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     const int rows_req = std::min(c.k_max + 1, MK_MAX_ROWS);
     const int n_qblk = (rows_req * gq + mk::ATT_QBLK - 1) / mk::ATT_QBLK;
     L->attn_units = c.max_requests * (2 * TC_GRID_MAX + 2 * hkv) * std::max(n_qblk, 1);
-    L->attn_part = take(t.wdtype == 1 ? (size_t)L->attn_units * mk::ATT_QBLK * (hdm + 2) * 4 : 0);
+    L->attn_part = take(t.wdtype == 1 ? (size_t)L->attn_units * mk::ATT_QBLK * (hdm + 4) * 4 : 0);
     auto prog = [&](const stairs_model& m, size_t* maps_off) {
       const size_t ph = align_up((size_t)(8 * std::max(m.n_layers, 1) + 4) * sizeof(mk::Phase), 128);
       *maps_off = ph;
@@ -485,6 +485,7 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
       p.norm_in = 1; p.u = aux_ptr(l, 0); p.c = aux_ptr(l, 1);
     }
     simple(mk::PH_ATTN, l, nullptr, M.kpool + (size_t)l * M.kv_layer_bytes, M.vpool + (size_t)l * M.kv_layer_bytes);
+    simple(mk::PH_COMBINE, l, nullptr, nullptr, nullptr);
     const int rd[1] = {d};
     {
       mk::Phase& p = gemm(l, b + 3, b + 3, b + 3, 1, rd, false, i_o, nq, tc::TC_ADD_F32, ws + L.x, d);
@@ -529,7 +530,7 @@ struct MkCall {
 };
 
 bool mk_eligible(const stairs_ctx* ctx, const DevModel& M, int T) {
-  return ctx->use_mk && M.m.n_layers >= 1 && T >= 1 && T <= MK_MAX_ROWS;
+  return ctx->use_mk && M.m.n_layers >= 1 && T >= 1 && T <= MK_MAX_ROWS && M.m.head_dim % 16 == 0 && M.m.head_dim <= 128;
 }
 
 int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, int n_logit_rows, const MkCall& c) {

@@ -36,7 +36,7 @@ namespace mk {
 
 using namespace tc;
 
-enum PhaseKind { PH_EMBED = 0, PH_GEMM = 2, PH_ATTN = 3, PH_ACCEPT = 6 };
+enum PhaseKind { PH_EMBED = 0, PH_GEMM = 2, PH_ATTN = 3, PH_COMBINE = 4, PH_ACCEPT = 6 };
 
 struct Phase {
   int kind, layer;
@@ -85,7 +85,7 @@ struct Params {
   int* target_tokens; int* accept_len; int commit; int* draft_out;
   // scratch
   float* partial; int* counters;
-  float* attn_part;         // [units][QBLK][hd + 2]
+  float* attn_part;         // [units][QBLK][hd + 4]: O, running max, running sum, pad
   int attn_part_units;
   unsigned long long* bar;  // [0] arrivals (monotonic), [1] abort word
   unsigned long long bar_base;
@@ -96,12 +96,28 @@ struct Params {
 constexpr int ATT_CHUNK = 64;
 constexpr int ATT_QBLK = 48;
 
-struct AttnSmem {   // carved after the GEMM ring
+struct AttnSmem {   // carved after the GEMM ring: Q block (bf16), K and V chunk tiles (bf16), merge buffer (fp32)
   static __host__ __device__ size_t k_pitch(int hd) { return (size_t)hd * 2 + 16; }
-  static __host__ __device__ size_t bytes(int hd) {
-    return (size_t)ATT_QBLK * hd * 4 + (size_t)ATT_QBLK * (hd + 2) * 4 + 2 * ATT_CHUNK * k_pitch(hd) + 64;
-  }
+  static __host__ __device__ size_t q_bytes(int hd) { return (size_t)ATT_QBLK * k_pitch(hd); }
+  static __host__ __device__ size_t kv_bytes(int hd) { return (size_t)ATT_CHUNK * k_pitch(hd); }
+  static __host__ __device__ size_t merge_bytes(int hd) { return (size_t)16 * (hd + 4) * 4 + 64; }
+  static __host__ __device__ size_t bytes(int hd) { return q_bytes(hd) + 2 * kv_bytes(hd) + merge_bytes(hd) + 64; }
 };
+
+// mma.sync m16n8k16 (bf16 in, fp32 accumulate) and its operand loads, for the attention tiles
+__device__ __forceinline__ void mma_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, const void* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
 
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
   unsigned long long v;
@@ -292,66 +308,79 @@ __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
 }
 
 
-// One attention unit, executed by the 128 compute threads.
+// One attention unit, executed by the 128 compute threads (4 warps), on the legacy tensor path
+// (mma.sync m16n8k16; the tiles are far too small for tcgen05).  The unit's queries are cut into
+// blocks of 16 (one MMA M tile); each 64-position chunk is staged once in shared memory and warp
+// w takes positions 16w..16w+15 of it for every block: S = Q.K^T (2 n-tiles x hd/16 k-steps),
+// online softmax per row with quad shuffles, O += P.V with P reused from the accumulator
+// registers and V fetched with ldmatrix.trans.  The four warps' (max, sum, O) states are merged
+// in warp order through a small shared buffer - a fixed order - and the block's result is either
+// final (the unit saw every visible position) or parked for the combine phase.
 __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot,
-                          int first_slot, int cnt_idx, uint8_t* att_smem, Ctl* ctl, uint32_t& att_parity, const Waiter& W, int et, bool& ok) {
+                          uint8_t* att_smem, Ctl* ctl, uint32_t& att_parity, const Waiter& W, int et, bool& ok) {
   const int hd = P.hd, G = P.Hq / P.Hkv, nkv = P.Hkv * hd, nq = P.Hq * hd, nqkv = nq + 2 * nkv;
-  const int lane = et & 31, w = et >> 5;
+  const int lane = et & 31, w = et >> 5, g = lane >> 2, t4 = lane & 3;
   const int Q = a.R * G;
   const int q0 = qblk * ATT_QBLK, nQ = min(ATT_QBLK, Q - q0);
-  float* qs = reinterpret_cast<float*>(att_smem);                       // [QBLK][hd] rotated, pre-scaled
-  float* state = qs + (size_t)ATT_QBLK * hd;                            // [QBLK][hd + 2]
   const size_t pitch = AttnSmem::k_pitch(hd);
-  uint8_t* ks = reinterpret_cast<uint8_t*>(state + (size_t)ATT_QBLK * (hd + 2));
-  uint8_t* vs = ks + ATT_CHUNK * pitch;
+  uint8_t* qs = att_smem;                                   // [QBLK][pitch] bf16, rotated and pre-scaled
+  uint8_t* ks = qs + AttnSmem::q_bytes(hd);                 // [CHUNK][pitch]
+  uint8_t* vs = ks + AttnSmem::kv_bytes(hd);
+  float* mrg = reinterpret_cast<float*>(vs + AttnSmem::kv_bytes(hd));   // [16][hd + 4]
   bf16* kc = reinterpret_cast<bf16*>(ph.kc);
   bf16* vc = reinterpret_cast<bf16*>(ph.vc);
   const int* pt = P.page_table + (size_t)a.slot * P.max_pages;
   const float scale = 1.0f / sqrtf((float)hd);
-  const int half = hd / 2;
+  const int half = hd / 2, ksteps = hd / 16, ntiles = hd / 8;
 
-  // queries of this block: query index q -> row r = q / G, head g = q % G
-  for (int idx = et; idx < nQ * half; idx += 128) {
+  // queries of this block: query index q -> row r = q / G, head = kvh * G + q % G
+  for (int idx = et; idx < ATT_QBLK * half; idx += 128) {
     const int ql = idx / half, i = idx % half, q = q0 + ql;
-    const int r = q / G, head = kvh * G + (q % G);
-    const float* src = P.qkv + (size_t)(a.off + r) * nqkv + (size_t)head * hd;
-    float x0 = src[i], x1 = src[i + half];
-    if (P.rope) {
-      const float ang = (float)(a.base + r) * P.rope_inv[i];
-      float s, c;
-      sincosf(ang, &s, &c);
-      const float r0 = x0 * c - x1 * s, r1 = x1 * c + x0 * s;
-      x0 = r0; x1 = r1;
+    float x0 = 0.f, x1 = 0.f;
+    if (ql < nQ) {
+      const int r = q / G, head = kvh * G + (q % G);
+      const float* src = P.qkv + (size_t)(a.off + r) * nqkv + (size_t)head * hd;
+      x0 = src[i]; x1 = src[i + half];
+      if (P.rope) {
+        const float ang = (float)(a.base + r) * P.rope_inv[i];
+        float sn, cs;
+        sincosf(ang, &sn, &cs);
+        const float r0 = x0 * cs - x1 * sn, r1 = x1 * cs + x0 * sn;
+        x0 = r0; x1 = r1;
+      }
     }
-    qs[(size_t)ql * hd + i] = x0 * scale;
-    qs[(size_t)ql * hd + i + half] = x1 * scale;
-  }
-  for (int idx = et; idx < nQ * (hd + 2); idx += 128) {
-    const int c = idx % (hd + 2);
-    state[idx] = (c == hd) ? -INFINITY : 0.f;   // [.. acc .., m, l]
+    bf16* qd = reinterpret_cast<bf16*>(qs + (size_t)ql * pitch);
+    qd[i] = __float2bfloat16_rn(x0 * scale);
+    qd[i + half] = __float2bfloat16_rn(x1 * scale);
   }
   epi_bar_sync();
 
   const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
-  for (int c = c_begin; c < c_end && ok; ++c) {
+  const bool single_chunk = (c_end - c_begin == 1);
+  const int n_mt = (nQ + 15) / 16;
+
+  // stages chunk c: one bulk async copy per cached row (K and V); rows of new positions are
+  // computed here (rotated k, v), patched into the tile and written to the cache
+  auto stage = [&](int c) {
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
-    // stage the chunk: one bulk async copy per cached row (K and V); rows of new positions are
-    // produced below instead
     if (et == 0) {
-      int cached = min(n_pos, max(0, a.base - p0));
+      const int cached = min(n_pos, max(0, a.base - p0));
       mbar_expect_tx(&ctl->att_bar, (uint32_t)(cached * 2 * hd * 2));
     }
     epi_bar_sync();
-    for (int j = et; j < n_pos; j += 128) {
+    for (int j = et; j < ATT_CHUNK; j += 128) {
       const int p = p0 + j;
-      if (p < a.base) {
+      if (j < n_pos && p < a.base) {
         const size_t slot = (size_t)pt[p / P.page_tokens] * P.page_tokens + (p % P.page_tokens);
         bulk_copy_g2s(ks + j * pitch, kc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
         bulk_copy_g2s(vs + j * pitch, vc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
+      } else if (j >= n_pos) {
+        // rows past the end of the sequence: zero V so that 0 * garbage cannot make a NaN
+        uint4* vz = reinterpret_cast<uint4*>(vs + j * pitch);
+        for (int q4 = 0; q4 < hd * 2 / 16; ++q4) vz[q4] = make_uint4(0, 0, 0, 0);
       }
     }
-    // new positions in this chunk: rotate k, round to bf16, patch the tile, write the cache
     {
       const int r_lo = max(0, p0 - a.base), r_hi = min(a.R, p0 + n_pos - a.base);
       for (int idx = et; idx < (r_hi - r_lo) * half; idx += 128) {
@@ -362,9 +391,9 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
         float x0 = ksrc[i], x1 = ksrc[i + half];
         if (P.rope) {
           const float ang = (float)p * P.rope_inv[i];
-          float s, cc;
-          sincosf(ang, &s, &cc);
-          const float r0 = x0 * cc - x1 * s, r1 = x1 * cc + x0 * s;
+          float sn, cs;
+          sincosf(ang, &sn, &cs);
+          const float r0 = x0 * cs - x1 * sn, r1 = x1 * cs + x0 * sn;
           x0 = r0; x1 = r1;
         }
         const bf16 k0 = __float2bfloat16_rn(x0), k1 = __float2bfloat16_rn(x1);
@@ -382,111 +411,148 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     }
     W.wait(&ctl->att_bar, att_parity);
     att_parity ^= 1;
-    ok = group_ok(ctl, et);
+    return group_ok(ctl, et);
+  };
+
+  for (int mt = 0; mt < n_mt && ok; ++mt) {
+    // rows of this warp's fragments: ql_a = mt*16 + g, ql_b = ql_a + 8
+    const int ql_a = mt * 16 + g, ql_b = ql_a + 8;
+    const int last_a = ql_a < nQ ? a.base + (q0 + ql_a) / G : -1;   // last visible position
+    const int last_b = ql_b < nQ ? a.base + (q0 + ql_b) / G : -1;
+    float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
+    float o[16][4];
+#pragma unroll
+    for (int nd = 0; nd < 16; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
+
+    for (int c = c_begin; c < c_end && ok; ++c) {
+      if (!(single_chunk && mt > 0)) {
+        ok = stage(c);
+        if (!ok) break;
+      }
+      const int p0 = c * ATT_CHUNK;
+      const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
+      const int sl0 = w * 16;                       // this warp's positions: p0 + sl0 .. + 15
+      if (sl0 < n_pos) {
+        float sc[2][4];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) { sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f; }
+        for (int kk = 0; kk < ksteps; ++kk) {
+          uint32_t af[4];
+          const uint8_t* qa = qs + (size_t)ql_a * pitch + (kk * 16 + t4 * 2) * 2;
+          af[0] = *reinterpret_cast<const uint32_t*>(qa);
+          af[1] = *reinterpret_cast<const uint32_t*>(qa + 8 * pitch);
+          af[2] = *reinterpret_cast<const uint32_t*>(qa + 16);
+          af[3] = *reinterpret_cast<const uint32_t*>(qa + 8 * pitch + 16);
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const uint8_t* kb = ks + (size_t)(sl0 + 8 * j + g) * pitch + (kk * 16 + t4 * 2) * 2;
+            mma_16816(sc[j], af, *reinterpret_cast<const uint32_t*>(kb), *reinterpret_cast<const uint32_t*>(kb + 16));
+          }
+        }
+        // staircase mask, row maxima
+        float mx_a = -INFINITY, mx_b = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int pj = p0 + sl0 + 8 * j + t4 * 2 + e;
+            const bool in = (pj - p0) < n_pos;
+            if (!(in && pj <= last_a)) sc[j][e] = -INFINITY;
+            if (!(in && pj <= last_b)) sc[j][2 + e] = -INFINITY;
+            mx_a = fmaxf(mx_a, sc[j][e]); mx_b = fmaxf(mx_b, sc[j][2 + e]);
+          }
+        }
+        mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1)); mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
+        mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1)); mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
+        const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
+        const float off_a = mn_a == -INFINITY ? 0.f : mn_a, off_b = mn_b == -INFINITY ? 0.f : mn_b;
+        const float corr_a = expf(m_a - off_a), corr_b = expf(m_b - off_b);   // exp(-inf) = 0
+        float sum_a = 0.f, sum_b = 0.f;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            sc[j][e] = expf(sc[j][e] - off_a); sc[j][2 + e] = expf(sc[j][2 + e] - off_b);
+            sum_a += sc[j][e]; sum_b += sc[j][2 + e];
+          }
+        }
+        sum_a += __shfl_xor_sync(0xffffffffu, sum_a, 1); sum_a += __shfl_xor_sync(0xffffffffu, sum_a, 2);
+        sum_b += __shfl_xor_sync(0xffffffffu, sum_b, 1); sum_b += __shfl_xor_sync(0xffffffffu, sum_b, 2);
+        l_a = l_a * corr_a + sum_a; l_b = l_b * corr_b + sum_b;
+        m_a = mn_a; m_b = mn_b;
+        uint32_t pf[4];
+        pf[0] = pack_bf16x2(sc[0][0], sc[0][1]); pf[1] = pack_bf16x2(sc[0][2], sc[0][3]);
+        pf[2] = pack_bf16x2(sc[1][0], sc[1][1]); pf[3] = pack_bf16x2(sc[1][2], sc[1][3]);
+        // V fragments: lane supplies the address of row (lane & 15) of the slice, column block (lane >> 4)
+        const uint8_t* vrow = vs + (size_t)(sl0 + (lane & 15)) * pitch + (lane >> 4) * 16;
+#pragma unroll
+        for (int nd = 0; nd < 16; nd += 2) {
+          if (nd < ntiles) {
+            o[nd][0] *= corr_a; o[nd][1] *= corr_a; o[nd][2] *= corr_b; o[nd][3] *= corr_b;
+            o[nd + 1][0] *= corr_a; o[nd + 1][1] *= corr_a; o[nd + 1][2] *= corr_b; o[nd + 1][3] *= corr_b;
+            uint32_t vf[4];
+            ldmatrix_x4_trans(vf, vrow + nd * 16);
+            mma_16816(o[nd], pf, vf[0], vf[1]);
+            mma_16816(o[nd + 1], pf, vf[2], vf[3]);
+          }
+        }
+      }
+      if (!(single_chunk) || mt == n_mt - 1) epi_bar_sync();   // tile may be overwritten next
+    }
     if (!ok) break;
 
-    // each warp takes queries w, w+4, ... of the block
-    for (int ql = w; ql < nQ; ql += 4) {
-      const int q = q0 + ql, r = q / G;
-      const int last = a.base + r;                 // last visible position of this query
-      const float* qv = qs + (size_t)ql * hd;
-      float s0 = -INFINITY, s1 = -INFINITY;
-      // scores: lane handles positions p0+lane and p0+lane+32
-      {
-        const int j0 = lane, j1 = lane + 32;
-        const bool v0 = (j0 < n_pos) && (p0 + j0 <= last), v1 = (j1 < n_pos) && (p0 + j1 <= last);
-        float d0 = 0.f, d1 = 0.f;
-        const uint8_t* k0p = ks + (size_t)(v0 ? j0 : 0) * pitch;
-        const uint8_t* k1p = ks + (size_t)(v1 ? j1 : 0) * pitch;
-        for (int d8 = 0; d8 < hd; d8 += 8) {
-          float ka[8], kb[8];
-          Vec16<bf16>::unpack(*reinterpret_cast<const uint4*>(k0p + d8 * 2), ka);
-          Vec16<bf16>::unpack(*reinterpret_cast<const uint4*>(k1p + d8 * 2), kb);
-          const float4 qa = *reinterpret_cast<const float4*>(qv + d8), qb = *reinterpret_cast<const float4*>(qv + d8 + 4);
-          d0 = fmaf(qa.x, ka[0], d0); d0 = fmaf(qa.y, ka[1], d0); d0 = fmaf(qa.z, ka[2], d0); d0 = fmaf(qa.w, ka[3], d0);
-          d0 = fmaf(qb.x, ka[4], d0); d0 = fmaf(qb.y, ka[5], d0); d0 = fmaf(qb.z, ka[6], d0); d0 = fmaf(qb.w, ka[7], d0);
-          d1 = fmaf(qa.x, kb[0], d1); d1 = fmaf(qa.y, kb[1], d1); d1 = fmaf(qa.z, kb[2], d1); d1 = fmaf(qa.w, kb[3], d1);
-          d1 = fmaf(qb.x, kb[4], d1); d1 = fmaf(qb.y, kb[5], d1); d1 = fmaf(qb.z, kb[6], d1); d1 = fmaf(qb.w, kb[7], d1);
+    // merge the four warps' states in warp order through `mrg` ([16][hd+4]: O, m, l)
+    for (int step = 0; step < 4; ++step) {
+      if (w == step) {
+        float* ra = mrg + (size_t)g * (hd + 4);
+        float* rb = mrg + (size_t)(g + 8) * (hd + 4);
+        float wa_buf = 0.f, wa_own = 1.f, wb_buf = 0.f, wb_own = 1.f, M_a = m_a, M_b = m_b;
+        if (step > 0) {
+          const float mb_a = ra[hd], mb_b = rb[hd];
+          M_a = fmaxf(mb_a, m_a); M_b = fmaxf(mb_b, m_b);
+          const float oa = M_a == -INFINITY ? 0.f : M_a, ob = M_b == -INFINITY ? 0.f : M_b;
+          wa_buf = expf(mb_a - oa); wa_own = expf(m_a - oa);
+          wb_buf = expf(mb_b - ob); wb_own = expf(m_b - ob);
+        } else {
+          if (m_a == -INFINITY) wa_own = 0.f;
+          if (m_b == -INFINITY) wb_own = 0.f;
         }
-        if (v0) s0 = d0;
-        if (v1) s1 = d1;
+        float nl_a = l_a * wa_own, nl_b = l_b * wb_own;
+        if (step > 0) { nl_a += ra[hd + 1] * wa_buf; nl_b += rb[hd + 1] * wb_buf; }
+        __syncwarp();
+#pragma unroll
+        for (int nd = 0; nd < 16; ++nd) {
+          if (nd < ntiles) {
+            const int col = nd * 8 + t4 * 2;
+            float2 va = make_float2(o[nd][0] * wa_own, o[nd][1] * wa_own);
+            float2 vb = make_float2(o[nd][2] * wb_own, o[nd][3] * wb_own);
+            if (step > 0) {
+              const float2 pa = *reinterpret_cast<const float2*>(ra + col), pb = *reinterpret_cast<const float2*>(rb + col);
+              va.x += pa.x * wa_buf; va.y += pa.y * wa_buf; vb.x += pb.x * wb_buf; vb.y += pb.y * wb_buf;
+            }
+            *reinterpret_cast<float2*>(ra + col) = va;
+            *reinterpret_cast<float2*>(rb + col) = vb;
+          }
+        }
+        __syncwarp();
+        if (t4 == 0) { ra[hd] = M_a; ra[hd + 1] = nl_a; rb[hd] = M_b; rb[hd + 1] = nl_b; }
       }
-      float* st = state + (size_t)ql * (hd + 2);
-      const float m_old = st[hd], l_old = st[hd + 1];
-      const float m_new = fmaxf(m_old, warp_max(fmaxf(s0, s1)));
-      if (m_new == -INFINITY) continue;            // nothing visible in this chunk (warp-uniform)
-      const float e0 = (s0 == -INFINITY) ? 0.f : expf(s0 - m_new), e1 = (s1 == -INFINITY) ? 0.f : expf(s1 - m_new);
-      const float corr = expf(m_old - m_new);
-      const float l_new = l_old * corr + warp_sum(e0 + e1);
-      // P.V: lane owns elements lane*? of head_dim in strides of 32 (pairs), up to 8 per lane
-      float acc[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) { const int dd = lane + 32 * i; acc[i] = dd < hd ? st[dd] * corr : 0.f; }
-      const int jmax = min(n_pos, last - p0 + 1);
-      for (int j = 0; j < jmax; ++j) {
-        const float pj = __shfl_sync(0xffffffffu, j < 32 ? e0 : e1, j & 31);
-        const bf16* vr = reinterpret_cast<const bf16*>(vs + (size_t)j * pitch);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { const int dd = lane + 32 * i; if (dd < hd) acc[i] = fmaf(pj, __bfloat162float(vr[dd]), acc[i]); }
-      }
-      __syncwarp();
-#pragma unroll
-      for (int i = 0; i < 8; ++i) { const int dd = lane + 32 * i; if (dd < hd) st[dd] = acc[i]; }
-      if (lane == 0) { st[hd] = m_new; st[hd + 1] = l_new; }
-      __syncwarp();
+      epi_bar_sync();
     }
-    epi_bar_sync();   // tile may be overwritten by the next chunk
-  }
-  if (!ok) return;
-  const int Hq = P.Hq;
-  if (a.n_ranges == 1) {
-    // the unit saw every visible position: normalise and write the attention output directly
-    for (int idx = et; idx < nQ * hd; idx += 128) {
-      const int ql = idx / hd, dd = idx % hd, q = q0 + ql;
-      const float* st = state + (size_t)ql * (hd + 2);
-      P.o[(size_t)(a.off + q / G) * Hq * hd + (size_t)(kvh * G + q % G) * hd + dd] = __float2bfloat16_rn(st[dd] / st[hd + 1]);
+    // write the block's 16 rows: final output, or state for the combine phase
+    const int rows = min(16, nQ - mt * 16);
+    if (a.n_ranges == 1) {
+      for (int idx = et; idx < rows * hd; idx += 128) {
+        const int row = idx / hd, dd = idx % hd, q = q0 + mt * 16 + row;
+        const float* st = mrg + (size_t)row * (hd + 4);
+        P.o[(size_t)(a.off + q / G) * P.Hq * hd + (size_t)(kvh * G + q % G) * hd + dd] = __float2bfloat16_rn(st[dd] / st[hd + 1]);
+      }
+    } else {
+      float* dst = P.attn_part + ((size_t)part_slot * ATT_QBLK + mt * 16) * (hd + 4);
+      for (int idx = et; idx < rows * (hd + 4); idx += 128) dst[idx] = mrg[idx];
     }
     epi_bar_sync();
-    return;
   }
-  // several units share the positions: park this unit's state; whichever unit of this
-  // (request, kv head, query block) arrives last merges all of them in position order
-  float* dst = P.attn_part + (size_t)part_slot * ATT_QBLK * (hd + 2);
-  for (int idx = et; idx < nQ * (hd + 2); idx += 128) dst[idx] = state[idx];
-  __threadfence();
-  epi_bar_sync();
-  if (et == 0) {
-    const int old = atomicAdd(P.attn_cnt + cnt_idx, 1);
-    ctl->last_flag = (old == a.n_ranges - 1) ? 1 : 0;
-    if (old == a.n_ranges - 1) P.attn_cnt[cnt_idx] = 0;
-  }
-  epi_bar_sync();
-  const bool last = ctl->last_flag != 0;
-  epi_bar_sync();
-  if (!last) return;
-  __threadfence();
-  for (int ql = w; ql < nQ; ql += 4) {
-    const int q = q0 + ql;
-    float M = -INFINITY;
-    for (int rg = 0; rg < a.n_ranges; ++rg)
-      M = fmaxf(M, __ldcg(P.attn_part + ((size_t)(first_slot + rg * a.n_qblk) * ATT_QBLK + ql) * (hd + 2) + hd));
-    float L = 0.f, acc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-    for (int rg = 0; rg < a.n_ranges; ++rg) {
-      const float* st = P.attn_part + ((size_t)(first_slot + rg * a.n_qblk) * ATT_QBLK + ql) * (hd + 2);
-      const float mu = __ldcg(st + hd);
-      if (mu == -INFINITY) continue;
-      const float wgt = expf(mu - M);
-      L += __ldcg(st + hd + 1) * wgt;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) { const int dd = lane + 32 * j; if (dd < hd) acc[j] += __ldcg(st + dd) * wgt; }
-    }
-    bf16* orow = P.o + (size_t)(a.off + q / G) * Hq * hd + (size_t)(kvh * G + q % G) * hd;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) { const int dd = lane + 32 * j; if (dd < hd) orow[dd] = __float2bfloat16_rn(acc[j] / L); }
-  }
-  epi_bar_sync();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -700,11 +766,54 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const int qblk = u % a.n_qblk, rest = u / a.n_qblk;
             const int range = rest % a.n_ranges, kvh = rest / a.n_ranges;
             const int slot = u0 + u;
-            const int first_slot = u0 + (kvh * a.n_ranges) * a.n_qblk + qblk;   // range 0 of this (kvh, qblk)
             if (slot < P.attn_part_units)
-              attn_unit(P, p, a, kvh, range, qblk, slot, first_slot, g0 + kvh * a.n_qblk + qblk, att_smem, ctl, att_parity, W, et, ok);
+              attn_unit(P, p, a, kvh, range, qblk, slot, att_smem, ctl, att_parity, W, et, ok);
           }
           u0 += a.units; g0 += P.Hkv * a.n_qblk;
+        }
+      } else if (p.kind == PH_COMBINE) {
+        // Requests whose positions were split over several units: merge the parked states of every
+        // (kv head, query) in position order.  One warp per item; each lane owns 4 consecutive
+        // elements of head_dim, so every partial is one 16-byte load per lane.
+        const int n_req = P.mode == CALL_VALIDATE ? P.n_req : 1;
+        const int hd = P.hd, Gq = P.Hq / P.Hkv;
+        int u0 = 0, item0 = 0;
+        for (int i = 0; i < n_req; ++i) {
+          const AttnReq a = attn_req(P, i, G);
+          if (a.n_ranges > 1) {
+            const int Q = a.R * Gq, items = P.Hkv * Q;
+            int it = ((cta * 4 + quad) - item0) % (G * 4);
+            if (it < 0) it += G * 4;
+            for (; it < items; it += G * 4) {
+              const int kvh = it / Q, q = it % Q, qblk = q / ATT_QBLK, ql = q % ATT_QBLK;
+              const int first_slot = u0 + (kvh * a.n_ranges) * a.n_qblk + qblk;
+              const size_t stride = (size_t)a.n_qblk * ATT_QBLK * (hd + 4);
+              const float* base = P.attn_part + ((size_t)first_slot * ATT_QBLK + ql) * (hd + 4);
+              float M = -INFINITY;
+              for (int rg = lane; rg < a.n_ranges; rg += 32) M = fmaxf(M, __ldcg(base + rg * stride + hd));
+              M = warp_max(M);
+              float L = 0.f;
+              float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+              const int dd = lane * 4;
+#pragma unroll 4
+              for (int rg = 0; rg < a.n_ranges; ++rg) {
+                const float* st = base + rg * stride;
+                const float mu = __ldcg(st + hd), lu = __ldcg(st + hd + 1);
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (dd < hd) v = __ldcg(reinterpret_cast<const float4*>(st + dd));
+                const float wgt = mu == -INFINITY ? 0.f : expf(mu - M);
+                L += lu * wgt;
+                acc.x += v.x * wgt; acc.y += v.y * wgt; acc.z += v.z * wgt; acc.w += v.w * wgt;
+              }
+              if (dd < hd) {
+                bf16* orow = P.o + (size_t)(a.off + q / Gq) * P.Hq * hd + (size_t)(kvh * Gq + q % Gq) * hd + dd;
+                const float inv = 1.0f / L;
+                *reinterpret_cast<uint2*>(orow) = make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
+              }
+            }
+            item0 += items;
+          }
+          u0 += a.units;
         }
       } else if (p.kind == PH_ACCEPT) {
         if (cta == 0) {
