@@ -243,3 +243,35 @@ def test_error_paths_return_codes_and_leave_the_context_usable():
     tt, al = eng.validate_host([1], [2], np.array([[7, 8, 0, 0]], np.int32))
     assert 0 <= int(al[0]) <= 2
     eng.close()
+
+
+@pytest.mark.parametrize("shape", [small_b(8, 2, 64), small_b(4, 4, 80, d=320, f=640), small_a()],
+                         ids=["gqa_hd64", "mha_hd80", "family_a"])
+def test_long_prefix_positions_split_over_several_units(shape):
+    # 333 cached positions span six 64-position chunks, so the softmax of every row is assembled
+    # from several units' partial states; pages of 32 tokens, ragged last page
+    st = _stairs()
+    shape = shape.replace(max_pos=512)
+    tsrc, dsrc = sources(shape)
+    tgt, _ = gu.oracle_pair(tsrc)
+    prompt = list(wl.zipf_tokens(334, shape.vocab, 77))
+    eng = st.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=400, k_max=8, kv_page_tokens=32, prefill_chunk=128)
+    eng.prefill(0, prompt)
+    k = 5
+    cont = so.greedy_generate(tgt, prompt, k + 1)
+    draft = wl.forced_draft(np.array(cont), 3, shape.vocab, 6)
+    d_dev = torch.zeros(8, dtype=torch.int32, device="cuda")
+    d_dev[:k] = torch.from_numpy(draft)
+    tt, al, logits = eng.validate([0], [k], d_dev, commit=False, want_logits=True)
+    eng.sync()
+    ref, _ = gu.oracle_stair_logits(tgt, prompt, draft)
+    gpu_tok = tt.cpu().numpy()[0]
+    gu.check_rows_against_oracle(logits.cpu().numpy(), gpu_tok, ref, gu.LOGIT_TOL_BF16)
+    assert int(al.cpu()[0]) == gu.first_mismatch(draft, gpu_tok)
+    # the per-launch tensor-core path (other attention kernel, explicit norms) agrees closely
+    eng2 = st.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=400, k_max=8, kv_page_tokens=32, prefill_chunk=128, gemm_impl=2)
+    eng2.prefill(0, prompt)
+    _, _, logits2 = eng2.validate([0], [k], d_dev, commit=False, want_logits=True)
+    eng2.sync()
+    assert float((logits2 - logits).abs().max()) < 0.03
+    eng.close(); eng2.close()
