@@ -166,6 +166,10 @@ def run_ours(args, rank, local_rank, world):
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
         dist.barrier()
     w, prefix, k = pick_workload(args.workload)
+    if args.layers > 0:
+        import dataclasses
+        w = dataclasses.replace(w, name=f"{w.name}_first{args.layers}layers", target=w.target.replace(n_layers=args.layers),
+                                draft_layers=min(w.draft_layers, args.layers))
     shape = w.target
     tsrc, dsrc = wl.make_sources(w, backend="torch-cuda")
     torch.cuda.set_device(local_rank)
@@ -331,6 +335,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--layers", type=int, default=0,
+                    help="use only the first N layers of the workload's target (small captures under a profiler)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--timed-only", action="store_true",
                     help="skip the end-to-end, generation and CPU legs (short runs under a profiler)")
