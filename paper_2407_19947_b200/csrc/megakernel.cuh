@@ -640,6 +640,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       uint32_t a_par = 0;
       unsigned int a_count = 0, b_count = 0, idle = 0;
       int ready_ph = -1;   // phases <= ready_ph have their inputs published
+      int traced_ph = -1;
       long long t_idle = clock64();
       while (B.valid) {
         bool progress = false;
@@ -663,6 +664,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           if (B.ph <= ready_ph) {
             uint8_t* b_dst = smem + (size_t)b_stage * stage_bytes + A_STAGE_BYTES;
             tma_load_2d(b_dst, P.maps + B.x_map, B.kk * BK, 0, ctl->full + b_stage, pol_x);
+            if (P.trace && cta == 0 && B.ph != traced_ph) { traced_ph = B.ph; P.trace[(size_t)B.ph * 8 + 7] = globaltimer_ns(); }
             ++b_count;
             if (++b_stage == stages) b_stage = 0;
             advance(B);
@@ -693,6 +695,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         if (remaining <= 0) continue;
         int kk = (int)(kr.begin % kblocks);
         bool seg_first = true;
+        unsigned long long* trm = (P.trace && cta == 0) ? P.trace + (size_t)ph * 8 : nullptr;
+        bool first_k = true;
         while (remaining > 0 && ok) {
           const bool seg_last = (remaining == 1) || (kk == kblocks - 1);
           if (seg_first) {
@@ -702,6 +706,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           }
           ok = W.wait(ctl->full + stage, phase);
           if (!ok) break;
+          if (trm && first_k) { trm[5] = globaltimer_ns(); first_k = false; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(smem + (size_t)stage * stage_bytes);
           const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + A_STAGE_BYTES);
@@ -717,6 +722,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           --remaining;
           if (++stage == stages) { stage = 0; phase ^= 1; }
         }
+        if (trm) trm[6] = globaltimer_ns();
       }
     }
   } else {
@@ -745,7 +751,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       }
 
       const bool tracing = P.trace && et == 0 && (cta == 0 || cta == G - 1);
-      unsigned long long* tr = tracing ? P.trace + ((size_t)(cta == 0 ? 0 : 1) * P.n_phases + ph) * 3 : nullptr;
+      unsigned long long* tr = tracing ? P.trace + ((size_t)(cta == 0 ? 0 : 1) * P.n_phases + ph) * 8 : nullptr;
       if (tracing) tr[0] = globaltimer_ns();
       if (p.kind == PH_EMBED) {
         if (cta == 0)
@@ -892,6 +898,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           epi_bar_sync();
         }
         const int tile_cols = BM;
+        if (tracing) tr[3] = globaltimer_ns();
+        bool first_seg = true;
         long long kb = kb_begin;
         while (kb < kb_end && ok) {
           const int tile = (int)(kb / p.kblocks), kk0 = (int)(kb % p.kblocks);
@@ -901,6 +909,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           W.wait(ctl->acc_full + buf, acc_phase[buf]);
           ok = group_ok(ctl, et);
           if (!ok) break;
+          if (tracing && first_seg) { tr[4] = globaltimer_ns(); first_seg = false; }
           acc_phase[buf] ^= 1;
           tc_fence_after();
           const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * P.t_box);
