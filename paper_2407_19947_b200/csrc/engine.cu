@@ -208,7 +208,7 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     L->prog_slot_d = (t.wdtype == 1 && has_draft) ? prog(d, &L->prog_maps_off_d) : 0;
     L->prog_t = take(L->prog_slot_t * MK_TBOX_SLOTS);
     L->prog_d = take(L->prog_slot_d * MK_TBOX_SLOTS);
-    L->mk_trace = take(t.wdtype == 1 ? (size_t)2 * (8 * std::max(t.n_layers, 1) + 4) * 8 * 8 : 0);
+    L->mk_trace = take(t.wdtype == 1 ? (size_t)(2 * 8 + TC_GRID_MAX) * (8 * std::max(t.n_layers, 1) + 4) * 8 : 0);
     L->stat_tiles = (t.d_model + tc::BM - 1) / tc::BM;
     L->mk_stats = take(t.wdtype == 1 ? (size_t)MK_MAX_ROWS * L->stat_tiles * 16 : 0);
     L->attn_cnt_n = c.max_requests * hkv * std::max(n_qblk, 1);
@@ -510,7 +510,8 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
   }
   simple(mk::PH_ACCEPT, -1, nullptr, nullptr, nullptr);
   for (const mk::Phase& p : ph)
-    if (p.kind == mk::PH_GEMM && p.n_tiles > TC_COUNTERS) return fail(ctx, STAIRS_EUNSUPPORTED, "too many tiles for the split bookkeeping");
+    if (p.kind == mk::PH_GEMM && (p.n_tiles > TC_COUNTERS || (long long)p.n_tiles * p.kblocks * TC_GRID_MAX >= (1ll << 32)))
+      return fail(ctx, STAIRS_EUNSUPPORTED, "too many tiles for the split bookkeeping");
   M.n_phases = (int)ph.size();
   char* base = M.prog_base + (size_t)slot * M.prog_slot_bytes;
   if (ph.size() * sizeof(mk::Phase) > M.prog_maps_off || M.prog_maps_off + maps.size() * sizeof(CUtensorMap) > M.prog_slot_bytes)

@@ -333,35 +333,13 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   const float scale = 1.0f / sqrtf((float)hd);
   const int half = hd / 2, ksteps = hd / 16, ntiles = hd / 8;
 
-  // queries of this block: query index q -> row r = q / G, head = kvh * G + q % G
-  for (int idx = et; idx < ATT_QBLK * half; idx += 128) {
-    const int ql = idx / half, i = idx % half, q = q0 + ql;
-    float x0 = 0.f, x1 = 0.f;
-    if (ql < nQ) {
-      const int r = q / G, head = kvh * G + (q % G);
-      const float* src = P.qkv + (size_t)(a.off + r) * nqkv + (size_t)head * hd;
-      x0 = src[i]; x1 = src[i + half];
-      if (P.rope) {
-        const float ang = (float)(a.base + r) * P.rope_inv[i];
-        float sn, cs;
-        sincosf(ang, &sn, &cs);
-        const float r0 = x0 * cs - x1 * sn, r1 = x1 * cs + x0 * sn;
-        x0 = r0; x1 = r1;
-      }
-    }
-    bf16* qd = reinterpret_cast<bf16*>(qs + (size_t)ql * pitch);
-    qd[i] = __float2bfloat16_rn(x0 * scale);
-    qd[i + half] = __float2bfloat16_rn(x1 * scale);
-  }
-  epi_bar_sync();
-
   const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
   const bool single_chunk = (c_end - c_begin == 1);
   const int n_mt = (nQ + 15) / 16;
 
   // stages chunk c: one bulk async copy per cached row (K and V); rows of new positions are
   // computed here (rotated k, v), patched into the tile and written to the cache
-  auto stage = [&](int c) {
+  auto stage_issue = [&](int c) {
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
     if (et == 0) {
@@ -409,10 +387,37 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
         }
       }
     }
+  };
+  auto stage_wait = [&]() {
     W.wait(&ctl->att_bar, att_parity);
     att_parity ^= 1;
     return group_ok(ctl, et);
   };
+
+  // the first chunk's copies fly while the queries are rotated
+  stage_issue(c_begin);
+  // queries of this block: query index q -> row r = q / G, head = kvh * G + q % G
+  for (int idx = et; idx < ATT_QBLK * half; idx += 128) {
+    const int ql = idx / half, i = idx % half, q = q0 + ql;
+    float x0 = 0.f, x1 = 0.f;
+    if (ql < nQ) {
+      const int r = q / G, head = kvh * G + (q % G);
+      const float* src = P.qkv + (size_t)(a.off + r) * nqkv + (size_t)head * hd;
+      x0 = src[i]; x1 = src[i + half];
+      if (P.rope) {
+        const float ang = (float)(a.base + r) * P.rope_inv[i];
+        float sn, cs;
+        sincosf(ang, &sn, &cs);
+        const float r0 = x0 * cs - x1 * sn, r1 = x1 * cs + x0 * sn;
+        x0 = r0; x1 = r1;
+      }
+    }
+    bf16* qd = reinterpret_cast<bf16*>(qs + (size_t)ql * pitch);
+    qd[i] = __float2bfloat16_rn(x0 * scale);
+    qd[i + half] = __float2bfloat16_rn(x1 * scale);
+  }
+  epi_bar_sync();
+
 
   for (int mt = 0; mt < n_mt && ok; ++mt) {
     // rows of this warp's fragments: ql_a = mt*16 + g, ql_b = ql_a + 8
@@ -426,7 +431,8 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
 
     for (int c = c_begin; c < c_end && ok; ++c) {
       if (!(single_chunk && mt > 0)) {
-        ok = stage(c);
+        if (!(mt == 0 && c == c_begin)) stage_issue(c);
+        ok = stage_wait();
         if (!ok) break;
       }
       const int p0 = c * ATT_CHUNK;
@@ -1016,7 +1022,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             }
           };
           if (whole) {
-            for (int c0 = 0; c0 < P.t_box; c0 += 16) {
+            for (int c0 = 0; c0 < Tvalid; c0 += 16) {
               float v[16];
               tmem_ld16(taddr + (uint32_t)c0, v);
               finish(c0, v);
@@ -1026,22 +1032,26 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           } else {
             const int slot = 2 * cta + (kb == kb_begin ? 0 : 1);
             float* mine = P.partial + (size_t)slot * P.t_box * BM;
-            for (int c0 = 0; c0 < P.t_box; c0 += 16) {
+            for (int c0 = 0; c0 < Tvalid; c0 += 16) {   // only rows that exist
               float v[16];
               tmem_ld16(taddr + (uint32_t)c0, v);
+              const int jn = min(16, Tvalid - c0);
 #pragma unroll
-              for (int j = 0; j < 16; ++j) mine[(size_t)(c0 + j) * BM + m] = v[j];
+              for (int j = 0; j < 16; ++j) if (j < jn) mine[(size_t)(c0 + j) * BM + m] = v[j];
             }
             tc_fence_before();
             if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
             __threadfence();
             epi_bar_sync();
-            int first_c = (int)((tile_first * Ge) / total);
-            while (range_begin(total, first_c + 1, Ge) <= tile_first) ++first_c;
-            while (first_c > 0 && range_begin(total, first_c, Ge) > tile_first) --first_c;
-            int last_c = first_c;
-            while (last_c + 1 < Ge && range_begin(total, last_c + 1, Ge) < tile_end) ++last_c;
-            const int nseg = last_c - first_c + 1;
+            // CTAs whose ranges touch this tile (32-bit arithmetic: total * Ge < 2^32, checked on the host)
+            const unsigned tot32 = (unsigned)total, ge32 = (unsigned)Ge, tf32 = (unsigned)tile_first, te32 = (unsigned)tile_end;
+            auto rb = [&](unsigned c) { return (tot32 * c) / ge32; };
+            unsigned first_c = (tf32 * ge32) / tot32;
+            while (rb(first_c + 1) <= tf32) ++first_c;
+            while (first_c > 0 && rb(first_c) > tf32) --first_c;
+            unsigned last_c = first_c;
+            while (last_c + 1 < ge32 && rb(last_c + 1) < te32) ++last_c;
+            const int nseg = (int)(last_c - first_c) + 1;
             if (et == 0) {
               const int old = atomicAdd(P.counters + tile, 1);
               ctl->last_flag = (old == nseg - 1) ? 1 : 0;
@@ -1052,16 +1062,28 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             epi_bar_sync();
             if (last) {
               __threadfence();
-              for (int c0 = 0; c0 < P.t_box; c0 += 16) {
+              for (int c0 = 0; c0 < Tvalid; c0 += 16) {
+                const int jn = min(16, Tvalid - c0);
                 float v[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j) v[j] = 0.f;
-                for (int c = first_c; c <= last_c; ++c) {
-                  const long long cb = range_begin(total, c, Ge);
-                  const int sl = 2 * c + (cb >= tile_first ? 0 : 1);
-                  const float* part = P.partial + (size_t)sl * P.t_box * BM;
+                // four segments' loads are issued together; the additions stay in k order
+                for (unsigned c = first_c; c <= last_c; c += 4) {
+                  float tmp[4][16];
 #pragma unroll
-                  for (int j = 0; j < 16; ++j) v[j] += __ldcg(part + (size_t)(c0 + j) * BM + m);
+                  for (int u = 0; u < 4; ++u) {
+                    const unsigned cc = c + u;
+                    const bool on = cc <= last_c;
+                    const int sl = 2 * (int)cc + (rb(cc) >= tf32 ? 0 : 1);
+                    const float* part = P.partial + (size_t)(on ? sl : 0) * P.t_box * BM;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) tmp[u][j] = (on && j < jn) ? __ldcg(part + (size_t)(c0 + j) * BM + m) : 0.f;
+                  }
+#pragma unroll
+                  for (int u = 0; u < 4; ++u) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] += tmp[u][j];
+                  }
                 }
                 finish(c0, v);
               }
@@ -1073,6 +1095,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       }
       if (!ok) break;
       if (tracing) tr[1] = globaltimer_ns();
+      // every CTA's completion time of the phase, after the two detailed traces
+      if (P.trace && et == 0) P.trace[(size_t)2 * P.n_phases * 8 + (size_t)cta * P.n_phases + ph] = globaltimer_ns();
       // Publish this CTA's part of the phase.  A CTA may arrive for phase ph only once every
       // CTA has arrived for phase ph-1: otherwise CTAs without work in two consecutive GEMM
       // phases would run ahead and their arrivals would be mistaken for the slower CTAs' ones
