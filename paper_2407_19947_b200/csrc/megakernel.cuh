@@ -101,7 +101,7 @@ struct AttnSmem {   // carved after the GEMM ring: Q block (bf16), K and V chunk
   static __host__ __device__ size_t q_bytes(int hd) { return (size_t)ATT_QBLK * k_pitch(hd); }
   static __host__ __device__ size_t kv_bytes(int hd) { return (size_t)ATT_CHUNK * k_pitch(hd); }
   static __host__ __device__ size_t merge_bytes(int hd) { return (size_t)16 * (hd + 4) * 4 + 64; }
-  static __host__ __device__ size_t bytes(int hd) { return q_bytes(hd) + 2 * kv_bytes(hd) + merge_bytes(hd) + 64; }
+  static __host__ __device__ size_t bytes(int hd) { return q_bytes(hd) + 2 * kv_bytes(hd) + 64; }
 };
 
 // mma.sync m16n8k16 (bf16 in, fp32 accumulate) and its operand loads, for the attention tiles
@@ -326,7 +326,6 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   uint8_t* qs = att_smem;                                   // [QBLK][pitch] bf16, rotated and pre-scaled
   uint8_t* ks = qs + AttnSmem::q_bytes(hd);                 // [CHUNK][pitch]
   uint8_t* vs = ks + AttnSmem::kv_bytes(hd);
-  float* mrg = reinterpret_cast<float*>(vs + AttnSmem::kv_bytes(hd));   // [16][hd + 4]
   bf16* kc = reinterpret_cast<bf16*>(ph.kc);
   bf16* vc = reinterpret_cast<bf16*>(ph.vc);
   const int* pt = P.page_table + (size_t)a.slot * P.max_pages;
@@ -334,7 +333,6 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   const int half = hd / 2, ksteps = hd / 16, ntiles = hd / 8;
 
   const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
-  const bool single_chunk = (c_end - c_begin == 1);
   const int n_mt = (nQ + 15) / 16;
 
   // stages chunk c: one bulk async copy per cached row (K and V); rows of new positions are
@@ -419,26 +417,26 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   epi_bar_sync();
 
 
-  for (int mt = 0; mt < n_mt && ok; ++mt) {
-    // rows of this warp's fragments: ql_a = mt*16 + g, ql_b = ql_a + 8
-    const int ql_a = mt * 16 + g, ql_b = ql_a + 8;
-    const int last_a = ql_a < nQ ? a.base + (q0 + ql_a) / G : -1;   // last visible position
-    const int last_b = ql_b < nQ ? a.base + (q0 + ql_b) / G : -1;
-    float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
-    float o[16][4];
+  // Warp w owns query block (MMA M tile) w of the unit and walks the chunk's four 16-position
+  // slices itself, so its softmax state and output accumulators never leave its registers.
+  const int mt = w;
+  const bool active = mt < n_mt;
+  const int ql_a = mt * 16 + g, ql_b = ql_a + 8;
+  const int last_a = (active && ql_a < nQ) ? a.base + (q0 + ql_a) / G : -1;   // last visible position
+  const int last_b = (active && ql_b < nQ) ? a.base + (q0 + ql_b) / G : -1;
+  float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
+  float o[16][4];
 #pragma unroll
-    for (int nd = 0; nd < 16; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
+  for (int nd = 0; nd < 16; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
 
-    for (int c = c_begin; c < c_end && ok; ++c) {
-      if (!(single_chunk && mt > 0)) {
-        if (!(mt == 0 && c == c_begin)) stage_issue(c);
-        ok = stage_wait();
-        if (!ok) break;
-      }
-      const int p0 = c * ATT_CHUNK;
-      const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
-      const int sl0 = w * 16;                       // this warp's positions: p0 + sl0 .. + 15
-      if (sl0 < n_pos) {
+  for (int c = c_begin; c < c_end && ok; ++c) {
+    if (c != c_begin) stage_issue(c);
+    ok = stage_wait();
+    if (!ok) break;
+    const int p0 = c * ATT_CHUNK;
+    const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
+    if (active) {
+      for (int sl0 = 0; sl0 < n_pos; sl0 += 16) {
         float sc[2][4];
 #pragma unroll
         for (int j = 0; j < 2; ++j) { sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f; }
@@ -503,61 +501,41 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
           }
         }
       }
-      if (!(single_chunk) || mt == n_mt - 1) epi_bar_sync();   // tile may be overwritten next
     }
-    if (!ok) break;
+    epi_bar_sync();   // tile may be overwritten by the next chunk or unit
+  }
+  if (!ok || !active) return;
 
-    // merge the four warps' states in warp order through `mrg` ([16][hd+4]: O, m, l)
-    for (int step = 0; step < 4; ++step) {
-      if (w == step) {
-        float* ra = mrg + (size_t)g * (hd + 4);
-        float* rb = mrg + (size_t)(g + 8) * (hd + 4);
-        float wa_buf = 0.f, wa_own = 1.f, wb_buf = 0.f, wb_own = 1.f, M_a = m_a, M_b = m_b;
-        if (step > 0) {
-          const float mb_a = ra[hd], mb_b = rb[hd];
-          M_a = fmaxf(mb_a, m_a); M_b = fmaxf(mb_b, m_b);
-          const float oa = M_a == -INFINITY ? 0.f : M_a, ob = M_b == -INFINITY ? 0.f : M_b;
-          wa_buf = expf(mb_a - oa); wa_own = expf(m_a - oa);
-          wb_buf = expf(mb_b - ob); wb_own = expf(m_b - ob);
-        } else {
-          if (m_a == -INFINITY) wa_own = 0.f;
-          if (m_b == -INFINITY) wb_own = 0.f;
-        }
-        float nl_a = l_a * wa_own, nl_b = l_b * wb_own;
-        if (step > 0) { nl_a += ra[hd + 1] * wa_buf; nl_b += rb[hd + 1] * wb_buf; }
-        __syncwarp();
+  // write this warp's 16 rows straight from the accumulator fragments: the final output when the
+  // unit saw every visible position, else the state (O, max, sum) for the combine phase
+  if (a.n_ranges == 1) {
+    const float ia = l_a > 0.f ? 1.0f / l_a : 0.f, ib = l_b > 0.f ? 1.0f / l_b : 0.f;
 #pragma unroll
-        for (int nd = 0; nd < 16; ++nd) {
-          if (nd < ntiles) {
-            const int col = nd * 8 + t4 * 2;
-            float2 va = make_float2(o[nd][0] * wa_own, o[nd][1] * wa_own);
-            float2 vb = make_float2(o[nd][2] * wb_own, o[nd][3] * wb_own);
-            if (step > 0) {
-              const float2 pa = *reinterpret_cast<const float2*>(ra + col), pb = *reinterpret_cast<const float2*>(rb + col);
-              va.x += pa.x * wa_buf; va.y += pa.y * wa_buf; vb.x += pb.x * wb_buf; vb.y += pb.y * wb_buf;
-            }
-            *reinterpret_cast<float2*>(ra + col) = va;
-            *reinterpret_cast<float2*>(rb + col) = vb;
-          }
-        }
-        __syncwarp();
-        if (t4 == 0) { ra[hd] = M_a; ra[hd + 1] = nl_a; rb[hd] = M_b; rb[hd + 1] = nl_b; }
+    for (int half_row = 0; half_row < 2; ++half_row) {
+      const int ql = half_row ? ql_b : ql_a;
+      if (ql < nQ) {
+        const int q = q0 + ql;
+        bf16* orow = P.o + (size_t)(a.off + q / G) * P.Hq * hd + (size_t)(kvh * G + q % G) * hd;
+        const float inv = half_row ? ib : ia;
+#pragma unroll
+        for (int nd = 0; nd < 16; ++nd)
+          if (nd < ntiles)
+            *reinterpret_cast<uint32_t*>(orow + nd * 8 + t4 * 2) = pack_bf16x2(o[nd][2 * half_row] * inv, o[nd][2 * half_row + 1] * inv);
       }
-      epi_bar_sync();
     }
-    // write the block's 16 rows: final output, or state for the combine phase
-    const int rows = min(16, nQ - mt * 16);
-    if (a.n_ranges == 1) {
-      for (int idx = et; idx < rows * hd; idx += 128) {
-        const int row = idx / hd, dd = idx % hd, q = q0 + mt * 16 + row;
-        const float* st = mrg + (size_t)row * (hd + 4);
-        P.o[(size_t)(a.off + q / G) * P.Hq * hd + (size_t)(kvh * G + q % G) * hd + dd] = __float2bfloat16_rn(st[dd] / st[hd + 1]);
+  } else {
+#pragma unroll
+    for (int half_row = 0; half_row < 2; ++half_row) {
+      const int ql = half_row ? ql_b : ql_a;
+      if (ql < nQ) {
+        float* dst = P.attn_part + ((size_t)part_slot * ATT_QBLK + ql) * (hd + 4);
+#pragma unroll
+        for (int nd = 0; nd < 16; ++nd)
+          if (nd < ntiles)
+            *reinterpret_cast<float2*>(dst + nd * 8 + t4 * 2) = make_float2(o[nd][2 * half_row], o[nd][2 * half_row + 1]);
+        if (t4 == 0) { dst[hd] = half_row ? m_b : m_a; dst[hd + 1] = half_row ? l_b : l_a; }
       }
-    } else {
-      float* dst = P.attn_part + ((size_t)part_slot * ATT_QBLK + mt * 16) * (hd + 4);
-      for (int idx = et; idx < rows * (hd + 4); idx += 128) dst[idx] = mrg[idx];
     }
-    epi_bar_sync();
   }
 }
 
@@ -928,6 +906,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const int src_n = (s + 1 < p.n_src ? p.src_col[s + 1] : p.N) - p.src_col[s];
             n_out = p.src_col[s] + in_src; n_valid = in_src < src_n;
           }
+          // old residual values and gain of the first 16 rows, fetched early on the split-tile path
+          // (before the arrival counter is known) so that the last arriver's chain is shorter
+          float xpre[16], gpre = 0.f;
+          bool have_pre = false;
           auto finish = [&](int c0, float* v) {
             if (p.norm_in) {
               // fold the normalisation in: y = rstd_t * (acc - mean_t * u[n]) + c[n]
@@ -974,32 +956,43 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             if (p.epi == TC_ADD_F32 && p.next_g) {
               // residual update; also the next GEMM's operand bf16(x * gain) and this tile's row
               // statistics (mean and centred sum of squares over the tile's columns)
-              const float gn = n_valid ? p.next_g[n_out] : 0.f;
+              const bool use_pre = have_pre && c0 == 0;
+              const float gn = use_pre ? gpre : (n_valid ? p.next_g[n_out] : 0.f);
               const int jn = min(16, Tvalid - c0);   // rows of this chunk that exist (uniform)
+              // all loads of the old residual values first (predicated, no early exit, so that
+              // they are in flight together), then the updates
+              float xo[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                xo[j] = use_pre ? xpre[j] : ((n_valid && j < jn) ? __ldcg(out_f32 + (size_t)(c0 + j) * p.ldo + n_out) : 0.f);
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
-                if (j >= jn) break;
-                const int t = c0 + j;
                 float xn = 0.f;
-                if (n_valid && t < Tvalid) {
-                  const size_t o = (size_t)t * p.ldo + n_out;
-                  xn = out_f32[o] + v[j];
+                if (n_valid && j < jn) {
+                  const size_t o = (size_t)(c0 + j) * p.ldo + n_out;
+                  xn = xo[j] + v[j];
                   out_f32[o] = xn;
                   P.h[o] = __float2bfloat16_rn(xn * gn);
                 }
                 v[j] = xn;
-                const float s1 = warp_sum(xn);
-                if (lane == 0) ctl->red[quad][j] = s1;
+              }
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                if (j < jn) {
+                  const float s1 = warp_sum(v[j]);
+                  if (lane == 0) ctl->red[quad][j] = s1;
+                }
               }
               epi_bar_sync();
               const int cnt = min(tile_cols, p.N - tile * BM);
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
-                if (j >= jn) break;
-                const float mean = (ctl->red[0][j] + ctl->red[1][j] + ctl->red[2][j] + ctl->red[3][j]) / (float)cnt;
-                const float dl = n_valid ? v[j] - mean : 0.f;
-                const float s2 = warp_sum(dl * dl);
-                if (lane == 0) ctl->red2[quad][j] = s2;
+                if (j < jn) {
+                  const float mean = (ctl->red[0][j] + ctl->red[1][j] + ctl->red[2][j] + ctl->red[3][j]) / (float)cnt;
+                  const float dl = n_valid ? v[j] - mean : 0.f;
+                  const float s2 = warp_sum(dl * dl);
+                  if (lane == 0) ctl->red2[quad][j] = s2;
+                }
               }
               epi_bar_sync();
               if (et < 16 && c0 + et < Tvalid) {
@@ -1011,14 +1004,23 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               return;
             }
             if (!n_valid) return;
+            if (p.epi == TC_ADD_F32) {
+              float xo[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                xo[j] = (have_pre && c0 == 0) ? xpre[j] : ((c0 + j < Tvalid) ? __ldcg(out_f32 + (size_t)(c0 + j) * p.ldo + n_out) : 0.f);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) if (c0 + j < Tvalid) out_f32[(size_t)(c0 + j) * p.ldo + n_out] = xo[j] + v[j];
+              return;
+            }
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               const int t = c0 + j;
-              if (t >= Tvalid) break;
-              const size_t o = (size_t)t * p.ldo + n_out;
-              if (p.epi == TC_STORE_F32) out_f32[o] = v[j];
-              else if (p.epi == TC_ADD_F32) out_f32[o] += v[j];
-              else out_act[o] = __float2bfloat16_rn(gelu_erf(v[j]));
+              if (t < Tvalid) {
+                const size_t o = (size_t)t * p.ldo + n_out;
+                if (p.epi == TC_STORE_F32) out_f32[o] = v[j];
+                else out_act[o] = __float2bfloat16_rn(gelu_erf(v[j]));
+              }
             }
           };
           if (whole) {
@@ -1041,6 +1043,12 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             }
             tc_fence_before();
             if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
+            if (p.epi == TC_ADD_F32) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) xpre[j] = (n_valid && j < Tvalid) ? __ldcg(out_f32 + (size_t)j * p.ldo + n_out) : 0.f;
+              gpre = (p.next_g && n_valid) ? p.next_g[n_out] : 0.f;
+              have_pre = true;
+            }
             __threadfence();
             epi_bar_sync();
             // CTAs whose ranges touch this tile (32-bit arithmetic: total * Ge < 2^32, checked on the host)
@@ -1060,7 +1068,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             epi_bar_sync();
             const bool last = ctl->last_flag != 0;
             epi_bar_sync();
+            unsigned long long* tra = (P.trace && et == 0) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 4 : nullptr;
             if (last) {
+              if (tra) tra[1] = globaltimer_ns();
               __threadfence();
               for (int c0 = 0; c0 < Tvalid; c0 += 16) {
                 const int jn = min(16, Tvalid - c0);
@@ -1085,8 +1095,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                     for (int j = 0; j < 16; ++j) v[j] += tmp[u][j];
                   }
                 }
+                if (tra) tra[2] = globaltimer_ns();
                 finish(c0, v);
               }
+              if (tra) tra[3] = globaltimer_ns();
             }
           }
           buf ^= 1;
@@ -1096,7 +1108,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       if (!ok) break;
       if (tracing) tr[1] = globaltimer_ns();
       // every CTA's completion time of the phase, after the two detailed traces
-      if (P.trace && et == 0) P.trace[(size_t)2 * P.n_phases * 8 + (size_t)cta * P.n_phases + ph] = globaltimer_ns();
+      if (P.trace && et == 0) P.trace[(size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 4] = globaltimer_ns();
       // Publish this CTA's part of the phase.  A CTA may arrive for phase ph only once every
       // CTA has arrived for phase ph-1: otherwise CTAs without work in two consecutive GEMM
       // phases would run ahead and their arrivals would be mistaken for the slower CTAs' ones
