@@ -1,6 +1,7 @@
 // Host engine and C-ABI of the stairs library: context, workspace layout, KV page
 // allocator, the per-pass kernel sequence, draft / validate / generate.
 #include <algorithm>
+#include <cmath>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -454,6 +455,22 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
       p.N = col;
     }
     p.n_tiles = tiles; p.epi = epi; p.out = out; p.ldo = ldo;
+    {
+      // How many CTAs to cut this GEMM over: more CTAs stream faster, but every tile is then
+      // finished from more partial tiles, which the finisher reads four at a time.  Model:
+      // stream time at ~44 GB/s per SM plus ~1.6 us per batch of four partials.
+      const int grid = std::min(ctx->sm_count, TC_GRID_MAX);
+      const double bytes = (double)tiles * p.kblocks * tc::A_STAGE_BYTES;
+      double best = 1e30; int best_ge = grid;
+      for (int s2 = 1; s2 <= 64; s2 *= 2) {
+        const int ge = std::min(grid, tiles * s2);
+        const double seg = (double)ge / tiles + (ge % tiles ? 1.0 : 0.0);
+        const double t_us = bytes / (ge * 44.0e3) + (seg > 1.0 ? std::ceil(seg / 4.0) * 1.6 + 2.0 : 0.0);
+        if (t_us < best - 1e-9) { best = t_us; best_ge = ge; }
+        if (ge == grid) break;
+      }
+      p.ge_max = best_ge;
+    }
     ph.push_back(p);
     return ph.back();
   };

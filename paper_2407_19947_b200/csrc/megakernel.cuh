@@ -49,6 +49,7 @@ struct Phase {
   // the epilogue applies y = rstd_t * (acc - mean_t * u[n]) + c[n] with u = W.gain, c = W.bias
   // (LayerNorm; both NULL for RMSNorm, where y = rstd_t * acc).  next_g: this residual GEMM's
   // finisher also writes bf16(x * next_g) for the following GEMM and per-tile row statistics.
+  int ge_max;                // CTAs this GEMM is cut over (0 = all): few tiles are not worth a wide split
   int norm_in;
   const float* u; const float* c;
   const float* next_g;
@@ -153,8 +154,9 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
 // k-block range of this CTA in a GEMM phase: the phase is cut over min(G, total) CTAs so that no
 // participating range is empty (the split-tile bookkeeping counts one segment per CTA touching a tile).
 struct KRange { long long begin, end; int ge; };
-__device__ __forceinline__ KRange phase_range(long long total, int cta, int G) {
+__device__ __forceinline__ KRange phase_range(long long total, int cta, int G, int ge_max) {
   KRange r;
+  if (ge_max > 0 && ge_max < G) G = ge_max;
   r.ge = (int)(total < (long long)G ? total : (long long)G);
   if (cta >= r.ge) { r.begin = r.end = 0; return r; }
   r.begin = range_begin(total, cta, r.ge); r.end = range_begin(total, cta + 1, r.ge);
@@ -601,7 +603,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         for (int ph = from; ph < P.n_phases; ++ph) {
           const Phase& p = P.phases[ph];
           if (p.kind != PH_GEMM) continue;
-          const KRange kr = phase_range((long long)p.n_tiles * p.kblocks, cta, G);
+          const KRange kr = phase_range((long long)p.n_tiles * p.kblocks, cta, G, p.ge_max);
           if (kr.begin >= kr.end) continue;
           c.ph = ph; c.kblocks = p.kblocks; c.dual = p.dual; c.n_src = p.n_src; c.x_map = p.x_map;
 #pragma unroll
@@ -674,7 +676,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         const Phase& p = P.phases[ph];
         if (p.kind != PH_GEMM) continue;
         const int kblocks = p.kblocks;
-        const KRange kr = phase_range((long long)p.n_tiles * kblocks, cta, G);
+        const KRange kr = phase_range((long long)p.n_tiles * kblocks, cta, G, p.ge_max);
         int remaining = (int)(kr.end - kr.begin);
         if (remaining <= 0) continue;
         int kk = (int)(kr.begin % kblocks);
@@ -833,7 +835,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       } else {
         // ---------------------------------------------------------------- GEMM epilogue
         const long long total = (long long)p.n_tiles * p.kblocks;
-        const KRange kr = phase_range(total, cta, G);
+        const KRange kr = phase_range(total, cta, G, p.ge_max);
         const long long kb_begin = kr.begin, kb_end = kr.end;
         const int Ge = kr.ge;
         const int Tvalid = P.T;
