@@ -115,6 +115,59 @@ def cpu_threads() -> int:
     return os.cpu_count() or 1
 
 
+def max_over_ranks(values, world, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (the job's time is its slowest rank's)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def kernel_source_hash() -> str:
+    """Hash of the kernel sources; a stored DRAM-traffic figure is only quoted while it matches."""
+    import hashlib
+    h = hashlib.sha1()
+    d = os.path.join(ROOT, "paper_2407_19947_b200", "csrc")
+    for f in sorted(os.listdir(d)):
+        with open(os.path.join(d, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def stored_traffic(workload_name: str):
+    """dram bytes per launch from the committed ncu capture of this workload, or None when the
+    kernels changed since it was taken."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(p):
+        return None
+    with open(p) as f:
+        t = json.load(f)
+    e = t.get(workload_name)
+    if not e or e.get("kernel_source_hash") != kernel_source_hash():
+        return None
+    return e.get("dram_bytes_per_launch")
+
+
+def time_validate(eng, torch, k, drafts_dev, steps, warmup):
+    """us per stairs_validate call (commit=0) with CUDA events on the engine's stream."""
+    tt = torch.zeros((1, eng.k_max + 1), dtype=torch.int32, device=eng.device)
+    al = torch.zeros((1,), dtype=torch.int32, device=eng.device)
+    n = drafts_dev.shape[0]
+    for i in range(warmup):
+        eng.validate([0], [k], drafts_dev[i % n], commit=False, out=(tt, al))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(eng.stream)
+    for i in range(steps):
+        eng.validate([0], [k], drafts_dev[i % n], commit=False, out=(tt, al))
+    e1.record(eng.stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / steps
+
+
 def run_reference(args, rank, world):
     """The oracle timed on the host cores.  Each step is one stair row (an independent no-cache
     fp32 forward) at a prefix shortened so that the whole run stays within a few minutes; the
@@ -245,13 +298,7 @@ def run_ours(args, rank, local_rank, world):
         eng.validate_host([0], [k], pin_d[i % len(a_list)].numpy()[None])
     e2e_s = time.perf_counter() - t0
 
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms, e2e_s * 1e3], device=eng.device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
-    else:
-        e2e_ms = e2e_s * 1e3
+    ms, e2e_ms = max_over_ranks([ms, e2e_s * 1e3], world, eng.device)
     if rank != 0:
         return
     total_calls = args.steps * world
@@ -287,7 +334,7 @@ def run_ours(args, rank, local_rank, world):
                      "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak if achieved else None,
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS if achieved else None,
-                     "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "peak_kind": f"of {peak_kind}", "traffic": stored_traffic(w.name) if gemm_n == 0 else None,
                      "launches_per_call": gemm_n / max(args.steps, 1),
                      "timing": roof_timing},
         "call": {"algorithmic_bytes": abytes, "hbm_gbs_whole_call": abytes / (us_per_call * 1e-6) / 1e9,
@@ -312,6 +359,56 @@ def run_ours(args, rank, local_rank, world):
                                                / line["generation"]["greedy_tokens_per_s"])
     except Exception as ex:  # reported, never hidden
         line["generation"] = {"error": str(ex)}
+    # the other points of the validation microbench (prefix x k), and the 7B-shaped target
+    if world == 1 and not args.timed_only and not args.no_extras:
+        try:
+            if args.workload == "cfg2" and args.layers == 0:
+                grid = {}
+                rng = np.random.default_rng(5)
+                for pfx in (128, 512, 2048):
+                    eng.prefill(0, prompt[: pfx + 1])
+                    for kk in (2, 4, 8):
+                        dd = torch.from_numpy(rng.integers(0, shape.vocab, size=(16, k)).astype(np.int32)).to(eng.device)
+                        us = time_validate(eng, torch, kk, dd, 100, 5)
+                        ab = algorithmic_bytes(shape, pfx, kk)
+                        grid[f"P{pfx}_k{kk}"] = {"us_per_call": us, "frac_of_measured_peak": ab / (us * 1e-6) / 1e9 / peak}
+                line["validate_grid"] = grid
+        except Exception as ex:
+            line["validate_grid"] = {"error": str(ex)}
+        try:
+            if args.workload == "cfg2" and args.layers == 0:
+                eng.close()
+                eng = None
+                del d_dev
+                tsrc.drop_cache()
+                torch.cuda.empty_cache()
+                w7, p7, k7 = pick_workload("cfg4")
+                t7, d7 = wl.make_sources(w7, backend="torch-cuda")
+                e7 = stairs.Stairs(t7, d7, max_requests=1, max_seq_len=p7 + 256, k_max=k7, kv_page_tokens=64,
+                                   device_index=local_rank)
+                e7.prefill(0, wl.prompt_tokens(w7, n=p7 + 1))
+                rng = np.random.default_rng(6)
+                per_k = {}
+                for kk in (0, 1, 2, 4, 8):
+                    dd = torch.from_numpy(rng.integers(0, w7.target.vocab, size=(16, k7)).astype(np.int32)).to(e7.device)
+                    us = time_validate(e7, torch, kk, dd, 30, 3)
+                    ab = algorithmic_bytes(w7.target, p7, kk)
+                    per_k[f"k{kk}"] = {"us_per_call": us, "hbm_gbs": ab / (us * 1e-6) / 1e9,
+                                       "frac_of_measured_peak": ab / (us * 1e-6) / 1e9 / peak,
+                                       "frac_of_nominal_8TBs": ab / (us * 1e-6) / 1e9 / NOMINAL_HBM_GBS}
+                g0, s0 = e7.generate(0, wl.prompt_tokens(w7, n=p7), 0, 32)
+                g4, s4 = e7.generate(0, wl.prompt_tokens(w7, n=p7), 4, 32)
+                line["target_7b"] = {"workload": f"{w7.name}: prefix {p7}", "validate": per_k,
+                                     "greedy_tokens_per_s": 32 / ((s0["total_ms"] - s0["prefill_ms"]) * 1e-3),
+                                     "stairs_k4_tokens_per_s": 32 / ((s4["total_ms"] - s4["prefill_ms"]) * 1e-3),
+                                     "acceptance_k4": s4["accepted"] / max(s4["drafted"], 1),
+                                     "identical_output": g0 == g4}
+                e7.close()
+                e7 = None
+                t7.drop_cache(); d7.drop_cache()
+                torch.cuda.empty_cache()
+        except Exception as ex:
+            line["target_7b"] = {"error": str(ex)}
     # the oracle beside it, on this host's cores, on a bounded sample
     if world == 1 and not args.no_cpu_baseline and not args.timed_only:
         cb_prefix = min(prefix, args.cpu_prefix)
@@ -325,7 +422,8 @@ def run_ours(args, rank, local_rank, world):
                                 "sample": f"{n_rows} of the {k + 1} stair rows at prefix {cb_prefix} "
                                           f"(no-cache fp32 forwards), scaled to {k + 1} rows"}
     print(json.dumps(line))
-    eng.close()
+    if eng is not None:
+        eng.close()
 
 
 def main():
@@ -338,6 +436,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0,
                     help="use only the first N layers of the workload's target (small captures under a profiler)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the (prefix, k) grid and the 7B-shaped target")
     ap.add_argument("--timed-only", action="store_true",
                     help="skip the end-to-end, generation and CPU legs (short runs under a profiler)")
     ap.add_argument("--cpu-prefix", type=int, default=2048, help="prefix length of the CPU-baseline sample")
