@@ -181,11 +181,12 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
   L->val_off = take((size_t)c.max_requests * 4);
   L->keys = take(R * 8);
   L->x = take(R * dm * 4);
-  L->h = take(R * dm * es);
+  const size_t parts = t.wdtype == 1 ? 2 : 1;   // bf16 GEMM operands are stored as hi + lo parts
+  L->h = take(parts * R * dm * es);
   L->qkv = take(R * nqkv * 4);
   L->q = take(R * nq * es);
-  L->o = take(R * nq * es);
-  L->ff = take(R * ff * es);
+  L->o = take(parts * R * nq * es);
+  L->ff = take(parts * R * ff * es);
   L->logits = take((size_t)L->logit_rows * t.vocab * 4);
   L->draft_buf = take((size_t)c.max_requests * std::max(c.k_max, 1) * 4);
   L->tt_buf = take((size_t)c.max_requests * (c.k_max + 1) * 4);
@@ -434,9 +435,9 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
   }
   const int i_head = 7 * m.n_layers, i_h = i_head + 1, i_o = i_head + 2, i_ff = i_head + 3;
   maps[i_head] = M.head_map;
-  bool ok = encode_map(ctx, &maps[i_h], ws + L.h, L.max_rows, d, t_box) &&
-            encode_map(ctx, &maps[i_o], ws + L.o, L.max_rows, nq, t_box) &&
-            encode_map(ctx, &maps[i_ff], ws + L.ff, L.max_rows, F, t_box);
+  bool ok = encode_map(ctx, &maps[i_h], ws + L.h, 2 * L.max_rows, d, t_box) &&
+            encode_map(ctx, &maps[i_o], ws + L.o, 2 * L.max_rows, nq, t_box) &&
+            encode_map(ctx, &maps[i_ff], ws + L.ff, 2 * L.max_rows, F, t_box);
   if (!ok) return fail(ctx, STAIRS_ECUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
   std::vector<mk::Phase> ph;
   auto gemm = [&](int layer, int w0, int w1, int w2, int n_src, const int* rows, bool dual, int xmap, int K, int epi, void* out, int ldo) -> mk::Phase& {
@@ -580,6 +581,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.page_table = reinterpret_cast<int*>(ws + L.page_table); P.page_tokens = ctx->cfg.kv_page_tokens; P.max_pages = L.max_pages;
   P.x = reinterpret_cast<float*>(ws + L.x); P.h = reinterpret_cast<bf16*>(ws + L.h); P.qkv = reinterpret_cast<float*>(ws + L.qkv);
   P.o = reinterpret_cast<bf16*>(ws + L.o); P.ff = reinterpret_cast<bf16*>(ws + L.ff);
+  P.lo_row = L.max_rows;
   P.keys = reinterpret_cast<unsigned long long*>(ws + L.keys); P.n_keys = L.max_rows;
   P.logits = c.logits;
   P.target_tokens = c.target_tokens; P.accept_len = c.accept_len; P.commit = c.commit; P.draft_out = c.draft_out;

@@ -77,6 +77,7 @@ struct Params {
   int* tok; int* pos; int* req;
   const int* page_table; int page_tokens, max_pages;
   float* x; bf16* h; float* qkv; bf16* o; bf16* ff;
+  int lo_row;               // GEMM operands are stored as bf16 hi + bf16 lo; the lo part sits lo_row rows further down
   unsigned long long* keys; int n_keys;
   float4* stats;            // [64 rows][stat_tiles] (mean, M2, count, -) per 128-column tile of x
   int stat_tiles;
@@ -161,6 +162,14 @@ __device__ __forceinline__ KRange phase_range(long long total, int cta, int G, i
   if (cta >= r.ge) { r.begin = r.end = 0; return r; }
   r.begin = range_begin(total, cta, r.ge); r.end = range_begin(total, cta + 1, r.ge);
   return r;
+}
+
+// GEMM activation operands keep ~16 mantissa bits: value = hi + lo with hi = bf16(value) and
+// lo = bf16(value - hi); the MMAs run once on each part into the same accumulator.
+__device__ __forceinline__ void store_split(bf16* base, size_t idx, size_t lo_off, float v) {
+  const bf16 hi = __float2bfloat16_rn(v);
+  base[idx] = hi;
+  base[idx + lo_off] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
 // Shared per-CTA control block.
@@ -269,7 +278,7 @@ __device__ void embed_row(const Params& P, int t, const RowInfo& r, const float*
       v = __bfloat162float(e[col]);
       if (pe) v += __bfloat162float(pe[col]);
       xr[col] = v;
-      hr[col] = __float2bfloat16_rn(v * g[col]);
+      store_split(hr, col, (size_t)P.lo_row * d, v * g[col]);
     }
     xv[i] = v; s1 += v;
   }
@@ -522,7 +531,13 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
 #pragma unroll
         for (int nd = 0; nd < 16; ++nd)
           if (nd < ntiles)
-            *reinterpret_cast<uint32_t*>(orow + nd * 8 + t4 * 2) = pack_bf16x2(o[nd][2 * half_row] * inv, o[nd][2 * half_row + 1] * inv);
+          {
+            const float v0 = o[nd][2 * half_row] * inv, v1 = o[nd][2 * half_row + 1] * inv;
+            const __nv_bfloat162 hi2 = __floats2bfloat162_rn(v0, v1);
+            *reinterpret_cast<__nv_bfloat162*>(orow + nd * 8 + t4 * 2) = hi2;
+            *reinterpret_cast<uint32_t*>(orow + (size_t)P.lo_row * P.Hq * hd + nd * 8 + t4 * 2) =
+                pack_bf16x2(v0 - __low2float(hi2), v1 - __high2float(hi2));
+          }
       }
     }
   } else {
@@ -548,8 +563,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int stages = P.stages;
-  const int b_stage_bytes = P.t_box * BK * 2;
-  const int stage_bytes = A_STAGE_BYTES + b_stage_bytes;
+  const int b_stage_bytes = P.t_box * BK * 2;               // one part (hi or lo) of the activation tile
+  const int stage_bytes = A_STAGE_BYTES + 2 * b_stage_bytes;
   uint8_t* tail = smem + (size_t)stages * stage_bytes;
   float* xch = reinterpret_cast<float*>(tail);
   Ctl* ctl = reinterpret_cast<Ctl*>(tail + XCH_BYTES);
@@ -650,6 +665,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           if (B.ph <= ready_ph) {
             uint8_t* b_dst = smem + (size_t)b_stage * stage_bytes + A_STAGE_BYTES;
             tma_load_2d(b_dst, P.maps + B.x_map, B.kk * BK, 0, ctl->full + b_stage, pol_x);
+            tma_load_2d(b_dst + b_stage_bytes, P.maps + B.x_map, B.kk * BK, P.lo_row, ctl->full + b_stage, pol_x);
             if (P.trace && cta == 0 && B.ph != traced_ph) { traced_ph = B.ph; P.trace[(size_t)B.ph * 8 + 7] = globaltimer_ns(); }
             ++b_count;
             if (++b_stage == stages) b_stage = 0;
@@ -696,11 +712,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           tc_fence_after();
           const uint32_t a_addr = smem_u32(smem + (size_t)stage * stage_bytes);
           const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + A_STAGE_BYTES);
+          const uint64_t b_desc_lo = smem_desc_sw128(a_addr + A_STAGE_BYTES + b_stage_bytes);
           const uint32_t d_tmem = tmem_base + (uint32_t)(buf * P.t_box);
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k)
+          for (int k = 0; k < BK / UMMA_K; ++k) {
             umma_bf16(d_tmem, a_desc + (uint64_t)(k * UMMA_K * 2 / 16), b_desc + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
                       (seg_first && k == 0) ? 0u : 1u);
+            umma_bf16(d_tmem, a_desc + (uint64_t)(k * UMMA_K * 2 / 16), b_desc_lo + (uint64_t)(k * UMMA_K * 2 / 16), idesc, 1u);
+          }
           umma_commit(ctl->empty + stage);
           if (seg_last) { umma_commit(ctl->acc_full + buf); acc_phase[buf] ^= 1; buf ^= 1; }
           seg_first = seg_last;
@@ -800,7 +819,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               if (dd < hd) {
                 bf16* orow = P.o + (size_t)(a.off + q / Gq) * P.Hq * hd + (size_t)(kvh * Gq + q % Gq) * hd + dd;
                 const float inv = 1.0f / L;
-                *reinterpret_cast<uint2*>(orow) = make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
+                const __nv_bfloat162 h01 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), h23 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+                *reinterpret_cast<uint2*>(orow) = make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
+                *reinterpret_cast<uint2*>(orow + (size_t)P.lo_row * P.Hq * hd) =
+                    make_uint2(pack_bf16x2(acc.x * inv - __low2float(h01), acc.y * inv - __high2float(h01)),
+                               pack_bf16x2(acc.z * inv - __low2float(h23), acc.w * inv - __high2float(h23)));
               }
             }
             item0 += items;
@@ -933,7 +956,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                   const int t = c0 + j;
-                  if (t < Tvalid) out_act[(size_t)t * p.ldo + n_out] = __float2bfloat16_rn(silu_f(v[j]) * xch[m * 16 + j]);
+                  if (t < Tvalid) store_split(out_act, (size_t)t * p.ldo + n_out, (size_t)P.lo_row * p.ldo, silu_f(v[j]) * xch[m * 16 + j]);
                 }
               }
               epi_bar_sync();
@@ -974,7 +997,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                   const size_t o = (size_t)(c0 + j) * p.ldo + n_out;
                   xn = xo[j] + v[j];
                   out_f32[o] = xn;
-                  P.h[o] = __float2bfloat16_rn(xn * gn);
+                  store_split(P.h, o, (size_t)P.lo_row * p.ldo, xn * gn);
                 }
                 v[j] = xn;
               }
@@ -1021,7 +1044,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               if (t < Tvalid) {
                 const size_t o = (size_t)t * p.ldo + n_out;
                 if (p.epi == TC_STORE_F32) out_f32[o] = v[j];
-                else out_act[o] = __float2bfloat16_rn(gelu_erf(v[j]));
+                else store_split(out_act, o, (size_t)P.lo_row * p.ldo, gelu_erf(v[j]));
               }
             }
           };
@@ -1156,7 +1179,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
 }
 
 inline size_t smem_bytes(int t_box, int stages, int hd) {
-  return 1024 + (size_t)stages * (A_STAGE_BYTES + (size_t)t_box * BK * 2) + XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127) +
+  return 1024 + (size_t)stages * (A_STAGE_BYTES + (size_t)2 * t_box * BK * 2) + XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127) +
          AttnSmem::bytes(hd) + 64;
 }
 inline int pick_stages(int t_box, int hd) {
