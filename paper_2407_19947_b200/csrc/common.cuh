@@ -1,6 +1,7 @@
 // Shared device helpers for the stairs kernels (sm_100a).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -15,7 +16,10 @@ template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f32<bf16>(bf16 v) { return __bfloat162float(v); }
 
+template <> __device__ __forceinline__ float to_f32<__half>(__half v) { return __half2float(v); }
+
 template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ __half from_f32<__half>(float v) { return __float2half_rn(v); }
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
 
@@ -47,6 +51,22 @@ template <> struct Vec16<bf16> {
     unpack(__ldcs(reinterpret_cast<const uint4*>(p)), out);
   }
 };
+
+template <> struct Vec16<__half> {
+  static constexpr int N = 8;
+  static __device__ __forceinline__ void load(const __half* p, float* out) {
+    const uint4 v = *reinterpret_cast<const uint4*>(p);
+    const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const float2 f = __half22float2(h[i]); out[2 * i] = f.x; out[2 * i + 1] = f.y; }
+  }
+};
+
+// Element type of the K/V cache for a weight type: fp32 models cache fp32; bf16 models cache fp16
+// (same 2 bytes as bf16 but 3 more mantissa bits; K/V of these models stay far inside its range).
+template <typename WT> struct KvType;
+template <> struct KvType<float> { typedef float type; };
+template <> struct KvType<bf16> { typedef __half type; };
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

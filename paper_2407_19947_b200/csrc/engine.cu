@@ -546,6 +546,7 @@ struct MkCall {
   const int* draft = nullptr;
   int* target_tokens = nullptr; int* accept_len = nullptr; int commit = 0; int* draft_out = nullptr;
   float* logits = nullptr;
+  bool skip_head = false;   // prefill: stop after the last layer (no LM head, no accept)
 };
 
 bool mk_eligible(const stairs_ctx* ctx, const DevModel& M, int T) {
@@ -565,7 +566,8 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   mk::Params P;
   memset(&P, 0, sizeof P);
   char* base = M.prog_base + (size_t)slot * M.prog_slot_bytes;
-  P.phases = reinterpret_cast<const mk::Phase*>(base); P.n_phases = M.n_phases;
+  const int n_run = c.skip_head ? M.n_phases - 2 : M.n_phases;
+  P.phases = reinterpret_cast<const mk::Phase*>(base); P.n_phases = n_run;
   P.maps = reinterpret_cast<const CUtensorMap*>(base + M.prog_maps_off);
   P.T = T; P.t_box = t_box; P.stages = mk::pick_stages(t_box, m.head_dim);
   P.logit_first_row = logit_first_row; P.n_logit_rows = n_logit_rows;
@@ -596,7 +598,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   void* args[] = {&P};
   CK(cudaLaunchCooperativeKernel((const void*)mk::k_forward, dim3(grid), dim3(tc::THREADS), args,
                                  mk::smem_bytes(t_box, P.stages, m.head_dim), ctx->stream));
-  ctx->bar_base += (unsigned long long)M.n_phases * grid;
+  ctx->bar_base += (unsigned long long)n_run * grid;
   ctx->launches++;
   return STAIRS_OK;
 }
@@ -642,8 +644,9 @@ int forward_rows(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, int n
   ctx->launches++;
   for (int l = 0; l < m.n_layers && !rc; ++l) {
     const stairs_layer_w& w = M.layers[l];
-    WT* kc = reinterpret_cast<WT*>(M.kpool + (size_t)l * M.kv_layer_bytes);
-    WT* vc = reinterpret_cast<WT*>(M.vpool + (size_t)l * M.kv_layer_bytes);
+    typedef typename KvType<WT>::type KT;
+    KT* kc = reinterpret_cast<KT*>(M.kpool + (size_t)l * M.kv_layer_bytes);
+    KT* vc = reinterpret_cast<KT*>(M.vpool + (size_t)l * M.kv_layer_bytes);
     k_norm<WT><<<T, 256, 0, st>>>(x, (const float*)w.norm1_w, (const float*)w.norm1_b, h, d, m.norm, m.norm_eps);
     {
       GemmTimer tm(ctx);
@@ -662,8 +665,8 @@ int forward_rows(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, int n
       }
     }
     if (rc) break;
-    k_rope_append<WT><<<T, 256, 0, st>>>(qkv, pos, req, page_table, q, kc, vc, hq, hkv, hd, m.pos, m.rope_theta, pt, L.max_pages);
-    k_attn_plain<WT, 8><<<dim3(hq, T), 128, (size_t)5 * hd * sizeof(float), st>>>(
+    k_rope_append<WT, KT><<<T, 256, 0, st>>>(qkv, pos, req, page_table, q, kc, vc, hq, hkv, hd, m.pos, m.rope_theta, pt, L.max_pages);
+    k_attn_plain<WT, KT, 8><<<dim3(hq, T), 128, (size_t)5 * hd * sizeof(float), st>>>(
         q, kc, vc, page_table, req, pos, o, hq, hkv, hd, pt, L.max_pages, 1.0f / sqrtf((float)hd));
     {
       GemmTimer tm(ctx);
@@ -773,6 +776,17 @@ int check_slot(stairs_ctx* ctx, int req, bool must_be_active) {
 }
 
 int prefill_model(stairs_ctx* ctx, DevModel& M, int slot, int n_ctx) {
+  if (mk_eligible(ctx, M, MK_MAX_ROWS)) {
+    // through the persistent kernel, 64 positions per pass: same arithmetic (hi+lo operands,
+    // fp16 attention tiles) as the validation pass, so cached K/V are as accurate as new ones
+    for (int c0 = 0; c0 < n_ctx; c0 += MK_MAX_ROWS) {
+      MkCall c;
+      c.mode = mk::CALL_PREFILL; c.slot = slot; c.draft_step = c0; c.skip_head = true;
+      int rc = launch_forward_mk(ctx, M, std::min(MK_MAX_ROWS, n_ctx - c0), 0, 0, c);
+      if (rc) return rc;
+    }
+    return STAIRS_OK;
+  }
   const int chunk = ctx->cfg.prefill_chunk > 0 ? ctx->cfg.prefill_chunk : 256;
   for (int c0 = 0; c0 < n_ctx; c0 += chunk) {
     const int n = std::min(chunk, n_ctx - c0);

@@ -113,10 +113,10 @@ __global__ void k_norm(const float* __restrict__ x, const float* __restrict__ g,
 // Rotary embedding of q and k, q to the attention operand buffer, k and v of the T new
 // positions into the slot's pages.  qkv is fp32 [T, (Hq+2Hkv)*hd].  Element i of a head
 // pairs with i + hd/2; angle = pos * theta^(-2i/hd).
-template <typename AT>
+template <typename AT, typename KT>
 __global__ void k_rope_append(const float* __restrict__ qkv, const int* __restrict__ pos,
                               const int* __restrict__ req, const int* __restrict__ page_table,
-                              AT* __restrict__ q_out, AT* __restrict__ kc, AT* __restrict__ vc,
+                              AT* __restrict__ q_out, KT* __restrict__ kc, KT* __restrict__ vc,
                               int Hq, int Hkv, int hd, int rope, float theta,
                               int page_tokens, int max_pages) {
   const int t = blockIdx.x;
@@ -142,21 +142,21 @@ __global__ void k_rope_append(const float* __restrict__ qkv, const int* __restri
       AT* dst = q_out + (size_t)t * nq + (size_t)head * hd;
       dst[i] = from_f32<AT>(a); dst[i + half] = from_f32<AT>(b2);
     } else {
-      AT* dst = kc + slot * nkv + (size_t)(head - Hq) * hd;
-      dst[i] = from_f32<AT>(a); dst[i + half] = from_f32<AT>(b2);
+      KT* dst = kc + slot * nkv + (size_t)(head - Hq) * hd;
+      dst[i] = from_f32<KT>(a); dst[i + half] = from_f32<KT>(b2);
     }
   }
   const float* vsrc = row + nq + nkv;
-  for (int i = threadIdx.x; i < nkv; i += blockDim.x) vc[slot * nkv + i] = from_f32<AT>(vsrc[i]);
+  for (int i = threadIdx.x; i < nkv; i += blockDim.x) vc[slot * nkv + i] = from_f32<KT>(vsrc[i]);
 }
 
 // Plain attention over the paged cache: one block per (query head, row), four warps; the
 // chunk of 32 positions starting at 32*c belongs to warp c % 4, whatever the batch, so a
 // row's result does not depend on which other rows are in the call.  Within a chunk each
 // lane scores one position; the four partial softmax states are merged in a fixed order.
-template <typename AT, int MAXD>
+template <typename AT, typename KT, int MAXD>
 __global__ void __launch_bounds__(128)
-k_attn_plain(const AT* __restrict__ q, const AT* __restrict__ kc, const AT* __restrict__ vc,
+k_attn_plain(const AT* __restrict__ q, const KT* __restrict__ kc, const KT* __restrict__ vc,
              const int* __restrict__ page_table, const int* __restrict__ req,
              const int* __restrict__ pos, AT* __restrict__ o, int Hq, int Hkv, int hd,
              int page_tokens, int max_pages, float scale) {
@@ -175,18 +175,18 @@ k_attn_plain(const AT* __restrict__ q, const AT* __restrict__ kc, const AT* __re
   float m = -INFINITY, l = 0.f, acc[MAXD];
 #pragma unroll
   for (int i = 0; i < MAXD; ++i) acc[i] = 0.f;
-  constexpr int VN = Vec16<AT>::N;
+  constexpr int VN = Vec16<KT>::N;
   for (int base = warp * 32; base <= last; base += 128) {
     const int p = base + lane;
     float s = -INFINITY;
     unsigned long long slot = 0;
     if (p <= last) {
       slot = (unsigned long long)pt[p / page_tokens] * page_tokens + (p % page_tokens);
-      const AT* kr = kc + slot * nkv + (size_t)kvh * hd;
+      const KT* kr = kc + slot * nkv + (size_t)kvh * hd;
       float dot = 0.f;
       for (int d0 = 0; d0 < hd; d0 += VN) {
         float kv[VN];
-        Vec16<AT>::load(kr + d0, kv);
+        Vec16<KT>::load(kr + d0, kv);
 #pragma unroll
         for (int j = 0; j < VN; ++j) dot = fmaf(qs[d0 + j], kv[j], dot);
       }
@@ -203,7 +203,7 @@ k_attn_plain(const AT* __restrict__ q, const AT* __restrict__ kc, const AT* __re
     for (int j = 0; j < cnt; ++j) {
       const float pj = __shfl_sync(0xffffffffu, pl, j);
       const unsigned long long sj = __shfl_sync(0xffffffffu, slot, j);
-      const AT* vr = vc + sj * nkv + (size_t)kvh * hd;
+      const KT* vr = vc + sj * nkv + (size_t)kvh * hd;
 #pragma unroll
       for (int i = 0; i < MAXD; ++i) {
         const int d = lane + 32 * i;

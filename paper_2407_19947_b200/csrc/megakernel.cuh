@@ -59,7 +59,7 @@ struct Phase {
   void* kc; void* vc;
 };
 
-enum CallMode { CALL_VALIDATE = 0, CALL_DRAFT_FIRST = 1, CALL_DRAFT_NEXT = 2 };
+enum CallMode { CALL_VALIDATE = 0, CALL_DRAFT_FIRST = 1, CALL_DRAFT_NEXT = 2, CALL_PREFILL = 3 };
 
 struct Params {
   const Phase* phases; int n_phases;
@@ -106,15 +106,20 @@ struct AttnSmem {   // carved after the GEMM ring: Q block (bf16), K and V chunk
   static __host__ __device__ size_t bytes(int hd) { return q_bytes(hd) + 2 * kv_bytes(hd) + 64; }
 };
 
-// mma.sync m16n8k16 (bf16 in, fp32 accumulate) and its operand loads, for the attention tiles
+// mma.sync m16n8k16 (fp16 in, fp32 accumulate) and its operand loads, for the attention tiles:
+// queries, cached K/V and the softmax weights are fp16 (11 significant bits)
 __device__ __forceinline__ void mma_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, const void* p) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)));
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -238,6 +243,11 @@ __device__ __forceinline__ RowInfo row_info(const Params& P, int t) {
     const int base = P.n_seq[r.slot] - 1;
     r.pos = base + rr;
     r.tok = clampv(rr == 0 ? P.seq[(size_t)r.slot * P.max_seq_len + base] : P.draft[i * P.k_max + rr - 1]);
+  } else if (P.mode == CALL_PREFILL) {
+    // T consecutive prompt positions starting at draft_step (no logits are taken)
+    r.slot = P.slot;
+    r.pos = P.draft_step + t;
+    r.tok = clampv(P.seq[(size_t)P.slot * P.max_seq_len + r.pos]);
   } else if (P.mode == CALL_DRAFT_FIRST) {
     r.slot = P.slot;
     const int n = P.n_seq[P.slot];
@@ -301,6 +311,8 @@ __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
   if (P.mode == CALL_VALIDATE) {
     a.slot = P.val_req[i]; a.R = P.val_k[i] + 1; a.off = P.val_off[i];
     a.base = P.n_seq[a.slot] - 1;
+  } else if (P.mode == CALL_PREFILL) {
+    a.slot = P.slot; a.R = P.T; a.off = 0; a.base = P.draft_step;
   } else if (P.mode == CALL_DRAFT_FIRST) {
     a.slot = P.slot; a.R = 2; a.off = 0; a.base = P.n_seq[P.slot] - 2;
   } else {
@@ -337,8 +349,8 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   uint8_t* qs = att_smem;                                   // [QBLK][pitch] bf16, rotated and pre-scaled
   uint8_t* ks = qs + AttnSmem::q_bytes(hd);                 // [CHUNK][pitch]
   uint8_t* vs = ks + AttnSmem::kv_bytes(hd);
-  bf16* kc = reinterpret_cast<bf16*>(ph.kc);
-  bf16* vc = reinterpret_cast<bf16*>(ph.vc);
+  __half* kc = reinterpret_cast<__half*>(ph.kc);
+  __half* vc = reinterpret_cast<__half*>(ph.vc);
   const int* pt = P.page_table + (size_t)a.slot * P.max_pages;
   const float scale = 1.0f / sqrtf((float)hd);
   const int half = hd / 2, ksteps = hd / 16, ntiles = hd / 8;
@@ -383,15 +395,15 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
           const float r0 = x0 * cs - x1 * sn, r1 = x1 * cs + x0 * sn;
           x0 = r0; x1 = r1;
         }
-        const bf16 k0 = __float2bfloat16_rn(x0), k1 = __float2bfloat16_rn(x1);
-        const bf16 v0 = __float2bfloat16_rn(vsrc[i]), v1 = __float2bfloat16_rn(vsrc[i + half]);
-        bf16* kd = reinterpret_cast<bf16*>(ks + j * pitch);
-        bf16* vd = reinterpret_cast<bf16*>(vs + j * pitch);
+        const __half k0 = __float2half_rn(x0), k1 = __float2half_rn(x1);
+        const __half v0 = __float2half_rn(vsrc[i]), v1 = __float2half_rn(vsrc[i + half]);
+        __half* kd = reinterpret_cast<__half*>(ks + j * pitch);
+        __half* vd = reinterpret_cast<__half*>(vs + j * pitch);
         kd[i] = k0; kd[i + half] = k1; vd[i] = v0; vd[i + half] = v1;
         if (qblk == 0) {
           const size_t slot = (size_t)pt[p / P.page_tokens] * P.page_tokens + (p % P.page_tokens);
-          bf16* kg = kc + slot * nkv + (size_t)kvh * hd;
-          bf16* vg = vc + slot * nkv + (size_t)kvh * hd;
+          __half* kg = kc + slot * nkv + (size_t)kvh * hd;
+          __half* vg = vc + slot * nkv + (size_t)kvh * hd;
           kg[i] = k0; kg[i + half] = k1; vg[i] = v0; vg[i + half] = v1;
         }
       }
@@ -421,9 +433,9 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
         x0 = r0; x1 = r1;
       }
     }
-    bf16* qd = reinterpret_cast<bf16*>(qs + (size_t)ql * pitch);
-    qd[i] = __float2bfloat16_rn(x0 * scale);
-    qd[i + half] = __float2bfloat16_rn(x1 * scale);
+    __half* qd = reinterpret_cast<__half*>(qs + (size_t)ql * pitch);
+    qd[i] = __float2half_rn(x0 * scale);
+    qd[i + half] = __float2half_rn(x1 * scale);
   }
   epi_bar_sync();
 
@@ -496,8 +508,8 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
         l_a = l_a * corr_a + sum_a; l_b = l_b * corr_b + sum_b;
         m_a = mn_a; m_b = mn_b;
         uint32_t pf[4];
-        pf[0] = pack_bf16x2(sc[0][0], sc[0][1]); pf[1] = pack_bf16x2(sc[0][2], sc[0][3]);
-        pf[2] = pack_bf16x2(sc[1][0], sc[1][1]); pf[3] = pack_bf16x2(sc[1][2], sc[1][3]);
+        pf[0] = pack_f16x2(sc[0][0], sc[0][1]); pf[1] = pack_f16x2(sc[0][2], sc[0][3]);
+        pf[2] = pack_f16x2(sc[1][0], sc[1][1]); pf[3] = pack_f16x2(sc[1][2], sc[1][3]);
         // V fragments: lane supplies the address of row (lane & 15) of the slice, column block (lane >> 4)
         const uint8_t* vrow = vs + (size_t)(sl0 + (lane & 15)) * pitch + (lane >> 4) * 16;
 #pragma unroll
@@ -851,7 +863,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                 P.n_seq[slot] = wpos;
               }
             }
-          } else if (et == 0) {
+          } else if (et == 0 && P.mode != CALL_PREFILL) {
             P.draft_out[P.draft_step] = argmax_key_index(__ldcg(P.keys + P.logit_first_row));
           }
         }
