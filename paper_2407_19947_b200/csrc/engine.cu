@@ -155,6 +155,7 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
   if (c.kv_pages < 0 || c.prefill_chunk < 0) { *why = "kv_pages and prefill_chunk must not be negative"; return false; }
   const int chunk = c.prefill_chunk > 0 ? c.prefill_chunk : 256;
   L->max_rows = (std::max(std::max(chunk, c.max_requests * (c.k_max + 1)), 2) + 15) / 16 * 16;
+  if (c.target.wdtype == 1) L->max_rows = std::max(L->max_rows, MK_MAX_ROWS);   // prefill passes of the persistent kernel
   L->t_box_max = std::min(256, L->max_rows);
   L->logit_rows = std::max(c.max_requests * (c.k_max + 1), 1);
   L->max_pages = (c.max_seq_len + pt - 1) / pt;
