@@ -140,7 +140,7 @@ def kernel_source_hash() -> str:
 def stored_traffic(workload_name: str):
     """dram bytes per launch from the committed ncu capture of this workload, or None when the
     kernels changed since it was taken."""
-    p = os.path.join(ROOT, "profiles", "traffic.json")
+    p = os.path.join(ROOT, "profiles", "traffic_k_forward.txt")
     if not os.path.exists(p):
         return None
     with open(p) as f:
