@@ -211,7 +211,7 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     L->prog_slot_d = (t.wdtype == 1 && has_draft) ? prog(d, &L->prog_maps_off_d) : 0;
     L->prog_t = take(L->prog_slot_t * MK_TBOX_SLOTS);
     L->prog_d = take(L->prog_slot_d * MK_TBOX_SLOTS);
-    L->mk_trace = take(t.wdtype == 1 ? (size_t)(2 * 8 + 4 * TC_GRID_MAX) * (8 * std::max(t.n_layers, 1) + 4) * 8 : 0);
+    L->mk_trace = take(t.wdtype == 1 ? (size_t)(2 * 8 + 8 * TC_GRID_MAX) * (8 * std::max(t.n_layers, 1) + 4) * 8 : 0);
     L->stat_tiles = (t.d_model + tc::BM - 1) / tc::BM;
     L->mk_stats = take(t.wdtype == 1 ? (size_t)MK_MAX_ROWS * L->stat_tiles * 16 : 0);
     L->attn_cnt_n = c.max_requests * hkv * std::max(n_qblk, 1);

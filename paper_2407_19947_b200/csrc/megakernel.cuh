@@ -947,6 +947,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           // (before the arrival counter is known) so that the last arriver's chain is shorter
           float xpre[16], gpre = 0.f;
           bool have_pre = false;
+          unsigned long long* tra = nullptr;   // this CTA's detail slots of the phase trace
           auto finish = [&](int c0, float* v) {
             if (p.norm_in) {
               // fold the normalisation in: y = rstd_t * (acc - mean_t * u[n]) + c[n]
@@ -1013,6 +1014,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                 }
                 v[j] = xn;
               }
+              if (tra) tra[6] = globaltimer_ns();
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
                 if (j < jn) {
@@ -1037,6 +1039,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                 const float m2 = ctl->red2[0][et] + ctl->red2[1][et] + ctl->red2[2][et] + ctl->red2[3][et];
                 P.stats[(size_t)(c0 + et) * P.stat_tiles + tile] = make_float4(mean, m2, (float)cnt, 0.f);
               }
+              if (tra) tra[7] = globaltimer_ns();
               epi_bar_sync();
               return;
             }
@@ -1070,6 +1073,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
           } else {
             const int slot = 2 * cta + (kb == kb_begin ? 0 : 1);
+            tra = (P.trace && et == 0) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
+            if (tra) tra[4] = globaltimer_ns();
             float* mine = P.partial + (size_t)slot * P.t_box * BM;
             for (int c0 = 0; c0 < Tvalid; c0 += 16) {   // only rows that exist
               float v[16];
@@ -1088,6 +1093,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             }
             __threadfence();
             epi_bar_sync();
+            if (tra) tra[5] = globaltimer_ns();
             // CTAs whose ranges touch this tile (32-bit arithmetic: total * Ge < 2^32, checked on the host)
             const unsigned tot32 = (unsigned)total, ge32 = (unsigned)Ge, tf32 = (unsigned)tile_first, te32 = (unsigned)tile_end;
             auto rb = [&](unsigned c) { return (tot32 * c) / ge32; };
@@ -1105,7 +1111,6 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             epi_bar_sync();
             const bool last = ctl->last_flag != 0;
             epi_bar_sync();
-            unsigned long long* tra = (P.trace && et == 0) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 4 : nullptr;
             if (last) {
               if (tra) tra[1] = globaltimer_ns();
               __threadfence();
@@ -1132,7 +1137,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                     for (int j = 0; j < 16; ++j) v[j] += tmp[u][j];
                   }
                 }
-                if (tra) tra[2] = globaltimer_ns();
+                if (tra) { asm volatile("" :: "f"(v[0]), "f"(v[1])); tra[2] = globaltimer_ns(); }
                 finish(c0, v);
               }
               if (tra) tra[3] = globaltimer_ns();
@@ -1145,7 +1150,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       if (!ok) break;
       if (tracing) tr[1] = globaltimer_ns();
       // every CTA's completion time of the phase, after the two detailed traces
-      if (P.trace && et == 0) P.trace[(size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 4] = globaltimer_ns();
+      if (P.trace && et == 0) P.trace[(size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8] = globaltimer_ns();
       // Publish this CTA's part of the phase.  A CTA may arrive for phase ph only once every
       // CTA has arrived for phase ph-1: otherwise CTAs without work in two consecutive GEMM
       // phases would run ahead and their arrivals would be mistaken for the slower CTAs' ones
