@@ -177,6 +177,23 @@ __device__ __forceinline__ void store_split(bf16* base, size_t idx, size_t lo_of
   base[idx + lo_off] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
+// Sums 32 per-lane values across the warp, all at once: on return lane l holds the warp-wide
+// total of a[l].  Each halving step exchanges the half a lane does not keep (31 shuffles in five
+// dependent steps, instead of 32 separate five-step reductions).
+__device__ __forceinline__ float warp_multi_sum32(float (&a)[32], int lane) {
+#pragma unroll
+  for (int h = 16; h >= 1; h >>= 1) {
+    const bool up = (lane & h) != 0;
+#pragma unroll
+    for (int i = 0; i < h; ++i) {
+      const float send = up ? a[i] : a[i + h];
+      const float keep = up ? a[i + h] : a[i];
+      a[i] = keep + __shfl_xor_sync(0xffffffffu, send, h);
+    }
+  }
+  return a[0];
+}
+
 // Shared per-CTA control block.
 struct Ctl {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2], att_bar;
@@ -185,7 +202,7 @@ struct Ctl {
   volatile int last_flag;
   volatile int bcast;
   float rstd[64], mu[64];       // per-row statistics of the current norm_in GEMM phase
-  float red[4][16], red2[4][16];
+  float red[4][16], red2[4][16], shift[4][16];
 };
 
 // Uniform verdict for the 128 compute threads after any of them may have timed out in a wait:
@@ -1015,28 +1032,39 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                 v[j] = xn;
               }
               if (tra) tra[6] = globaltimer_ns();
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                if (j < jn) {
-                  const float s1 = warp_sum(v[j]);
-                  if (lane == 0) ctl->red[quad][j] = s1;
-                }
-              }
-              epi_bar_sync();
+              // Row statistics of this tile's columns.  Each warp reduces, for its 32 columns, the
+              // sums of d and d*d of all 16 rows at once (d = x minus the warp's first column, a
+              // shift that keeps the subtraction below free of cancellation); one thread per row
+              // then merges the four warps' (mean, M2, count).
               const int cnt = min(tile_cols, p.N - tile * BM);
+              {
+                float bf[32];
 #pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                if (j < jn) {
-                  const float mean = (ctl->red[0][j] + ctl->red[1][j] + ctl->red[2][j] + ctl->red[3][j]) / (float)cnt;
-                  const float dl = n_valid ? v[j] - mean : 0.f;
-                  const float s2 = warp_sum(dl * dl);
-                  if (lane == 0) ctl->red2[quad][j] = s2;
+                for (int j = 0; j < 16; ++j) {
+                  const float sh = __shfl_sync(0xffffffffu, v[j], 0);
+                  if (lane == 0) ctl->shift[quad][j] = sh;
+                  const float dl = n_valid ? v[j] - sh : 0.f;
+                  bf[j] = dl; bf[16 + j] = dl * dl;
                 }
+                const float tot = warp_multi_sum32(bf, lane);   // lane l: total of bf[l]
+                if (lane < 16) ctl->red[quad][lane] = tot; else ctl->red2[quad][lane - 16] = tot;
               }
               epi_bar_sync();
               if (et < 16 && c0 + et < Tvalid) {
-                const float mean = (ctl->red[0][et] + ctl->red[1][et] + ctl->red[2][et] + ctl->red[3][et]) / (float)cnt;
-                const float m2 = ctl->red2[0][et] + ctl->red2[1][et] + ctl->red2[2][et] + ctl->red2[3][et];
+                float mean = 0.f, m2 = 0.f, n = 0.f;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                  const float nw = (float)max(0, min(32, cnt - 32 * w));
+                  if (nw > 0.f) {
+                    const float sd = ctl->red[w][et];
+                    const float mw = ctl->shift[w][et] + sd / nw;
+                    const float m2w = fmaxf(ctl->red2[w][et] - sd * sd / nw, 0.f);
+                    const float dm = mw - mean, nn = n + nw;
+                    m2 += m2w + dm * dm * (n * nw / nn);
+                    mean += dm * (nw / nn);
+                    n = nn;
+                  }
+                }
                 P.stats[(size_t)(c0 + et) * P.stat_tiles + tile] = make_float4(mean, m2, (float)cnt, 0.f);
               }
               if (tra) tra[7] = globaltimer_ns();
@@ -1063,15 +1091,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               }
             }
           };
-          if (whole) {
-            for (int c0 = 0; c0 < Tvalid; c0 += 16) {
-              float v[16];
-              tmem_ld16(taddr + (uint32_t)c0, v);
-              finish(c0, v);
-            }
-            tc_fence_before();
-            if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
-          } else {
+          // A whole tile is finished straight from TMEM.  A split tile's segment goes to this CTA's
+          // partial slot; whichever CTA arrives last at the tile's counter sums the partials in
+          // k order (a fixed order: results do not depend on timing) and finishes the tile.
+          bool last = false;
+          unsigned first_c = 0, last_c = 0;
+          const unsigned tot32 = (unsigned)total, ge32 = (unsigned)Ge, tf32 = (unsigned)tile_first, te32 = (unsigned)tile_end;
+          auto rb = [&](unsigned c) { return (tot32 * c) / ge32; };   // total * Ge < 2^32, checked on the host
+          if (!whole) {
             const int slot = 2 * cta + (kb == kb_begin ? 0 : 1);
             tra = (P.trace && et == 0) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
             if (tra) tra[4] = globaltimer_ns();
@@ -1094,13 +1121,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             __threadfence();
             epi_bar_sync();
             if (tra) tra[5] = globaltimer_ns();
-            // CTAs whose ranges touch this tile (32-bit arithmetic: total * Ge < 2^32, checked on the host)
-            const unsigned tot32 = (unsigned)total, ge32 = (unsigned)Ge, tf32 = (unsigned)tile_first, te32 = (unsigned)tile_end;
-            auto rb = [&](unsigned c) { return (tot32 * c) / ge32; };
-            unsigned first_c = (tf32 * ge32) / tot32;
+            // CTAs whose ranges touch this tile
+            first_c = (tf32 * ge32) / tot32;
             while (rb(first_c + 1) <= tf32) ++first_c;
             while (first_c > 0 && rb(first_c) > tf32) --first_c;
-            unsigned last_c = first_c;
+            last_c = first_c;
             while (last_c + 1 < ge32 && rb(last_c + 1) < te32) ++last_c;
             const int nseg = (int)(last_c - first_c) + 1;
             if (et == 0) {
@@ -1109,14 +1134,20 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               if (old == nseg - 1) P.counters[tile] = 0;
             }
             epi_bar_sync();
-            const bool last = ctl->last_flag != 0;
+            last = ctl->last_flag != 0;
             epi_bar_sync();
             if (last) {
               if (tra) tra[1] = globaltimer_ns();
               __threadfence();
-              for (int c0 = 0; c0 < Tvalid; c0 += 16) {
+            }
+          }
+          if (whole || last) {
+            for (int c0 = 0; c0 < Tvalid; c0 += 16) {
+              float v[16];
+              if (whole) {
+                tmem_ld16(taddr + (uint32_t)c0, v);
+              } else {
                 const int jn = min(16, Tvalid - c0);
-                float v[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j) v[j] = 0.f;
                 // four segments' loads are issued together; the additions stay in k order
@@ -1138,10 +1169,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                   }
                 }
                 if (tra) { asm volatile("" :: "f"(v[0]), "f"(v[1])); tra[2] = globaltimer_ns(); }
-                finish(c0, v);
               }
-              if (tra) tra[3] = globaltimer_ns();
+              finish(c0, v);
             }
+            if (!whole && tra) tra[3] = globaltimer_ns();
+          }
+          if (whole) {
+            tc_fence_before();
+            if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
           }
           buf ^= 1;
           kb = seg_end;
