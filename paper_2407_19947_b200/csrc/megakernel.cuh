@@ -689,8 +689,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           advance(A);
           progress = true;
         }
-        const bool chain_wait = B.valid && B.ph > ready_ph && !progress;   // MMAs stalled on a phase's inputs
-        for (int burst = 0; burst < 4 && chain_wait && C.valid && (int)(c_count - a_count) < P.l2_ahead; ++burst) {
+        for (int burst = 0; burst < 4 && C.valid && (int)(c_count - a_count) < P.l2_ahead; ++burst) {
           if ((int)(c_count - a_count) >= 0) {   // a tile the ring has already asked for needs no prefetch
             tma_prefetch_l2_2d(C.wm0, C.kk * BK, C.row);
             if (C.dual) tma_prefetch_l2_2d(C.wm1, C.kk * BK, C.row);
