@@ -4,7 +4,6 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <new>
@@ -572,7 +571,6 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.phases = reinterpret_cast<const mk::Phase*>(base); P.n_phases = n_run;
   P.maps = reinterpret_cast<const CUtensorMap*>(base + M.prog_maps_off);
   P.T = T; P.t_box = t_box; P.stages = mk::pick_stages(t_box, m.head_dim);
-  { const char* e = getenv("STAIRS_L2_AHEAD"); P.l2_ahead = e ? atoi(e) : 24; }
   P.logit_first_row = logit_first_row; P.n_logit_rows = n_logit_rows;
   P.d = m.d_model; P.Hq = m.n_heads; P.Hkv = m.n_kv_heads; P.hd = m.head_dim; P.F = m.d_ff; P.vocab = m.vocab;
   P.norm_kind = m.norm; P.rope = m.pos; P.rope_theta = m.rope_theta; P.eps = m.norm_eps;

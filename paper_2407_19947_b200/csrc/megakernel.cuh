@@ -65,7 +65,6 @@ struct Params {
   const Phase* phases; int n_phases;
   const CUtensorMap* maps;
   int T, t_box, stages;
-  int l2_ahead;            // weight tiles asked of L2 ahead of the shared-memory ring, per CTA
   int logit_first_row, n_logit_rows;
   // model
   int d, Hq, Hkv, hd, F, vocab, norm_kind, rope; float rope_theta, eps;
@@ -665,11 +664,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         if (--c.remaining == 0) { enter(c, c.ph + 1); return; }
         if (++c.kk == c.kblocks) { c.kk = 0; ++c.n_tile; locate(c); }
       };
-      // C runs ahead of A and only asks L2 for the weight tiles: HBM keeps streaming while the
-      // ring is full and the MMAs wait for a phase's inputs, and the ring then fills from L2.
-      Cursor A, B, C;
-      enter(A, 0); enter(B, 0); enter(C, 0);
-      unsigned int c_count = 0;
+      Cursor A, B;
+      enter(A, 0); enter(B, 0);
       int a_stage = 0, b_stage = 0;
       uint32_t a_par = 0;
       unsigned int a_count = 0, b_count = 0, idle = 0;
@@ -688,14 +684,6 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           p_stage = a_stage; p_phase = a_par;
           advance(A);
           progress = true;
-        }
-        for (int burst = 0; burst < 4 && C.valid && (int)(c_count - a_count) < P.l2_ahead; ++burst) {
-          if ((int)(c_count - a_count) >= 0) {   // a tile the ring has already asked for needs no prefetch
-            tma_prefetch_l2_2d(C.wm0, C.kk * BK, C.row);
-            if (C.dual) tma_prefetch_l2_2d(C.wm1, C.kk * BK, C.row);
-          }
-          ++c_count;
-          advance(C);
         }
         if (b_count != a_count) {
           // inputs of phase B.ph are published once every CTA has finished phase B.ph - 1; the
