@@ -216,8 +216,8 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     L->mk_stats = take(t.wdtype == 1 ? (size_t)MK_MAX_ROWS * L->stat_tiles * 16 : 0);
     L->attn_cnt_n = c.max_requests * hkv * std::max(n_qblk, 1);
     L->attn_cnt = take(t.wdtype == 1 ? (size_t)L->attn_cnt_n * 4 : 0);
-    L->rope_t = take(t.wdtype == 1 ? (size_t)t.head_dim * 2 : 0);
-    L->rope_d = take((t.wdtype == 1 && has_draft) ? (size_t)d.head_dim * 2 : 0);
+    L->rope_t = take(t.wdtype == 1 ? (size_t)t.head_dim * 2 * (1 + 2 * 64) : 0);   // inverse frequencies, then cos and sin of 64 rows
+    L->rope_d = take((t.wdtype == 1 && has_draft) ? (size_t)d.head_dim * 2 * (1 + 2 * 64) : 0);
     // LayerNorm models: u = W.gain and c = W.bias per normalised GEMM (fp32)
     auto aux = [&](const stairs_model& m) {
       if (m.norm != 0) return (size_t)0;
@@ -591,7 +591,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.partial = reinterpret_cast<float*>(ws + L.gemm_partial); P.counters = reinterpret_cast<int*>(ws + L.gemm_counters);
   P.attn_part = reinterpret_cast<float*>(ws + L.attn_part); P.attn_part_units = L.attn_units;
   P.stats = reinterpret_cast<float4*>(ws + L.mk_stats); P.stat_tiles = L.stat_tiles;
-  P.rope_inv = M.rope_inv; P.attn_cnt = reinterpret_cast<int*>(ws + L.attn_cnt);
+  P.rope_inv = M.rope_inv; P.rope_cs = M.rope_inv + m.head_dim / 2; P.rope_sn = P.rope_cs + 64 * (m.head_dim / 2); P.attn_cnt = reinterpret_cast<int*>(ws + L.attn_cnt);
   P.bar = reinterpret_cast<unsigned long long*>(ws + L.mk_bar); P.bar_base = ctx->bar_base;
   P.status = ctx->status_dev; P.wait_limit = ctx->wait_limit;
   P.trace = (ctx->profile && &M == &ctx->target) ? reinterpret_cast<unsigned long long*>(ws + L.mk_trace) : nullptr;

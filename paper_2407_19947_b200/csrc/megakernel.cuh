@@ -81,7 +81,9 @@ struct Params {
   unsigned long long* keys; int n_keys;
   float4* stats;            // [64 rows][stat_tiles] (mean, M2, count, -) per 128-column tile of x
   int stat_tiles;
-  const float* rope_inv;    // [hd/2] theta^(-2i/hd)
+  const float* rope_inv;
+  float* rope_cs; float* rope_sn;   // [row][hd/2] cos and sin of the call's row positions, written by the embedding phase
+     // [hd/2] theta^(-2i/hd)
   int* attn_cnt;            // split-KV arrival counters per (request, kv head, query block)
   float* logits;            // optional dump
   int* target_tokens; int* accept_len; int commit; int* draft_out;
@@ -316,6 +318,12 @@ __device__ void embed_row(const Params& P, int t, const RowInfo& r, const float*
   const float m2 = group_sum(s2, red, et);
   for (int tile = et; tile < P.stat_tiles; tile += 128)
     P.stats[(size_t)t * P.stat_tiles + tile] = tile == 0 ? make_float4(mean, m2, (float)d, 0.f) : make_float4(0.f, 0.f, 0.f, 0.f);
+  if (P.rope && et < P.hd / 2) {   // rotation table of this row's position, shared by every layer
+    float sn, cs;
+    sincosf((float)r.pos * P.rope_inv[et], &sn, &cs);
+    P.rope_cs[(size_t)t * (P.hd / 2) + et] = cs;
+    P.rope_sn[(size_t)t * (P.hd / 2) + et] = sn;
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -398,30 +406,58 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
       }
     }
     {
+      // rows of new positions: four column pairs (i, i + hd/2) per item, the item's six
+      // vector loads in flight together (each is an L2 round trip)
       const int r_lo = max(0, p0 - a.base), r_hi = min(a.R, p0 + n_pos - a.base);
-      for (int idx = et; idx < (r_hi - r_lo) * half; idx += 128) {
-        const int r = r_lo + idx / half, i = idx % half, p = a.base + r, j = p - p0;
-        const float* row = P.qkv + (size_t)(a.off + r) * nqkv;
-        const float* ksrc = row + nq + (size_t)kvh * hd;
-        const float* vsrc = row + nq + nkv + (size_t)kvh * hd;
-        float x0 = ksrc[i], x1 = ksrc[i + half];
-        if (P.rope) {
-          const float ang = (float)p * P.rope_inv[i];
-          float sn, cs;
-          sincosf(ang, &sn, &cs);
-          const float r0 = x0 * cs - x1 * sn, r1 = x1 * cs + x0 * sn;
-          x0 = r0; x1 = r1;
+      const int hq = half / 4, n_items = (r_hi - r_lo) * hq;
+      for (int b0 = et; b0 < n_items; b0 += 128) {
+        float4 kl[1], kh[1], vl[1], vh[1], cs4[1], sn4[1];
+#pragma unroll
+        for (int u = 0; u < 1; ++u) {
+          const int idx = b0 + 128 * u;
+          if (idx < n_items) {
+            const int r = r_lo + idx / hq, i4 = (idx % hq) * 4;
+            const float* row = P.qkv + (size_t)(a.off + r) * nqkv;
+            const float* ksrc = row + nq + (size_t)kvh * hd + i4;
+            const float* vsrc = row + nq + nkv + (size_t)kvh * hd + i4;
+            kl[u] = __ldcg(reinterpret_cast<const float4*>(ksrc)); kh[u] = __ldcg(reinterpret_cast<const float4*>(ksrc + half));
+            vl[u] = __ldcg(reinterpret_cast<const float4*>(vsrc)); vh[u] = __ldcg(reinterpret_cast<const float4*>(vsrc + half));
+            if (P.rope) {
+              cs4[u] = __ldcg(reinterpret_cast<const float4*>(P.rope_cs + (size_t)(a.off + r) * half + i4));
+              sn4[u] = __ldcg(reinterpret_cast<const float4*>(P.rope_sn + (size_t)(a.off + r) * half + i4));
+            }
+          }
         }
-        const __half k0 = __float2half_rn(x0), k1 = __float2half_rn(x1);
-        const __half v0 = __float2half_rn(vsrc[i]), v1 = __float2half_rn(vsrc[i + half]);
-        __half* kd = reinterpret_cast<__half*>(ks + j * pitch);
-        __half* vd = reinterpret_cast<__half*>(vs + j * pitch);
-        kd[i] = k0; kd[i + half] = k1; vd[i] = v0; vd[i + half] = v1;
-        if (qblk == 0) {
-          const size_t slot = (size_t)pt[p / P.page_tokens] * P.page_tokens + (p % P.page_tokens);
-          __half* kg = kc + slot * nkv + (size_t)kvh * hd;
-          __half* vg = vc + slot * nkv + (size_t)kvh * hd;
-          kg[i] = k0; kg[i + half] = k1; vg[i] = v0; vg[i + half] = v1;
+#pragma unroll
+        for (int u = 0; u < 1; ++u) {
+          const int idx = b0 + 128 * u;
+          if (idx < n_items) {
+            const int r = r_lo + idx / hq, i4 = (idx % hq) * 4, p = a.base + r, j = p - p0;
+            float x0[4] = {kl[u].x, kl[u].y, kl[u].z, kl[u].w}, x1[4] = {kh[u].x, kh[u].y, kh[u].z, kh[u].w};
+            if (P.rope) {
+              const float cs[4] = {cs4[u].x, cs4[u].y, cs4[u].z, cs4[u].w}, sn[4] = {sn4[u].x, sn4[u].y, sn4[u].z, sn4[u].w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float r0 = x0[e] * cs[e] - x1[e] * sn[e], r1 = x1[e] * cs[e] + x0[e] * sn[e];
+                x0[e] = r0; x1[e] = r1;
+              }
+            }
+            const uint2 k_lo = make_uint2(pack_f16x2(x0[0], x0[1]), pack_f16x2(x0[2], x0[3]));
+            const uint2 k_hi = make_uint2(pack_f16x2(x1[0], x1[1]), pack_f16x2(x1[2], x1[3]));
+            const uint2 v_lo = make_uint2(pack_f16x2(vl[u].x, vl[u].y), pack_f16x2(vl[u].z, vl[u].w));
+            const uint2 v_hi = make_uint2(pack_f16x2(vh[u].x, vh[u].y), pack_f16x2(vh[u].z, vh[u].w));
+            __half* kd = reinterpret_cast<__half*>(ks + j * pitch);
+            __half* vd = reinterpret_cast<__half*>(vs + j * pitch);
+            *reinterpret_cast<uint2*>(kd + i4) = k_lo; *reinterpret_cast<uint2*>(kd + half + i4) = k_hi;
+            *reinterpret_cast<uint2*>(vd + i4) = v_lo; *reinterpret_cast<uint2*>(vd + half + i4) = v_hi;
+            if (qblk == 0) {
+              const size_t slot = (size_t)pt[p / P.page_tokens] * P.page_tokens + (p % P.page_tokens);
+              __half* kg = kc + slot * nkv + (size_t)kvh * hd;
+              __half* vg = vc + slot * nkv + (size_t)kvh * hd;
+              *reinterpret_cast<uint2*>(kg + i4) = k_lo; *reinterpret_cast<uint2*>(kg + half + i4) = k_hi;
+              *reinterpret_cast<uint2*>(vg + i4) = v_lo; *reinterpret_cast<uint2*>(vg + half + i4) = v_hi;
+            }
+          }
         }
       }
     }
@@ -435,24 +471,50 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   // the first chunk's copies fly while the queries are rotated
   stage_issue(c_begin);
   // queries of this block: query index q -> row r = q / G, head = kvh * G + q % G
-  for (int idx = et; idx < ATT_QBLK * half; idx += 128) {
-    const int ql = idx / half, i = idx % half, q = q0 + ql;
-    float x0 = 0.f, x1 = 0.f;
-    if (ql < nQ) {
-      const int r = q / G, head = kvh * G + (q % G);
-      const float* src = P.qkv + (size_t)(a.off + r) * nqkv + (size_t)head * hd;
-      x0 = src[i]; x1 = src[i + half];
-      if (P.rope) {
-        const float ang = (float)(a.base + r) * P.rope_inv[i];
-        float sn, cs;
-        sincosf(ang, &sn, &cs);
-        const float r0 = x0 * cs - x1 * sn, r1 = x1 * cs + x0 * sn;
-        x0 = r0; x1 = r1;
+  {
+    // two items' loads in flight together (at most six items of four column pairs per thread
+    // at hd = 128): each load is an L2 round trip
+    const int hq = half / 4, n_items = nQ * hq, n_all = ATT_QBLK * hq;
+    for (int u0 = 0; u0 < 6 && et + 128 * u0 < n_all; u0 += 2) {
+      float4 xa[2], xb[2], qc[2], qn[2];
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int idx = et + 128 * (u0 + u);
+        if (idx < n_items) {
+          const int ql = idx / hq, i4 = (idx % hq) * 4, q = q0 + ql;
+          const int r = q / G, head = kvh * G + (q % G);
+          const float* src = P.qkv + (size_t)(a.off + r) * nqkv + (size_t)head * hd + i4;
+          xa[u] = __ldcg(reinterpret_cast<const float4*>(src)); xb[u] = __ldcg(reinterpret_cast<const float4*>(src + half));
+          if (P.rope) {
+            qc[u] = __ldcg(reinterpret_cast<const float4*>(P.rope_cs + (size_t)(a.off + r) * half + i4));
+            qn[u] = __ldcg(reinterpret_cast<const float4*>(P.rope_sn + (size_t)(a.off + r) * half + i4));
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int idx = et + 128 * (u0 + u);
+        if (idx < n_all) {
+          const int ql = idx / hq, i4 = (idx % hq) * 4;
+          uint2 lo = make_uint2(0u, 0u), hi = make_uint2(0u, 0u);   // rows past the unit's queries stay zero
+          if (idx < n_items) {
+            float x0[4] = {xa[u].x, xa[u].y, xa[u].z, xa[u].w}, x1[4] = {xb[u].x, xb[u].y, xb[u].z, xb[u].w};
+            if (P.rope) {
+              const float cs[4] = {qc[u].x, qc[u].y, qc[u].z, qc[u].w}, sn[4] = {qn[u].x, qn[u].y, qn[u].z, qn[u].w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float r0 = x0[e] * cs[e] - x1[e] * sn[e], r1 = x1[e] * cs[e] + x0[e] * sn[e];
+                x0[e] = r0; x1[e] = r1;
+              }
+            }
+            lo = make_uint2(pack_f16x2(x0[0] * scale, x0[1] * scale), pack_f16x2(x0[2] * scale, x0[3] * scale));
+            hi = make_uint2(pack_f16x2(x1[0] * scale, x1[1] * scale), pack_f16x2(x1[2] * scale, x1[3] * scale));
+          }
+          __half* qd = reinterpret_cast<__half*>(qs + (size_t)ql * pitch);
+          *reinterpret_cast<uint2*>(qd + i4) = lo; *reinterpret_cast<uint2*>(qd + half + i4) = hi;
+        }
       }
     }
-    __half* qd = reinterpret_cast<__half*>(qs + (size_t)ql * pitch);
-    qd[i] = __float2half_rn(x0 * scale);
-    qd[i + half] = __float2half_rn(x1 * scale);
   }
   epi_bar_sync();
 
@@ -944,13 +1006,6 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           const long long tile_first = (long long)tile * p.kblocks, tile_end = tile_first + p.kblocks;
           const long long seg_end = tile_end < kb_end ? tile_end : kb_end;
           const bool whole = (kk0 == 0) && (seg_end == tile_end);
-          W.wait(ctl->acc_full + buf, acc_phase[buf]);
-          ok = group_ok(ctl, et);
-          if (!ok) break;
-          if (tracing && first_seg) { tr[4] = globaltimer_ns(); first_seg = false; }
-          acc_phase[buf] ^= 1;
-          tc_fence_after();
-          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * P.t_box);
           int n_out, n_valid;
           if (p.dual) { n_out = tile * 64 + (m & 63); n_valid = n_out < p.N; }
           else {
@@ -960,16 +1015,33 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const int src_n = (s + 1 < p.n_src ? p.src_col[s + 1] : p.N) - p.src_col[s];
             n_out = p.src_col[s] + in_src; n_valid = in_src < src_n;
           }
-          // old residual values and gain of the first 16 rows, fetched early on the split-tile path
-          // (before the arrival counter is known) so that the last arriver's chain is shorter
-          float xpre[16], gpre = 0.f;
-          bool have_pre = false;
+          // Per-column constants of the epilogue and the old residual values of the first 16 rows
+          // are fetched before the accumulator is waited for: their round trips then overlap the
+          // MMAs instead of extending the chain that ends the phase.  (Nobody else writes this
+          // tile's columns of the residual during the phase.)
+          float xpre[16], gpre = 0.f, un = 0.f, cn = 0.f;
+          const bool have_pre = p.epi == TC_ADD_F32;
+          if (p.norm_in && n_valid) {
+            const int ncol = (p.dual && m >= 64) ? p.N + n_out : n_out;
+            if (p.u) un = p.u[ncol];
+            if (p.c) cn = p.c[ncol];
+          }
+          if (have_pre) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) xpre[j] = (n_valid && j < Tvalid) ? __ldcg(out_f32 + (size_t)j * p.ldo + n_out) : 0.f;
+            gpre = (p.next_g && n_valid) ? p.next_g[n_out] : 0.f;
+          }
+          W.wait(ctl->acc_full + buf, acc_phase[buf]);
+          ok = group_ok(ctl, et);
+          if (!ok) break;
+          if (tracing && first_seg) { tr[4] = globaltimer_ns(); first_seg = false; }
+          acc_phase[buf] ^= 1;
+          tc_fence_after();
+          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * P.t_box);
           unsigned long long* tra = nullptr;   // this CTA's detail slots of the phase trace
           auto finish = [&](int c0, float* v) {
             if (p.norm_in) {
               // fold the normalisation in: y = rstd_t * (acc - mean_t * u[n]) + c[n]
-              const int ncol = (p.dual && m >= 64) ? p.N + n_out : n_out;
-              const float un = (p.u && n_valid) ? p.u[ncol] : 0.f, cn = (p.c && n_valid) ? p.c[ncol] : 0.f;
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
                 const int t = c0 + j;
@@ -1012,7 +1084,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               // residual update; also the next GEMM's operand bf16(x * gain) and this tile's row
               // statistics (mean and centred sum of squares over the tile's columns)
               const bool use_pre = have_pre && c0 == 0;
-              const float gn = use_pre ? gpre : (n_valid ? p.next_g[n_out] : 0.f);
+              const float gn = gpre;
               const int jn = min(16, Tvalid - c0);   // rows of this chunk that exist (uniform)
               // all loads of the old residual values first (predicated, no early exit, so that
               // they are in flight together), then the updates
@@ -1112,12 +1184,6 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             }
             tc_fence_before();
             if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
-            if (p.epi == TC_ADD_F32) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) xpre[j] = (n_valid && j < Tvalid) ? __ldcg(out_f32 + (size_t)j * p.ldo + n_out) : 0.f;
-              gpre = (p.next_g && n_valid) ? p.next_g[n_out] : 0.f;
-              have_pre = true;
-            }
             __threadfence();
             epi_bar_sync();
             if (tra) tra[5] = globaltimer_ns();
