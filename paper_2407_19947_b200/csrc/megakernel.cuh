@@ -99,6 +99,8 @@ struct Params {
 
 constexpr int ATT_CHUNK = 64;
 constexpr int ATT_QBLK = 48;
+constexpr int VT_LD = 132;                      // row pitch (floats) of the epilogue's 16 x 128 exchange tile
+constexpr int MK_XCH_BYTES = 16 * VT_LD * 4;     // the tile itself
 
 struct AttnSmem {   // carved after the GEMM ring: Q block (bf16), K and V chunk tiles (bf16), merge buffer (fp32)
   static __host__ __device__ size_t k_pitch(int hd) { return (size_t)hd * 2 + 16; }
@@ -179,6 +181,14 @@ __device__ __forceinline__ void store_split(bf16* base, size_t idx, size_t lo_of
   base[idx + lo_off] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
+// Four consecutive values as bf16 hi parts and bf16 lo parts (8-byte stores; idx a multiple of 4).
+__device__ __forceinline__ void store_split4(bf16* base, size_t idx, size_t lo_off, float4 v) {
+  const __nv_bfloat162 h01 = __floats2bfloat162_rn(v.x, v.y), h23 = __floats2bfloat162_rn(v.z, v.w);
+  *reinterpret_cast<uint2*>(base + idx) = make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
+  *reinterpret_cast<uint2*>(base + idx + lo_off) =
+      make_uint2(pack_bf16x2(v.x - __low2float(h01), v.y - __high2float(h01)), pack_bf16x2(v.z - __low2float(h23), v.w - __high2float(h23)));
+}
+
 // Sums 32 per-lane values across the warp, all at once: on return lane l holds the warp-wide
 // total of a[l].  Each halving step exchanges the half a lane does not keep (31 shuffles in five
 // dependent steps, instead of 32 separate five-step reductions).
@@ -204,7 +214,7 @@ struct Ctl {
   volatile int last_flag;
   volatile int bcast;
   float rstd[64], mu[64];       // per-row statistics of the current norm_in GEMM phase
-  float red[4][16], red2[4][16], shift[4][16];
+  float gtile[128];             // next operand's gain for the current tile's columns
 };
 
 // Uniform verdict for the 128 compute threads after any of them may have timed out in a wait:
@@ -657,9 +667,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
   const int b_stage_bytes = P.t_box * BK * 2;               // one part (hi or lo) of the activation tile
   const int stage_bytes = A_STAGE_BYTES + 2 * b_stage_bytes;
   uint8_t* tail = smem + (size_t)stages * stage_bytes;
-  float* xch = reinterpret_cast<float*>(tail);
-  Ctl* ctl = reinterpret_cast<Ctl*>(tail + XCH_BYTES);
-  uint8_t* att_smem = tail + XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127);
+  float* vt = reinterpret_cast<float*>(tail);   // epilogue exchange tile [16][VT_LD]
+  Ctl* ctl = reinterpret_cast<Ctl*>(tail + MK_XCH_BYTES);
+  uint8_t* att_smem = tail + MK_XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = gridDim.x, cta = blockIdx.x;
@@ -826,7 +836,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     const int quad = warp & 3;
     const int m = quad * 32 + lane;
     const int et = threadIdx.x - 64;
-    float* red = xch;   // 4 floats of scratch for group sums (xch is free outside SwiGLU epilogues)
+    float* red = vt;    // 4 floats of scratch for group sums (the exchange tile is free outside GEMM epilogues)
     int buf = 0; uint32_t acc_phase[2] = {0, 0};
     uint32_t att_parity = 0;
     bool ok = true;
@@ -1015,11 +1025,27 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const int src_n = (s + 1 < p.n_src ? p.src_col[s + 1] : p.N) - p.src_col[s];
             n_out = p.src_col[s] + in_src; n_valid = in_src < src_n;
           }
-          // Per-column constants of the epilogue and the old residual values of the first 16 rows
-          // are fetched before the accumulator is waited for: their round trips then overlap the
-          // MMAs instead of extending the chain that ends the phase.  (Nobody else writes this
-          // tile's columns of the residual during the phase.)
-          float xpre[16], gpre = 0.f, un = 0.f, cn = 0.f;
+          // First output column of the tile and how many of its columns exist (a tile never
+          // straddles two sources).
+          int n0, ncols;
+          if (p.dual) { n0 = tile * 64; ncols = min(64, p.N - n0); }
+          else {
+            int s = 0, local = tile;
+            while (s + 1 < p.n_src && local >= p.src_tiles[s]) { local -= p.src_tiles[s]; ++s; }
+            const int src_n = (s + 1 < p.n_src ? p.src_col[s + 1] : p.N) - p.src_col[s];
+            n0 = p.src_col[s] + local * BM; ncols = min(BM, src_n - local * BM);
+          }
+          // The epilogue works in two thread mappings: per feature (thread m owns feature m of
+          // the tile, as the accumulator is laid out) for the normalisation fold, then, after a
+          // transpose through shared memory, per row: thread (er, cg) owns row er of a 16-row
+          // chunk and the float4 column groups cg, cg + 8, ... - compact code with vector
+          // accesses.  What the second mapping needs from memory (old residual values of the
+          // first chunk, gains) is fetched here, before the accumulator is waited for, so that
+          // the round trips overlap the MMAs instead of extending the chain that ends the phase.
+          // (Nobody else writes this tile's columns of the residual during the phase.)
+          const int er = et >> 3, cg = et & 7;
+          float4 xq[4];
+          float un = 0.f, cn = 0.f;
           const bool have_pre = p.epi == TC_ADD_F32;
           if (p.norm_in && n_valid) {
             const int ncol = (p.dual && m >= 64) ? p.N + n_out : n_out;
@@ -1028,8 +1054,12 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           }
           if (have_pre) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) xpre[j] = (n_valid && j < Tvalid) ? __ldcg(out_f32 + (size_t)j * p.ldo + n_out) : 0.f;
-            gpre = (p.next_g && n_valid) ? p.next_g[n_out] : 0.f;
+            for (int q = 0; q < 4; ++q) {
+              const int col = (cg + 8 * q) * 4;
+              xq[q] = (er < Tvalid && col < ncols) ? __ldcg(reinterpret_cast<const float4*>(out_f32 + (size_t)er * p.ldo + n0 + col))
+                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            ctl->gtile[m] = (p.next_g && n_valid) ? p.next_g[n_out] : 0.f;   // read after the barriers below
           }
           W.wait(ctl->acc_full + buf, acc_phase[buf]);
           ok = group_ok(ctl, et);
@@ -1048,22 +1078,6 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                 if (t < Tvalid) v[j] = ctl->rstd[t] * (v[j] - ctl->mu[t] * un) + cn;
               }
             }
-            if (p.epi == TC_SWIGLU) {
-              if (m >= 64) {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) xch[(m - 64) * 16 + j] = v[j];
-              }
-              epi_bar_sync();
-              if (m < 64 && n_valid) {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                  const int t = c0 + j;
-                  if (t < Tvalid) store_split(out_act, (size_t)t * p.ldo + n_out, (size_t)P.lo_row * p.ldo, silu_f(v[j]) * xch[m * 16 + j]);
-                }
-              }
-              epi_bar_sync();
-              return;
-            }
             if (p.epi == TC_LMHEAD) {
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
@@ -1080,88 +1094,83 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               }
               return;
             }
-            if (p.epi == TC_ADD_F32 && p.next_g) {
-              // residual update; also the next GEMM's operand bf16(x * gain) and this tile's row
-              // statistics (mean and centred sum of squares over the tile's columns)
-              const bool use_pre = have_pre && c0 == 0;
-              const float gn = gpre;
-              const int jn = min(16, Tvalid - c0);   // rows of this chunk that exist (uniform)
-              // all loads of the old residual values first (predicated, no early exit, so that
-              // they are in flight together), then the updates
-              float xo[16];
+            // transpose: vt[row of the chunk][feature]
 #pragma unroll
-              for (int j = 0; j < 16; ++j)
-                xo[j] = use_pre ? xpre[j] : ((n_valid && j < jn) ? __ldcg(out_f32 + (size_t)(c0 + j) * p.ldo + n_out) : 0.f);
+            for (int j = 0; j < 16; ++j) vt[j * VT_LD + m] = v[j];
+            epi_bar_sync();
+            const int t = c0 + er;
+            const float* vrow = vt + er * VT_LD;
+            if (p.epi == TC_ADD_F32) {
+              // residual update; with a following normalised GEMM also its operand bf16(x * gain)
+              // and this tile's row statistics (count, mean, centred sum of squares)
+              float xn[16];
+              float cnt = 0.f, sum = 0.f;
 #pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                float xn = 0.f;
-                if (n_valid && j < jn) {
-                  const size_t o = (size_t)(c0 + j) * p.ldo + n_out;
-                  xn = xo[j] + v[j];
-                  out_f32[o] = xn;
-                  store_split(P.h, o, (size_t)P.lo_row * p.ldo, xn * gn);
+              for (int q = 0; q < 4; ++q) {
+                const int col = (cg + 8 * q) * 4;
+                const bool on = t < Tvalid && col < ncols;
+                float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (on) {
+                  const float4 v4 = *reinterpret_cast<const float4*>(vrow + col);
+                  const size_t o = (size_t)t * p.ldo + n0 + col;
+                  const float4 x4 = (have_pre && c0 == 0) ? xq[q] : __ldcg(reinterpret_cast<const float4*>(out_f32 + o));
+                  a4 = make_float4(x4.x + v4.x, x4.y + v4.y, x4.z + v4.z, x4.w + v4.w);
+                  *reinterpret_cast<float4*>(out_f32 + o) = a4;
+                  if (p.next_g) {
+                    const float4 g4 = *reinterpret_cast<const float4*>(ctl->gtile + col);
+                    store_split4(P.h, o, (size_t)P.lo_row * p.ldo, make_float4(a4.x * g4.x, a4.y * g4.y, a4.z * g4.z, a4.w * g4.w));
+                  }
+                  cnt += 4.f; sum += (a4.x + a4.y) + (a4.z + a4.w);
                 }
-                v[j] = xn;
+                xn[4 * q] = a4.x; xn[4 * q + 1] = a4.y; xn[4 * q + 2] = a4.z; xn[4 * q + 3] = a4.w;
               }
-              if (tra) tra[6] = globaltimer_ns();
-              // Row statistics of this tile's columns.  Each warp reduces, for its 32 columns, the
-              // sums of d and d*d of all 16 rows at once (d = x minus the warp's first column, a
-              // shift that keeps the subtraction below free of cancellation); one thread per row
-              // then merges the four warps' (mean, M2, count).
-              const int cnt = min(tile_cols, p.N - tile * BM);
-              {
-                float bf[32];
+              if (p.next_g) {
+                float mean = cnt > 0.f ? sum / cnt : 0.f, m2 = 0.f;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                  const float sh = __shfl_sync(0xffffffffu, v[j], 0);
-                  if (lane == 0) ctl->shift[quad][j] = sh;
-                  const float dl = n_valid ? v[j] - sh : 0.f;
-                  bf[j] = dl; bf[16 + j] = dl * dl;
-                }
-                const float tot = warp_multi_sum32(bf, lane);   // lane l: total of bf[l]
-                if (lane < 16) ctl->red[quad][lane] = tot; else ctl->red2[quad][lane - 16] = tot;
-              }
-              epi_bar_sync();
-              if (et < 16 && c0 + et < Tvalid) {
-                float mean = 0.f, m2 = 0.f, n = 0.f;
+                for (int q = 0; q < 4; ++q) {
+                  if ((float)(4 * q) < cnt) {   // a thread's valid groups come first (columns ascend with q)
 #pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                  const float nw = (float)max(0, min(32, cnt - 32 * w));
-                  if (nw > 0.f) {
-                    const float sd = ctl->red[w][et];
-                    const float mw = ctl->shift[w][et] + sd / nw;
-                    const float m2w = fmaxf(ctl->red2[w][et] - sd * sd / nw, 0.f);
-                    const float dm = mw - mean, nn = n + nw;
-                    m2 += m2w + dm * dm * (n * nw / nn);
-                    mean += dm * (nw / nn);
-                    n = nn;
+                    for (int e = 0; e < 4; ++e) { const float dl = xn[4 * q + e] - mean; m2 += dl * dl; }
                   }
                 }
-                P.stats[(size_t)(c0 + et) * P.stat_tiles + tile] = make_float4(mean, m2, (float)cnt, 0.f);
+                // merge the eight threads of the row, pairwise and symmetrically
+#pragma unroll
+                for (int o = 1; o < 8; o <<= 1) {
+                  const float c2 = __shfl_xor_sync(0xffffffffu, cnt, o), mean2 = __shfl_xor_sync(0xffffffffu, mean, o),
+                              m22 = __shfl_xor_sync(0xffffffffu, m2, o);
+                  const float tot = cnt + c2;
+                  if (tot > 0.f) {
+                    const float delta = mean2 - mean;
+                    const float mm = (cnt * mean + c2 * mean2) / tot;
+                    m2 = m2 + m22 + delta * delta * cnt * c2 / tot;
+                    mean = mm; cnt = tot;
+                  }
+                }
+                if (cg == 0 && t < Tvalid) P.stats[(size_t)t * P.stat_tiles + tile] = make_float4(mean, m2, cnt, 0.f);
               }
-              if (tra) tra[7] = globaltimer_ns();
-              epi_bar_sync();
-              return;
-            }
-            if (!n_valid) return;
-            if (p.epi == TC_ADD_F32) {
-              float xo[16];
+            } else if (p.epi == TC_SWIGLU) {
 #pragma unroll
-              for (int j = 0; j < 16; ++j)
-                xo[j] = (have_pre && c0 == 0) ? xpre[j] : ((c0 + j < Tvalid) ? __ldcg(out_f32 + (size_t)(c0 + j) * p.ldo + n_out) : 0.f);
+              for (int q = 0; q < 2; ++q) {
+                const int col = (cg + 8 * q) * 4;
+                if (t < Tvalid && col < ncols) {
+                  const float4 g4 = *reinterpret_cast<const float4*>(vrow + col), u4 = *reinterpret_cast<const float4*>(vrow + 64 + col);
+                  store_split4(out_act, (size_t)t * p.ldo + n0 + col, (size_t)P.lo_row * p.ldo,
+                               make_float4(silu_f(g4.x) * u4.x, silu_f(g4.y) * u4.y, silu_f(g4.z) * u4.z, silu_f(g4.w) * u4.w));
+                }
+              }
+            } else {
 #pragma unroll
-              for (int j = 0; j < 16; ++j) if (c0 + j < Tvalid) out_f32[(size_t)(c0 + j) * p.ldo + n_out] = xo[j] + v[j];
-              return;
-            }
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int t = c0 + j;
-              if (t < Tvalid) {
-                const size_t o = (size_t)t * p.ldo + n_out;
-                if (p.epi == TC_STORE_F32) out_f32[o] = v[j];
-                else store_split(out_act, o, (size_t)P.lo_row * p.ldo, gelu_erf(v[j]));
+              for (int q = 0; q < 4; ++q) {
+                const int col = (cg + 8 * q) * 4;
+                if (t < Tvalid && col < ncols) {
+                  const float4 v4 = *reinterpret_cast<const float4*>(vrow + col);
+                  const size_t o = (size_t)t * p.ldo + n0 + col;
+                  if (p.epi == TC_STORE_F32) *reinterpret_cast<float4*>(out_f32 + o) = v4;
+                  else store_split4(out_act, o, (size_t)P.lo_row * p.ldo, make_float4(gelu_erf(v4.x), gelu_erf(v4.y), gelu_erf(v4.z), gelu_erf(v4.w)));
+                }
               }
             }
+            epi_bar_sync();   // the exchange tile is reused by the next chunk
           };
           // A whole tile is finished straight from TMEM.  A split tile's segment goes to this CTA's
           // partial slot; whichever CTA arrives last at the tile's counter sums the partials in
@@ -1297,7 +1306,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
 }
 
 inline size_t smem_bytes(int t_box, int stages, int hd) {
-  return 1024 + (size_t)stages * (A_STAGE_BYTES + (size_t)2 * t_box * BK * 2) + XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127) +
+  return 1024 + (size_t)stages * (A_STAGE_BYTES + (size_t)2 * t_box * BK * 2) + MK_XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127) +
          AttnSmem::bytes(hd) + 64;
 }
 inline int pick_stages(int t_box, int hd) {
