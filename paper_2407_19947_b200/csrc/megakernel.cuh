@@ -214,7 +214,7 @@ struct Ctl {
   volatile int last_flag;
   volatile int bcast;
   float rstd[64], mu[64];       // per-row statistics of the current norm_in GEMM phase
-  float gtile[128];             // next operand's gain for the current tile's columns
+  alignas(16) float gtile[128]; // next operand's gain for the current tile's columns
 };
 
 // Uniform verdict for the 128 compute threads after any of them may have timed out in a wait:
