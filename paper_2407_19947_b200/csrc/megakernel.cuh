@@ -88,6 +88,7 @@ struct Params {
   float* logits;            // optional dump
   int* target_tokens; int* accept_len; int commit; int* draft_out;
   // scratch
+  unsigned long long* seg_flags;   // one flag per CTA: the tag of the phase whose partial its slot holds
   float* partial; int* counters;
   float* attn_part;         // [units][QBLK][hd + 4]: O, running max, running sum, pad
   int attn_part_units;
@@ -134,6 +135,9 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
   unsigned long long v;
   asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
   return v;
+}
+__device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 __device__ __forceinline__ void red_release_add_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
@@ -215,6 +219,8 @@ struct Ctl {
   volatile int bcast;
   float rstd[64], mu[64];       // per-row statistics of the current norm_in GEMM phase
   alignas(16) float gtile[128]; // next operand's gain for the current tile's columns
+  alignas(16) float utile[128]; // folded-normalisation constants u[n], c[n] of the tile's columns
+  alignas(16) float ctile[128];
 };
 
 // Uniform verdict for the 128 compute threads after any of them may have timed out in a wait:
@@ -1007,26 +1013,26 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           }
           epi_bar_sync();
         }
-        const int tile_cols = BM;
         if (tracing) tr[3] = globaltimer_ns();
         bool first_seg = true;
         long long kb = kb_begin;
+        const unsigned long long seg_tag = P.bar_base + (unsigned long long)ph + 1ull;   // unique per launch and phase
+        const unsigned tot32 = (unsigned)total, ge32 = (unsigned)Ge;
+        auto rb = [&](unsigned c) { return (tot32 * c) / ge32; };   // total * Ge < 2^32, checked on the host
+        const int er = et >> 3, cg = et & 7;
         while (kb < kb_end && ok) {
           const int tile = (int)(kb / p.kblocks), kk0 = (int)(kb % p.kblocks);
           const long long tile_first = (long long)tile * p.kblocks, tile_end = tile_first + p.kblocks;
           const long long seg_end = tile_end < kb_end ? tile_end : kb_end;
-          const bool whole = (kk0 == 0) && (seg_end == tile_end);
-          int n_out, n_valid;
-          if (p.dual) { n_out = tile * 64 + (m & 63); n_valid = n_out < p.N; }
-          else {
-            int s = 0, local = tile;
-            while (s + 1 < p.n_src && local >= p.src_tiles[s]) { local -= p.src_tiles[s]; ++s; }
-            const int in_src = local * BM + m;
-            const int src_n = (s + 1 < p.n_src ? p.src_col[s + 1] : p.N) - p.src_col[s];
-            n_out = p.src_col[s] + in_src; n_valid = in_src < src_n;
-          }
-          // First output column of the tile and how many of its columns exist (a tile never
-          // straddles two sources).
+          // The CTA that owns a tile's first k-block finishes the tile; a CTA whose segment starts
+          // inside a tile (always the first segment of its range, so at most one per phase) parks
+          // the partial sums in its slot and raises its flag.  The finisher's segment is the
+          // last thing its range holds, so it reaches the tile when the others are done or
+          // nearly so, and it adds their partials to its own in k order - a fixed order: results
+          // do not depend on timing.
+          const bool finisher = kk0 == 0, whole = finisher && seg_end == tile_end;
+          // first output column of the tile and how many of its columns exist (a tile never
+          // straddles two sources)
           int n0, ncols;
           if (p.dual) { n0 = tile * 64; ncols = min(64, p.N - n0); }
           else {
@@ -1035,155 +1041,44 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const int src_n = (s + 1 < p.n_src ? p.src_col[s + 1] : p.N) - p.src_col[s];
             n0 = p.src_col[s] + local * BM; ncols = min(BM, src_n - local * BM);
           }
-          // The epilogue works in two thread mappings: per feature (thread m owns feature m of
-          // the tile, as the accumulator is laid out) for the normalisation fold, then, after a
-          // transpose through shared memory, per row: thread (er, cg) owns row er of a 16-row
-          // chunk and the float4 column groups cg, cg + 8, ... - compact code with vector
-          // accesses.  What the second mapping needs from memory (old residual values of the
-          // first chunk, gains) is fetched here, before the accumulator is waited for, so that
+          // The epilogue runs in a per-row mapping: thread (er, cg) owns row er of a 16-row chunk
+          // and the float4 column groups cg, cg + 8, cg + 16, cg + 24 of the tile (for a gate/up
+          // tile: two gate groups and the matching two up groups) - compact code with vector
+          // accesses.  What it needs from memory (per-column constants, the old residual values
+          // of the first chunk) is fetched here, before the accumulator is waited for, so that
           // the round trips overlap the MMAs instead of extending the chain that ends the phase.
           // (Nobody else writes this tile's columns of the residual during the phase.)
-          const int er = et >> 3, cg = et & 7;
           float4 xq[4];
-          float un = 0.f, cn = 0.f;
           const bool have_pre = p.epi == TC_ADD_F32;
-          if (p.norm_in && n_valid) {
-            const int ncol = (p.dual && m >= 64) ? p.N + n_out : n_out;
-            if (p.u) un = p.u[ncol];
-            if (p.c) cn = p.c[ncol];
-          }
-          if (have_pre) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const int col = (cg + 8 * q) * 4;
-              xq[q] = (er < Tvalid && col < ncols) ? __ldcg(reinterpret_cast<const float4*>(out_f32 + (size_t)er * p.ldo + n0 + col))
-                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+          if (finisher) {
+            const int mc = p.dual ? (m & 63) : m;
+            const bool m_on = mc < ncols;
+            if (p.norm_in) {
+              const int ncol = (p.dual && m >= 64) ? p.N + n0 + mc : n0 + mc;
+              ctl->utile[m] = (p.u && m_on) ? p.u[ncol] : 0.f;
+              ctl->ctile[m] = (p.c && m_on) ? p.c[ncol] : 0.f;
             }
-            ctl->gtile[m] = (p.next_g && n_valid) ? p.next_g[n_out] : 0.f;   // read after the barriers below
+            if (have_pre) {
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const int col = (cg + 8 * q) * 4;
+                xq[q] = (er < Tvalid && col < ncols) ? __ldcg(reinterpret_cast<const float4*>(out_f32 + (size_t)er * p.ldo + n0 + col))
+                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+              }
+              ctl->gtile[m] = (p.next_g && m_on) ? p.next_g[n0 + mc] : 0.f;
+            }
           }
           W.wait(ctl->acc_full + buf, acc_phase[buf]);
-          ok = group_ok(ctl, et);
+          ok = group_ok(ctl, et);   // (its barriers also publish the staged constants)
           if (!ok) break;
           if (tracing && first_seg) { tr[4] = globaltimer_ns(); first_seg = false; }
           acc_phase[buf] ^= 1;
           tc_fence_after();
           const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * P.t_box);
-          unsigned long long* tra = nullptr;   // this CTA's detail slots of the phase trace
-          auto finish = [&](int c0, float* v) {
-            if (p.norm_in) {
-              // fold the normalisation in: y = rstd_t * (acc - mean_t * u[n]) + c[n]
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const int t = c0 + j;
-                if (t < Tvalid) v[j] = ctl->rstd[t] * (v[j] - ctl->mu[t] * un) + cn;
-              }
-            }
-            if (p.epi == TC_LMHEAD) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const int t = c0 + j;
-                if (t >= Tvalid) break;
-                if (out_f32 && n_valid) out_f32[(size_t)t * p.ldo + n_out] = v[j];
-                unsigned long long key = n_valid ? argmax_key(v[j], (uint32_t)n_out) : 0ull;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                  const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
-                  key = other > key ? other : key;
-                }
-                if (lane == 0 && key) atomicMax(keys + t, key);
-              }
-              return;
-            }
-            // transpose: vt[row of the chunk][feature]
-#pragma unroll
-            for (int j = 0; j < 16; ++j) vt[j * VT_LD + m] = v[j];
-            epi_bar_sync();
-            const int t = c0 + er;
-            const float* vrow = vt + er * VT_LD;
-            if (p.epi == TC_ADD_F32) {
-              // residual update; with a following normalised GEMM also its operand bf16(x * gain)
-              // and this tile's row statistics (count, mean, centred sum of squares)
-              float xn[16];
-              float cnt = 0.f, sum = 0.f;
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const int col = (cg + 8 * q) * 4;
-                const bool on = t < Tvalid && col < ncols;
-                float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (on) {
-                  const float4 v4 = *reinterpret_cast<const float4*>(vrow + col);
-                  const size_t o = (size_t)t * p.ldo + n0 + col;
-                  const float4 x4 = (have_pre && c0 == 0) ? xq[q] : __ldcg(reinterpret_cast<const float4*>(out_f32 + o));
-                  a4 = make_float4(x4.x + v4.x, x4.y + v4.y, x4.z + v4.z, x4.w + v4.w);
-                  *reinterpret_cast<float4*>(out_f32 + o) = a4;
-                  if (p.next_g) {
-                    const float4 g4 = *reinterpret_cast<const float4*>(ctl->gtile + col);
-                    store_split4(P.h, o, (size_t)P.lo_row * p.ldo, make_float4(a4.x * g4.x, a4.y * g4.y, a4.z * g4.z, a4.w * g4.w));
-                  }
-                  cnt += 4.f; sum += (a4.x + a4.y) + (a4.z + a4.w);
-                }
-                xn[4 * q] = a4.x; xn[4 * q + 1] = a4.y; xn[4 * q + 2] = a4.z; xn[4 * q + 3] = a4.w;
-              }
-              if (p.next_g) {
-                float mean = cnt > 0.f ? sum / cnt : 0.f, m2 = 0.f;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  if ((float)(4 * q) < cnt) {   // a thread's valid groups come first (columns ascend with q)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) { const float dl = xn[4 * q + e] - mean; m2 += dl * dl; }
-                  }
-                }
-                // merge the eight threads of the row, pairwise and symmetrically
-#pragma unroll
-                for (int o = 1; o < 8; o <<= 1) {
-                  const float c2 = __shfl_xor_sync(0xffffffffu, cnt, o), mean2 = __shfl_xor_sync(0xffffffffu, mean, o),
-                              m22 = __shfl_xor_sync(0xffffffffu, m2, o);
-                  const float tot = cnt + c2;
-                  if (tot > 0.f) {
-                    const float delta = mean2 - mean;
-                    const float mm = (cnt * mean + c2 * mean2) / tot;
-                    m2 = m2 + m22 + delta * delta * cnt * c2 / tot;
-                    mean = mm; cnt = tot;
-                  }
-                }
-                if (cg == 0 && t < Tvalid) P.stats[(size_t)t * P.stat_tiles + tile] = make_float4(mean, m2, cnt, 0.f);
-              }
-            } else if (p.epi == TC_SWIGLU) {
-#pragma unroll
-              for (int q = 0; q < 2; ++q) {
-                const int col = (cg + 8 * q) * 4;
-                if (t < Tvalid && col < ncols) {
-                  const float4 g4 = *reinterpret_cast<const float4*>(vrow + col), u4 = *reinterpret_cast<const float4*>(vrow + 64 + col);
-                  store_split4(out_act, (size_t)t * p.ldo + n0 + col, (size_t)P.lo_row * p.ldo,
-                               make_float4(silu_f(g4.x) * u4.x, silu_f(g4.y) * u4.y, silu_f(g4.z) * u4.z, silu_f(g4.w) * u4.w));
-                }
-              }
-            } else {
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const int col = (cg + 8 * q) * 4;
-                if (t < Tvalid && col < ncols) {
-                  const float4 v4 = *reinterpret_cast<const float4*>(vrow + col);
-                  const size_t o = (size_t)t * p.ldo + n0 + col;
-                  if (p.epi == TC_STORE_F32) *reinterpret_cast<float4*>(out_f32 + o) = v4;
-                  else store_split4(out_act, o, (size_t)P.lo_row * p.ldo, make_float4(gelu_erf(v4.x), gelu_erf(v4.y), gelu_erf(v4.z), gelu_erf(v4.w)));
-                }
-              }
-            }
-            epi_bar_sync();   // the exchange tile is reused by the next chunk
-          };
-          // A whole tile is finished straight from TMEM.  A split tile's segment goes to this CTA's
-          // partial slot; whichever CTA arrives last at the tile's counter sums the partials in
-          // k order (a fixed order: results do not depend on timing) and finishes the tile.
-          bool last = false;
-          unsigned first_c = 0, last_c = 0;
-          const unsigned tot32 = (unsigned)total, ge32 = (unsigned)Ge, tf32 = (unsigned)tile_first, te32 = (unsigned)tile_end;
-          auto rb = [&](unsigned c) { return (tot32 * c) / ge32; };   // total * Ge < 2^32, checked on the host
-          if (!whole) {
-            const int slot = 2 * cta + (kb == kb_begin ? 0 : 1);
-            tra = (P.trace && et == 0) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
+          unsigned long long* tra = (P.trace && et == 0 && !whole) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
+          if (!finisher) {
             if (tra) tra[4] = globaltimer_ns();
-            float* mine = P.partial + (size_t)slot * P.t_box * BM;
+            float* mine = P.partial + (size_t)cta * P.t_box * BM;
             for (int c0 = 0; c0 < Tvalid; c0 += 16) {   // only rows that exist
               float v[16];
               tmem_ld16(taddr + (uint32_t)c0, v);
@@ -1193,66 +1088,184 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             }
             tc_fence_before();
             if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
-            __threadfence();
             epi_bar_sync();
+            // release: cumulative over the group's stores, which the barrier ordered before it
+            if (et == 0) st_release_u64(P.seg_flags + cta, seg_tag);
             if (tra) tra[5] = globaltimer_ns();
-            // CTAs whose ranges touch this tile
-            first_c = (tf32 * ge32) / tot32;
-            while (rb(first_c + 1) <= tf32) ++first_c;
-            while (first_c > 0 && rb(first_c) > tf32) --first_c;
-            last_c = first_c;
-            while (last_c + 1 < ge32 && rb(last_c + 1) < te32) ++last_c;
-            const int nseg = (int)(last_c - first_c) + 1;
-            if (et == 0) {
-              const int old = atomicAdd(P.counters + tile, 1);
-              ctl->last_flag = (old == nseg - 1) ? 1 : 0;
-              if (old == nseg - 1) P.counters[tile] = 0;
-            }
-            epi_bar_sync();
-            last = ctl->last_flag != 0;
-            epi_bar_sync();
-            if (last) {
-              if (tra) tra[1] = globaltimer_ns();
-              __threadfence();
-            }
-          }
-          if (whole || last) {
+          } else {
+            unsigned last_c = (unsigned)cta;   // CTAs cta + 1 .. last_c hold the tile's other segments
+            if (!whole) while (last_c + 1 < ge32 && rb(last_c + 1) < (unsigned)tile_end) ++last_c;
             for (int c0 = 0; c0 < Tvalid; c0 += 16) {
-              float v[16];
-              if (whole) {
+              {
+                float v[16];
                 tmem_ld16(taddr + (uint32_t)c0, v);
+                if (c0 + 16 >= Tvalid) {   // accumulator drained: the MMA warp may reuse it
+                  tc_fence_before();
+                  if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) vt[j * VT_LD + m] = v[j];
+              }
+              if (!whole && c0 == 0) {
+                if (tra) tra[1] = globaltimer_ns();
+                if (et < 32) {
+                  // one lane per other segment: wait (bounded) until its flag carries this phase's tag
+                  const long long t0 = clock64();
+                  bool all_set;
+                  do {
+                    bool mine_set = true;
+                    for (unsigned cc = (unsigned)cta + 1 + (unsigned)lane; cc <= last_c; cc += 32)
+                      if (ld_acquire_u64(P.seg_flags + cc) != seg_tag) mine_set = false;
+                    all_set = __all_sync(0xffffffffu, mine_set);
+                    if (!all_set) {
+                      bool give_up = false;
+                      if (lane == 0) give_up = W.poll_abort(t0);
+                      if (__shfl_sync(0xffffffffu, give_up ? 1 : 0, 0)) break;
+                    }
+                  } while (!all_set);
+                  if (lane == 0 && !all_set) ctl->abort_flag = 1;
+                }
+                ok = group_ok(ctl, et);   // also orders the other threads' partial reads after the acquires
+                if (tra) tra[2] = globaltimer_ns();
               } else {
-                const int jn = min(16, Tvalid - c0);
+                epi_bar_sync();
+              }
+              if (ok) {
+                const int t = c0 + er;
+                const bool row_on = t < Tvalid;
+                const float* vrow = vt + er * VT_LD;
+                float4 a[4];
+                bool on[4];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] = 0.f;
-                // four segments' loads are issued together; the additions stay in k order
-                for (unsigned c = first_c; c <= last_c; c += 4) {
-                  float tmp[4][16];
+                for (int q = 0; q < 4; ++q) {
+                  const int col = (cg + 8 * q) * 4;
+                  on[q] = row_on && (p.dual ? (col & 63) < ncols : col < ncols);
+                  a[q] = on[q] ? *reinterpret_cast<const float4*>(vrow + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                if (!whole) {
+                  // the other segments' partial sums: six segments' loads in flight together, the
+                  // additions in k order
+                  for (unsigned c = (unsigned)cta + 1; c <= last_c; c += 6) {
+                    float4 tmp[6][4];
 #pragma unroll
-                  for (int u = 0; u < 4; ++u) {
-                    const unsigned cc = c + u;
-                    const bool on = cc <= last_c;
-                    const int sl = 2 * (int)cc + (rb(cc) >= tf32 ? 0 : 1);
-                    const float* part = P.partial + (size_t)(on ? sl : 0) * P.t_box * BM;
+                    for (int u = 0; u < 6; ++u) {
+                      const float* part = P.partial + ((size_t)min(c + u, last_c) * P.t_box + (row_on ? t : 0)) * BM;
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) tmp[u][j] = (on && j < jn) ? __ldcg(part + (size_t)(c0 + j) * BM + m) : 0.f;
-                  }
+                      for (int q = 0; q < 4; ++q)
+                        tmp[u][q] = (on[q] && c + u <= last_c) ? __ldcg(reinterpret_cast<const float4*>(part + (cg + 8 * q) * 4))
+                                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
 #pragma unroll
-                  for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < 6; ++u) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] += tmp[u][j];
+                      for (int q = 0; q < 4; ++q) { a[q].x += tmp[u][q].x; a[q].y += tmp[u][q].y; a[q].z += tmp[u][q].z; a[q].w += tmp[u][q].w; }
+                    }
                   }
                 }
-                if (tra) { asm volatile("" :: "f"(v[0]), "f"(v[1])); tra[2] = globaltimer_ns(); }
+                if (p.norm_in && row_on) {
+                  // fold the normalisation in: y = rstd_t * (acc - mean_t * u[n]) + c[n]
+                  const float rs = ctl->rstd[t], mu = ctl->mu[t];
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    const float4 u4 = *reinterpret_cast<const float4*>(ctl->utile + (cg + 8 * q) * 4);
+                    const float4 c4 = *reinterpret_cast<const float4*>(ctl->ctile + (cg + 8 * q) * 4);
+                    a[q].x = rs * (a[q].x - mu * u4.x) + c4.x; a[q].y = rs * (a[q].y - mu * u4.y) + c4.y;
+                    a[q].z = rs * (a[q].z - mu * u4.z) + c4.z; a[q].w = rs * (a[q].w - mu * u4.w) + c4.w;
+                  }
+                }
+                if (p.epi == TC_ADD_F32) {
+                  // residual update; with a following normalised GEMM also its operand bf16(x * gain)
+                  // and this tile's row statistics (count, mean, centred sum of squares)
+                  float cnt = 0.f, sum = 0.f;
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    if (on[q]) {
+                      const int col = (cg + 8 * q) * 4;
+                      const size_t o = (size_t)t * p.ldo + n0 + col;
+                      const float4 x4 = c0 == 0 ? xq[q] : __ldcg(reinterpret_cast<const float4*>(out_f32 + o));
+                      a[q] = make_float4(x4.x + a[q].x, x4.y + a[q].y, x4.z + a[q].z, x4.w + a[q].w);
+                      *reinterpret_cast<float4*>(out_f32 + o) = a[q];
+                      if (p.next_g) {
+                        const float4 g4 = *reinterpret_cast<const float4*>(ctl->gtile + col);
+                        store_split4(P.h, o, (size_t)P.lo_row * p.ldo, make_float4(a[q].x * g4.x, a[q].y * g4.y, a[q].z * g4.z, a[q].w * g4.w));
+                      }
+                      cnt += 4.f; sum += (a[q].x + a[q].y) + (a[q].z + a[q].w);
+                    }
+                  }
+                  if (p.next_g) {
+                    float mean = cnt > 0.f ? sum / cnt : 0.f, m2 = 0.f;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                      if (on[q]) {
+                        const float d0 = a[q].x - mean, d1 = a[q].y - mean, d2 = a[q].z - mean, d3 = a[q].w - mean;
+                        m2 += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+                      }
+                    }
+                    // merge the eight threads of the row, pairwise and symmetrically
+#pragma unroll
+                    for (int o = 1; o < 8; o <<= 1) {
+                      const float c2 = __shfl_xor_sync(0xffffffffu, cnt, o), mean2 = __shfl_xor_sync(0xffffffffu, mean, o),
+                                  m22 = __shfl_xor_sync(0xffffffffu, m2, o);
+                      const float tot = cnt + c2;
+                      if (tot > 0.f) {
+                        const float delta = mean2 - mean;
+                        const float mm = (cnt * mean + c2 * mean2) / tot;
+                        m2 = m2 + m22 + delta * delta * cnt * c2 / tot;
+                        mean = mm; cnt = tot;
+                      }
+                    }
+                    if (cg == 0 && row_on) P.stats[(size_t)t * P.stat_tiles + tile] = make_float4(mean, m2, cnt, 0.f);
+                  }
+                } else if (p.epi == TC_SWIGLU) {
+#pragma unroll
+                  for (int q = 0; q < 2; ++q) {
+                    if (on[q]) {
+                      const float4 g4 = a[q], u4 = a[q + 2];
+                      store_split4(out_act, (size_t)t * p.ldo + n0 + (cg + 8 * q) * 4, (size_t)P.lo_row * p.ldo,
+                                   make_float4(silu_f(g4.x) * u4.x, silu_f(g4.y) * u4.y, silu_f(g4.z) * u4.z, silu_f(g4.w) * u4.w));
+                    }
+                  }
+                } else if (p.epi == TC_LMHEAD) {
+                  // logits (optional) and the row's running argmax; the vocabulary need not be a
+                  // multiple of 4, so validity and stores are per element
+                  unsigned long long key = 0ull;
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    const int col = (cg + 8 * q) * 4;
+                    const float e4[4] = {a[q].x, a[q].y, a[q].z, a[q].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                      if (row_on && col + e < ncols) {
+                        if (out_f32) out_f32[(size_t)t * p.ldo + n0 + col + e] = e4[e];
+                        const unsigned long long k2 = argmax_key(e4[e], (uint32_t)(n0 + col + e));
+                        key = k2 > key ? k2 : key;
+                      }
+                    }
+                  }
+#pragma unroll
+                  for (int o = 1; o < 8; o <<= 1) {
+                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+                    key = other > key ? other : key;
+                  }
+                  if (cg == 0 && key) atomicMax(keys + t, key);
+                } else {
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    if (on[q]) {
+                      const size_t o = (size_t)t * p.ldo + n0 + (cg + 8 * q) * 4;
+                      if (p.epi == TC_STORE_F32) *reinterpret_cast<float4*>(out_f32 + o) = a[q];
+                      else store_split4(out_act, o, (size_t)P.lo_row * p.ldo,
+                                        make_float4(gelu_erf(a[q].x), gelu_erf(a[q].y), gelu_erf(a[q].z), gelu_erf(a[q].w)));
+                    }
+                  }
+                }
               }
-              finish(c0, v);
+              epi_bar_sync();   // the exchange tile is reused by the next chunk
+              if (!ok) break;
             }
-            if (!whole && tra) tra[3] = globaltimer_ns();
+            if (tra) tra[3] = globaltimer_ns();
           }
-          if (whole) {
-            tc_fence_before();
-            if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
-          }
+          if (!ok) break;
           buf ^= 1;
           kb = seg_end;
         }
