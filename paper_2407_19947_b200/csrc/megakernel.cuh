@@ -381,7 +381,8 @@ __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
 // in warp order through a small shared buffer - a fixed order - and the block's result is either
 // final (the unit saw every visible position) or parked for the combine phase.
 __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot,
-                          uint8_t* att_smem, Ctl* ctl, uint32_t& att_parity, const Waiter& W, int et, bool& ok) {
+                          uint8_t* att_smem, Ctl* ctl, uint32_t& att_parity, const Waiter& W, int et, bool& ok,
+                          unsigned long long* tra) {
   const int hd = P.hd, G = P.Hq / P.Hkv, nkv = P.Hkv * hd, nq = P.Hq * hd, nqkv = nq + 2 * nkv;
   const int lane = et & 31, w = et >> 5, g = lane >> 2, t4 = lane & 3;
   const int Q = a.R * G;
@@ -485,7 +486,9 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   };
 
   // the first chunk's copies fly while the queries are rotated
+  if (tra) tra[1] = globaltimer_ns();
   stage_issue(c_begin);
+  if (tra) tra[2] = globaltimer_ns();
   // queries of this block: query index q -> row r = q / G, head = kvh * G + q % G
   {
     // two items' loads in flight together (at most six items of four column pairs per thread
@@ -533,7 +536,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     }
   }
   epi_bar_sync();
-
+  if (tra) tra[3] = globaltimer_ns();
 
   // Warp w owns query block (MMA M tile) w of the unit and walks the chunk's four 16-position
   // slices itself, so its softmax state and output accumulators never leave its registers.
@@ -551,6 +554,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     if (c != c_begin) stage_issue(c);
     ok = stage_wait();
     if (!ok) break;
+    if (tra && c == c_begin) tra[4] = globaltimer_ns();
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
     if (active) {
@@ -621,6 +625,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
       }
     }
     epi_bar_sync();   // tile may be overwritten by the next chunk or unit
+    if (tra && c == c_begin) tra[5] = globaltimer_ns();
   }
   if (!ok || !active) return;
 
@@ -862,6 +867,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         if (!ok) break;
       }
 
+      bool gemm_worked = false;
       const bool tracing = P.trace && et == 0 && (cta == 0 || cta == G - 1);
       unsigned long long* tr = tracing ? P.trace + ((size_t)(cta == 0 ? 0 : 1) * P.n_phases + ph) * 8 : nullptr;
       if (tracing) tr[0] = globaltimer_ns();
@@ -885,7 +891,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const int range = rest % a.n_ranges, kvh = rest / a.n_ranges;
             const int slot = u0 + u;
             if (slot < P.attn_part_units)
-              attn_unit(P, p, a, kvh, range, qblk, slot, att_smem, ctl, att_parity, W, et, ok);
+              attn_unit(P, p, a, kvh, range, qblk, slot, att_smem, ctl, att_parity, W, et, ok,
+                        (P.trace && et == 0 && u == first) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr);
           }
           u0 += a.units; g0 += P.Hkv * a.n_qblk;
         }
@@ -968,6 +975,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         const KRange kr = phase_range(total, cta, G, p.ge_max);
         const long long kb_begin = kr.begin, kb_end = kr.end;
         const int Ge = kr.ge;
+        gemm_worked = kb_begin < kb_end;
         const int Tvalid = P.T;
         float* out_f32 = (p.epi == TC_LMHEAD) ? P.logits : reinterpret_cast<float*>(p.out);
         bf16* out_act = reinterpret_cast<bf16*>(p.out);
@@ -1279,9 +1287,12 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       // phases would run ahead and their arrivals would be mistaken for the slower CTAs' ones
       // (one monotonic counter serves all phases).  For a CTA that had GEMM work the wait is
       // already satisfied - its own activation tiles were gated on the same count.
-      __threadfence();
+      // The release below is cumulative: it covers the other compute threads' stores, which the
+      // barrier orders before it.  A CTA that had GEMM work in this phase already knows that
+      // barrier ph-1 completed (its activation tiles were loaded after that), so only idle CTAs
+      // look at the counter.
       fence_proxy_async();   // later TMA (async proxy) reads of these generic-proxy writes
-      if (ph > 0 && p.kind == PH_GEMM) {
+      if (ph > 0 && p.kind == PH_GEMM && !gemm_worked) {
         if (et == 0) ctl->bcast = W.wait_grid(bar_count, P.bar_base + (unsigned long long)ph * G) ? 1 : 0;
         epi_bar_sync();
         ok = ctl->bcast != 0;
