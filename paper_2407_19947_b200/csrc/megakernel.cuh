@@ -669,159 +669,6 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
 }
 
 // ---------------------------------------------------------------------------------------------
-// GEMM epilogue of one 16-row chunk of a tile, in the per-row mapping (thread = row of the
-// chunk x float4 column groups cg, cg + 8, cg + 16, cg + 24).  Deliberately one out-of-line
-// copy, written as straight-line code in which only the memory accesses are predicated: a CTA
-// runs it once per phase at the very end of the phase's critical path, where every instruction
-// cache miss counts, and a dry pass (row_on = false, no segments) executed while the MMAs are
-// still running fetches the same instructions ahead of time.
-// ---------------------------------------------------------------------------------------------
-struct EpiArgs {
-  int t, ncols, n0, tile, cg;
-  bool row_on, first_chunk;
-  unsigned seg_first, seg_last;     // CTAs whose partial sums are added (none if seg_first > seg_last)
-  float* out_f32; bf16* out_act; unsigned long long* keys;
-};
-
-__device__ __noinline__ void epilogue_rows(const Params& P, const Phase& p, Ctl* ctl, const float* vrow, const EpiArgs& ea,
-                                           const float4* xq) {
-  const int t = ea.t, cg = ea.cg, ncols = ea.ncols, n0 = ea.n0;
-  const bool row_on = ea.row_on;
-  const int tr = row_on ? t : 0;   // a row that exists, for addresses that are formed but not used
-  float4 a[4];
-  bool on[4];
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int col = (cg + 8 * q) * 4;
-    on[q] = row_on && (p.dual ? (col & 63) < ncols : col < ncols);
-    a[q] = on[q] ? *reinterpret_cast<const float4*>(vrow + col) : make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  // the other segments' partial sums: six segments' loads in flight together, the additions in
-  // k order (a dry pass makes one round with every load switched off)
-  for (unsigned c = ea.seg_first; c <= ea.seg_last || (!row_on && c == ea.seg_first && ea.seg_first > ea.seg_last); c += 6) {
-    float4 tmp[6][4];
-#pragma unroll
-    for (int u = 0; u < 6; ++u) {
-      const bool seg_on = c + u <= ea.seg_last;
-      const float* part = P.partial + ((size_t)(seg_on ? c + u : 0) * P.t_box + tr) * BM;
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        tmp[u][q] = (on[q] && seg_on) ? __ldcg(reinterpret_cast<const float4*>(part + (cg + 8 * q) * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-#pragma unroll
-    for (int u = 0; u < 6; ++u) {
-#pragma unroll
-      for (int q = 0; q < 4; ++q) { a[q].x += tmp[u][q].x; a[q].y += tmp[u][q].y; a[q].z += tmp[u][q].z; a[q].w += tmp[u][q].w; }
-    }
-    if (!row_on) break;
-  }
-  if (p.norm_in) {
-    // fold the normalisation in: y = rstd_t * (acc - mean_t * u[n]) + c[n]
-    const float rs = ctl->rstd[tr], mu = ctl->mu[tr];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const float4 u4 = *reinterpret_cast<const float4*>(ctl->utile + (cg + 8 * q) * 4);
-      const float4 c4 = *reinterpret_cast<const float4*>(ctl->ctile + (cg + 8 * q) * 4);
-      a[q].x = rs * (a[q].x - mu * u4.x) + c4.x; a[q].y = rs * (a[q].y - mu * u4.y) + c4.y;
-      a[q].z = rs * (a[q].z - mu * u4.z) + c4.z; a[q].w = rs * (a[q].w - mu * u4.w) + c4.w;
-    }
-  }
-  if (p.epi == TC_ADD_F32) {
-    // residual update; with a following normalised GEMM also its operand bf16(x * gain) and this
-    // tile's row statistics (count, mean, centred sum of squares)
-    float cnt = 0.f, sum = 0.f;
-    const bool with_next = p.next_g != nullptr;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int col = (cg + 8 * q) * 4;
-      const size_t o = (size_t)tr * p.ldo + n0 + (on[q] ? col : 0);
-      float4 x4 = xq[q];
-      if (!ea.first_chunk) x4 = on[q] ? __ldcg(reinterpret_cast<const float4*>(ea.out_f32 + o)) : make_float4(0.f, 0.f, 0.f, 0.f);
-      a[q] = make_float4(x4.x + a[q].x, x4.y + a[q].y, x4.z + a[q].z, x4.w + a[q].w);
-      if (on[q]) *reinterpret_cast<float4*>(ea.out_f32 + o) = a[q];
-      const float4 g4 = *reinterpret_cast<const float4*>(ctl->gtile + col);
-      const float4 h4 = make_float4(a[q].x * g4.x, a[q].y * g4.y, a[q].z * g4.z, a[q].w * g4.w);
-      const __nv_bfloat162 h01 = __floats2bfloat162_rn(h4.x, h4.y), h23 = __floats2bfloat162_rn(h4.z, h4.w);
-      const uint2 hi = make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
-      const uint2 lo = make_uint2(pack_bf16x2(h4.x - __low2float(h01), h4.y - __high2float(h01)),
-                                  pack_bf16x2(h4.z - __low2float(h23), h4.w - __high2float(h23)));
-      if (on[q] && with_next) {
-        *reinterpret_cast<uint2*>(P.h + o) = hi;
-        *reinterpret_cast<uint2*>(P.h + o + (size_t)P.lo_row * p.ldo) = lo;
-      }
-      const float w = on[q] ? 1.f : 0.f;
-      cnt += 4.f * w; sum += w * ((a[q].x + a[q].y) + (a[q].z + a[q].w));
-    }
-    float mean = sum / fmaxf(cnt, 1.f), m2 = 0.f;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const float d0 = a[q].x - mean, d1 = a[q].y - mean, d2 = a[q].z - mean, d3 = a[q].w - mean;
-      m2 += (on[q] ? 1.f : 0.f) * ((d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3));
-    }
-    // merge the eight threads of the row, pairwise and symmetrically
-#pragma unroll
-    for (int o = 1; o < 8; o <<= 1) {
-      const float c2 = __shfl_xor_sync(0xffffffffu, cnt, o), mean2 = __shfl_xor_sync(0xffffffffu, mean, o),
-                  m22 = __shfl_xor_sync(0xffffffffu, m2, o);
-      const float tot = cnt + c2, inv = 1.f / fmaxf(tot, 1.f);
-      const float delta = mean2 - mean;
-      m2 = m2 + m22 + delta * delta * cnt * c2 * inv;
-      mean = (cnt * mean + c2 * mean2) * inv;
-      cnt = tot;
-    }
-    if (cg == 0 && row_on && with_next) P.stats[(size_t)t * P.stat_tiles + ea.tile] = make_float4(mean, m2, cnt, 0.f);
-  } else if (p.epi == TC_SWIGLU) {
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-      const float4 g4 = a[q], u4 = a[q + 2];
-      const float4 y = make_float4(silu_f(g4.x) * u4.x, silu_f(g4.y) * u4.y, silu_f(g4.z) * u4.z, silu_f(g4.w) * u4.w);
-      const __nv_bfloat162 h01 = __floats2bfloat162_rn(y.x, y.y), h23 = __floats2bfloat162_rn(y.z, y.w);
-      const uint2 hi = make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
-      const uint2 lo = make_uint2(pack_bf16x2(y.x - __low2float(h01), y.y - __high2float(h01)),
-                                  pack_bf16x2(y.z - __low2float(h23), y.w - __high2float(h23)));
-      const size_t o = (size_t)tr * p.ldo + n0 + (on[q] ? (cg + 8 * q) * 4 : 0);
-      if (on[q]) {
-        *reinterpret_cast<uint2*>(ea.out_act + o) = hi;
-        *reinterpret_cast<uint2*>(ea.out_act + o + (size_t)P.lo_row * p.ldo) = lo;
-      }
-    }
-  } else if (p.epi == TC_LMHEAD) {
-    // logits (optional) and the row's running argmax; the vocabulary need not be a multiple of
-    // 4, so validity and stores are per element
-    unsigned long long key = 0ull;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int col = (cg + 8 * q) * 4;
-      const float e4[4] = {a[q].x, a[q].y, a[q].z, a[q].w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (row_on && col + e < ncols) {
-          if (ea.out_f32) ea.out_f32[(size_t)t * p.ldo + n0 + col + e] = e4[e];
-          const unsigned long long k2 = argmax_key(e4[e], (uint32_t)(n0 + col + e));
-          key = k2 > key ? k2 : key;
-        }
-      }
-    }
-#pragma unroll
-    for (int o = 1; o < 8; o <<= 1) {
-      const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
-      key = other > key ? other : key;
-    }
-    if (cg == 0 && key) atomicMax(ea.keys + t, key);
-  } else {
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      if (on[q]) {
-        const size_t o = (size_t)t * p.ldo + n0 + (cg + 8 * q) * 4;
-        if (p.epi == TC_STORE_F32) *reinterpret_cast<float4*>(ea.out_f32 + o) = a[q];
-        else store_split4(ea.out_act, o, (size_t)P.lo_row * p.ldo,
-                          make_float4(gelu_erf(a[q].x), gelu_erf(a[q].y), gelu_erf(a[q].z), gelu_erf(a[q].w)));
-      }
-    }
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ Params P) {
@@ -1229,15 +1076,6 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               ctl->gtile[m] = (p.next_g && m_on) ? p.next_g[n0 + mc] : 0.f;
             }
           }
-          if (finisher && seg_end == kb_end) {
-            // dry pass of the epilogue while the MMAs of the CTA's last segment are still running
-            EpiArgs ea;
-            ea.t = er; ea.row_on = false; ea.first_chunk = true;
-            ea.ncols = ncols; ea.n0 = n0; ea.tile = tile; ea.cg = cg;
-            ea.seg_first = 1; ea.seg_last = 0;
-            ea.out_f32 = out_f32; ea.out_act = out_act; ea.keys = keys;
-            epilogue_rows(P, p, ctl, vt + er * VT_LD, ea, xq);
-          }
           W.wait(ctl->acc_full + buf, acc_phase[buf]);
           ok = group_ok(ctl, et);   // (its barriers also publish the staged constants)
           if (!ok) break;
@@ -1301,12 +1139,134 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                 epi_bar_sync();
               }
               if (ok) {
-                EpiArgs ea;
-                ea.t = c0 + er; ea.row_on = ea.t < Tvalid; ea.first_chunk = c0 == 0;
-                ea.ncols = ncols; ea.n0 = n0; ea.tile = tile; ea.cg = cg;
-                ea.seg_first = (unsigned)cta + 1; ea.seg_last = whole ? (unsigned)cta : last_c;
-                ea.out_f32 = out_f32; ea.out_act = out_act; ea.keys = keys;
-                epilogue_rows(P, p, ctl, vt + er * VT_LD, ea, xq);
+                const int t = c0 + er;
+                const bool row_on = t < Tvalid;
+                const float* vrow = vt + er * VT_LD;
+                float4 a[4];
+                bool on[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const int col = (cg + 8 * q) * 4;
+                  on[q] = row_on && (p.dual ? (col & 63) < ncols : col < ncols);
+                  a[q] = on[q] ? *reinterpret_cast<const float4*>(vrow + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                if (!whole) {
+                  // the other segments' partial sums: six segments' loads in flight together, the
+                  // additions in k order
+                  for (unsigned c = (unsigned)cta + 1; c <= last_c; c += 6) {
+                    float4 tmp[6][4];
+#pragma unroll
+                    for (int u = 0; u < 6; ++u) {
+                      const float* part = P.partial + ((size_t)min(c + u, last_c) * P.t_box + (row_on ? t : 0)) * BM;
+#pragma unroll
+                      for (int q = 0; q < 4; ++q)
+                        tmp[u][q] = (on[q] && c + u <= last_c) ? __ldcg(reinterpret_cast<const float4*>(part + (cg + 8 * q) * 4))
+                                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 6; ++u) {
+#pragma unroll
+                      for (int q = 0; q < 4; ++q) { a[q].x += tmp[u][q].x; a[q].y += tmp[u][q].y; a[q].z += tmp[u][q].z; a[q].w += tmp[u][q].w; }
+                    }
+                  }
+                }
+                if (p.norm_in && row_on) {
+                  // fold the normalisation in: y = rstd_t * (acc - mean_t * u[n]) + c[n]
+                  const float rs = ctl->rstd[t], mu = ctl->mu[t];
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    const float4 u4 = *reinterpret_cast<const float4*>(ctl->utile + (cg + 8 * q) * 4);
+                    const float4 c4 = *reinterpret_cast<const float4*>(ctl->ctile + (cg + 8 * q) * 4);
+                    a[q].x = rs * (a[q].x - mu * u4.x) + c4.x; a[q].y = rs * (a[q].y - mu * u4.y) + c4.y;
+                    a[q].z = rs * (a[q].z - mu * u4.z) + c4.z; a[q].w = rs * (a[q].w - mu * u4.w) + c4.w;
+                  }
+                }
+                if (p.epi == TC_ADD_F32) {
+                  // residual update; with a following normalised GEMM also its operand bf16(x * gain)
+                  // and this tile's row statistics (count, mean, centred sum of squares)
+                  float cnt = 0.f, sum = 0.f;
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    if (on[q]) {
+                      const int col = (cg + 8 * q) * 4;
+                      const size_t o = (size_t)t * p.ldo + n0 + col;
+                      const float4 x4 = c0 == 0 ? xq[q] : __ldcg(reinterpret_cast<const float4*>(out_f32 + o));
+                      a[q] = make_float4(x4.x + a[q].x, x4.y + a[q].y, x4.z + a[q].z, x4.w + a[q].w);
+                      *reinterpret_cast<float4*>(out_f32 + o) = a[q];
+                      if (p.next_g) {
+                        const float4 g4 = *reinterpret_cast<const float4*>(ctl->gtile + col);
+                        store_split4(P.h, o, (size_t)P.lo_row * p.ldo, make_float4(a[q].x * g4.x, a[q].y * g4.y, a[q].z * g4.z, a[q].w * g4.w));
+                      }
+                      cnt += 4.f; sum += (a[q].x + a[q].y) + (a[q].z + a[q].w);
+                    }
+                  }
+                  if (p.next_g) {
+                    float mean = cnt > 0.f ? sum / cnt : 0.f, m2 = 0.f;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                      if (on[q]) {
+                        const float d0 = a[q].x - mean, d1 = a[q].y - mean, d2 = a[q].z - mean, d3 = a[q].w - mean;
+                        m2 += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+                      }
+                    }
+                    // merge the eight threads of the row, pairwise and symmetrically
+#pragma unroll
+                    for (int o = 1; o < 8; o <<= 1) {
+                      const float c2 = __shfl_xor_sync(0xffffffffu, cnt, o), mean2 = __shfl_xor_sync(0xffffffffu, mean, o),
+                                  m22 = __shfl_xor_sync(0xffffffffu, m2, o);
+                      const float tot = cnt + c2;
+                      if (tot > 0.f) {
+                        const float delta = mean2 - mean;
+                        const float mm = (cnt * mean + c2 * mean2) / tot;
+                        m2 = m2 + m22 + delta * delta * cnt * c2 / tot;
+                        mean = mm; cnt = tot;
+                      }
+                    }
+                    if (cg == 0 && row_on) P.stats[(size_t)t * P.stat_tiles + tile] = make_float4(mean, m2, cnt, 0.f);
+                  }
+                } else if (p.epi == TC_SWIGLU) {
+#pragma unroll
+                  for (int q = 0; q < 2; ++q) {
+                    if (on[q]) {
+                      const float4 g4 = a[q], u4 = a[q + 2];
+                      store_split4(out_act, (size_t)t * p.ldo + n0 + (cg + 8 * q) * 4, (size_t)P.lo_row * p.ldo,
+                                   make_float4(silu_f(g4.x) * u4.x, silu_f(g4.y) * u4.y, silu_f(g4.z) * u4.z, silu_f(g4.w) * u4.w));
+                    }
+                  }
+                } else if (p.epi == TC_LMHEAD) {
+                  // logits (optional) and the row's running argmax; the vocabulary need not be a
+                  // multiple of 4, so validity and stores are per element
+                  unsigned long long key = 0ull;
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    const int col = (cg + 8 * q) * 4;
+                    const float e4[4] = {a[q].x, a[q].y, a[q].z, a[q].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                      if (row_on && col + e < ncols) {
+                        if (out_f32) out_f32[(size_t)t * p.ldo + n0 + col + e] = e4[e];
+                        const unsigned long long k2 = argmax_key(e4[e], (uint32_t)(n0 + col + e));
+                        key = k2 > key ? k2 : key;
+                      }
+                    }
+                  }
+#pragma unroll
+                  for (int o = 1; o < 8; o <<= 1) {
+                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+                    key = other > key ? other : key;
+                  }
+                  if (cg == 0 && key) atomicMax(keys + t, key);
+                } else {
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    if (on[q]) {
+                      const size_t o = (size_t)t * p.ldo + n0 + (cg + 8 * q) * 4;
+                      if (p.epi == TC_STORE_F32) *reinterpret_cast<float4*>(out_f32 + o) = a[q];
+                      else store_split4(out_act, o, (size_t)P.lo_row * p.ldo,
+                                        make_float4(gelu_erf(a[q].x), gelu_erf(a[q].y), gelu_erf(a[q].z), gelu_erf(a[q].w)));
+                    }
+                  }
+                }
               }
               epi_bar_sync();   // the exchange tile is reused by the next chunk
               if (!ok) break;
