@@ -503,6 +503,8 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
     {
       mk::Phase& p = gemm(l, b + 0, b + 1, b + 2, 3, r3, false, i_h, d, tc::TC_STORE_F32, ws + L.qkv, nqkv);
       p.norm_in = 1; p.u = aux_ptr(l, 0); p.c = aux_ptr(l, 1);
+      p.qkv_prep = 1;   // q to the query buffer, k and v (fp16) to this layer's cache rows
+      p.kc = M.kpool + (size_t)l * M.kv_layer_bytes; p.vc = M.vpool + (size_t)l * M.kv_layer_bytes;
     }
     simple(mk::PH_ATTN, l, nullptr, M.kpool + (size_t)l * M.kv_layer_bytes, M.vpool + (size_t)l * M.kv_layer_bytes);
     simple(mk::PH_COMBINE, l, nullptr, nullptr, nullptr);
@@ -554,7 +556,8 @@ struct MkCall {
 bool mk_eligible(const stairs_ctx* ctx, const DevModel& M, int T) {
   // (the epilogue's vector stores want every GEMM width but the vocabulary to be a multiple of 4)
   return ctx->use_mk && M.m.n_layers >= 1 && T >= 1 && T <= MK_MAX_ROWS && M.m.head_dim % 16 == 0 && M.m.head_dim <= 128 &&
-         M.m.d_model % 4 == 0 && M.m.d_ff % 4 == 0;
+         M.m.d_model % 4 == 0 && M.m.d_ff % 4 == 0 &&
+         (M.m.pos == 0 || M.m.head_dim == 64 || M.m.head_dim == 128);   // rotation pairs must sit in one thread of the QKV epilogue
 }
 
 int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, int n_logit_rows, const MkCall& c) {
@@ -586,6 +589,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.tok = reinterpret_cast<int*>(ws + L.tok); P.pos = reinterpret_cast<int*>(ws + L.pos); P.req = reinterpret_cast<int*>(ws + L.req);
   P.page_table = reinterpret_cast<int*>(ws + L.page_table); P.page_tokens = ctx->cfg.kv_page_tokens; P.max_pages = L.max_pages;
   P.x = reinterpret_cast<float*>(ws + L.x); P.h = reinterpret_cast<bf16*>(ws + L.h); P.qkv = reinterpret_cast<float*>(ws + L.qkv);
+  P.q16 = reinterpret_cast<__half*>(ws + L.q);
   P.o = reinterpret_cast<bf16*>(ws + L.o); P.ff = reinterpret_cast<bf16*>(ws + L.ff);
   P.lo_row = L.max_rows;
   P.keys = reinterpret_cast<unsigned long long*>(ws + L.keys); P.n_keys = L.max_rows;

@@ -51,6 +51,7 @@ struct Phase {
   // finisher also writes bf16(x * next_g) for the following GEMM and per-tile row statistics.
   int ge_max;                // CTAs this GEMM is cut over (0 = all): few tiles are not worth a wide split
   int norm_in;
+  int qkv_prep;              // QKV projection: the epilogue rotates, converts and files q, k, v (see epilogue)
   const float* u; const float* c;
   const float* next_g;
   // PH_EMBED
@@ -82,6 +83,7 @@ struct Params {
   float4* stats;            // [64 rows][stat_tiles] (mean, M2, count, -) per 128-column tile of x
   int stat_tiles;
   const float* rope_inv;
+  __half* q16;               // [row][Hq*hd] queries, rotated and scaled by 1/sqrt(hd), written by the QKV epilogue
   float* rope_cs; float* rope_sn;   // [row][hd/2] cos and sin of the call's row positions, written by the embedding phase
      // [hd/2] theta^(-2i/hd)
   int* attn_cnt;            // split-KV arrival counters per (request, kv head, query block)
@@ -383,7 +385,7 @@ __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
 __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot,
                           uint8_t* att_smem, Ctl* ctl, uint32_t& att_parity, const Waiter& W, int et, bool& ok,
                           unsigned long long* tra) {
-  const int hd = P.hd, G = P.Hq / P.Hkv, nkv = P.Hkv * hd, nq = P.Hq * hd, nqkv = nq + 2 * nkv;
+  const int hd = P.hd, G = P.Hq / P.Hkv, nkv = P.Hkv * hd, nq = P.Hq * hd;
   const int lane = et & 31, w = et >> 5, g = lane >> 2, t4 = lane & 3;
   const int Q = a.R * G;
   const int q0 = qblk * ATT_QBLK, nQ = min(ATT_QBLK, Q - q0);
@@ -394,88 +396,39 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   __half* kc = reinterpret_cast<__half*>(ph.kc);
   __half* vc = reinterpret_cast<__half*>(ph.vc);
   const int* pt = P.page_table + (size_t)a.slot * P.max_pages;
-  const float scale = 1.0f / sqrtf((float)hd);
-  const int half = hd / 2, ksteps = hd / 16, ntiles = hd / 8;
+  const int ksteps = hd / 16, ntiles = hd / 8;
 
   const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
   const int n_mt = (nQ + 15) / 16;
 
-  // stages chunk c: one bulk async copy per cached row (K and V); rows of new positions are
-  // computed here (rotated k, v), patched into the tile and written to the cache
-  auto stage_issue = [&](int c) {
+  // stages chunk c: one bulk async copy per cached row of K and of V (the rows of this call's
+  // new positions are in the cache already - the QKV epilogue put them there), and with the
+  // unit's first chunk one per query row
+  auto stage_issue = [&](int c, bool with_q) {
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
-    if (et == 0) {
-      const int cached = min(n_pos, max(0, a.base - p0));
-      mbar_expect_tx(&ctl->att_bar, (uint32_t)(cached * 2 * hd * 2));
-    }
+    if (et == 0) mbar_expect_tx(&ctl->att_bar, (uint32_t)(n_pos * 2 * hd * 2 + (with_q ? nQ * hd * 2 : 0)));
     epi_bar_sync();
-    for (int j = et; j < ATT_CHUNK; j += 128) {
-      const int p = p0 + j;
-      if (j < n_pos && p < a.base) {
+    if (et < ATT_CHUNK) {
+      const int j = et, p = p0 + j;
+      if (j < n_pos) {
         const size_t slot = (size_t)pt[p / P.page_tokens] * P.page_tokens + (p % P.page_tokens);
         bulk_copy_g2s(ks + j * pitch, kc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
         bulk_copy_g2s(vs + j * pitch, vc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
-      } else if (j >= n_pos) {
+      } else {
         // rows past the end of the sequence: zero V so that 0 * garbage cannot make a NaN
         uint4* vz = reinterpret_cast<uint4*>(vs + j * pitch);
         for (int q4 = 0; q4 < hd * 2 / 16; ++q4) vz[q4] = make_uint4(0, 0, 0, 0);
       }
-    }
-    {
-      // rows of new positions: four column pairs (i, i + hd/2) per item, the item's six
-      // vector loads in flight together (each is an L2 round trip)
-      const int r_lo = max(0, p0 - a.base), r_hi = min(a.R, p0 + n_pos - a.base);
-      const int hq = half / 4, n_items = (r_hi - r_lo) * hq;
-      for (int b0 = et; b0 < n_items; b0 += 128) {
-        float4 kl[1], kh[1], vl[1], vh[1], cs4[1], sn4[1];
-#pragma unroll
-        for (int u = 0; u < 1; ++u) {
-          const int idx = b0 + 128 * u;
-          if (idx < n_items) {
-            const int r = r_lo + idx / hq, i4 = (idx % hq) * 4;
-            const float* row = P.qkv + (size_t)(a.off + r) * nqkv;
-            const float* ksrc = row + nq + (size_t)kvh * hd + i4;
-            const float* vsrc = row + nq + nkv + (size_t)kvh * hd + i4;
-            kl[u] = __ldcg(reinterpret_cast<const float4*>(ksrc)); kh[u] = __ldcg(reinterpret_cast<const float4*>(ksrc + half));
-            vl[u] = __ldcg(reinterpret_cast<const float4*>(vsrc)); vh[u] = __ldcg(reinterpret_cast<const float4*>(vsrc + half));
-            if (P.rope) {
-              cs4[u] = __ldcg(reinterpret_cast<const float4*>(P.rope_cs + (size_t)(a.off + r) * half + i4));
-              sn4[u] = __ldcg(reinterpret_cast<const float4*>(P.rope_sn + (size_t)(a.off + r) * half + i4));
-            }
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 1; ++u) {
-          const int idx = b0 + 128 * u;
-          if (idx < n_items) {
-            const int r = r_lo + idx / hq, i4 = (idx % hq) * 4, p = a.base + r, j = p - p0;
-            float x0[4] = {kl[u].x, kl[u].y, kl[u].z, kl[u].w}, x1[4] = {kh[u].x, kh[u].y, kh[u].z, kh[u].w};
-            if (P.rope) {
-              const float cs[4] = {cs4[u].x, cs4[u].y, cs4[u].z, cs4[u].w}, sn[4] = {sn4[u].x, sn4[u].y, sn4[u].z, sn4[u].w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float r0 = x0[e] * cs[e] - x1[e] * sn[e], r1 = x1[e] * cs[e] + x0[e] * sn[e];
-                x0[e] = r0; x1[e] = r1;
-              }
-            }
-            const uint2 k_lo = make_uint2(pack_f16x2(x0[0], x0[1]), pack_f16x2(x0[2], x0[3]));
-            const uint2 k_hi = make_uint2(pack_f16x2(x1[0], x1[1]), pack_f16x2(x1[2], x1[3]));
-            const uint2 v_lo = make_uint2(pack_f16x2(vl[u].x, vl[u].y), pack_f16x2(vl[u].z, vl[u].w));
-            const uint2 v_hi = make_uint2(pack_f16x2(vh[u].x, vh[u].y), pack_f16x2(vh[u].z, vh[u].w));
-            __half* kd = reinterpret_cast<__half*>(ks + j * pitch);
-            __half* vd = reinterpret_cast<__half*>(vs + j * pitch);
-            *reinterpret_cast<uint2*>(kd + i4) = k_lo; *reinterpret_cast<uint2*>(kd + half + i4) = k_hi;
-            *reinterpret_cast<uint2*>(vd + i4) = v_lo; *reinterpret_cast<uint2*>(vd + half + i4) = v_hi;
-            if (qblk == 0) {
-              const size_t slot = (size_t)pt[p / P.page_tokens] * P.page_tokens + (p % P.page_tokens);
-              __half* kg = kc + slot * nkv + (size_t)kvh * hd;
-              __half* vg = vc + slot * nkv + (size_t)kvh * hd;
-              *reinterpret_cast<uint2*>(kg + i4) = k_lo; *reinterpret_cast<uint2*>(kg + half + i4) = k_hi;
-              *reinterpret_cast<uint2*>(vg + i4) = v_lo; *reinterpret_cast<uint2*>(vg + half + i4) = v_hi;
-            }
-          }
-        }
+    } else if (with_q && et - ATT_CHUNK < ATT_QBLK) {
+      // query index q -> row r = q / G, head = kvh * G + q % G; rows past the unit's queries are zero
+      const int ql = et - ATT_CHUNK, q = q0 + ql;
+      if (ql < nQ) {
+        bulk_copy_g2s(qs + (size_t)ql * pitch, P.q16 + (size_t)(a.off + q / G) * nq + (size_t)(kvh * G + q % G) * hd,
+                      (uint32_t)(hd * 2), &ctl->att_bar);
+      } else {
+        uint4* qz = reinterpret_cast<uint4*>(qs + (size_t)ql * pitch);
+        for (int q4 = 0; q4 < hd * 2 / 16; ++q4) qz[q4] = make_uint4(0, 0, 0, 0);
       }
     }
   };
@@ -485,58 +438,10 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     return group_ok(ctl, et);
   };
 
-  // the first chunk's copies fly while the queries are rotated
   if (tra) tra[1] = globaltimer_ns();
-  stage_issue(c_begin);
+  fence_proxy_async();   // the rows copied below were written (generic proxy) earlier in this launch
+  stage_issue(c_begin, true);
   if (tra) tra[2] = globaltimer_ns();
-  // queries of this block: query index q -> row r = q / G, head = kvh * G + q % G
-  {
-    // two items' loads in flight together (at most six items of four column pairs per thread
-    // at hd = 128): each load is an L2 round trip
-    const int hq = half / 4, n_items = nQ * hq, n_all = ATT_QBLK * hq;
-    for (int u0 = 0; u0 < 6 && et + 128 * u0 < n_all; u0 += 2) {
-      float4 xa[2], xb[2], qc[2], qn[2];
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const int idx = et + 128 * (u0 + u);
-        if (idx < n_items) {
-          const int ql = idx / hq, i4 = (idx % hq) * 4, q = q0 + ql;
-          const int r = q / G, head = kvh * G + (q % G);
-          const float* src = P.qkv + (size_t)(a.off + r) * nqkv + (size_t)head * hd + i4;
-          xa[u] = __ldcg(reinterpret_cast<const float4*>(src)); xb[u] = __ldcg(reinterpret_cast<const float4*>(src + half));
-          if (P.rope) {
-            qc[u] = __ldcg(reinterpret_cast<const float4*>(P.rope_cs + (size_t)(a.off + r) * half + i4));
-            qn[u] = __ldcg(reinterpret_cast<const float4*>(P.rope_sn + (size_t)(a.off + r) * half + i4));
-          }
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const int idx = et + 128 * (u0 + u);
-        if (idx < n_all) {
-          const int ql = idx / hq, i4 = (idx % hq) * 4;
-          uint2 lo = make_uint2(0u, 0u), hi = make_uint2(0u, 0u);   // rows past the unit's queries stay zero
-          if (idx < n_items) {
-            float x0[4] = {xa[u].x, xa[u].y, xa[u].z, xa[u].w}, x1[4] = {xb[u].x, xb[u].y, xb[u].z, xb[u].w};
-            if (P.rope) {
-              const float cs[4] = {qc[u].x, qc[u].y, qc[u].z, qc[u].w}, sn[4] = {qn[u].x, qn[u].y, qn[u].z, qn[u].w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float r0 = x0[e] * cs[e] - x1[e] * sn[e], r1 = x1[e] * cs[e] + x0[e] * sn[e];
-                x0[e] = r0; x1[e] = r1;
-              }
-            }
-            lo = make_uint2(pack_f16x2(x0[0] * scale, x0[1] * scale), pack_f16x2(x0[2] * scale, x0[3] * scale));
-            hi = make_uint2(pack_f16x2(x1[0] * scale, x1[1] * scale), pack_f16x2(x1[2] * scale, x1[3] * scale));
-          }
-          __half* qd = reinterpret_cast<__half*>(qs + (size_t)ql * pitch);
-          *reinterpret_cast<uint2*>(qd + i4) = lo; *reinterpret_cast<uint2*>(qd + half + i4) = hi;
-        }
-      }
-    }
-  }
-  epi_bar_sync();
-  if (tra) tra[3] = globaltimer_ns();
 
   // Warp w owns query block (MMA M tile) w of the unit and walks the chunk's four 16-position
   // slices itself, so its softmax state and output accumulators never leave its registers.
@@ -551,7 +456,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   for (int nd = 0; nd < 16; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
 
   for (int c = c_begin; c < c_end && ok; ++c) {
-    if (c != c_begin) stage_issue(c);
+    if (c != c_begin) stage_issue(c, false);
     ok = stage_wait();
     if (!ok) break;
     if (tra && c == c_begin) tra[4] = globaltimer_ns();
@@ -988,35 +893,55 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           ok = ctl->bcast != 0;
           epi_bar_sync();
           if (!ok) break;
-          // one warp per row, one lane per tile entry (all loads of a row in flight at once), then
-          // a shuffle tree merges (count, mean, M2) triples pairwise
-          for (int t = quad; t < Tvalid; t += 4) {
-            float n = 0.f, mean = 0.f, m2 = 0.f;
+          // One warp per row, four rows per warp at a time; a lane first folds the tile entries
+          // lane, lane + 32, ... of each row (all loads of the four rows in flight together), then
+          // a shuffle tree merges the lanes' (count, mean, M2) triples pairwise.
+          for (int tb = quad; tb < Tvalid; tb += 16) {
+            float n[4], mean[4], m2[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) { n[r] = 0.f; mean[r] = 0.f; m2[r] = 0.f; }
             for (int tl = lane; tl < P.stat_tiles; tl += 32) {
-              const float4 sv = __ldcg(P.stats + (size_t)t * P.stat_tiles + tl);
-              if (sv.z > 0.f) {
-                const float delta = sv.x - mean, tot = n + sv.z;
-                mean += delta * sv.z / tot;
-                m2 += sv.y + delta * delta * n * sv.z / tot;
-                n = tot;
+              float4 sv[4];
+#pragma unroll
+              for (int r = 0; r < 4; ++r) {
+                const int t = tb + 4 * r;
+                sv[r] = t < Tvalid ? __ldcg(P.stats + (size_t)t * P.stat_tiles + tl) : make_float4(0.f, 0.f, 0.f, 0.f);
+              }
+#pragma unroll
+              for (int r = 0; r < 4; ++r) {
+                if (sv[r].z > 0.f) {
+                  const float delta = sv[r].x - mean[r], tot = n[r] + sv[r].z;
+                  mean[r] += delta * sv[r].z / tot;
+                  m2[r] += sv[r].y + delta * delta * n[r] * sv[r].z / tot;
+                  n[r] = tot;
+                }
               }
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
-              const float n2 = __shfl_xor_sync(0xffffffffu, n, o), mean2 = __shfl_xor_sync(0xffffffffu, mean, o),
-                          m22 = __shfl_xor_sync(0xffffffffu, m2, o);
-              const float tot = n + n2;
-              if (tot > 0.f) {
-                // symmetric form so that both partners compute the same merged triple
-                const float delta = mean2 - mean;
-                const float mm = (n * mean + n2 * mean2) / tot;
-                m2 = m2 + m22 + delta * delta * n * n2 / tot;
-                mean = mm; n = tot;
+#pragma unroll
+              for (int r = 0; r < 4; ++r) {
+                const float n2 = __shfl_xor_sync(0xffffffffu, n[r], o), mean2 = __shfl_xor_sync(0xffffffffu, mean[r], o),
+                            m22 = __shfl_xor_sync(0xffffffffu, m2[r], o);
+                const float tot = n[r] + n2;
+                if (tot > 0.f) {
+                  // symmetric form so that both partners compute the same merged triple
+                  const float delta = mean2 - mean[r];
+                  const float mm = (n[r] * mean[r] + n2 * mean2) / tot;
+                  m2[r] = m2[r] + m22 + delta * delta * n[r] * n2 / tot;
+                  mean[r] = mm; n[r] = tot;
+                }
               }
             }
             if (lane == 0) {
-              if (P.norm_kind == 0) { ctl->mu[t] = mean; ctl->rstd[t] = 1.0f / sqrtf(m2 / (float)P.d + P.eps); }
-              else { ctl->mu[t] = 0.f; ctl->rstd[t] = 1.0f / sqrtf((m2 + n * mean * mean) / (float)P.d + P.eps); }
+#pragma unroll
+              for (int r = 0; r < 4; ++r) {
+                const int t = tb + 4 * r;
+                if (t < Tvalid) {
+                  if (P.norm_kind == 0) { ctl->mu[t] = mean[r]; ctl->rstd[t] = 1.0f / sqrtf(m2[r] / (float)P.d + P.eps); }
+                  else { ctl->mu[t] = 0.f; ctl->rstd[t] = 1.0f / sqrtf((m2[r] + n[r] * mean[r] * mean[r]) / (float)P.d + P.eps); }
+                }
+              }
             }
           }
           epi_bar_sync();
@@ -1041,13 +966,13 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           const bool finisher = kk0 == 0, whole = finisher && seg_end == tile_end;
           // first output column of the tile and how many of its columns exist (a tile never
           // straddles two sources)
-          int n0, ncols;
+          int n0, ncols, src_s = 0;
           if (p.dual) { n0 = tile * 64; ncols = min(64, p.N - n0); }
           else {
-            int s = 0, local = tile;
-            while (s + 1 < p.n_src && local >= p.src_tiles[s]) { local -= p.src_tiles[s]; ++s; }
-            const int src_n = (s + 1 < p.n_src ? p.src_col[s + 1] : p.N) - p.src_col[s];
-            n0 = p.src_col[s] + local * BM; ncols = min(BM, src_n - local * BM);
+            int local = tile;
+            while (src_s + 1 < p.n_src && local >= p.src_tiles[src_s]) { local -= p.src_tiles[src_s]; ++src_s; }
+            const int src_n = (src_s + 1 < p.n_src ? p.src_col[src_s + 1] : p.N) - p.src_col[src_s];
+            n0 = p.src_col[src_s] + local * BM; ncols = min(BM, src_n - local * BM);
           }
           // The epilogue runs in a per-row mapping: thread (er, cg) owns row er of a 16-row chunk
           // and the float4 column groups cg, cg + 8, cg + 16, cg + 24 of the tile (for a gate/up
@@ -1058,6 +983,35 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           // (Nobody else writes this tile's columns of the residual during the phase.)
           float4 xq[4];
           const bool have_pre = p.epi == TC_ADD_F32;
+          // QKV projection: cache row of this thread's row (k and v tiles) and the rotation
+          // table entries of its column groups (q and k tiles), for the first chunk
+          int kv_row0 = 0;
+          float4 rc0[2], rs0[2];
+          auto kv_row_of = [&](int t) {
+            int slot, pos;
+            if (P.mode == CALL_VALIDATE) {
+              int i = 0;
+              while (i + 1 < P.n_req && P.val_off[i + 1] <= t) ++i;
+              slot = P.val_req[i]; pos = P.n_seq[slot] - 1 + (t - P.val_off[i]);
+            } else if (P.mode == CALL_PREFILL) { slot = P.slot; pos = P.draft_step + t; }
+            else if (P.mode == CALL_DRAFT_FIRST) { slot = P.slot; pos = P.n_seq[slot] - 2 + t; }
+            else { slot = P.slot; pos = P.n_seq[slot] - 1 + P.draft_step; }
+            return P.page_table[(size_t)slot * P.max_pages + pos / P.page_tokens] * P.page_tokens + pos % P.page_tokens;
+          };
+          auto rope_of = [&](int t, float4* rc, float4* rs) {
+            // hd = 128: groups (0, 2) and (1, 3) pair up, at table columns cg*4 and 32 + cg*4;
+            // hd = 64: groups (0, 1) and (2, 3), both at table column cg*4
+            const int hh = P.hd / 2;
+            const int i1 = P.hd == 128 ? 32 + cg * 4 : cg * 4;
+            rc[0] = __ldcg(reinterpret_cast<const float4*>(P.rope_cs + (size_t)t * hh + cg * 4));
+            rs[0] = __ldcg(reinterpret_cast<const float4*>(P.rope_sn + (size_t)t * hh + cg * 4));
+            rc[1] = __ldcg(reinterpret_cast<const float4*>(P.rope_cs + (size_t)t * hh + i1));
+            rs[1] = __ldcg(reinterpret_cast<const float4*>(P.rope_sn + (size_t)t * hh + i1));
+          };
+          if (finisher && p.qkv_prep && er < Tvalid) {
+            if (src_s >= 1) kv_row0 = kv_row_of(er);
+            if (P.rope && src_s < 2) rope_of(er, rc0, rs0);
+          }
           if (finisher) {
             const int mc = p.dual ? (m & 63) : m;
             const bool m_on = mc < ncols;
@@ -1256,6 +1210,37 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                     key = other > key ? other : key;
                   }
                   if (cg == 0 && key) atomicMax(keys + t, key);
+                } else if (p.qkv_prep) {
+                  // q: rotate, scale by 1/sqrt(hd), fp16, to the query buffer; k: rotate, fp16, to
+                  // its row of the cache; v: fp16 to the cache.  The rotation pairs column i with
+                  // i + hd/2 of a head; with hd = 128 (a tile is one head) or 64 (two heads) both
+                  // columns of a pair belong to the same thread.
+                  int kv_row = kv_row0;
+                  float4 rc[2] = {rc0[0], rc0[1]}, rs[2] = {rs0[0], rs0[1]};
+                  if (c0 != 0 && row_on) {
+                    if (src_s >= 1) kv_row = kv_row_of(t);
+                    if (P.rope && src_s < 2) rope_of(t, rc, rs);
+                  }
+                  if (P.rope && src_s < 2) {
+                    auto rot = [](float4& lo, float4& hi, const float4& cs, const float4& sn) {
+                      const float4 l = lo, h = hi;
+                      lo = make_float4(l.x * cs.x - h.x * sn.x, l.y * cs.y - h.y * sn.y, l.z * cs.z - h.z * sn.z, l.w * cs.w - h.w * sn.w);
+                      hi = make_float4(h.x * cs.x + l.x * sn.x, h.y * cs.y + l.y * sn.y, h.z * cs.z + l.z * sn.z, h.w * cs.w + l.w * sn.w);
+                    };
+                    if (P.hd == 128) { rot(a[0], a[2], rc[0], rs[0]); rot(a[1], a[3], rc[1], rs[1]); }
+                    else { rot(a[0], a[1], rc[0], rs[0]); rot(a[2], a[3], rc[1], rs[1]); }
+                  }
+                  const float qscale = src_s == 0 ? 1.0f / sqrtf((float)P.hd) : 1.0f;
+                  const int nq_all = P.Hq * P.hd, nkv_all = P.Hkv * P.hd;
+                  __half* dst = src_s == 0 ? P.q16 + (size_t)t * nq_all
+                                           : reinterpret_cast<__half*>(src_s == 1 ? p.kc : p.vc) + (size_t)kv_row * nkv_all;
+                  const int colsrc0 = n0 - p.src_col[src_s];
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    if (on[q])
+                      *reinterpret_cast<uint2*>(dst + colsrc0 + (cg + 8 * q) * 4) =
+                          make_uint2(pack_f16x2(a[q].x * qscale, a[q].y * qscale), pack_f16x2(a[q].z * qscale, a[q].w * qscale));
+                  }
                 } else {
 #pragma unroll
                   for (int q = 0; q < 4; ++q) {
