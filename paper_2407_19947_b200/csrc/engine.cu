@@ -556,7 +556,7 @@ struct MkCall {
 bool mk_eligible(const stairs_ctx* ctx, const DevModel& M, int T) {
   // (the epilogue's vector stores want every GEMM width but the vocabulary to be a multiple of 4)
   return ctx->use_mk && M.m.n_layers >= 1 && T >= 1 && T <= MK_MAX_ROWS && M.m.head_dim % 16 == 0 && M.m.head_dim <= 128 &&
-         M.m.d_model % 4 == 0 && M.m.d_ff % 4 == 0 &&
+         M.m.d_model % 4 == 0 && M.m.d_ff % 4 == 0 && M.m.d_model <= 8192 &&
          (M.m.pos == 0 || M.m.head_dim == 64 || M.m.head_dim == 128);   // rotation pairs must sit in one thread of the QKV epilogue
 }
 

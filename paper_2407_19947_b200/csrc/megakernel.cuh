@@ -463,10 +463,12 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
     if (active) {
-      for (int sl0 = 0; sl0 < n_pos; sl0 += 16) {
-        float sc[2][4];
+      // 32 positions (two MMA k-steps of P.V, four n-tiles of S) per round: four independent
+      // accumulator chains hide the MMA latency, and the softmax bookkeeping is done once per 32
+      for (int sl0 = 0; sl0 < n_pos; sl0 += 32) {
+        float sc[4][4];
 #pragma unroll
-        for (int j = 0; j < 2; ++j) { sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f; }
+        for (int j = 0; j < 4; ++j) { sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f; }
         for (int kk = 0; kk < ksteps; ++kk) {
           uint32_t af[4];
           const uint8_t* qa = qs + (size_t)ql_a * pitch + (kk * 16 + t4 * 2) * 2;
@@ -475,19 +477,20 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
           af[2] = *reinterpret_cast<const uint32_t*>(qa + 16);
           af[3] = *reinterpret_cast<const uint32_t*>(qa + 8 * pitch + 16);
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
+          for (int j = 0; j < 4; ++j) {
             const uint8_t* kb = ks + (size_t)(sl0 + 8 * j + g) * pitch + (kk * 16 + t4 * 2) * 2;
             mma_16816(sc[j], af, *reinterpret_cast<const uint32_t*>(kb), *reinterpret_cast<const uint32_t*>(kb + 16));
           }
         }
-        // staircase mask, row maxima
+        // staircase mask (rows past the chunk's last position hold stale data: assigned, never
+        // computed with), row maxima
         float mx_a = -INFINITY, mx_b = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
+        for (int j = 0; j < 4; ++j) {
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
-            const int pj = p0 + sl0 + 8 * j + t4 * 2 + e;
-            const bool in = (pj - p0) < n_pos;
+            const int jl = sl0 + 8 * j + t4 * 2 + e, pj = p0 + jl;
+            const bool in = jl < n_pos;
             if (!(in && pj <= last_a)) sc[j][e] = -INFINITY;
             if (!(in && pj <= last_b)) sc[j][2 + e] = -INFINITY;
             mx_a = fmaxf(mx_a, sc[j][e]); mx_b = fmaxf(mx_b, sc[j][2 + e]);
@@ -500,7 +503,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
         const float corr_a = expf(m_a - off_a), corr_b = expf(m_b - off_b);   // exp(-inf) = 0
         float sum_a = 0.f, sum_b = 0.f;
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
+        for (int j = 0; j < 4; ++j) {
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
             sc[j][e] = expf(sc[j][e] - off_a); sc[j][2 + e] = expf(sc[j][2 + e] - off_b);
@@ -511,20 +514,29 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
         sum_b += __shfl_xor_sync(0xffffffffu, sum_b, 1); sum_b += __shfl_xor_sync(0xffffffffu, sum_b, 2);
         l_a = l_a * corr_a + sum_a; l_b = l_b * corr_b + sum_b;
         m_a = mn_a; m_b = mn_b;
-        uint32_t pf[4];
-        pf[0] = pack_f16x2(sc[0][0], sc[0][1]); pf[1] = pack_f16x2(sc[0][2], sc[0][3]);
-        pf[2] = pack_f16x2(sc[1][0], sc[1][1]); pf[3] = pack_f16x2(sc[1][2], sc[1][3]);
-        // V fragments: lane supplies the address of row (lane & 15) of the slice, column block (lane >> 4)
+        uint32_t pf[2][4];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          pf[h][0] = pack_f16x2(sc[2 * h][0], sc[2 * h][1]); pf[h][1] = pack_f16x2(sc[2 * h][2], sc[2 * h][3]);
+          pf[h][2] = pack_f16x2(sc[2 * h + 1][0], sc[2 * h + 1][1]); pf[h][3] = pack_f16x2(sc[2 * h + 1][2], sc[2 * h + 1][3]);
+        }
+        // V fragments: lane supplies the address of row (lane & 15) of a 16-position slice, column block (lane >> 4)
         const uint8_t* vrow = vs + (size_t)(sl0 + (lane & 15)) * pitch + (lane >> 4) * 16;
+        const bool second = sl0 + 16 < ATT_CHUNK;   // (always true for 64-position chunks walked in steps of 32)
 #pragma unroll
         for (int nd = 0; nd < 16; nd += 2) {
           if (nd < ntiles) {
             o[nd][0] *= corr_a; o[nd][1] *= corr_a; o[nd][2] *= corr_b; o[nd][3] *= corr_b;
             o[nd + 1][0] *= corr_a; o[nd + 1][1] *= corr_a; o[nd + 1][2] *= corr_b; o[nd + 1][3] *= corr_b;
-            uint32_t vf[4];
+            uint32_t vf[4], vg[4];
             ldmatrix_x4_trans(vf, vrow + nd * 16);
-            mma_16816(o[nd], pf, vf[0], vf[1]);
-            mma_16816(o[nd + 1], pf, vf[2], vf[3]);
+            if (second) ldmatrix_x4_trans(vg, vrow + 16 * pitch + nd * 16);
+            mma_16816(o[nd], pf[0], vf[0], vf[1]);
+            mma_16816(o[nd + 1], pf[0], vf[2], vf[3]);
+            if (second) {
+              mma_16816(o[nd], pf[1], vg[0], vg[1]);
+              mma_16816(o[nd + 1], pf[1], vg[2], vg[3]);
+            }
           }
         }
       }
@@ -893,53 +905,51 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           ok = ctl->bcast != 0;
           epi_bar_sync();
           if (!ok) break;
-          // One warp per row, four rows per warp at a time; a lane first folds the tile entries
-          // lane, lane + 32, ... of each row (all loads of the four rows in flight together), then
-          // a shuffle tree merges the lanes' (count, mean, M2) triples pairwise.
+          // One warp per row, four rows per warp at a time.  A lane holds the tile entries lane and
+          // lane + 32 of each row (all loads of the four rows in flight together; at most 64 tiles,
+          // d <= 8192).  The merged mean is the count-weighted mean of the tiles' means, and the
+          // merged M2 the sum of the tiles' M2 plus count * (tile mean - mean)^2: two warp sums
+          // of non-negative or well-scaled terms, identical on every lane.
           for (int tb = quad; tb < Tvalid; tb += 16) {
-            float n[4], mean[4], m2[4];
+            float4 sv[4][2];
 #pragma unroll
-            for (int r = 0; r < 4; ++r) { n[r] = 0.f; mean[r] = 0.f; m2[r] = 0.f; }
-            for (int tl = lane; tl < P.stat_tiles; tl += 32) {
-              float4 sv[4];
+            for (int r = 0; r < 4; ++r) {
+              const int t = tb + 4 * r;
 #pragma unroll
-              for (int r = 0; r < 4; ++r) {
-                const int t = tb + 4 * r;
-                sv[r] = t < Tvalid ? __ldcg(P.stats + (size_t)t * P.stat_tiles + tl) : make_float4(0.f, 0.f, 0.f, 0.f);
+              for (int e = 0; e < 2; ++e) {
+                const int tl = lane + 32 * e;
+                sv[r][e] = (t < Tvalid && tl < P.stat_tiles) ? __ldcg(P.stats + (size_t)t * P.stat_tiles + tl) : make_float4(0.f, 0.f, 0.f, 0.f);
               }
+            }
+            float n[4], s1[4], m2[4];
 #pragma unroll
-              for (int r = 0; r < 4; ++r) {
-                if (sv[r].z > 0.f) {
-                  const float delta = sv[r].x - mean[r], tot = n[r] + sv[r].z;
-                  mean[r] += delta * sv[r].z / tot;
-                  m2[r] += sv[r].y + delta * delta * n[r] * sv[r].z / tot;
-                  n[r] = tot;
-                }
-              }
+            for (int r = 0; r < 4; ++r) {
+              n[r] = sv[r][0].z + sv[r][1].z;
+              s1[r] = sv[r][0].z * sv[r][0].x + sv[r][1].z * sv[r][1].x;
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-              for (int r = 0; r < 4; ++r) {
-                const float n2 = __shfl_xor_sync(0xffffffffu, n[r], o), mean2 = __shfl_xor_sync(0xffffffffu, mean[r], o),
-                            m22 = __shfl_xor_sync(0xffffffffu, m2[r], o);
-                const float tot = n[r] + n2;
-                if (tot > 0.f) {
-                  // symmetric form so that both partners compute the same merged triple
-                  const float delta = mean2 - mean[r];
-                  const float mm = (n[r] * mean[r] + n2 * mean2) / tot;
-                  m2[r] = m2[r] + m22 + delta * delta * n[r] * n2 / tot;
-                  mean[r] = mm; n[r] = tot;
-                }
-              }
+              for (int r = 0; r < 4; ++r) { n[r] += __shfl_xor_sync(0xffffffffu, n[r], o); s1[r] += __shfl_xor_sync(0xffffffffu, s1[r], o); }
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+              s1[r] = s1[r] / fmaxf(n[r], 1.f);   // the row's mean
+              const float d0 = sv[r][0].x - s1[r], d1 = sv[r][1].x - s1[r];
+              m2[r] = (sv[r][0].y + sv[r][0].z * d0 * d0) + (sv[r][1].y + sv[r][1].z * d1 * d1);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+              for (int r = 0; r < 4; ++r) m2[r] += __shfl_xor_sync(0xffffffffu, m2[r], o);
             }
             if (lane == 0) {
 #pragma unroll
               for (int r = 0; r < 4; ++r) {
                 const int t = tb + 4 * r;
                 if (t < Tvalid) {
-                  if (P.norm_kind == 0) { ctl->mu[t] = mean[r]; ctl->rstd[t] = 1.0f / sqrtf(m2[r] / (float)P.d + P.eps); }
-                  else { ctl->mu[t] = 0.f; ctl->rstd[t] = 1.0f / sqrtf((m2[r] + n[r] * mean[r] * mean[r]) / (float)P.d + P.eps); }
+                  if (P.norm_kind == 0) { ctl->mu[t] = s1[r]; ctl->rstd[t] = 1.0f / sqrtf(m2[r] / (float)P.d + P.eps); }
+                  else { ctl->mu[t] = 0.f; ctl->rstd[t] = 1.0f / sqrtf((m2[r] + n[r] * s1[r] * s1[r]) / (float)P.d + P.eps); }
                 }
               }
             }
