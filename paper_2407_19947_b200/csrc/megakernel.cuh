@@ -365,7 +365,7 @@ __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
   // chunks per unit: from the first row's position only (so it is the same for any draft length)
   const int c0 = (a.base + ATT_CHUNK) / ATT_CHUNK;
   int cpu = 1;
-  while (cpu < 64 && (c0 * P.Hkv) / cpu > 2 * G) cpu <<= 1;
+  while (cpu < 64 && (c0 * P.Hkv) / cpu > G) cpu <<= 1;   // one unit per CTA where possible: a unit's fixed cost exceeds a chunk's
   a.cpu = cpu;
   a.n_ranges = (a.n_chunks + cpu - 1) / cpu;
   a.n_qblk = (a.R * (P.Hq / P.Hkv) + ATT_QBLK - 1) / ATT_QBLK;
@@ -407,12 +407,14 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   auto stage_issue = [&](int c, bool with_q) {
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
+    // (the page-table entry is fetched before the barrier so that its round trip overlaps it)
+    size_t slot = 0;
+    if (et < n_pos) slot = (size_t)pt[(p0 + et) / P.page_tokens] * P.page_tokens + ((p0 + et) % P.page_tokens);
     if (et == 0) mbar_expect_tx(&ctl->att_bar, (uint32_t)(n_pos * 2 * hd * 2 + (with_q ? nQ * hd * 2 : 0)));
     epi_bar_sync();
     if (et < ATT_CHUNK) {
-      const int j = et, p = p0 + j;
+      const int j = et;
       if (j < n_pos) {
-        const size_t slot = (size_t)pt[p / P.page_tokens] * P.page_tokens + (p % P.page_tokens);
         bulk_copy_g2s(ks + j * pitch, kc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
         bulk_copy_g2s(vs + j * pitch, vc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
       } else {
