@@ -401,58 +401,48 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
   const int n_mt = (nQ + 15) / 16;
 
-  // Stages chunk c (and, with the unit's first chunk, its queries) with plain 16-byte loads, all
-  // of a thread's loads in flight together, then the stores.  (One bulk async copy per row was
-  // tried first: ~180 small copies per chunk queue up in the copy engine for microseconds.)
-  // The rows of this call's new positions are in the cache already: the QKV epilogue put them
-  // there, as it put the rotated and scaled queries into the query buffer.
-  const int pieces = hd * 2 / 16;   // 16-byte pieces per row: 8 (hd = 64) .. 16 (hd = 128)
-  auto stage = [&](int c, bool with_q) {
+  // stages chunk c: one bulk async copy per cached row of K and of V (the rows of this call's
+  // new positions are in the cache already - the QKV epilogue put them there), and with the
+  // unit's first chunk one per query row
+  auto stage_issue = [&](int c, bool with_q) {
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
-    uint4 kreg[8], vreg[8], qreg[6];
-    // K and V: item = (row, piece); a thread takes items et, et + 128, ... (at most 8 of each)
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int item = et + 128 * u, j = item / pieces, pc = item % pieces;
-      kreg[u] = vreg[u] = make_uint4(0u, 0u, 0u, 0u);   // rows past the end of the sequence are zero
-      if (j < n_pos) {
-        const int pz = p0 + j;
-        const size_t slot = (size_t)pt[pz / P.page_tokens] * P.page_tokens + (pz % P.page_tokens);
-        kreg[u] = __ldcg(reinterpret_cast<const uint4*>(kc + slot * nkv + (size_t)kvh * hd) + pc);
-        vreg[u] = __ldcg(reinterpret_cast<const uint4*>(vc + slot * nkv + (size_t)kvh * hd) + pc);
-      }
-    }
-    if (with_q) {
-      // query index q -> row r = q / G, head = kvh * G + q % G; rows past the unit's queries are zero
-#pragma unroll
-      for (int u = 0; u < 6; ++u) {
-        const int item = et + 128 * u, ql = item / pieces, pc = item % pieces, q = q0 + ql;
-        qreg[u] = make_uint4(0u, 0u, 0u, 0u);
-        if (ql < nQ)
-          qreg[u] = __ldcg(reinterpret_cast<const uint4*>(P.q16 + (size_t)(a.off + q / G) * nq + (size_t)(kvh * G + q % G) * hd) + pc);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int item = et + 128 * u, j = item / pieces, pc = item % pieces;
-      if (j < ATT_CHUNK) {
-        *reinterpret_cast<uint4*>(ks + j * pitch + pc * 16) = kreg[u];
-        *reinterpret_cast<uint4*>(vs + j * pitch + pc * 16) = vreg[u];
-      }
-    }
-    if (with_q) {
-#pragma unroll
-      for (int u = 0; u < 6; ++u) {
-        const int item = et + 128 * u, ql = item / pieces, pc = item % pieces;
-        if (ql < ATT_QBLK) *reinterpret_cast<uint4*>(qs + (size_t)ql * pitch + pc * 16) = qreg[u];
-      }
-    }
+    // (the page-table entry is fetched before the barrier so that its round trip overlaps it)
+    size_t slot = 0;
+    if (et < n_pos) slot = (size_t)pt[(p0 + et) / P.page_tokens] * P.page_tokens + ((p0 + et) % P.page_tokens);
+    if (et == 0) mbar_expect_tx(&ctl->att_bar, (uint32_t)(n_pos * 2 * hd * 2 + (with_q ? nQ * hd * 2 : 0)));
     epi_bar_sync();
+    if (et < ATT_CHUNK) {
+      const int j = et;
+      if (j < n_pos) {
+        bulk_copy_g2s(ks + j * pitch, kc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
+        bulk_copy_g2s(vs + j * pitch, vc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
+      } else {
+        // rows past the end of the sequence: zero V so that 0 * garbage cannot make a NaN
+        uint4* vz = reinterpret_cast<uint4*>(vs + j * pitch);
+        for (int q4 = 0; q4 < hd * 2 / 16; ++q4) vz[q4] = make_uint4(0, 0, 0, 0);
+      }
+    } else if (with_q && et - ATT_CHUNK < ATT_QBLK) {
+      // query index q -> row r = q / G, head = kvh * G + q % G; rows past the unit's queries are zero
+      const int ql = et - ATT_CHUNK, q = q0 + ql;
+      if (ql < nQ) {
+        bulk_copy_g2s(qs + (size_t)ql * pitch, P.q16 + (size_t)(a.off + q / G) * nq + (size_t)(kvh * G + q % G) * hd,
+                      (uint32_t)(hd * 2), &ctl->att_bar);
+      } else {
+        uint4* qz = reinterpret_cast<uint4*>(qs + (size_t)ql * pitch);
+        for (int q4 = 0; q4 < hd * 2 / 16; ++q4) qz[q4] = make_uint4(0, 0, 0, 0);
+      }
+    }
+  };
+  auto stage_wait = [&]() {
+    W.wait(&ctl->att_bar, att_parity);
+    att_parity ^= 1;
+    return group_ok(ctl, et);
   };
 
   if (tra) tra[1] = globaltimer_ns();
-  stage(c_begin, true);
+  fence_proxy_async();   // the rows copied below were written (generic proxy) earlier in this launch
+  stage_issue(c_begin, true);
   if (tra) tra[2] = globaltimer_ns();
 
   // Warp w owns query block (MMA M tile) w of the unit and walks the chunk's four 16-position
@@ -468,7 +458,9 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   for (int nd = 0; nd < 16; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
 
   for (int c = c_begin; c < c_end && ok; ++c) {
-    if (c != c_begin) stage(c, false);
+    if (c != c_begin) stage_issue(c, false);
+    ok = stage_wait();
+    if (!ok) break;
     if (tra && c == c_begin) tra[4] = globaltimer_ns();
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
