@@ -113,6 +113,13 @@ struct AttnSmem {   // carved after the GEMM ring: Q block (bf16), K and V chunk
   static __host__ __device__ size_t bytes(int hd) { return q_bytes(hd) + 2 * kv_bytes(hd) + 64; }
 };
 
+// 16-byte asynchronous copy global -> shared; `on` false writes zeros and reads nothing
+__device__ __forceinline__ void cp_async16(void* dst, const void* src, bool on) {
+  const uint32_t n = on ? 16u : 0u;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 // mma.sync m16n8k16 (fp16 in, fp32 accumulate) and its operand loads, for the attention tiles:
 // queries, cached K/V and the softmax weights are fp16 (11 significant bits)
 __device__ __forceinline__ void mma_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
@@ -401,48 +408,40 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
   const int n_mt = (nQ + 15) / 16;
 
-  // stages chunk c: one bulk async copy per cached row of K and of V (the rows of this call's
-  // new positions are in the cache already - the QKV epilogue put them there), and with the
-  // unit's first chunk one per query row
-  auto stage_issue = [&](int c, bool with_q) {
+  // Stages chunk c (and, with the unit's first chunk, its queries) with 16-byte asynchronous
+  // copies issued by all 128 threads (no registers held, so all of a thread's copies are in
+  // flight together; rows past the end are zero-filled by the copy itself).  One bulk copy per
+  // row was tried first: ~180 small copies per chunk queue up in the copy engine for
+  // microseconds.  The rows of this call's new positions are in the cache already: the QKV
+  // epilogue put them there, as it put the rotated and scaled queries into the query buffer.
+  const int pieces = hd * 2 / 16;   // 16-byte pieces per row
+  auto stage = [&](int c, bool with_q) {
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
-    // (the page-table entry is fetched before the barrier so that its round trip overlaps it)
-    size_t slot = 0;
-    if (et < n_pos) slot = (size_t)pt[(p0 + et) / P.page_tokens] * P.page_tokens + ((p0 + et) % P.page_tokens);
-    if (et == 0) mbar_expect_tx(&ctl->att_bar, (uint32_t)(n_pos * 2 * hd * 2 + (with_q ? nQ * hd * 2 : 0)));
-    epi_bar_sync();
-    if (et < ATT_CHUNK) {
-      const int j = et;
-      if (j < n_pos) {
-        bulk_copy_g2s(ks + j * pitch, kc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
-        bulk_copy_g2s(vs + j * pitch, vc + slot * nkv + (size_t)kvh * hd, (uint32_t)(hd * 2), &ctl->att_bar);
-      } else {
-        // rows past the end of the sequence: zero V so that 0 * garbage cannot make a NaN
-        uint4* vz = reinterpret_cast<uint4*>(vs + j * pitch);
-        for (int q4 = 0; q4 < hd * 2 / 16; ++q4) vz[q4] = make_uint4(0, 0, 0, 0);
-      }
-    } else if (with_q && et - ATT_CHUNK < ATT_QBLK) {
+    for (int item = et; item < ATT_CHUNK * pieces; item += 128) {
+      const int j = item / pieces, pc = item % pieces;
+      const bool on = j < n_pos;
+      const int pz = on ? p0 + j : 0;
+      const size_t slot = (size_t)pt[pz / P.page_tokens] * P.page_tokens + (pz % P.page_tokens);
+      cp_async16(ks + j * pitch + pc * 16, reinterpret_cast<const uint4*>(kc + slot * nkv + (size_t)kvh * hd) + pc, on);
+      cp_async16(vs + j * pitch + pc * 16, reinterpret_cast<const uint4*>(vc + slot * nkv + (size_t)kvh * hd) + pc, on);
+    }
+    if (with_q) {
       // query index q -> row r = q / G, head = kvh * G + q % G; rows past the unit's queries are zero
-      const int ql = et - ATT_CHUNK, q = q0 + ql;
-      if (ql < nQ) {
-        bulk_copy_g2s(qs + (size_t)ql * pitch, P.q16 + (size_t)(a.off + q / G) * nq + (size_t)(kvh * G + q % G) * hd,
-                      (uint32_t)(hd * 2), &ctl->att_bar);
-      } else {
-        uint4* qz = reinterpret_cast<uint4*>(qs + (size_t)ql * pitch);
-        for (int q4 = 0; q4 < hd * 2 / 16; ++q4) qz[q4] = make_uint4(0, 0, 0, 0);
+      for (int item = et; item < ATT_QBLK * pieces; item += 128) {
+        const int ql = item / pieces, pc = item % pieces;
+        const bool on = ql < nQ;
+        const int q = on ? q0 + ql : q0;
+        cp_async16(qs + (size_t)ql * pitch + pc * 16,
+                   reinterpret_cast<const uint4*>(P.q16 + (size_t)(a.off + q / G) * nq + (size_t)(kvh * G + q % G) * hd) + pc, on);
       }
     }
-  };
-  auto stage_wait = [&]() {
-    W.wait(&ctl->att_bar, att_parity);
-    att_parity ^= 1;
-    return group_ok(ctl, et);
+    cp_async_wait_all();
+    epi_bar_sync();
   };
 
   if (tra) tra[1] = globaltimer_ns();
-  fence_proxy_async();   // the rows copied below were written (generic proxy) earlier in this launch
-  stage_issue(c_begin, true);
+  stage(c_begin, true);
   if (tra) tra[2] = globaltimer_ns();
 
   // Warp w owns query block (MMA M tile) w of the unit and walks the chunk's four 16-position
@@ -458,9 +457,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   for (int nd = 0; nd < 16; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
 
   for (int c = c_begin; c < c_end && ok; ++c) {
-    if (c != c_begin) stage_issue(c, false);
-    ok = stage_wait();
-    if (!ok) break;
+    if (c != c_begin) stage(c, false);
     if (tra && c == c_begin) tra[4] = globaltimer_ns();
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
