@@ -227,6 +227,7 @@ struct Ctl {
   volatile int last_flag;
   volatile int bcast;
   float rstd[64], mu[64];       // per-row statistics of the current norm_in GEMM phase
+  int rowbase[64];              // attention staging: cache row of each position of the chunk
   alignas(16) float gtile[128]; // next operand's gain for the current tile's columns
   alignas(16) float utile[128]; // folded-normalisation constants u[n], c[n] of the tile's columns
   alignas(16) float ctile[128];
@@ -418,22 +419,38 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   auto stage = [&](int c, bool with_q) {
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
-    for (int item = et; item < ATT_CHUNK * pieces; item += 128) {
-      const int j = item / pieces, pc = item % pieces;
-      const bool on = j < n_pos;
-      const int pz = on ? p0 + j : 0;
-      const size_t slot = (size_t)pt[pz / P.page_tokens] * P.page_tokens + (pz % P.page_tokens);
-      cp_async16(ks + j * pitch + pc * 16, reinterpret_cast<const uint4*>(kc + slot * nkv + (size_t)kvh * hd) + pc, on);
-      cp_async16(vs + j * pitch + pc * 16, reinterpret_cast<const uint4*>(vc + slot * nkv + (size_t)kvh * hd) + pc, on);
+    // cache row of each position of the chunk, looked up once (-1: past the end)
+    if (et < ATT_CHUNK) {
+      const int pz = p0 + et;
+      ctl->rowbase[et] = et < n_pos ? pt[pz / P.page_tokens] * P.page_tokens + (pz % P.page_tokens) : -1;
+    }
+    epi_bar_sync();
+    {
+      // items (row, 16-byte piece) et, et + 128, ...; row and piece advance without divisions
+      const int dj = 128 / pieces, dp = 128 % pieces;
+      int jr = et / pieces, pc = et % pieces;
+      const size_t head_off = (size_t)kvh * hd;
+      while (jr < ATT_CHUNK) {
+        const int rb = ctl->rowbase[jr];
+        const bool on = rb >= 0;
+        const size_t off = (size_t)(on ? rb : 0) * nkv + head_off;
+        cp_async16(ks + jr * pitch + pc * 16, reinterpret_cast<const uint4*>(kc + off) + pc, on);
+        cp_async16(vs + jr * pitch + pc * 16, reinterpret_cast<const uint4*>(vc + off) + pc, on);
+        jr += dj; pc += dp;
+        if (pc >= pieces) { pc -= pieces; ++jr; }
+      }
     }
     if (with_q) {
       // query index q -> row r = q / G, head = kvh * G + q % G; rows past the unit's queries are zero
-      for (int item = et; item < ATT_QBLK * pieces; item += 128) {
-        const int ql = item / pieces, pc = item % pieces;
+      const int dj = 128 / pieces, dp = 128 % pieces;
+      int ql = et / pieces, pc = et % pieces;
+      while (ql < ATT_QBLK) {
         const bool on = ql < nQ;
         const int q = on ? q0 + ql : q0;
         cp_async16(qs + (size_t)ql * pitch + pc * 16,
                    reinterpret_cast<const uint4*>(P.q16 + (size_t)(a.off + q / G) * nq + (size_t)(kvh * G + q % G) * hd) + pc, on);
+        ql += dj; pc += dp;
+        if (pc >= pieces) { pc -= pieces; ++ql; }
       }
     }
     cp_async_wait_all();
