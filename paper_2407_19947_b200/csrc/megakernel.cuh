@@ -463,7 +463,11 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
 
   // Warp w owns query block (MMA M tile) w of the unit and walks the chunk's four 16-position
   // slices itself, so its softmax state and output accumulators never leave its registers.
-  const int mt = w;
+  // With one or two query blocks the four warps also split each chunk's positions in two (warps
+  // 0, 1 take the first 32 positions, warps 2, 3 the last 32) and the two states of a block are
+  // merged once, at the end of the unit.
+  const int ps = (n_mt <= 2 && hd >= 64) ? 2 : 1;
+  const int mt = ps == 2 ? (w & 1) : w, part = ps == 2 ? (w >> 1) : 0;
   const bool active = mt < n_mt;
   const int ql_a = mt * 16 + g, ql_b = ql_a + 8;
   const int last_a = (active && ql_a < nQ) ? a.base + (q0 + ql_a) / G : -1;   // last visible position
@@ -481,7 +485,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     if (active) {
       // 32 positions (two MMA k-steps of P.V, four n-tiles of S) per round: four independent
       // accumulator chains hide the MMA latency, and the softmax bookkeeping is done once per 32
-      for (int sl0 = 0; sl0 < n_pos; sl0 += 32) {
+      for (int sl0 = 32 * part; sl0 < n_pos; sl0 += 32 * ps) {
         float sc[4][4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) { sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f; }
@@ -560,7 +564,35 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     epi_bar_sync();   // tile may be overwritten by the next chunk or unit
     if (tra && c == c_begin) tra[5] = globaltimer_ns();
   }
-  if (!ok || !active) return;
+  if (!ok) return;
+  if (ps == 2) {
+    // second half's state -> shared memory (the K/V tiles are free now) -> merged into the first's
+    float4* mb = reinterpret_cast<float4*>(ks);
+    if (active && part == 1) {
+#pragma unroll
+      for (int nd = 0; nd < 16; ++nd)
+        if (nd < ntiles) mb[(mt * 17 + nd) * 32 + lane] = make_float4(o[nd][0], o[nd][1], o[nd][2], o[nd][3]);
+      mb[(mt * 17 + 16) * 32 + lane] = make_float4(m_a, m_b, l_a, l_b);
+    }
+    epi_bar_sync();
+    if (active && part == 0) {
+      const float4 st = mb[(mt * 17 + 16) * 32 + lane];
+      const float M_a = fmaxf(m_a, st.x), M_b = fmaxf(m_b, st.y);
+      const float off_a = M_a == -INFINITY ? 0.f : M_a, off_b = M_b == -INFINITY ? 0.f : M_b;
+      const float wa = expf(m_a - off_a), wa2 = expf(st.x - off_a), wb = expf(m_b - off_b), wb2 = expf(st.y - off_b);
+      l_a = l_a * wa + st.z * wa2; l_b = l_b * wb + st.w * wb2;
+      m_a = M_a; m_b = M_b;
+#pragma unroll
+      for (int nd = 0; nd < 16; ++nd)
+        if (nd < ntiles) {
+          const float4 v = mb[(mt * 17 + nd) * 32 + lane];
+          o[nd][0] = o[nd][0] * wa + v.x * wa2; o[nd][1] = o[nd][1] * wa + v.y * wa2;
+          o[nd][2] = o[nd][2] * wb + v.z * wb2; o[nd][3] = o[nd][3] * wb + v.w * wb2;
+        }
+    }
+    // (the next unit's staging starts with a barrier of its own before it overwrites the tiles)
+  }
+  if (!active || part != 0) return;
 
   // write this warp's 16 rows straight from the accumulator fragments: the final output when the
   // unit saw every visible position, else the state (O, max, sum) for the combine phase
