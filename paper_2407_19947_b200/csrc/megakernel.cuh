@@ -219,6 +219,9 @@ __device__ __forceinline__ float warp_multi_sum32(float (&a)[32], int lane) {
   return a[0];
 }
 
+// Geometry of one request's attention units.
+struct AttnReq { int slot, base, R, off, n_chunks, cpu, n_ranges, n_qblk, units; };
+
 // Shared per-CTA control block.
 struct Ctl {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2], att_bar;
@@ -228,6 +231,9 @@ struct Ctl {
   volatile int bcast;
   float rstd[64], mu[64];       // per-row statistics of the current norm_in GEMM phase
   int rowbase[64];              // attention staging: cache row of each position of the chunk
+  AttnReq areq[64];             // per request, filled once per launch (a request has at least one row: <= 64)
+  alignas(16) uint32_t phc[2][(sizeof(Phase) + 3) / 4];   // this and the next phase's descriptor (global memory is a
+                                                          // long round trip with the L1 carved down to almost nothing)
   alignas(16) float gtile[128]; // next operand's gain for the current tile's columns
   alignas(16) float utile[128]; // folded-normalisation constants u[n], c[n] of the tile's columns
   alignas(16) float ctile[128];
@@ -355,7 +361,6 @@ __device__ void embed_row(const Params& P, int t, const RowInfo& r, const float*
 // ---------------------------------------------------------------------------------------------
 // Attention units
 // ---------------------------------------------------------------------------------------------
-struct AttnReq { int slot, base, R, off, n_chunks, cpu, n_ranges, n_qblk, units; };
 
 __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
   AttnReq a;
@@ -818,8 +823,19 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     bool ok = true;
     bool waited = true;   // true when every earlier phase is known complete grid-wide
 
+    constexpr int PH_WORDS = (int)((sizeof(Phase) + 3) / 4);
+    static_assert(PH_WORDS <= 128, "one descriptor word per compute thread");
+    {
+      // descriptor of phase 0 and the requests' attention geometry, once
+      if (et < PH_WORDS) ctl->phc[0][et] = __ldcg(reinterpret_cast<const uint32_t*>(P.phases) + et);
+      const int n_req0 = P.mode == CALL_VALIDATE ? P.n_req : 1;
+      if (et < n_req0 && et < 64) ctl->areq[et] = attn_req(P, et, G);
+      epi_bar_sync();
+    }
     for (int ph = 0; ph < P.n_phases && ok; ++ph) {
-      const Phase& p = P.phases[ph];
+      const Phase& p = *reinterpret_cast<const Phase*>(ctl->phc[ph & 1]);
+      // the next phase's descriptor: fetched now, parked in shared memory at the end of this phase
+      const uint32_t next_word = (et < PH_WORDS && ph + 1 < P.n_phases) ? __ldcg(reinterpret_cast<const uint32_t*>(P.phases + ph + 1) + et) : 0u;
       if (p.kind != PH_GEMM && !waited) {
         // inputs come from other CTAs: wait until all of them finished phase ph - 1
         if (et == 0) {
@@ -848,7 +864,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         const int n_req = P.mode == CALL_VALIDATE ? P.n_req : 1;
         int u0 = 0, g0 = 0;
         for (int i = 0; i < n_req && ok; ++i) {
-          const AttnReq a = attn_req(P, i, G);
+          const AttnReq a = ctl->areq[i];
           // units of this request: index = ((kvh * n_ranges) + range) * n_qblk + qblk
           int first = (cta - u0 % G + G) % G;
           for (int u = first; u < a.units && ok; u += G) {
@@ -869,7 +885,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         const int hd = P.hd, Gq = P.Hq / P.Hkv;
         int u0 = 0, item0 = 0;
         for (int i = 0; i < n_req; ++i) {
-          const AttnReq a = attn_req(P, i, G);
+          const AttnReq a = ctl->areq[i];
           if (a.n_ranges > 1) {
             const int Q = a.R * Gq, items = P.Hkv * Q;
             int it = ((cta * 4 + quad) - item0) % (G * 4);
@@ -1182,6 +1198,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                     }
                   }
                 }
+                if (tra) {
+                  asm volatile("" ::"f"(a[0].x), "f"(a[0].w), "f"(a[1].x), "f"(a[1].w), "f"(a[2].x), "f"(a[2].w), "f"(a[3].x), "f"(a[3].w));
+                  tra[6] = globaltimer_ns();
+                }
                 if (p.norm_in && row_on) {
                   // fold the normalisation in: y = rstd_t * (acc - mean_t * u[n]) + c[n]
                   const float rs = ctl->rstd[t], mu = ctl->mu[t];
@@ -1212,6 +1232,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                       cnt += 4.f; sum += (a[q].x + a[q].y) + (a[q].z + a[q].w);
                     }
                   }
+                  if (tra) { asm volatile("" ::"f"(sum), "f"(cnt)); tra[7] = globaltimer_ns(); }
                   if (p.next_g) {
                     float mean = cnt > 0.f ? sum / cnt : 0.f, m2 = 0.f;
 #pragma unroll
@@ -1335,6 +1356,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       // barrier ph-1 completed (its activation tiles were loaded after that), so only idle CTAs
       // look at the counter.
       fence_proxy_async();   // later TMA (async proxy) reads of these generic-proxy writes
+      if (et < PH_WORDS) ctl->phc[(ph + 1) & 1][et] = next_word;   // (the barriers below publish it)
       if (ph > 0 && p.kind == PH_GEMM && !gemm_worked) {
         if (et == 0) ctl->bcast = W.wait_grid(bar_count, P.bar_base + (unsigned long long)ph * G) ? 1 : 0;
         epi_bar_sync();
