@@ -459,19 +459,16 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
     }
     p.n_tiles = tiles; p.epi = epi; p.out = out; p.ldo = ldo;
     {
-      // How many CTAs to cut this GEMM over.  More CTAs stream faster - up to the point where
-      // HBM, not the CTA's own ring of tiles in flight, is the limit - but a split tile costs a
-      // fix-up chain (partials parked, flags raised, the finisher's wait and reads) that a whole
-      // tile does not have.  Model, from device timestamps: a CTA streams at most ~120 GB/s, all
-      // CTAs together ~6 TB/s; a split costs ~3 us plus ~0.6 us per six partial tiles read.
+      // How many CTAs to cut this GEMM over: more CTAs stream faster, but every tile is then
+      // finished from more partial tiles, which the finisher reads four at a time.  Model:
+      // stream time at ~44 GB/s per SM plus ~1.6 us per batch of four partials.
       const int grid = std::min(ctx->sm_count, TC_GRID_MAX);
       const double bytes = (double)tiles * p.kblocks * tc::A_STAGE_BYTES;
       double best = 1e30; int best_ge = grid;
       for (int s2 = 1; s2 <= 64; s2 *= 2) {
         const int ge = std::min(grid, tiles * s2);
         const double seg = (double)ge / tiles + (ge % tiles ? 1.0 : 0.0);
-        const double rate = std::min(120.0e3, 6000.0e3 / ge);   // bytes per us per CTA
-        const double t_us = bytes / (ge * rate) + (seg > 1.0 ? 3.0 + std::ceil((seg - 1.0) / 6.0) * 0.6 : 0.0);
+        const double t_us = bytes / (ge * 44.0e3) + (seg > 1.0 ? std::ceil(seg / 4.0) * 1.6 + 2.0 : 0.0);
         if (t_us < best - 1e-9) { best = t_us; best_ge = ge; }
         if (ge == grid) break;
       }
