@@ -655,7 +655,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = gridDim.x, cta = blockIdx.x;
   uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < 2 * P.t_box) tmem_cols <<= 1;
+  while ((int)tmem_cols < 4 * P.t_box) tmem_cols <<= 1;   // two accumulators, each with hi-part and lo-part columns
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) { mbar_init(ctl->full + s, 1); mbar_init(ctl->empty + s, 1); }
@@ -755,9 +755,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             progress = true;
           }
         }
-        if (progress) { idle = 0; t_idle = clock64(); }
+        if (progress) idle = 0;
         else {
-          ++idle;
+          if (idle++ == 0) t_idle = clock64();   // (the clock is only read once the producer goes idle)
           if (W.poll_abort(t_idle)) break;
           if ((idle & 4095u) == 0 && ld_acquire_u64(P.bar + 1)) { ctl->abort_flag = 1; break; }
         }
@@ -766,7 +766,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
   } else if (warp == 1) {
     // ================================================================== MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = instr_desc_bf16(P.t_box);
+      // One MMA covers the hi and the lo rows of the activation tile (they are adjacent in the
+      // stage: N = 2 * t_box); the two halves of the accumulator are added when it is drained.
+      const uint32_t idesc = instr_desc_bf16(2 * P.t_box);
       int stage = 0; uint32_t phase = 0;
       int buf = 0; uint32_t acc_phase[2] = {0, 0};
       bool ok = true;
@@ -794,14 +796,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           tc_fence_after();
           const uint32_t a_addr = smem_u32(smem + (size_t)stage * stage_bytes);
           const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + A_STAGE_BYTES);
-          const uint64_t b_desc_lo = smem_desc_sw128(a_addr + A_STAGE_BYTES + b_stage_bytes);
-          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * P.t_box);
+          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 2 * P.t_box);
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
+          for (int k = 0; k < BK / UMMA_K; ++k)
             umma_bf16(d_tmem, a_desc + (uint64_t)(k * UMMA_K * 2 / 16), b_desc + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
                       (seg_first && k == 0) ? 0u : 1u);
-            umma_bf16(d_tmem, a_desc + (uint64_t)(k * UMMA_K * 2 / 16), b_desc_lo + (uint64_t)(k * UMMA_K * 2 / 16), idesc, 1u);
-          }
           umma_commit(ctl->empty + stage);
           if (seg_last) { umma_commit(ctl->acc_full + buf); acc_phase[buf] ^= 1; buf ^= 1; }
           seg_first = seg_last;
@@ -1110,7 +1109,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           if (tracing && first_seg) { tr[4] = globaltimer_ns(); first_seg = false; }
           acc_phase[buf] ^= 1;
           tc_fence_after();
-          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * P.t_box);
+          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * 2 * P.t_box);
           unsigned long long* tra = (P.trace && et == 0 && !whole) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
           if (!finisher) {
             if (tra) tra[4] = globaltimer_ns();
@@ -1118,6 +1117,12 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             for (int c0 = 0; c0 < Tvalid; c0 += 16) {   // only rows that exist
               float v[16];
               tmem_ld16(taddr + (uint32_t)c0, v);
+              {
+                float vl[16];
+                tmem_ld16(taddr + (uint32_t)(P.t_box + c0), vl);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] += vl[j];
+              }
               const int jn = min(16, Tvalid - c0);
 #pragma unroll
               for (int j = 0; j < 16; ++j) if (j < jn) mine[(size_t)(c0 + j) * BM + m] = v[j];
@@ -1135,6 +1140,12 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               {
                 float v[16];
                 tmem_ld16(taddr + (uint32_t)c0, v);
+                {
+                  float vl[16];
+                  tmem_ld16(taddr + (uint32_t)(P.t_box + c0), vl);
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) v[j] += vl[j];
+                }
                 if (c0 + 16 >= Tvalid) {   // accumulator drained: the MMA warp may reuse it
                   tc_fence_before();
                   if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
