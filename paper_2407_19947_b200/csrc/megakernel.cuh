@@ -682,18 +682,23 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
       // Cursor over this CTA's k-blocks of all GEMM phases, in program order.  Per-phase fields
       // are hoisted into registers on phase entry; tile and k indices advance incrementally.
+      // (scalar fields only: an array indexed at run time would put the cursor in local memory,
+      // and with the L1 carved down for shared memory every such access is an L2 round trip)
       struct Cursor {
         int ph, kk, n_tile, remaining, kblocks, dual, n_src, x_map;
-        int src_tiles[3], w_map[3];
+        int st0, st1, wmap0, wmap1, wmap2;   // tiles of sources 0 and 1; tensor-map indices of the (up to) three sources
         const CUtensorMap* wm0; const CUtensorMap* wm1; int row;
         bool valid;
       };
       auto locate = [&](Cursor& c) {   // source map and row coordinate of tile c.n_tile
-        if (c.dual) { c.wm0 = P.maps + c.w_map[0]; c.wm1 = P.maps + c.w_map[1]; c.row = c.n_tile * 64; }
+        if (c.dual) { c.wm0 = P.maps + c.wmap0; c.wm1 = P.maps + c.wmap1; c.row = c.n_tile * 64; }
         else {
-          int s2 = 0, local = c.n_tile;
-          while (s2 + 1 < c.n_src && local >= c.src_tiles[s2]) { local -= c.src_tiles[s2]; ++s2; }
-          c.wm0 = P.maps + c.w_map[s2]; c.row = local * BM;
+          int local = c.n_tile, wm = c.wmap0;
+          if (c.n_src > 1 && local >= c.st0) {
+            local -= c.st0; wm = c.wmap1;
+            if (c.n_src > 2 && local >= c.st1) { local -= c.st1; wm = c.wmap2; }
+          }
+          c.wm0 = P.maps + wm; c.row = local * BM;
         }
       };
       auto enter = [&](Cursor& c, int from) {   // first GEMM phase >= from in which this CTA has work
@@ -703,8 +708,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           const KRange kr = phase_range((long long)p.n_tiles * p.kblocks, cta, G, p.ge_max);
           if (kr.begin >= kr.end) continue;
           c.ph = ph; c.kblocks = p.kblocks; c.dual = p.dual; c.n_src = p.n_src; c.x_map = p.x_map;
-#pragma unroll
-          for (int q = 0; q < 3; ++q) { c.src_tiles[q] = p.src_tiles[q]; c.w_map[q] = p.w_map[q]; }
+          c.st0 = p.src_tiles[0]; c.st1 = p.src_tiles[1];
+          c.wmap0 = p.w_map[0]; c.wmap1 = p.w_map[1]; c.wmap2 = p.w_map[2];
           c.n_tile = (int)(kr.begin / p.kblocks); c.kk = (int)(kr.begin % p.kblocks);
           c.remaining = (int)(kr.end - kr.begin);
           locate(c);
@@ -770,7 +775,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       // stage: N = 2 * t_box); the two halves of the accumulator are added when it is drained.
       const uint32_t idesc = instr_desc_bf16(2 * P.t_box);
       int stage = 0; uint32_t phase = 0;
-      int buf = 0; uint32_t acc_phase[2] = {0, 0};
+      int buf = 0; uint32_t acc_bits = 0;   // bit b: parity of accumulator b (no run-time indexed array: see the cursor)
       bool ok = true;
       for (int ph = 0; ph < P.n_phases && ok; ++ph) {
         const Phase& p = P.phases[ph];
@@ -786,7 +791,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         while (remaining > 0 && ok) {
           const bool seg_last = (remaining == 1) || (kk == kblocks - 1);
           if (seg_first) {
-            ok = W.wait(ctl->acc_empty + buf, acc_phase[buf] ^ 1);
+            ok = W.wait(ctl->acc_empty + buf, ((acc_bits >> buf) & 1u) ^ 1u);
             if (!ok) break;
             tc_fence_after();
           }
@@ -802,7 +807,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             umma_bf16(d_tmem, a_desc + (uint64_t)(k * UMMA_K * 2 / 16), b_desc + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
                       (seg_first && k == 0) ? 0u : 1u);
           umma_commit(ctl->empty + stage);
-          if (seg_last) { umma_commit(ctl->acc_full + buf); acc_phase[buf] ^= 1; buf ^= 1; }
+          if (seg_last) { umma_commit(ctl->acc_full + buf); acc_bits ^= 1u << buf; buf ^= 1; }
           seg_first = seg_last;
           if (++kk == kblocks) kk = 0;
           --remaining;
@@ -817,7 +822,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     const int m = quad * 32 + lane;
     const int et = threadIdx.x - 64;
     float* red = vt;    // 4 floats of scratch for group sums (the exchange tile is free outside GEMM epilogues)
-    int buf = 0; uint32_t acc_phase[2] = {0, 0};
+    int buf = 0; uint32_t acc_bits = 0;
     uint32_t att_parity = 0;
     bool ok = true;
     bool waited = true;   // true when every earlier phase is known complete grid-wide
@@ -1039,13 +1044,16 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           const bool finisher = kk0 == 0, whole = finisher && seg_end == tile_end;
           // first output column of the tile and how many of its columns exist (a tile never
           // straddles two sources)
-          int n0, ncols, src_s = 0;
+          int n0, ncols, src_s = 0, src_col0 = 0;
           if (p.dual) { n0 = tile * 64; ncols = min(64, p.N - n0); }
           else {
-            int local = tile;
-            while (src_s + 1 < p.n_src && local >= p.src_tiles[src_s]) { local -= p.src_tiles[src_s]; ++src_s; }
-            const int src_n = (src_s + 1 < p.n_src ? p.src_col[src_s + 1] : p.N) - p.src_col[src_s];
-            n0 = p.src_col[src_s] + local * BM; ncols = min(BM, src_n - local * BM);
+            int local = tile, col0 = 0, col1 = p.n_src > 1 ? p.src_col[1] : p.N;
+            if (p.n_src > 1 && local >= p.src_tiles[0]) {
+              local -= p.src_tiles[0]; src_s = 1; col0 = p.src_col[1]; col1 = p.n_src > 2 ? p.src_col[2] : p.N;
+              if (p.n_src > 2 && local >= p.src_tiles[1]) { local -= p.src_tiles[1]; src_s = 2; col0 = p.src_col[2]; col1 = p.N; }
+            }
+            src_col0 = col0;
+            n0 = col0 + local * BM; ncols = min(BM, (col1 - col0) - local * BM);
           }
           // The epilogue runs in a per-row mapping: thread (er, cg) owns row er of a 16-row chunk
           // and the float4 column groups cg, cg + 8, cg + 16, cg + 24 of the tile (for a gate/up
@@ -1059,7 +1067,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           // QKV projection: cache row of this thread's row (k and v tiles) and the rotation
           // table entries of its column groups (q and k tiles), for the first chunk
           int kv_row0 = 0;
-          float4 rc0[2], rs0[2];
+          float4 rc0a, rc0b, rs0a, rs0b;
           auto kv_row_of = [&](int t) {
             int slot, pos;
             if (P.mode == CALL_VALIDATE) {
@@ -1071,19 +1079,19 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             else { slot = P.slot; pos = P.n_seq[slot] - 1 + P.draft_step; }
             return P.page_table[(size_t)slot * P.max_pages + pos / P.page_tokens] * P.page_tokens + pos % P.page_tokens;
           };
-          auto rope_of = [&](int t, float4* rc, float4* rs) {
+          auto rope_of = [&](int t, float4& c0, float4& s0, float4& c1, float4& s1) {
             // hd = 128: groups (0, 2) and (1, 3) pair up, at table columns cg*4 and 32 + cg*4;
             // hd = 64: groups (0, 1) and (2, 3), both at table column cg*4
             const int hh = P.hd / 2;
             const int i1 = P.hd == 128 ? 32 + cg * 4 : cg * 4;
-            rc[0] = __ldcg(reinterpret_cast<const float4*>(P.rope_cs + (size_t)t * hh + cg * 4));
-            rs[0] = __ldcg(reinterpret_cast<const float4*>(P.rope_sn + (size_t)t * hh + cg * 4));
-            rc[1] = __ldcg(reinterpret_cast<const float4*>(P.rope_cs + (size_t)t * hh + i1));
-            rs[1] = __ldcg(reinterpret_cast<const float4*>(P.rope_sn + (size_t)t * hh + i1));
+            c0 = __ldcg(reinterpret_cast<const float4*>(P.rope_cs + (size_t)t * hh + cg * 4));
+            s0 = __ldcg(reinterpret_cast<const float4*>(P.rope_sn + (size_t)t * hh + cg * 4));
+            c1 = __ldcg(reinterpret_cast<const float4*>(P.rope_cs + (size_t)t * hh + i1));
+            s1 = __ldcg(reinterpret_cast<const float4*>(P.rope_sn + (size_t)t * hh + i1));
           };
           if (finisher && p.qkv_prep && er < Tvalid) {
             if (src_s >= 1) kv_row0 = kv_row_of(er);
-            if (P.rope && src_s < 2) rope_of(er, rc0, rs0);
+            if (P.rope && src_s < 2) rope_of(er, rc0a, rs0a, rc0b, rs0b);
           }
           if (finisher) {
             const int mc = p.dual ? (m & 63) : m;
@@ -1103,11 +1111,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               ctl->gtile[m] = (p.next_g && m_on) ? p.next_g[n0 + mc] : 0.f;
             }
           }
-          W.wait(ctl->acc_full + buf, acc_phase[buf]);
+          W.wait(ctl->acc_full + buf, (acc_bits >> buf) & 1u);
           ok = group_ok(ctl, et);   // (its barriers also publish the staged constants)
           if (!ok) break;
           if (tracing && first_seg) { tr[4] = globaltimer_ns(); first_seg = false; }
-          acc_phase[buf] ^= 1;
+          acc_bits ^= 1u << buf;
           tc_fence_after();
           const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * 2 * P.t_box);
           unsigned long long* tra = (P.trace && et == 0 && !whole) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
@@ -1306,10 +1314,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                   // i + hd/2 of a head; with hd = 128 (a tile is one head) or 64 (two heads) both
                   // columns of a pair belong to the same thread.
                   int kv_row = kv_row0;
-                  float4 rc[2] = {rc0[0], rc0[1]}, rs[2] = {rs0[0], rs0[1]};
+                  float4 rca = rc0a, rcb = rc0b, rsa = rs0a, rsb = rs0b;
                   if (c0 != 0 && row_on) {
                     if (src_s >= 1) kv_row = kv_row_of(t);
-                    if (P.rope && src_s < 2) rope_of(t, rc, rs);
+                    if (P.rope && src_s < 2) rope_of(t, rca, rsa, rcb, rsb);
                   }
                   if (P.rope && src_s < 2) {
                     auto rot = [](float4& lo, float4& hi, const float4& cs, const float4& sn) {
@@ -1317,14 +1325,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                       lo = make_float4(l.x * cs.x - h.x * sn.x, l.y * cs.y - h.y * sn.y, l.z * cs.z - h.z * sn.z, l.w * cs.w - h.w * sn.w);
                       hi = make_float4(h.x * cs.x + l.x * sn.x, h.y * cs.y + l.y * sn.y, h.z * cs.z + l.z * sn.z, h.w * cs.w + l.w * sn.w);
                     };
-                    if (P.hd == 128) { rot(a[0], a[2], rc[0], rs[0]); rot(a[1], a[3], rc[1], rs[1]); }
-                    else { rot(a[0], a[1], rc[0], rs[0]); rot(a[2], a[3], rc[1], rs[1]); }
+                    if (P.hd == 128) { rot(a[0], a[2], rca, rsa); rot(a[1], a[3], rcb, rsb); }
+                    else { rot(a[0], a[1], rca, rsa); rot(a[2], a[3], rcb, rsb); }
                   }
                   const float qscale = src_s == 0 ? 1.0f / sqrtf((float)P.hd) : 1.0f;
                   const int nq_all = P.Hq * P.hd, nkv_all = P.Hkv * P.hd;
                   __half* dst = src_s == 0 ? P.q16 + (size_t)t * nq_all
                                            : reinterpret_cast<__half*>(src_s == 1 ? p.kc : p.vc) + (size_t)kv_row * nkv_all;
-                  const int colsrc0 = n0 - p.src_col[src_s];
+                  const int colsrc0 = n0 - src_col0;
 #pragma unroll
                   for (int q = 0; q < 4; ++q) {
                     if (on[q])
