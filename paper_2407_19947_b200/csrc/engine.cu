@@ -437,9 +437,11 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
   }
   const int i_head = 7 * m.n_layers, i_h = i_head + 1, i_o = i_head + 2, i_ff = i_head + 3;
   maps[i_head] = M.head_map;
-  bool ok = encode_map(ctx, &maps[i_h], ws + L.h, 2 * L.max_rows, d, t_box) &&
-            encode_map(ctx, &maps[i_o], ws + L.o, 2 * L.max_rows, nq, t_box) &&
-            encode_map(ctx, &maps[i_ff], ws + L.ff, 2 * L.max_rows, F, t_box);
+  // activation operands: the lo parts' rows follow the hi parts' t_box rows, so one box of
+  // 2 * t_box rows brings both
+  bool ok = encode_map(ctx, &maps[i_h], ws + L.h, 2 * L.max_rows, d, 2 * t_box) &&
+            encode_map(ctx, &maps[i_o], ws + L.o, 2 * L.max_rows, nq, 2 * t_box) &&
+            encode_map(ctx, &maps[i_ff], ws + L.ff, 2 * L.max_rows, F, 2 * t_box);
   if (!ok) return fail(ctx, STAIRS_ECUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
   std::vector<mk::Phase> ph;
   auto gemm = [&](int layer, int w0, int w1, int w2, int n_src, const int* rows, bool dual, int xmap, int K, int epi, void* out, int ldo) -> mk::Phase& {
@@ -591,7 +593,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.x = reinterpret_cast<float*>(ws + L.x); P.h = reinterpret_cast<bf16*>(ws + L.h); P.qkv = reinterpret_cast<float*>(ws + L.qkv);
   P.q16 = reinterpret_cast<__half*>(ws + L.q);
   P.o = reinterpret_cast<bf16*>(ws + L.o); P.ff = reinterpret_cast<bf16*>(ws + L.ff);
-  P.lo_row = L.max_rows;
+  P.lo_row = t_box;   // lo parts directly after the hi parts of this launch's row box
   P.keys = reinterpret_cast<unsigned long long*>(ws + L.keys); P.n_keys = L.max_rows;
   P.logits = c.logits;
   P.target_tokens = c.target_tokens; P.accept_len = c.accept_len; P.commit = c.commit; P.draft_out = c.draft_out;

@@ -751,8 +751,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           }
           if (B.ph <= ready_ph) {
             uint8_t* b_dst = smem + (size_t)b_stage * stage_bytes + A_STAGE_BYTES;
-            tma_load_2d(b_dst, P.maps + B.x_map, B.kk * BK, 0, ctl->full + b_stage, pol_x);
-            tma_load_2d(b_dst + b_stage_bytes, P.maps + B.x_map, B.kk * BK, P.lo_row, ctl->full + b_stage, pol_x);
+            tma_load_2d(b_dst, P.maps + B.x_map, B.kk * BK, 0, ctl->full + b_stage, pol_x);   // hi and lo rows in one box
             if (P.trace && cta == 0 && B.ph != traced_ph) { traced_ph = B.ph; P.trace[(size_t)B.ph * 8 + 7] = globaltimer_ns(); }
             ++b_count;
             if (++b_stage == stages) b_stage = 0;
