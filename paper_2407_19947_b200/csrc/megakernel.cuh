@@ -728,6 +728,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       uint32_t a_par = 0;
       unsigned int a_count = 0, b_count = 0, idle = 0;
       int ready_ph = -1;   // phases <= ready_ph have their inputs published
+      unsigned long long poll_val = 0; bool poll_pending = false;
       int traced_ph = -1;
       long long t_idle = clock64();
       while (B.valid) {
@@ -744,10 +745,13 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           progress = true;
         }
         if (b_count != a_count) {
-          // inputs of phase B.ph are published once every CTA has finished phase B.ph - 1; the
-          // poll is a global acquire load, so it is only made when no weight tile could be issued
-          if (B.ph > ready_ph && !progress) {
-            if (ld_acquire_u64(bar_count) >= P.bar_base + (unsigned long long)B.ph * G) { ready_ph = B.ph; fence_proxy_async(); }
+          // Inputs of phase B.ph are published once every CTA has finished phase B.ph - 1.  The
+          // poll is a global acquire load (a long round trip): it is issued in one pass of this
+          // loop and looked at in the next, so that weight tiles keep being issued under it.
+          if (B.ph > ready_ph) {
+            if (poll_pending && poll_val >= P.bar_base + (unsigned long long)B.ph * G) { ready_ph = B.ph; fence_proxy_async(); }
+            poll_pending = false;
+            if (B.ph > ready_ph) { poll_val = ld_acquire_u64(bar_count); poll_pending = true; }
           }
           if (B.ph <= ready_ph) {
             uint8_t* b_dst = smem + (size_t)b_stage * stage_bytes + A_STAGE_BYTES;
@@ -898,22 +902,45 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
               const int first_slot = u0 + (kvh * a.n_ranges) * a.n_qblk + qblk;
               const size_t stride = (size_t)a.n_qblk * ATT_QBLK * (hd + 4);
               const float* base = P.attn_part + ((size_t)first_slot * ATT_QBLK + ql) * (hd + 4);
-              float M = -INFINITY;
-              for (int rg = lane; rg < a.n_ranges; rg += 32) M = fmaxf(M, __ldcg(base + rg * stride + hd));
+              // (max, sum) of range lane, lane + 32, ...: one load round for up to 32 ranges, then
+              // the ranges' output vectors sixteen loads at a time; weights travel by shuffle and
+              // the accumulation stays in range order
+              const int nr = a.n_ranges, dd = lane * 4;
+              float M = -INFINITY, m0 = -INFINITY, l0 = 0.f;
+              for (int rb = 0; rb < nr; rb += 32) {
+                const int r = rb + lane;
+                float mu = -INFINITY, lu = 0.f;
+                if (r < nr) { mu = __ldcg(base + r * stride + hd); lu = __ldcg(base + r * stride + hd + 1); }
+                if (rb == 0) { m0 = mu; l0 = lu; }
+                M = fmaxf(M, mu);
+              }
               M = warp_max(M);
               float L = 0.f;
               float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-              const int dd = lane * 4;
-#pragma unroll 4
-              for (int rg = 0; rg < a.n_ranges; ++rg) {
-                const float* st = base + rg * stride;
-                const float mu = __ldcg(st + hd), lu = __ldcg(st + hd + 1);
-                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (dd < hd) v = __ldcg(reinterpret_cast<const float4*>(st + dd));
-                const float wgt = mu == -INFINITY ? 0.f : expf(mu - M);
+              for (int rb = 0; rb < nr; rb += 32) {
+                const int r = rb + lane;
+                float mu = m0, lu = l0;
+                if (rb != 0) {
+                  mu = -INFINITY; lu = 0.f;
+                  if (r < nr) { mu = __ldcg(base + r * stride + hd); lu = __ldcg(base + r * stride + hd + 1); }
+                }
+                const float wgt = mu == -INFINITY ? 0.f : expf(mu - M);   // 0 for lanes past the last range
                 L += lu * wgt;
-                acc.x += v.x * wgt; acc.y += v.y * wgt; acc.z += v.z * wgt; acc.w += v.w * wgt;
+                const int nb = min(32, nr - rb);
+                for (int g0 = 0; g0 < nb; g0 += 16) {
+                  float4 v[16];
+#pragma unroll
+                  for (int u = 0; u < 16; ++u)
+                    v[u] = (g0 + u < nb && dd < hd) ? __ldcg(reinterpret_cast<const float4*>(base + (size_t)(rb + g0 + u) * stride + dd))
+                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                  for (int u = 0; u < 16; ++u) {
+                    const float wu = __shfl_sync(0xffffffffu, wgt, (g0 + u) & 31);
+                    acc.x += v[u].x * wu; acc.y += v[u].y * wu; acc.z += v[u].z * wu; acc.w += v[u].w * wu;
+                  }
+                }
               }
+              L = warp_sum(L);
               if (dd < hd) {
                 bf16* orow = P.o + (size_t)(a.off + q / Gq) * P.Hq * hd + (size_t)(kvh * Gq + q % Gq) * hd + dd;
                 const float inv = 1.0f / L;
