@@ -41,15 +41,18 @@ def measured_peaks():
 
 
 def pick_workload(name: str):
-    idx = {"cfg2": 2, "cfg3": 3, "cfg4": 4}[name]
+    """(workload, prefix tokens in the cache, draft length k, requests per call)"""
+    idx = {"cfg2": 2, "cfg3": 3, "cfg4": 4, "cfg5": 5}[name]
     w = wl.workload(idx)
     if idx == 2:
-        prefix, k = 2048, 8
+        prefix, k, n_req = 2048, 8, 1
     elif idx == 3:
-        prefix, k = 512, 4
+        prefix, k, n_req = 512, 4, 1
+    elif idx == 4:
+        prefix, k, n_req = 1024, 8, 1
     else:
-        prefix, k = 1024, 8
-    return w, prefix, k
+        prefix, k, n_req = 16384, 8, 4     # four long requests validated in one call (36 stair rows)
+    return w, prefix, k, n_req
 
 
 class ClockSampler(threading.Thread):
@@ -89,9 +92,9 @@ class ClockSampler(threading.Thread):
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def algorithmic_bytes(shape, prefix: int, k: int) -> int:
-    """Bytes one validate call must move: every weight matrix once plus the visible K/V once."""
-    return shape.weight_bytes_per_call() + shape.kv_bytes_per_token() * (prefix + k + 1)
+def algorithmic_bytes(shape, prefix: int, k: int, n_req: int = 1) -> int:
+    """Bytes one validate call must move: every weight matrix once plus each request's visible K/V once."""
+    return shape.weight_bytes_per_call() + n_req * shape.kv_bytes_per_token() * (prefix + k + 1)
 
 
 def oracle_row_seconds(w, tsrc, prompt, draft, rows):
@@ -176,7 +179,7 @@ def run_reference(args, rank, world):
     if rank != 0:
         return
     from oracle import stairs_oracle as so
-    w, prefix, k = pick_workload(args.workload)
+    w, prefix, k, n_req = pick_workload(args.workload)
     tsrc, _ = wl.make_sources(w, backend="numpy")
     tgt = so.OracleModel(w.target, tsrc, keep=True)
     prompt = list(wl.prompt_tokens(w, n=prefix + 1))
@@ -196,13 +199,13 @@ def run_reference(args, rank, world):
         if i >= args.warmup:
             times.append((time.perf_counter() - t0) * (prefix + 1 + r) / len(row))
     row_s = float(np.mean(times))
-    value = row_s * (k + 1) * 1e6
+    value = row_s * (k + 1) * n_req * 1e6
     sample = (f"{args.steps} stair rows at prefix {p_s} of {prefix + 1}, one no-cache fp32 forward each, "
-              f"scaled linearly in tokens to the full prefix and to {k + 1} rows per call")
+              f"scaled linearly in tokens to the full prefix and to {n_req * (k + 1)} rows per call")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(np.mean(times)) * 1e3,
             "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"{w.name}: prefix {prefix}, k {k}, {k + 1} stair rows, 1 request"},
+            "config": {"workload": f"{w.name}: prefix {prefix}, k {k}, {n_req * (k + 1)} stair rows, {n_req} request{'s' if n_req > 1 else ''}"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -218,7 +221,7 @@ def run_ours(args, rank, local_rank, world):
         torch.cuda.set_device(local_rank)
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
         dist.barrier()
-    w, prefix, k = pick_workload(args.workload)
+    w, prefix, k, n_req = pick_workload(args.workload)
     if args.layers > 0:
         import dataclasses
         w = dataclasses.replace(w, name=f"{w.name}_first{args.layers}layers", target=w.target.replace(n_layers=args.layers),
@@ -227,32 +230,40 @@ def run_ours(args, rank, local_rank, world):
     tsrc, dsrc = wl.make_sources(w, backend="torch-cuda")
     torch.cuda.set_device(local_rank)
     max_seq = prefix + 256 if shape.pos == wl.POS_ROPE else min(prefix + 256, shape.max_pos)
-    eng = stairs.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=max_seq, k_max=k, kv_page_tokens=64,
+    eng = stairs.Stairs(tsrc, dsrc, max_requests=n_req, max_seq_len=max_seq, k_max=k, kv_page_tokens=64,
                         device_index=local_rank)
-    prompt = wl.prompt_tokens(w, n=prefix + 1)     # prefix tokens in the cache + the last committed token
-    eng.prefill(0, prompt)
+    reqs = list(range(n_req))
+    prompts = [wl.prompt_tokens(w, request=r, n=prefix + 1) for r in reqs]   # prefix in the cache + the last committed token
+    prompt = prompts[0]
+    for r in reqs:
+        eng.prefill(r, prompts[r])
     eng.sync()
-    # forced draft (first a tokens equal the target's own continuation, then a mismatch)
-    cont = []
-    for _ in range(k + 1):                       # k+1 plain greedy steps, then roll the request back
-        t_host, _ = eng.validate_host([0], [0], None, commit=True)
-        cont.append(int(t_host[0, 0]))
-    eng.truncate(0, len(prompt))
-    a_list = wl.forced_accept_lengths(k, 64, 1234)
-    drafts = np.stack([wl.forced_draft(np.array(cont), a, shape.vocab, 50 + i) for i, a in enumerate(a_list)])
+    # forced drafts (first a tokens equal the target's own continuation, then a mismatch), per request
+    n_var = 64 if n_req == 1 else 8
+    a_list = wl.forced_accept_lengths(k, n_var * n_req, 1234)
+    drafts = np.zeros((n_var, n_req, k), np.int32)
+    for r in reqs:
+        cont = []
+        for _ in range(k + 1):                   # k+1 plain greedy steps, then roll the request back
+            t_host, _ = eng.validate_host([r], [0], None, commit=True)
+            cont.append(int(t_host[0, 0]))
+        eng.truncate(r, len(prompts[r]))
+        for i in range(n_var):
+            drafts[i, r] = wl.forced_draft(np.array(cont), a_list[i * n_req + r], shape.vocab, 50 + i * n_req + r)
     d_dev = torch.from_numpy(drafts).to(eng.device)
-    tt = torch.zeros((1, k + 1), dtype=torch.int32, device=eng.device)
-    al = torch.zeros((1,), dtype=torch.int32, device=eng.device)
+    tt = torch.zeros((n_req, k + 1), dtype=torch.int32, device=eng.device)
+    al = torch.zeros((n_req,), dtype=torch.int32, device=eng.device)
     stream = eng.stream
 
     def step(i):
-        eng.validate([0], [k], d_dev[i % len(a_list)], commit=False, out=(tt, al))
+        eng.validate(reqs, [k] * n_req, d_dev[i % n_var], commit=False, out=(tt, al))
 
     # accept lengths must come out as forced (checks the path end to end before timing it)
-    for i in range(min(8, len(a_list))):
+    for i in range(min(8, n_var)):
         step(i)
         eng.sync()
-        assert int(al.cpu()[0]) == a_list[i], (int(al.cpu()[0]), a_list[i])
+        got = [int(x) for x in al.cpu()]
+        assert got == a_list[i * n_req:(i + 1) * n_req], (got, a_list[i * n_req:(i + 1) * n_req])
 
     def barrier():
         torch.cuda.synchronize()
@@ -291,11 +302,11 @@ def run_ours(args, rank, local_rank, world):
     # end to end through the host-buffer entry point (drafts in, tokens and accept length out)
     pin_d = torch.from_numpy(drafts).pin_memory()
     for i in range(0 if args.timed_only else 3):
-        eng.validate_host([0], [k], pin_d[i].numpy()[None])
+        eng.validate_host(reqs, [k] * n_req, pin_d[i].numpy())
     torch.cuda.synchronize()
     t0 = time.perf_counter()
     for i in range(0 if args.timed_only else args.steps):
-        eng.validate_host([0], [k], pin_d[i % len(a_list)].numpy()[None])
+        eng.validate_host(reqs, [k] * n_req, pin_d[i % n_var].numpy())
     e2e_s = time.perf_counter() - t0
 
     ms, e2e_ms = max_over_ranks([ms, e2e_s * 1e3], world, eng.device)
@@ -306,7 +317,7 @@ def run_ours(args, rank, local_rank, world):
     peaks, peak_kind = measured_peaks()
     peak = float(peaks["hbm_gbs"])
     wbytes = shape.weight_bytes_per_call()
-    abytes = algorithmic_bytes(shape, prefix, k)
+    abytes = algorithmic_bytes(shape, prefix, k, n_req)
     gemm_s_per_call = gemm_ms * 1e-3 / args.steps
     if gemm_n > 0:
         dominant = "k_gemm_tc: weight-streaming GEMMs (QKV, O, MLP, LM head), one launch each"
@@ -323,19 +334,19 @@ def run_ours(args, rank, local_rank, world):
         "metric": METRIC, "value": us_per_call, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{w.name}: prefix {prefix}, k {k}, {k + 1} stair rows, 1 request per GPU, commit=0",
+        "config": {"workload": f"{w.name}: prefix {prefix}, k {k}, {n_req * (k + 1)} stair rows, {n_req} request{'s' if n_req > 1 else ''} per GPU, commit=0",
                    "l2": "inputs larger than L2 (weights %.2f GB per call)" % (wbytes / 1e9),
                    "replicas": world},
         "clocks": clocks,
         "gpu_launches": int(launches),
         "e2e": {"value": e2e_ms * 1e3 / total_calls, "unit": UNIT,
-                "h2d_bytes_per_step": int(k * 4 + 3 * 4), "d2h_bytes_per_step": int((k + 1) * 4 + 4)},
+                "h2d_bytes_per_step": int(n_req * (k * 4 + 2 * 4) + 4), "d2h_bytes_per_step": int(n_req * ((k + 1) * 4 + 4))},
         "roofline": {"bound": "hbm", "kernel": dominant, "bytes_per_launch": roof_bytes,
                      "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak if achieved else None,
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS if achieved else None,
                      "peak_kind": f"of {peak_kind}", "traffic": stored_traffic(w.name) if gemm_n == 0 else None,
-                     "launches_per_call": gemm_n / max(args.steps, 1),
+                     "launches_per_call": (gemm_n if gemm_n > 0 else launches) / max(args.steps, 1),
                      "timing": roof_timing},
         "call": {"algorithmic_bytes": abytes, "hbm_gbs_whole_call": abytes / (us_per_call * 1e-6) / 1e9,
                  "frac_of_measured_peak": abytes / (us_per_call * 1e-6) / 1e9 / peak,
@@ -344,8 +355,8 @@ def run_ours(args, rank, local_rank, world):
     }
     # generation: tokens/s with stairs against k=0 greedy on the same kernels (short run)
     try:
-        if args.timed_only:
-            raise RuntimeError('skipped (--timed-only)')
+        if args.timed_only or n_req > 1:
+            raise RuntimeError('skipped (--timed-only, or a multi-request workload)')
         gen_prompt = prompt[: min(len(prompt), 512)]
         n_new = 48
         out0, st0 = eng.generate(0, gen_prompt, 0, n_new)
@@ -382,7 +393,7 @@ def run_ours(args, rank, local_rank, world):
                 del d_dev
                 tsrc.drop_cache()
                 torch.cuda.empty_cache()
-                w7, p7, k7 = pick_workload("cfg4")
+                w7, p7, k7, _ = pick_workload("cfg4")
                 t7, d7 = wl.make_sources(w7, backend="torch-cuda")
                 e7 = stairs.Stairs(t7, d7, max_requests=1, max_seq_len=p7 + 256, k_max=k7, kv_page_tokens=64,
                                    device_index=local_rank)
@@ -414,13 +425,13 @@ def run_ours(args, rank, local_rank, world):
         cb_prefix = min(prefix, args.cpu_prefix)
         osrc = tsrc
         cb_prompt = list(prompt[: cb_prefix + 1])
-        row_s, _ = oracle_row_seconds(w, osrc, cb_prompt, list(drafts[0]), [0])
+        row_s, _ = oracle_row_seconds(w, osrc, cb_prompt, list(drafts[0][0]), [0])
         n_rows = int(max(1, min(k + 1, 15.0 // max(row_s, 1e-3))))
         if n_rows > 1:
-            row_s, _ = oracle_row_seconds(w, osrc, cb_prompt, list(drafts[0]), list(range(n_rows)))
-        line["cpu_baseline"] = {"value": row_s * (k + 1) * 1e6, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
-                                "sample": f"{n_rows} of the {k + 1} stair rows at prefix {cb_prefix} "
-                                          f"(no-cache fp32 forwards), scaled to {k + 1} rows"}
+            row_s, _ = oracle_row_seconds(w, osrc, cb_prompt, list(drafts[0][0]), list(range(n_rows)))
+        line["cpu_baseline"] = {"value": row_s * (k + 1) * n_req * 1e6, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                "sample": f"{n_rows} of the {n_req * (k + 1)} stair rows at prefix {cb_prefix} "
+                                          f"(no-cache fp32 forwards), scaled to {n_req * (k + 1)} rows"}
     print(json.dumps(line))
     if eng is not None:
         eng.close()
@@ -432,7 +443,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--layers", type=int, default=0,
                     help="use only the first N layers of the workload's target (small captures under a profiler)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
