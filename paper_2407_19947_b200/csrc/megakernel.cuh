@@ -127,6 +127,10 @@ __device__ __forceinline__ void mma_16816(float* c, const uint32_t* a, uint32_t 
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void ldmatrix_x4(uint32_t* r, const void* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)));
+}
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, const void* p) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)));
@@ -494,17 +498,23 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
         float sc[4][4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) { sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f; }
-        for (int kk = 0; kk < ksteps; ++kk) {
-          uint32_t af[4];
-          const uint8_t* qa = qs + (size_t)ql_a * pitch + (kk * 16 + t4 * 2) * 2;
-          af[0] = *reinterpret_cast<const uint32_t*>(qa);
-          af[1] = *reinterpret_cast<const uint32_t*>(qa + 8 * pitch);
-          af[2] = *reinterpret_cast<const uint32_t*>(qa + 16);
-          af[3] = *reinterpret_cast<const uint32_t*>(qa + 8 * pitch + 16);
+        // Operand fragments by ldmatrix: for the queries one x4 per k-step (rows 0-7 / 8-15 of
+        // the block x the k-step's two 8-column halves), for K one x4 per pair of 8-position
+        // n-tiles (positions x the two halves).  Lane l supplies the address of matrix l / 8,
+        // row l % 8.
+        const uint8_t* q_lane = qs + (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * pitch + (lane >> 4) * 16;
+        const uint8_t* k_lane = ks + (size_t)(sl0 + (lane & 7) + (lane >> 4) * 8) * pitch + ((lane >> 3) & 1) * 16;
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint8_t* kb = ks + (size_t)(sl0 + 8 * j + g) * pitch + (kk * 16 + t4 * 2) * 2;
-            mma_16816(sc[j], af, *reinterpret_cast<const uint32_t*>(kb), *reinterpret_cast<const uint32_t*>(kb + 16));
+        for (int kk = 0; kk < 8; ++kk) {
+          if (kk < ksteps) {
+            uint32_t af[4], kf0[4], kf1[4];
+            ldmatrix_x4(af, q_lane + kk * 32);
+            ldmatrix_x4(kf0, k_lane + kk * 32);
+            ldmatrix_x4(kf1, k_lane + 16 * pitch + kk * 32);
+            mma_16816(sc[0], af, kf0[0], kf0[1]);
+            mma_16816(sc[1], af, kf0[2], kf0[3]);
+            mma_16816(sc[2], af, kf1[0], kf1[1]);
+            mma_16816(sc[3], af, kf1[2], kf1[3]);
           }
         }
         // staircase mask (rows past the chunk's last position hold stale data: assigned, never
