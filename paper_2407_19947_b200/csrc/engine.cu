@@ -502,12 +502,16 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
     const stairs_layer_w& w = M.layers[l];
     const int b = 7 * l;
     const int r3[3] = {nq, nkv, nkv};
+    const bool in_epilogue = m.pos == 0 || m.head_dim == 64 || m.head_dim == 128;
     {
       mk::Phase& p = gemm(l, b + 0, b + 1, b + 2, 3, r3, false, i_h, d, tc::TC_STORE_F32, ws + L.qkv, nqkv);
       p.norm_in = 1; p.u = aux_ptr(l, 0); p.c = aux_ptr(l, 1);
-      p.qkv_prep = 1;   // q to the query buffer, k and v (fp16) to this layer's cache rows
+      // q to the query buffer, k and v (fp16) to this layer's cache rows: in the epilogue where a
+      // rotation pair sits in one thread (head size 64 or 128, or no rotation), else in a phase of its own
+      p.qkv_prep = in_epilogue ? 1 : 0;
       p.kc = M.kpool + (size_t)l * M.kv_layer_bytes; p.vc = M.vpool + (size_t)l * M.kv_layer_bytes;
     }
+    if (!in_epilogue) simple(mk::PH_PREP, l, nullptr, M.kpool + (size_t)l * M.kv_layer_bytes, M.vpool + (size_t)l * M.kv_layer_bytes);
     simple(mk::PH_ATTN, l, nullptr, M.kpool + (size_t)l * M.kv_layer_bytes, M.vpool + (size_t)l * M.kv_layer_bytes);
     simple(mk::PH_COMBINE, l, nullptr, nullptr, nullptr);
     const int rd[1] = {d};
@@ -558,8 +562,7 @@ struct MkCall {
 bool mk_eligible(const stairs_ctx* ctx, const DevModel& M, int T) {
   // (the epilogue's vector stores want every GEMM width but the vocabulary to be a multiple of 4)
   return ctx->use_mk && M.m.n_layers >= 1 && T >= 1 && T <= MK_MAX_ROWS && M.m.head_dim % 16 == 0 && M.m.head_dim <= 128 &&
-         M.m.d_model % 4 == 0 && M.m.d_ff % 4 == 0 && M.m.d_model <= 8192 &&
-         (M.m.pos == 0 || M.m.head_dim == 64 || M.m.head_dim == 128);   // rotation pairs must sit in one thread of the QKV epilogue
+         M.m.d_model % 4 == 0 && M.m.d_ff % 4 == 0 && M.m.d_model <= 8192;
 }
 
 int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, int n_logit_rows, const MkCall& c) {

@@ -36,7 +36,7 @@ namespace mk {
 
 using namespace tc;
 
-enum PhaseKind { PH_EMBED = 0, PH_GEMM = 2, PH_ATTN = 3, PH_COMBINE = 4, PH_ACCEPT = 6 };
+enum PhaseKind { PH_EMBED = 0, PH_GEMM = 2, PH_ATTN = 3, PH_COMBINE = 4, PH_PREP = 5, PH_ACCEPT = 6 };
 
 struct Phase {
   int kind, layer;
@@ -314,6 +314,19 @@ __device__ __forceinline__ RowInfo row_info(const Params& P, int t) {
     r.tok = clampv(P.draft[P.draft_step - 1]);
   }
   return r;
+}
+
+// Row of the K/V pools that holds the position of the call's row t.
+__device__ __forceinline__ int cache_row_of(const Params& P, int t) {
+  int slot, pos;
+  if (P.mode == CALL_VALIDATE) {
+    int i = 0;
+    while (i + 1 < P.n_req && P.val_off[i + 1] <= t) ++i;
+    slot = P.val_req[i]; pos = P.n_seq[slot] - 1 + (t - P.val_off[i]);
+  } else if (P.mode == CALL_PREFILL) { slot = P.slot; pos = P.draft_step + t; }
+  else if (P.mode == CALL_DRAFT_FIRST) { slot = P.slot; pos = P.n_seq[slot] - 2 + t; }
+  else { slot = P.slot; pos = P.n_seq[slot] - 1 + P.draft_step; }
+  return P.page_table[(size_t)slot * P.max_pages + pos / P.page_tokens] * P.page_tokens + pos % P.page_tokens;
 }
 
 // sum over the 128 compute threads (4 warps); red = 4 floats
@@ -965,6 +978,32 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           }
           u0 += a.units;
         }
+      } else if (p.kind == PH_PREP) {
+        // Models whose head size is neither 64 nor 128: a rotation pair (i, i + hd/2) need not sit in
+        // one thread (or one tile) of the QKV epilogue, so that epilogue stores fp32 and this extra
+        // phase rotates, converts and files q, k and v.  One item = one pair of one head of one row.
+        const int hd = P.hd, half = hd / 2, nq = P.Hq * hd, nkv = P.Hkv * hd, nqkv = nq + 2 * nkv, heads = P.Hq + 2 * P.Hkv;
+        const int items = P.T * heads * half;
+        const float qscale = 1.0f / sqrtf((float)hd);
+        for (int it = cta * 128 + et; it < items; it += G * 128) {
+          const int i = it % half, hs = (it / half) % heads, t = it / (half * heads);
+          const float* row = P.qkv + (size_t)t * nqkv + (size_t)hs * hd;   // q heads, then k heads, then v heads
+          float x0 = __ldcg(row + i), x1 = __ldcg(row + i + half);
+          if (P.rope && hs < P.Hq + P.Hkv) {
+            const float cs = __ldcg(P.rope_cs + (size_t)t * half + i), sn = __ldcg(P.rope_sn + (size_t)t * half + i);
+            const float r0 = x0 * cs - x1 * sn, r1 = x1 * cs + x0 * sn;
+            x0 = r0; x1 = r1;
+          }
+          if (hs < P.Hq) {
+            __half* dst = P.q16 + (size_t)t * nq + (size_t)hs * hd;
+            dst[i] = __float2half_rn(x0 * qscale); dst[i + half] = __float2half_rn(x1 * qscale);
+          } else {
+            const bool is_k = hs < P.Hq + P.Hkv;
+            __half* dst = reinterpret_cast<__half*>(is_k ? p.kc : p.vc) + (size_t)cache_row_of(P, t) * nkv +
+                          (size_t)(hs - P.Hq - (is_k ? 0 : P.Hkv)) * hd;
+            dst[i] = __float2half_rn(x0); dst[i + half] = __float2half_rn(x1);
+          }
+        }
       } else if (p.kind == PH_ACCEPT) {
         if (cta == 0) {
           if (P.mode == CALL_VALIDATE) {
@@ -1104,17 +1143,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           // table entries of its column groups (q and k tiles), for the first chunk
           int kv_row0 = 0;
           float4 rc0a, rc0b, rs0a, rs0b;
-          auto kv_row_of = [&](int t) {
-            int slot, pos;
-            if (P.mode == CALL_VALIDATE) {
-              int i = 0;
-              while (i + 1 < P.n_req && P.val_off[i + 1] <= t) ++i;
-              slot = P.val_req[i]; pos = P.n_seq[slot] - 1 + (t - P.val_off[i]);
-            } else if (P.mode == CALL_PREFILL) { slot = P.slot; pos = P.draft_step + t; }
-            else if (P.mode == CALL_DRAFT_FIRST) { slot = P.slot; pos = P.n_seq[slot] - 2 + t; }
-            else { slot = P.slot; pos = P.n_seq[slot] - 1 + P.draft_step; }
-            return P.page_table[(size_t)slot * P.max_pages + pos / P.page_tokens] * P.page_tokens + pos % P.page_tokens;
-          };
+          auto kv_row_of = [&](int t) { return cache_row_of(P, t); };
           auto rope_of = [&](int t, float4& c0, float4& s0, float4& c1, float4& s1) {
             // hd = 128: groups (0, 2) and (1, 3) pair up, at table columns cg*4 and 32 + cg*4;
             // hd = 64: groups (0, 1) and (2, 3), both at table column cg*4
