@@ -395,7 +395,7 @@ __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
   // chunks per unit: from the first row's position only (so it is the same for any draft length)
   const int c0 = (a.base + ATT_CHUNK) / ATT_CHUNK;
   int cpu = 1;
-  while (cpu < 64 && (c0 * P.Hkv) / cpu > G) cpu <<= 1;   // one unit per CTA where possible: a unit's fixed cost exceeds a chunk's
+  while (cpu < 64 && P.Hkv * ((c0 + cpu - 1) / cpu) > G) cpu <<= 1;   // one unit per CTA where possible: a unit's fixed cost exceeds a chunk's
   a.cpu = cpu;
   a.n_ranges = (a.n_chunks + cpu - 1) / cpu;
   a.n_qblk = (a.R * (P.Hq / P.Hkv) + ATT_QBLK - 1) / ATT_QBLK;
