@@ -581,7 +581,9 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   const int n_run = c.skip_head ? M.n_phases - 2 : M.n_phases;
   P.phases = reinterpret_cast<const mk::Phase*>(base); P.n_phases = n_run;
   P.maps = reinterpret_cast<const CUtensorMap*>(base + M.prog_maps_off);
-  P.T = T; P.t_box = t_box; P.stages = mk::pick_stages(t_box, m.head_dim);
+  P.T = T; P.t_box = t_box; // two K/V chunk buffers where they are cheap (small heads) or needed (contexts so long that a unit walks several chunks)
+  P.att_dbl = (m.head_dim <= 64 || (long long)ctx->cfg.max_seq_len * m.n_kv_heads / mk::ATT_CHUNK > ctx->sm_count) ? 1 : 0;
+  P.stages = mk::pick_stages(t_box, m.head_dim, P.att_dbl);
   P.logit_first_row = logit_first_row; P.n_logit_rows = n_logit_rows;
   P.d = m.d_model; P.Hq = m.n_heads; P.Hkv = m.n_kv_heads; P.hd = m.head_dim; P.F = m.d_ff; P.vocab = m.vocab;
   P.norm_kind = m.norm; P.rope = m.pos; P.rope_theta = m.rope_theta; P.eps = m.norm_eps;
@@ -611,7 +613,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   const int grid = std::min(ctx->sm_count, TC_GRID_MAX);
   void* args[] = {&P};
   CK(cudaLaunchCooperativeKernel((const void*)mk::k_forward, dim3(grid), dim3(tc::THREADS), args,
-                                 mk::smem_bytes(t_box, P.stages, m.head_dim), ctx->stream));
+                                 mk::smem_bytes(t_box, P.stages, m.head_dim, P.att_dbl), ctx->stream));
   ctx->bar_base += (unsigned long long)n_run * grid;
   ctx->launches++;
   return STAIRS_OK;
@@ -939,7 +941,7 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
       const int hdm = has_draft ? std::max(cfg->target.head_dim, cfg->draft.head_dim) : cfg->target.head_dim;
       const long long worst_chunks = ((long long)cfg->max_seq_len + mk::ATT_CHUNK - 1) / mk::ATT_CHUNK;
       const int hkvm = has_draft ? std::max(cfg->target.n_kv_heads, cfg->draft.n_kv_heads) : cfg->target.n_kv_heads;
-      const bool fits = mk::pick_stages(MK_MAX_ROWS, hdm) >= 3 && worst_chunks * hkvm / 64 <= 2 * std::min(ctx->sm_count, TC_GRID_MAX);
+      const bool fits = mk::pick_stages(MK_MAX_ROWS, hdm, 1) >= 3 && worst_chunks * hkvm / 64 <= 2 * std::min(ctx->sm_count, TC_GRID_MAX);
       if (coop && fits && cfg->gemm_impl == 0) {
         e = cudaFuncSetAttribute(mk::k_forward, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_LIMIT);
         if (e == cudaSuccess) {

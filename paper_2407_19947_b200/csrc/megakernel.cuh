@@ -83,6 +83,7 @@ struct Params {
   float4* stats;            // [64 rows][stat_tiles] (mean, M2, count, -) per 128-column tile of x
   int stat_tiles;
   const float* rope_inv;
+  int att_dbl;               // attention: two K/V chunk buffers, the next chunk's copies fly under the current chunk's MMAs
   __half* q16;               // [row][Hq*hd] queries, rotated and scaled by 1/sqrt(hd), written by the QKV epilogue
   float* rope_cs; float* rope_sn;   // [row][hd/2] cos and sin of the call's row positions, written by the embedding phase
      // [hd/2] theta^(-2i/hd)
@@ -110,7 +111,7 @@ struct AttnSmem {   // carved after the GEMM ring: Q block (bf16), K and V chunk
   static __host__ __device__ size_t q_bytes(int hd) { return (size_t)ATT_QBLK * k_pitch(hd); }
   static __host__ __device__ size_t kv_bytes(int hd) { return (size_t)ATT_CHUNK * k_pitch(hd); }
   static __host__ __device__ size_t merge_bytes(int hd) { return (size_t)16 * (hd + 4) * 4 + 64; }
-  static __host__ __device__ size_t bytes(int hd) { return q_bytes(hd) + 2 * kv_bytes(hd) + 64; }
+  static __host__ __device__ size_t bytes(int hd, int dbl) { return q_bytes(hd) + (dbl ? 4 : 2) * kv_bytes(hd) + 64; }   // dbl: two K/V chunk buffers
 };
 
 // 16-byte asynchronous copy global -> shared; `on` false writes zeros and reads nothing
@@ -119,6 +120,8 @@ __device__ __forceinline__ void cp_async16(void* dst, const void* src, bool on) 
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(n) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
 // mma.sync m16n8k16 (fp16 in, fp32 accumulate) and its operand loads, for the attention tiles:
 // queries, cached K/V and the softmax weights are fp16 (11 significant bits)
@@ -234,7 +237,7 @@ struct Ctl {
   volatile int last_flag;
   volatile int bcast;
   float rstd[64], mu[64];       // per-row statistics of the current norm_in GEMM phase
-  int rowbase[64];              // attention staging: cache row of each position of the chunk
+  int rowbase[2][64];           // attention staging: cache row of each position of the chunk (per chunk buffer)
   AttnReq areq[64];             // per request, filled once per launch (a request has at least one row: <= 64)
   alignas(16) uint32_t phc[2][(sizeof(Phase) + 3) / 4];   // this and the next phase's descriptor (global memory is a
                                                           // long round trip with the L1 carved down to almost nothing)
@@ -421,8 +424,10 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   const int q0 = qblk * ATT_QBLK, nQ = min(ATT_QBLK, Q - q0);
   const size_t pitch = AttnSmem::k_pitch(hd);
   uint8_t* qs = att_smem;                                   // [QBLK][pitch] bf16, rotated and pre-scaled
-  uint8_t* ks = qs + AttnSmem::q_bytes(hd);                 // [CHUNK][pitch]
-  uint8_t* vs = ks + AttnSmem::kv_bytes(hd);
+  uint8_t* kv0 = qs + AttnSmem::q_bytes(hd);                // chunk buffer b: K [CHUNK][pitch] then V, at kv0 + b * 2 * kv_bytes
+  const size_t kvb = AttnSmem::kv_bytes(hd);
+  uint8_t* ks = kv0;                                        // the buffer being computed on
+  uint8_t* vs = ks + kvb;
   __half* kc = reinterpret_cast<__half*>(ph.kc);
   __half* vc = reinterpret_cast<__half*>(ph.vc);
   const int* pt = P.page_table + (size_t)a.slot * P.max_pages;
@@ -438,13 +443,16 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   // microseconds.  The rows of this call's new positions are in the cache already: the QKV
   // epilogue put them there, as it put the rotated and scaled queries into the query buffer.
   const int pieces = hd * 2 / 16;   // 16-byte pieces per row
-  auto stage = [&](int c, bool with_q) {
+  auto stage_issue = [&](int c, int b, bool with_q) {
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
+    uint8_t* kd = kv0 + (size_t)b * 2 * kvb;
+    uint8_t* vd = kd + kvb;
+    int* rowbase = ctl->rowbase[b];
     // cache row of each position of the chunk, looked up once (-1: past the end)
     if (et < ATT_CHUNK) {
       const int pz = p0 + et;
-      ctl->rowbase[et] = et < n_pos ? pt[pz / P.page_tokens] * P.page_tokens + (pz % P.page_tokens) : -1;
+      rowbase[et] = et < n_pos ? pt[pz / P.page_tokens] * P.page_tokens + (pz % P.page_tokens) : -1;
     }
     epi_bar_sync();
     {
@@ -453,11 +461,11 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
       int jr = et / pieces, pc = et % pieces;
       const size_t head_off = (size_t)kvh * hd;
       while (jr < ATT_CHUNK) {
-        const int rb = ctl->rowbase[jr];
+        const int rb = rowbase[jr];
         const bool on = rb >= 0;
         const size_t off = (size_t)(on ? rb : 0) * nkv + head_off;
-        cp_async16(ks + jr * pitch + pc * 16, reinterpret_cast<const uint4*>(kc + off) + pc, on);
-        cp_async16(vs + jr * pitch + pc * 16, reinterpret_cast<const uint4*>(vc + off) + pc, on);
+        cp_async16(kd + jr * pitch + pc * 16, reinterpret_cast<const uint4*>(kc + off) + pc, on);
+        cp_async16(vd + jr * pitch + pc * 16, reinterpret_cast<const uint4*>(vc + off) + pc, on);
         jr += dj; pc += dp;
         if (pc >= pieces) { pc -= pieces; ++jr; }
       }
@@ -475,12 +483,11 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
         if (pc >= pieces) { pc -= pieces; ++ql; }
       }
     }
-    cp_async_wait_all();
-    epi_bar_sync();
+    cp_async_commit();
   };
 
   if (tra) tra[1] = globaltimer_ns();
-  stage(c_begin, true);
+  stage_issue(c_begin, 0, true);
   if (tra) tra[2] = globaltimer_ns();
 
   // Warp w owns query block (MMA M tile) w of the unit and walks the chunk's four 16-position
@@ -499,8 +506,14 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
 #pragma unroll
   for (int nd = 0; nd < 16; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
 
+  int cur = 0;
   for (int c = c_begin; c < c_end && ok; ++c) {
-    if (c != c_begin) stage(c, false);
+    // with two chunk buffers the next chunk's copies are issued before this chunk is waited for
+    const bool ahead = P.att_dbl && c + 1 < c_end;
+    if (ahead) { stage_issue(c + 1, cur ^ 1, false); cp_async_wait_but_one(); }
+    else cp_async_wait_all();
+    epi_bar_sync();
+    ks = kv0 + (size_t)cur * 2 * kvb; vs = ks + kvb;
     if (tra && c == c_begin) tra[4] = globaltimer_ns();
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
@@ -591,7 +604,10 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     }
     epi_bar_sync();   // tile may be overwritten by the next chunk or unit
     if (tra && c == c_begin) tra[5] = globaltimer_ns();
+    if (P.att_dbl) cur ^= 1;
+    else if (c + 1 < c_end) stage_issue(c + 1, 0, false);
   }
+  ks = kv0; vs = ks + kvb;   // (buffer 0 serves the merge below)
   if (!ok) return;
   if (ps == 2) {
     // second half's state -> shared memory (the K/V tiles are free now) -> merged into the first's
@@ -1478,13 +1494,13 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, tmem_cols); }
 }
 
-inline size_t smem_bytes(int t_box, int stages, int hd) {
+inline size_t smem_bytes(int t_box, int stages, int hd, int dbl) {
   return 1024 + (size_t)stages * (A_STAGE_BYTES + (size_t)2 * t_box * BK * 2) + MK_XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127) +
-         AttnSmem::bytes(hd) + 64;
+         AttnSmem::bytes(hd, dbl) + 64;
 }
-inline int pick_stages(int t_box, int hd) {
+inline int pick_stages(int t_box, int hd, int dbl) {
   int s = MAX_STAGES;
-  while (s > 1 && smem_bytes(t_box, s, hd) > (size_t)SMEM_LIMIT) --s;
+  while (s > 1 && smem_bytes(t_box, s, hd, dbl) > (size_t)SMEM_LIMIT) --s;
   return s;
 }
 
