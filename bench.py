@@ -407,11 +407,34 @@ def run_ours(args, rank, local_rank, world):
                     per_k[f"k{kk}"] = {"us_per_call": us, "hbm_gbs": ab / (us * 1e-6) / 1e9,
                                        "frac_of_measured_peak": ab / (us * 1e-6) / 1e9 / peak,
                                        "frac_of_nominal_8TBs": ab / (us * 1e-6) / 1e9 / NOMINAL_HBM_GBS}
-                g0, s0 = e7.generate(0, wl.prompt_tokens(w7, n=p7), 0, 32)
-                g4, s4 = e7.generate(0, wl.prompt_tokens(w7, n=p7), 4, 32)
+                g0, s0 = e7.generate(0, wl.prompt_tokens(w7, n=p7), 0, 96)
+                g4, s4 = e7.generate(0, wl.prompt_tokens(w7, n=p7), 4, 96)
+                # forced-acceptance sweep: drafts come from the known greedy continuation, each token
+                # corrupted with probability 1 - alpha; tokens/s of the validate loop alone (no draft
+                # model), against its own alpha = 0 and against k = 0 greedy
+                sweep = {}
+                kf, n_gen = 4, 64
+                base_prompt = wl.prompt_tokens(w7, n=p7)
+                rngf = np.random.default_rng(7)
+                for alpha in (0.0, 0.5, 0.8, 1.0):
+                    e7.prefill(0, base_prompt)
+                    produced, calls = 0, 0
+                    torch.cuda.synchronize()
+                    t0 = time.perf_counter()
+                    while produced < n_gen:
+                        want = np.array(g0[produced:produced + kf] + [0] * kf, dtype=np.int32)[:kf]
+                        bad = rngf.random(kf) >= alpha
+                        want = np.where(bad, (want + 1) % w7.target.vocab, want).astype(np.int32)
+                        _, acc = e7.validate_host([0], [kf], want[None], commit=True)
+                        produced += int(acc[0]) + 1
+                        calls += 1
+                    dt = time.perf_counter() - t0
+                    sweep[f"alpha_{alpha}"] = {"tokens_per_s": produced / dt, "validate_calls": calls,
+                                               "tokens_per_call": produced / calls}
                 line["target_7b"] = {"workload": f"{w7.name}: prefix {p7}", "validate": per_k,
-                                     "greedy_tokens_per_s": 32 / ((s0["total_ms"] - s0["prefill_ms"]) * 1e-3),
-                                     "stairs_k4_tokens_per_s": 32 / ((s4["total_ms"] - s4["prefill_ms"]) * 1e-3),
+                                     "forced_acceptance_k4": sweep,
+                                     "greedy_tokens_per_s": 96 / ((s0["total_ms"] - s0["prefill_ms"]) * 1e-3),
+                                     "stairs_k4_tokens_per_s": 96 / ((s4["total_ms"] - s4["prefill_ms"]) * 1e-3),
                                      "acceptance_k4": s4["accepted"] / max(s4["drafted"], 1),
                                      "identical_output": g0 == g4}
                 e7.close()
