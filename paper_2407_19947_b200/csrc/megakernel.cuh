@@ -1480,12 +1480,16 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       atomicExch(P.bar + 1, 1ull);   // tell the other CTAs
       *reinterpret_cast<volatile unsigned int*>(P.status + STATUS_ERROR) = 5u;  // STAIRS_ETIMEOUT
       __threadfence_system();
+      // let the copies in flight land before the CTA's shared memory is given up (a stage whose
+      // activation tile was never issued cannot complete: the loop is bounded, by at least ~1 ms so
+      // that a very short wait limit still leaves the copies time to finish)
       const long long t0 = clock64();
+      const unsigned long long drain_limit = P.wait_limit > 2000000ull ? P.wait_limit : 2000000ull;
       int s = p_stage; uint32_t phs = p_phase;
       for (int i = 0; i < stages && i < issued; ++i) {
         if (--s < 0) { s = stages - 1; phs ^= 1; }
         while (!mbar_try(ctl->full + s, phs)) {
-          if ((unsigned long long)(clock64() - t0) > P.wait_limit) break;
+          if ((unsigned long long)(clock64() - t0) > drain_limit) break;
         }
       }
     }

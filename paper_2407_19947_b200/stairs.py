@@ -145,7 +145,8 @@ class Stairs:
     """One library context: a target model, an optional draft model, request slots."""
 
     def __init__(self, target_source, draft_source=None, *, max_requests=1, max_seq_len=512, k_max=8,
-                 kv_page_tokens=64, kv_pages=0, prefill_chunk=0, device_index=0, gemm_impl=0, stream=None):
+                 kv_page_tokens=64, kv_pages=0, prefill_chunk=0, device_index=0, gemm_impl=0, stream=None,
+                 wait_limit_cycles=0):
         import torch
         self.torch = torch
         self.lib = load_library()
@@ -165,6 +166,7 @@ class Stairs:
         cfg.max_requests, cfg.max_seq_len, cfg.k_max = max_requests, max_seq_len, k_max
         cfg.kv_page_tokens, cfg.kv_pages, cfg.prefill_chunk = kv_page_tokens, kv_pages, prefill_chunk
         cfg.device, cfg.gemm_impl = device_index, gemm_impl
+        cfg.wait_limit_cycles = int(wait_limit_cycles)   # 0: the library's default bound for device-side waits
         self.stream = stream if stream is not None else torch.cuda.current_stream()
         cfg.stream = self.stream.cuda_stream
         need = self.lib.stairs_workspace_bytes(C.byref(cfg))

@@ -245,6 +245,27 @@ def test_error_paths_return_codes_and_leave_the_context_usable():
     eng.close()
 
 
+def test_expired_device_wait_is_reported_and_the_gpu_stays_usable():
+    """Every wait inside the persistent kernel is bounded.  With the bound set to about a microsecond the
+    waits of a healthy call run out: the kernel must drain and exit by itself, the next sync must
+    report STAIRS_ETIMEOUT (5), and a context with the default bound must work afterwards."""
+    st = _stairs()
+    shape = small_b()
+    tsrc, dsrc = sources(shape)
+    prompt = list(wl.uniform_tokens(40, shape.vocab, 3))
+    eng = st.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=128, k_max=4, wait_limit_cycles=2000)
+    with pytest.raises(st.StairsError) as e:
+        eng.prefill(0, prompt)
+        eng.sync()
+    assert e.value.code == 5
+    eng.close()
+    eng = st.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=128, k_max=4)
+    eng.prefill(0, prompt)
+    tt, al = eng.validate_host([0], [2], np.array([[7, 8, 0, 0]], np.int32))
+    assert 0 <= int(al[0]) <= 2
+    eng.close()
+
+
 @pytest.mark.parametrize("shape", [small_b(8, 2, 64), small_b(4, 4, 80, d=320, f=640), small_a()],
                          ids=["gqa_hd64", "mha_hd80", "family_a"])
 def test_long_prefix_positions_split_over_several_units(shape):
