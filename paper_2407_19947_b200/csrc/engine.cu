@@ -1207,14 +1207,20 @@ int stairs_sync(stairs_ctx* ctx) {
   CK(cudaStreamSynchronize(ctx->stream));
   if (ctx->status_host && ctx->status_host[STATUS_ERROR]) {
     const unsigned int code = ctx->status_host[STATUS_ERROR];
+    const unsigned int where[5] = {ctx->status_host[STATUS_WHERE], ctx->status_host[2], ctx->status_host[3], ctx->status_host[4],
+                                   ctx->status_host[5]};
     ctx->status_host[STATUS_ERROR] = 0;
+    for (int i = 1; i <= 5; ++i) ctx->status_host[i] = 0;
     cudaMemsetAsync(ctx->ws + ctx->lay.mk_bar, 0, 64, ctx->stream);   // barrier count and abort word
     cudaMemsetAsync(ctx->ws + ctx->lay.gemm_counters, 0, (size_t)TC_COUNTERS * 4, ctx->stream);
     cudaMemsetAsync(ctx->ws + ctx->lay.mk_partial, 0xff, ctx->lay.mk_partial_bytes, ctx->stream);   // every word empty again
     cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)ctx->lay.attn_cnt_n * 4, ctx->stream);
     cudaStreamSynchronize(ctx->stream);
     ctx->bar_base = 0;
-    return fail(ctx, (int)code, "a device-side bounded wait expired (code %u); results of the last calls are invalid", code);
+    // kind: 1 shared-memory barrier (block, thread, parity), 2 grid barrier (block, thread, target),
+    // 3 split-tile partial sums (phase, block, first segment awaited, tile << 8 | row)
+    return fail(ctx, (int)code, "a device-side bounded wait expired (code %u; first: kind %u at %u, %u, %u, %u); results of the last calls are invalid",
+                code, where[0], where[1], where[2], where[3], where[4]);
   }
   return STAIRS_OK;
 }

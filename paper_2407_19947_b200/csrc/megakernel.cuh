@@ -263,6 +263,12 @@ __device__ __forceinline__ bool group_ok(Ctl* ctl, int et) {
 
 struct Waiter {
   volatile int* abort_flag; const unsigned long long* gabort; unsigned long long limit;
+  unsigned int* status;   // host-visible status words: [1] kind of the first wait that ran out, [2..5] where
+  // first expired wait of the launch leaves a note for the host's error text
+  __device__ __forceinline__ void note(unsigned int kind, unsigned int a, unsigned int b, unsigned int c, unsigned int d) const {
+    volatile unsigned int* s = status;   // (plain accesses: the words live in mapped host memory; a lost race only costs detail)
+    if (s[STATUS_WHERE] == 0u) { s[STATUS_WHERE] = kind; s[2] = a; s[3] = b; s[4] = c; s[5] = d; }
+  }
   __device__ __forceinline__ bool poll_abort(long long t0) const {
     if (*abort_flag) return true;
     if ((unsigned long long)(clock64() - t0) > limit) { *abort_flag = 1; return true; }
@@ -275,7 +281,10 @@ struct Waiter {
     int spins = 0;
     while (true) {
       if (mbar_try(bar, parity)) return true;
-      if (poll_abort(t0)) return false;
+      if (poll_abort(t0)) {
+        if ((unsigned long long)(clock64() - t0) > limit) note(1u, (unsigned)blockIdx.x, (unsigned)threadIdx.x, parity, 0u);
+        return false;
+      }
       if ((++spins & 255) == 0 && ld_acquire_u64(gabort)) { *abort_flag = 1; return false; }
     }
   }
@@ -284,7 +293,10 @@ struct Waiter {
     const long long t0 = clock64();
     int spins = 0;
     while (ld_acquire_u64(counter) < target) {
-      if (poll_abort(t0)) return false;
+      if (poll_abort(t0)) {
+        if ((unsigned long long)(clock64() - t0) > limit) note(2u, (unsigned)blockIdx.x, (unsigned)threadIdx.x, (unsigned)target, 0u);
+        return false;
+      }
       if ((++spins & 63) == 0 && ld_acquire_u64(gabort)) { *abort_flag = 1; return false; }
     }
     return true;
@@ -715,7 +727,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_slot;
-  const Waiter W{&ctl->abort_flag, P.bar + 1, P.wait_limit};
+  const Waiter W{&ctl->abort_flag, P.bar + 1, P.wait_limit, P.status};
   const unsigned long long* bar_count = P.bar;
   // producer bookkeeping for the abort path
   int issued = 0, p_stage = 0;
@@ -1294,6 +1306,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                         }
                       }
                     } while (!all_there && !W.poll_abort(t0));
+                    if (!all_there && (unsigned long long)(clock64() - t0) > P.wait_limit)
+                      W.note(3u, (unsigned)ph, (unsigned)cta, c, ((unsigned)tile << 8) | (unsigned)t);
                     const float4 empty4 = make_float4(__uint_as_float(PARTIAL_EMPTY), __uint_as_float(PARTIAL_EMPTY),
                                                       __uint_as_float(PARTIAL_EMPTY), __uint_as_float(PARTIAL_EMPTY));
 #pragma unroll
