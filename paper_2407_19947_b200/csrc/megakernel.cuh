@@ -267,7 +267,8 @@ struct Waiter {
   // first expired wait of the launch leaves a note for the host's error text
   __device__ __forceinline__ void note(unsigned int kind, unsigned int a, unsigned int b, unsigned int c, unsigned int d) const {
     volatile unsigned int* s = status;   // (plain accesses: the words live in mapped host memory; a lost race only costs detail)
-    if (s[STATUS_WHERE] == 0u) { s[STATUS_WHERE] = kind; s[2] = a; s[3] = b; s[4] = c; s[5] = d; }
+    // a wait for partial sums (kind 3) is the likelier root cause than the barrier waits stuck behind it
+    if (s[STATUS_WHERE] == 0u || (kind == 3u && s[STATUS_WHERE] != 3u)) { s[STATUS_WHERE] = kind; s[2] = a; s[3] = b; s[4] = c; s[5] = d; }
   }
   __device__ __forceinline__ bool poll_abort(long long t0) const {
     if (*abort_flag) return true;
