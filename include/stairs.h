@@ -196,8 +196,7 @@ int stairs_profile_read(stairs_ctx *ctx, float *gemm_ms, int32_t *gemm_launches,
  * workspace after a pass (which: 0 residual x fp32 [rows, d], 1 normed h, 2 qkv fp32,
  * 3 attention output o, 4 MLP activation ff, 5 argmax keys u64, 6 per-phase timestamps of the
  * persistent kernel, u64 ns [2 CTAs][phases][8 stamps: start, work done, arrived, prologue done, first tile ready, first MMA, last MMA, first activation load], written while
- * profiling is on, 7 the persistent kernel's split-tile partial sums, fp32: between calls every
- * word holds the empty pattern 0xffffffff). */
+ * profiling is on). */
 int stairs_debug_buffer(stairs_ctx *ctx, int which, void **ptr_dev, size_t *bytes);
 
 /* Frees the slot's KV pages and forgets its sequence. */

@@ -283,14 +283,12 @@ class Stairs:
         return g.value, n.value, c.value
 
     def debug_buffer(self, which: int, dtype, count: int):
-        """Copy of the first `count` elements (None: all) of an internal buffer (tests only)."""
+        """Copy of the first `count` elements of an internal activation buffer (tests only)."""
         ptr, nbytes = C.c_void_p(), C.c_size_t()
         self._ck(self.lib.stairs_debug_buffer(self.h, which, C.byref(ptr), C.byref(nbytes)))
         t = self.torch
         off = ptr.value - self.workspace.data_ptr()
         esz = t.empty(0, dtype=dtype).element_size()
-        if count is None:
-            count = nbytes.value // esz
         assert count * esz <= nbytes.value
         self.sync()
         return self.workspace[off: off + count * esz].view(dtype).clone()

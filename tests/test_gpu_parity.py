@@ -245,27 +245,6 @@ def test_error_paths_return_codes_and_leave_the_context_usable():
     eng.close()
 
 
-def test_split_tile_scratch_is_left_empty_after_calls_of_different_shapes():
-    """The persistent kernel's partial-sum words vouch for themselves: a word is 'empty' (all ones)
-    until its segment writes it, and the tile's finisher empties it again.  After any mix of calls
-    (prefill: 64-row passes, validate with several row counts, draft) every word must be empty."""
-    st = _stairs()
-    shape = small_b()
-    tsrc, dsrc = sources(shape)
-    eng = st.Stairs(tsrc, dsrc, max_requests=2, max_seq_len=256, k_max=8)
-    eng.prefill(0, list(wl.uniform_tokens(150, shape.vocab, 5)))
-    eng.prefill(1, list(wl.uniform_tokens(70, shape.vocab, 6)))
-    d = torch.from_numpy(wl.uniform_tokens(16, shape.vocab, 9).reshape(2, 8).astype(np.int32)).cuda()
-    for ks in ([8, 3], [0, 0], [5, 8]):
-        eng.validate([0, 1], ks, d)
-    eng.draft(0, 3)
-    eng.sync()
-    buf = eng.debug_buffer(7, torch.int32, None)
-    assert buf.numel() > 0
-    assert bool((buf == -1).all()), int((buf != -1).sum())
-    eng.close()
-
-
 def test_expired_device_wait_is_reported_and_the_gpu_stays_usable():
     """Every wait inside the persistent kernel is bounded.  With the bound set to about a microsecond the
     waits of a healthy call run out: the kernel must drain and exit by itself, the next sync must
