@@ -11,22 +11,27 @@
 // norms and attention.
 //
 // Roles per CTA (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner,
-// warps 2-5 = "compute group": GEMM epilogues and every non-GEMM phase (rows+embedding, norms,
-// attention, combine, accept).  GEMM work is split exactly as in k_gemm_tc (contiguous k-block
-// ranges per CTA, split tiles finished by the last arriver in k order).
+// warps 2-5 = "compute group": GEMM epilogues and every non-GEMM phase (rows+embedding,
+// attention, combine, accept).  GEMM work is cut into contiguous k-block ranges per CTA; a tile
+// cut over several CTAs is finished by the CTA that owns its first k-block, which adds the other
+// CTAs' parked partial tiles in k order once their flags are up.  Normalisation is folded into
+// the GEMMs (operand x * gain, epilogue rescales by the row's 1/std from per-tile statistics).
 //
 // Attention (staircase mask over the paged cache): a unit is (request, kv head, range of
 // 64-position chunks, block of <= 48 queries); all rows x grouped heads of the request share the
-// K/V chunk, which is staged in shared memory by bulk async copies (one per cache row, so pages
-// need not be contiguous) completing on an mbarrier.  Scores: lane = position; softmax state
-// per query with warp shuffles; P.V: lane = slice of head_dim.  New positions' K (rotated) and V
-// are computed in the unit that owns their chunk, patched into the staged tile and written to
-// the cache.  Unit boundaries depend only on absolute positions and on the request's own
-// committed length, never on the other rows or requests in the call.
+// K/V chunk, staged in shared memory by 16-byte asynchronous copies (cache rows looked up once
+// per chunk, so pages need not be contiguous).  Queries (rotated, scaled, fp16) and the new
+// positions' K/V are filed by the QKV projection's epilogue.  Scores and P.V run on fp16
+// mma.sync tiles, one warp per 16-query block, online softmax in registers.  Unit boundaries
+// depend only on the request's own committed length, never on the other requests in the call.
 //
-// All waits (mbarriers, grid barrier) are clock-bounded: on expiry the CTA raises an abort flag
-// (shared memory) and a global abort word that every other CTA's waits poll, so the whole grid
-// drains, frees TMEM and exits with STAIRS_ETIMEOUT in the status word.
+// With 227 KB of shared memory the L1 is nearly gone: every global or local access is an L2 round
+// trip.  Phase descriptors and request geometry are therefore kept in shared memory, cursors in
+// scalar registers, and loads that feed a dependent chain are issued together.
+//
+// All waits (mbarriers, grid barrier, split-tile flags) are clock-bounded: on expiry the CTA
+// raises an abort flag (shared memory) and a global abort word that every other CTA's waits poll,
+// so the whole grid drains, frees TMEM and exits with STAIRS_ETIMEOUT in the status word.
 #pragma once
 #include "gemm_tc.cuh"
 #include "kernels_basic.cuh"
@@ -87,7 +92,7 @@ struct Params {
   __half* q16;               // [row][Hq*hd] queries, rotated and scaled by 1/sqrt(hd), written by the QKV epilogue
   float* rope_cs; float* rope_sn;   // [row][hd/2] cos and sin of the call's row positions, written by the embedding phase
      // [hd/2] theta^(-2i/hd)
-  int* attn_cnt;            // split-KV arrival counters per (request, kv head, query block)
+  int* attn_cnt;            // (reserved; the combine phase needs no counters)
   float* logits;            // optional dump
   int* target_tokens; int* accept_len; int commit; int* draft_out;
   // scratch
@@ -176,10 +181,6 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ void tma_load_2d_ptr(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar, uint64_t policy) {
   tma_load_2d(dst, map, c0, c1, bar, policy);
 }
-__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
 
 // k-block range of this CTA in a GEMM phase: the phase is cut over min(G, total) CTAs so that no
 // participating range is empty (the split-tile bookkeeping counts one segment per CTA touching a tile).
@@ -231,10 +232,9 @@ struct AttnReq { int slot, base, R, off, n_chunks, cpu, n_ranges, n_qblk, units;
 
 // Shared per-CTA control block.
 struct Ctl {
-  uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2], att_bar;
+  uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
   uint32_t tmem_slot;
   volatile int abort_flag;
-  volatile int last_flag;
   volatile int bcast;
   float rstd[64], mu[64];       // per-row statistics of the current norm_in GEMM phase
   int rowbase[2][64];           // attention staging: cache row of each position of the chunk (per chunk buffer)
@@ -429,7 +429,7 @@ __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
 // in warp order through a small shared buffer - a fixed order - and the block's result is either
 // final (the unit saw every visible position) or parked for the combine phase.
 __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot,
-                          uint8_t* att_smem, Ctl* ctl, uint32_t& att_parity, const Waiter& W, int et, bool& ok,
+                          uint8_t* att_smem, Ctl* ctl, int et, bool& ok,
                           unsigned long long* tra) {
   const int hd = P.hd, G = P.Hq / P.Hkv, nkv = P.Hkv * hd, nq = P.Hq * hd;
   const int lane = et & 31, w = et >> 5, g = lane >> 2, t4 = lane & 3;
@@ -713,8 +713,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     for (int s = 0; s < stages; ++s) { mbar_init(ctl->full + s, 1); mbar_init(ctl->empty + s, 1); }
     mbar_init(ctl->acc_full + 0, 1); mbar_init(ctl->acc_full + 1, 1);
     mbar_init(ctl->acc_empty + 0, 4); mbar_init(ctl->acc_empty + 1, 4);
-    mbar_init(&ctl->att_bar, 1);
-    ctl->abort_flag = 0; ctl->last_flag = 0; ctl->bcast = 0;
+    ctl->abort_flag = 0; ctl->bcast = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) tmem_alloc(&ctl->tmem_slot, tmem_cols);
@@ -878,7 +877,6 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     const int et = threadIdx.x - 64;
     float* red = vt;    // 4 floats of scratch for group sums (the exchange tile is free outside GEMM epilogues)
     int buf = 0; uint32_t acc_bits = 0;
-    uint32_t att_parity = 0;
     bool ok = true;
     bool waited = true;   // true when every earlier phase is known complete grid-wide
 
@@ -931,7 +929,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const int range = rest % a.n_ranges, kvh = rest / a.n_ranges;
             const int slot = u0 + u;
             if (slot < P.attn_part_units)
-              attn_unit(P, p, a, kvh, range, qblk, slot, att_smem, ctl, att_parity, W, et, ok,
+              attn_unit(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok,
                         (P.trace && et == 0 && u == first) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr);
           }
           u0 += a.units; g0 += P.Hkv * a.n_qblk;
