@@ -57,8 +57,7 @@ struct DevModel {
 
 struct Layout {
   size_t status, seq, n_seq, page_table, tok, pos, req, val_req, val_k, val_off, keys, x, h, qkv, q,
-      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_partial, mk_bar, attn_part, prog_t, prog_d, mk_trace, mk_stats, attn_cnt, rope_t, rope_d, aux_t, aux_d, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
-  size_t mk_partial_bytes = 0;
+      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_flags, mk_bar, attn_part, prog_t, prog_d, mk_trace, mk_stats, attn_cnt, rope_t, rope_d, aux_t, aux_d, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
   int max_rows, logit_rows, max_pages, n_pages, t_box_max, attn_units, stat_tiles, attn_cnt_n;
   size_t prog_slot_t, prog_slot_d, prog_maps_off_t, prog_maps_off_d;
   size_t kv_t_layer, kv_d_layer;
@@ -195,10 +194,7 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
   L->al_buf = take((size_t)c.max_requests * 4);
   L->gemm_partial = take(t.wdtype == 1 ? (size_t)TC_GRID_MAX * 2 * L->t_box_max * tc::BM * 4 : 0);
   L->gemm_counters = take(t.wdtype == 1 ? (size_t)TC_COUNTERS * 4 : 0);
-  // split-tile partial sums of the persistent kernel: one slot per CTA; a word holds the empty pattern
-  // (all ones) whenever nobody has written it
-  L->mk_partial_bytes = t.wdtype == 1 ? (size_t)TC_GRID_MAX * MK_MAX_ROWS * tc::BM * 4 : 0;
-  L->mk_partial = take(L->mk_partial_bytes);
+  L->mk_flags = take(t.wdtype == 1 ? (size_t)TC_GRID_MAX * 8 : 0);   // split-tile flags of the persistent kernel
   {
     // persistent-kernel scratch: attention unit states and the per-(model, row box) programs
     const int hkv = mx(t.n_kv_heads, d.n_kv_heads), hdm = mx(t.head_dim, d.head_dim);
@@ -606,7 +602,8 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.keys = reinterpret_cast<unsigned long long*>(ws + L.keys); P.n_keys = L.max_rows;
   P.logits = c.logits;
   P.target_tokens = c.target_tokens; P.accept_len = c.accept_len; P.commit = c.commit; P.draft_out = c.draft_out;
-  P.partial = reinterpret_cast<float*>(ws + L.mk_partial); P.counters = reinterpret_cast<int*>(ws + L.gemm_counters);
+  P.partial = reinterpret_cast<float*>(ws + L.gemm_partial); P.counters = reinterpret_cast<int*>(ws + L.gemm_counters);
+  P.seg_flags = reinterpret_cast<unsigned long long*>(ws + L.mk_flags);
   P.attn_part = reinterpret_cast<float*>(ws + L.attn_part); P.attn_part_units = L.attn_units;
   P.stats = reinterpret_cast<float4*>(ws + L.mk_stats); P.stat_tiles = L.stat_tiles;
   P.rope_inv = M.rope_inv; P.rope_cs = M.rope_inv + m.head_dim / 2; P.rope_sn = P.rope_cs + 64 * (m.head_dim / 2); P.attn_cnt = reinterpret_cast<int*>(ws + L.attn_cnt);
@@ -890,7 +887,6 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
   e = cudaMemsetAsync(ctx->ws, 0, L.tok, ctx->stream);
   if (e == cudaSuccess && L.kv_t_k > L.gemm_counters)  // split-tile counters start at zero and return to zero
     e = cudaMemsetAsync(ctx->ws + L.gemm_counters, 0, L.kv_t_k - L.gemm_counters, ctx->stream);
-  if (e == cudaSuccess && L.mk_partial_bytes) e = cudaMemsetAsync(ctx->ws + L.mk_partial, 0xff, L.mk_partial_bytes, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
   if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_begin);
   if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_end);
@@ -1213,7 +1209,7 @@ int stairs_sync(stairs_ctx* ctx) {
     for (int i = 1; i <= 5; ++i) ctx->status_host[i] = 0;
     cudaMemsetAsync(ctx->ws + ctx->lay.mk_bar, 0, 64, ctx->stream);   // barrier count and abort word
     cudaMemsetAsync(ctx->ws + ctx->lay.gemm_counters, 0, (size_t)TC_COUNTERS * 4, ctx->stream);
-    cudaMemsetAsync(ctx->ws + ctx->lay.mk_partial, 0xff, ctx->lay.mk_partial_bytes, ctx->stream);   // every word empty again
+    cudaMemsetAsync(ctx->ws + ctx->lay.mk_flags, 0, (size_t)TC_GRID_MAX * 8, ctx->stream);   // tags restart with the barrier count
     cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)ctx->lay.attn_cnt_n * 4, ctx->stream);
     cudaStreamSynchronize(ctx->stream);
     ctx->bar_base = 0;

@@ -96,6 +96,7 @@ struct Params {
   float* logits;            // optional dump
   int* target_tokens; int* accept_len; int commit; int* draft_out;
   // scratch
+  unsigned long long* seg_flags;   // one flag per CTA: the tag of the phase whose partial its slot holds
   float* partial; int* counters;
   float* attn_part;         // [units][QBLK][hd + 4]: O, running max, running sum, pad
   int attn_part_units;
@@ -156,13 +157,6 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
   asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
   return v;
 }
-// 16-byte load through L2 that the compiler must repeat every time it is written (polling)
-__device__ __forceinline__ float4 ld_cg_poll_f4(const float* p) {
-  float4 v;
-  asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
-  return v;
-}
-constexpr unsigned int PARTIAL_EMPTY = 0xffffffffu;   // bit pattern of a partial-sum word nobody has written yet
 __device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
@@ -1135,6 +1129,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         if (tracing) tr[3] = globaltimer_ns();
         bool first_seg = true;
         long long kb = kb_begin;
+        const unsigned long long seg_tag = P.bar_base + (unsigned long long)ph + 1ull;   // unique per launch and phase
         const unsigned tot32 = (unsigned)total, ge32 = (unsigned)Ge;
         auto rb = [&](unsigned c) { return (tot32 * c) / ge32; };   // total * Ge < 2^32, checked on the host
         const int er = et >> 3, cg = et & 7;
@@ -1190,10 +1185,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             if (src_s >= 1) kv_row0 = kv_row_of(er);
             if (P.rope && src_s < 2) rope_of(er, rc0a, rs0a, rc0b, rs0b);
           }
-          const int mc = p.dual ? (m & 63) : m;
-          const bool m_on = mc < ncols;
-          const bool m_store = mc < ((ncols + 3) & ~3);   // partial sums are read four columns at a time
           if (finisher) {
+            const int mc = p.dual ? (m & 63) : m;
+            const bool m_on = mc < ncols;
             if (p.norm_in) {
               const int ncol = (p.dual && m >= 64) ? p.N + n0 + mc : n0 + mc;
               ctl->utile[m] = (p.u && m_on) ? p.u[ncol] : 0.f;
@@ -1230,12 +1224,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                 for (int j = 0; j < 16; ++j) v[j] += vl[j];
               }
               const int jn = min(16, Tvalid - c0);
-              // (only words that exist: the finisher reads, and empties again, exactly these)
 #pragma unroll
-              for (int j = 0; j < 16; ++j) if (j < jn && m_store) mine[(size_t)(c0 + j) * BM + m] = v[j];
+              for (int j = 0; j < 16; ++j) if (j < jn) mine[(size_t)(c0 + j) * BM + m] = v[j];
             }
             tc_fence_before();
             if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
+            epi_bar_sync();
+            // release: cumulative over the group's stores, which the barrier ordered before it
+            if (et == 0) st_release_u64(P.seg_flags + cta, seg_tag);
             if (tra) tra[5] = globaltimer_ns();
           } else {
             unsigned last_c = (unsigned)cta;   // CTAs cta + 1 .. last_c hold the tile's other segments
@@ -1257,8 +1253,30 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
 #pragma unroll
                 for (int j = 0; j < 16; ++j) vt[j * VT_LD + m] = v[j];
               }
-              if (tra && !whole && c0 == 0) tra[1] = globaltimer_ns();
-              epi_bar_sync();
+              if (!whole && c0 == 0) {
+                if (tra) tra[1] = globaltimer_ns();
+                if (et < 32) {
+                  // one lane per other segment: wait (bounded) until its flag carries this phase's tag
+                  const long long t0 = clock64();
+                  bool all_set;
+                  do {
+                    bool mine_set = true;
+                    for (unsigned cc = (unsigned)cta + 1 + (unsigned)lane; cc <= last_c; cc += 32)
+                      if (ld_acquire_u64(P.seg_flags + cc) != seg_tag) mine_set = false;
+                    all_set = __all_sync(0xffffffffu, mine_set);
+                    if (!all_set) {
+                      bool give_up = false;
+                      if (lane == 0) give_up = W.poll_abort(t0);
+                      if (__shfl_sync(0xffffffffu, give_up ? 1 : 0, 0)) break;
+                    }
+                  } while (!all_set);
+                  if (lane == 0 && !all_set) { ctl->abort_flag = 1; W.note(3u, (unsigned)ph, (unsigned)cta, last_c, (unsigned)tile); }
+                }
+                ok = group_ok(ctl, et);   // also orders the other threads' partial reads after the acquires
+                if (tra) tra[2] = globaltimer_ns();
+              } else {
+                epi_bar_sync();
+              }
               if (ok) {
                 const int t = c0 + er;
                 const bool row_on = t < Tvalid;
@@ -1272,59 +1290,24 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                   a[q] = on[q] ? *reinterpret_cast<const float4*>(vrow + col) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
                 if (!whole) {
-                  // The other segments' partial sums, four segments' loads in flight together, the
-                  // additions in k order.  A word still holding the empty pattern has not been
-                  // written yet: the loads are repeated (bounded) until every word is there - no
-                  // flag, no fence: each word vouches for itself - and the words are emptied again
-                  // for the slot's next use (a later phase, behind at least one grid barrier).
-                  for (unsigned c = (unsigned)cta + 1; c <= last_c; c += 4) {
-                    float4 tmp[4][4];
-                    const long long t0 = clock64();
-                    bool all_there;
-                    do {
-                      all_there = true;
+                  // the other segments' partial sums: six segments' loads in flight together, the
+                  // additions in k order
+                  for (unsigned c = (unsigned)cta + 1; c <= last_c; c += 6) {
+                    float4 tmp[6][4];
 #pragma unroll
-                      for (int u = 0; u < 4; ++u) {
-                        const float* part = P.partial + ((size_t)min(c + u, last_c) * P.t_box + (row_on ? t : 0)) * BM;
+                    for (int u = 0; u < 6; ++u) {
+                      const float* part = P.partial + ((size_t)min(c + u, last_c) * P.t_box + (row_on ? t : 0)) * BM;
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                          if (on[q] && c + u <= last_c) {
-                            tmp[u][q] = ld_cg_poll_f4(part + (cg + 8 * q) * 4);
-                          } else {
-                            tmp[u][q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                          }
-                        }
-                      }
+                      for (int q = 0; q < 4; ++q)
+                        tmp[u][q] = (on[q] && c + u <= last_c) ? __ldcg(reinterpret_cast<const float4*>(part + (cg + 8 * q) * 4))
+                                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
 #pragma unroll
-                      for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < 6; ++u) {
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                          if (__float_as_uint(tmp[u][q].x) == PARTIAL_EMPTY || __float_as_uint(tmp[u][q].y) == PARTIAL_EMPTY ||
-                              __float_as_uint(tmp[u][q].z) == PARTIAL_EMPTY || __float_as_uint(tmp[u][q].w) == PARTIAL_EMPTY)
-                            all_there = false;
-                        }
-                      }
-                    } while (!all_there && !W.poll_abort(t0));
-                    if (!all_there && (unsigned long long)(clock64() - t0) > P.wait_limit)
-                      W.note(3u, (unsigned)ph, (unsigned)cta, c, ((unsigned)tile << 8) | (unsigned)t);
-                    // The lanes leave the loop at different times.  bar.sync counts a warp as arrived
-                    // when ANY of its lanes gets there, so the warp must be whole again before the
-                    // next barrier (a barrier met by a split warp completes early and the stragglers
-                    // then count towards the following one: the group's barriers drift apart).
-                    __syncwarp();
-                    const float4 empty4 = make_float4(__uint_as_float(PARTIAL_EMPTY), __uint_as_float(PARTIAL_EMPTY),
-                                                      __uint_as_float(PARTIAL_EMPTY), __uint_as_float(PARTIAL_EMPTY));
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                      float* part = P.partial + ((size_t)min(c + u, last_c) * P.t_box + (row_on ? t : 0)) * BM;
-#pragma unroll
-                      for (int q = 0; q < 4; ++q) {
-                        if (on[q] && c + u <= last_c) *reinterpret_cast<float4*>(part + (cg + 8 * q) * 4) = empty4;
-                        a[q].x += tmp[u][q].x; a[q].y += tmp[u][q].y; a[q].z += tmp[u][q].z; a[q].w += tmp[u][q].w;
-                      }
+                      for (int q = 0; q < 4; ++q) { a[q].x += tmp[u][q].x; a[q].y += tmp[u][q].y; a[q].z += tmp[u][q].z; a[q].w += tmp[u][q].w; }
                     }
                   }
-                  if (tra) tra[2] = globaltimer_ns();
                 }
                 if (tra) {
                   asm volatile("" ::"f"(a[0].x), "f"(a[0].w), "f"(a[1].x), "f"(a[1].w), "f"(a[2].x), "f"(a[2].w), "f"(a[3].x), "f"(a[3].w));
@@ -1460,8 +1443,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
                   }
                 }
               }
-              if (whole) epi_bar_sync();   // the exchange tile is reused by the next chunk
-              else ok = ok && group_ok(ctl, et);   // (a thread's wait for partial sums may have run out)
+              epi_bar_sync();   // the exchange tile is reused by the next chunk
               if (!ok) break;
             }
             if (tra) tra[3] = globaltimer_ns();
