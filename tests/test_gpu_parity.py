@@ -245,6 +245,30 @@ def test_error_paths_return_codes_and_leave_the_context_usable():
     eng.close()
 
 
+@pytest.mark.parametrize("lengths", [[10], [17, 30], [65, 10], [33], [40, 10], [129]], ids=str)
+def test_fresh_contexts_with_varied_call_shapes_complete(lengths):
+    """Every row-box size as the very first launch of a context, then validate calls of several row
+    counts and a draft: no device wait may run out (the sync would raise) and the library's own
+    accept rule must hold for every request."""
+    st = _stairs()
+    shape = small_b()
+    tsrc, dsrc = sources(shape)
+    n = len(lengths)
+    eng = st.Stairs(tsrc, dsrc, max_requests=n, max_seq_len=192, k_max=8, wait_limit_cycles=400000000)
+    for r, length in enumerate(lengths):
+        eng.prefill(r, list(wl.uniform_tokens(length, shape.vocab, 20 + r)))
+    d = torch.from_numpy(wl.uniform_tokens(8 * n, shape.vocab, 31).reshape(n, 8).astype(np.int32)).cuda()
+    for ks in ([8] * n, [0] * n, [3] * n):
+        tt, al, _ = eng.validate(list(range(n)), ks, d)
+        eng.sync()
+        tt_h, al_h = tt.cpu().numpy(), al.cpu().numpy()
+        for i in range(n):
+            assert int(al_h[i]) == gu.first_mismatch(d[i, :ks[i]].cpu().numpy(), tt_h[i])
+    eng.draft(0, 3)
+    eng.sync()
+    eng.close()
+
+
 def test_expired_device_wait_is_reported_and_the_gpu_stays_usable():
     """Every wait inside the persistent kernel is bounded.  With the bound set to about a microsecond the
     waits of a healthy call run out: the kernel must drain and exit by itself, the next sync must
