@@ -1204,6 +1204,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             }
           }
           W.wait(ctl->acc_full + buf, (acc_bits >> buf) & 1u);
+          __syncwarp();   // lanes may leave the wait an iteration apart; the barriers below want whole warps
           ok = group_ok(ctl, et);   // (its barriers also publish the staged constants)
           if (!ok) break;
           if (tracing && first_seg) { tr[4] = globaltimer_ns(); first_seg = false; }
