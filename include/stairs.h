@@ -1,8 +1,8 @@
 /*
  * stairs.h - C-ABI of the B200 (sm_100a) "stairs" assisted greedy generation library.
  *
- * Method (Zhydik et al., "Inference acceleration for large language models using
- * 'stairs' assisted greedy generation", Section 3.3, Fig. 4 and Fig. 5): a small
+ * Method (D. Grigaliunas and M. Lukosevicius, "Inference acceleration for large language
+ * models using 'stairs' assisted greedy generation", Section 3.3, Fig. 4 and Fig. 5): a small
  * assistant model greedily drafts k tokens; the k+1 sub-sequences
  * context+draft[:r], r = 0..k, are given to the main model as one batch; the main
  * model's greedy token is taken for every row; rows are then walked in order and a
@@ -184,20 +184,6 @@ int stairs_sync(stairs_ctx *ctx);
 
 /* Number of kernels this context has launched so far. */
 int64_t stairs_launch_count(const stairs_ctx *ctx);
-
-/* Per-call device timing.  With profiling on, stairs_validate brackets the call and each
- * weight-streaming GEMM launch with events; stairs_profile_read waits and returns the
- * summed GEMM time, the number of GEMM launches and the whole call's time (ms) of the
- * most recent stairs_validate. */
-int stairs_profile(stairs_ctx *ctx, int enable);
-int stairs_profile_read(stairs_ctx *ctx, float *gemm_ms, int32_t *gemm_launches, float *call_ms);
-
-/* Inspection hook for tests: device address and size of one activation buffer inside the
- * workspace after a pass (which: 0 residual x fp32 [rows, d], 1 normed h, 2 qkv fp32,
- * 3 attention output o, 4 MLP activation ff, 5 argmax keys u64, 6 per-phase timestamps of the
- * persistent kernel, u64 ns [2 CTAs][phases][8 stamps: start, work done, arrived, prologue done, first tile ready, first MMA, last MMA, first activation load], written while
- * profiling is on). */
-int stairs_debug_buffer(stairs_ctx *ctx, int which, void **ptr_dev, size_t *bytes);
 
 /* Frees the slot's KV pages and forgets its sequence. */
 int stairs_reset(stairs_ctx *ctx, int req);

@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "../../include/stairs.h"
+#include "../../include/stairs_debug.h"
 #include "common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
@@ -91,6 +92,11 @@ struct stairs_ctx {
   std::map<std::tuple<const void*, int, int>, CUtensorMap> act_maps;
   unsigned int* status_host = nullptr;  // pinned, device-visible status words
   unsigned int* status_dev = nullptr;
+  // pinned, device-visible block of the host-buffer entry points: drafts in (staged for one
+  // asynchronous copy), target tokens and accept lengths out (written by the kernel itself)
+  int* io_host = nullptr;
+  int* io_dev = nullptr;
+  size_t io_draft = 0, io_tt = 0, io_al = 0;   // offsets in ints
   unsigned long long wait_limit = 0;
   bool use_mk = false;
   unsigned long long bar_base = 0;   // grid-barrier arrivals consumed by earlier launches
@@ -130,6 +136,15 @@ const char* check_model(const stairs_model& m) {
   if (m.wdtype < 0 || m.wdtype > 1) return "wdtype must be 0 (fp32) or 1 (bf16)";
   if (m.pos == 0 && m.max_pos <= 0) return "max_pos must be positive with learned positions";
   return nullptr;
+}
+
+// Upper bound of the attention units of one request with `rows` rows in the persistent kernel: the
+// kernel picks chunks per unit so that kv heads x position ranges fit the grid (or, for contexts
+// too long for that, at most twice the grid: stairs_init checks this); the rows of the call can
+// add one more range per kv head.
+int attn_unit_bound(int hkv, int gq, int rows) {
+  const int n_qblk = (rows * gq + mk::ATT_QBLK - 1) / mk::ATT_QBLK;
+  return (2 * TC_GRID_MAX + 2 * hkv) * std::max(n_qblk, 1);
 }
 
 bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
@@ -199,9 +214,12 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     // persistent-kernel scratch: attention unit states and the per-(model, row box) programs
     const int hkv = mx(t.n_kv_heads, d.n_kv_heads), hdm = mx(t.head_dim, d.head_dim);
     const int gq = mx(t.n_heads / t.n_kv_heads, has_draft ? d.n_heads / d.n_kv_heads : 1);
+    // A request with R rows has at most (2 * grid + 2 * Hkv) * ceil(R * G / query block) units (see
+    // attn_unit_bound).  A validate call holds up to max_requests requests of k_max + 1 rows; a
+    // prefill pass of the persistent kernel is one request of MK_MAX_ROWS rows.
     const int rows_req = std::min(c.k_max + 1, MK_MAX_ROWS);
     const int n_qblk = (rows_req * gq + mk::ATT_QBLK - 1) / mk::ATT_QBLK;
-    L->attn_units = c.max_requests * (2 * TC_GRID_MAX + 2 * hkv) * std::max(n_qblk, 1);
+    L->attn_units = std::max(c.max_requests * attn_unit_bound(hkv, gq, rows_req), attn_unit_bound(hkv, gq, MK_MAX_ROWS));
     L->attn_part = take(t.wdtype == 1 ? (size_t)L->attn_units * mk::ATT_QBLK * (hdm + 4) * 4 : 0);
     auto prog = [&](const stairs_model& m, size_t* maps_off) {
       const size_t ph = align_up((size_t)(8 * std::max(m.n_layers, 1) + 4) * sizeof(mk::Phase), 128);
@@ -557,6 +575,9 @@ struct MkCall {
   int* target_tokens = nullptr; int* accept_len = nullptr; int commit = 0; int* draft_out = nullptr;
   float* logits = nullptr;
   bool skip_head = false;   // prefill: stop after the last layer (no LM head, no accept)
+  const int* req_host = nullptr; // validate: slot, draft length and first row per request (travel as kernel parameters)
+  const int* k_host = nullptr;
+  const int* off_host = nullptr;
 };
 
 bool mk_eligible(const stairs_ctx* ctx, const DevModel& M, int T) {
@@ -575,6 +596,15 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
     int rc = build_program(ctx, M, t_box);
     if (rc) return rc;
   }
+  {
+    // attention scratch: refuse a call whose units might not fit rather than compute part of it
+    const int hkv = m.n_kv_heads, gq = m.n_heads / m.n_kv_heads;
+    long long need = 0;
+    if (c.mode == mk::CALL_VALIDATE) for (int i = 0; i < c.n_req; ++i) need += attn_unit_bound(hkv, gq, c.k_host[i] + 1);
+    else need = attn_unit_bound(hkv, gq, T);
+    if (need > L.attn_units)
+      return fail(ctx, STAIRS_ENOSPC, "attention scratch holds %d units, this call may need %lld", L.attn_units, need);
+  }
   mk::Params P;
   memset(&P, 0, sizeof P);
   char* base = M.prog_base + (size_t)slot * M.prog_slot_bytes;
@@ -589,8 +619,8 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.norm_kind = m.norm; P.rope = m.pos; P.rope_theta = m.rope_theta; P.eps = m.norm_eps;
   P.tok_emb = (const bf16*)M.w.tok_emb; P.pos_emb = (const bf16*)M.w.pos_emb;
   P.mode = c.mode; P.n_req = c.n_req; P.slot = c.slot; P.draft_step = c.draft_step;
-  P.val_req = reinterpret_cast<int*>(ws + L.val_req); P.val_k = reinterpret_cast<int*>(ws + L.val_k);
-  P.val_off = reinterpret_cast<int*>(ws + L.val_off);
+  if (c.mode == mk::CALL_VALIDATE)
+    for (int i = 0; i < c.n_req; ++i) { P.val_req[i] = c.req_host[i]; P.val_k[i] = c.k_host[i]; P.val_off[i] = c.off_host[i]; }
   P.draft = c.draft; P.k_max = ctx->cfg.k_max;
   P.seq = reinterpret_cast<int*>(ws + L.seq); P.n_seq = reinterpret_cast<int*>(ws + L.n_seq); P.max_seq_len = ctx->cfg.max_seq_len;
   P.tok = reinterpret_cast<int*>(ws + L.tok); P.pos = reinterpret_cast<int*>(ws + L.pos); P.req = reinterpret_cast<int*>(ws + L.req);
@@ -906,8 +936,16 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
       memset(ctx->status_host, 0, STATUS_WORDS * 4);
       e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&ctx->status_dev), ctx->status_host, 0);
     }
+    if (e == cudaSuccess) {
+      const size_t nd = (size_t)cfg->max_requests * std::max(cfg->k_max, 1), ntt = (size_t)cfg->max_requests * (cfg->k_max + 1);
+      ctx->io_draft = 0; ctx->io_tt = nd; ctx->io_al = nd + ntt;
+      e = cudaHostAlloc(reinterpret_cast<void**>(&ctx->io_host), (nd + ntt + cfg->max_requests) * 4, cudaHostAllocMapped);
+      if (e == cudaSuccess) e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&ctx->io_dev), ctx->io_host, 0);
+    }
     if (e != cudaSuccess) {
-      int rc = fail(nullptr, STAIRS_ECUDA, "status word set-up failed: %s", cudaGetErrorString(e));
+      int rc = fail(nullptr, STAIRS_ECUDA, "pinned status / result block set-up failed: %s", cudaGetErrorString(e));
+      if (ctx->status_host) cudaFreeHost(ctx->status_host);
+      if (ctx->io_host) cudaFreeHost(ctx->io_host);
       delete ctx;
       return rc;
     }
@@ -1046,13 +1084,11 @@ int stairs_validate(stairs_ctx* ctx, int n_req, const int32_t* req_ids_host, con
   }
   char* ws = ctx->ws;
   const Layout& L = ctx->lay;
-  CK(cudaMemcpyAsync(ws + L.val_req, req_ids_host, (size_t)n_req * 4, cudaMemcpyHostToDevice, ctx->stream));
-  CK(cudaMemcpyAsync(ws + L.val_k, k_host, (size_t)n_req * 4, cudaMemcpyHostToDevice, ctx->stream));
-  CK(cudaMemcpyAsync(ws + L.val_off, off.data(), (size_t)n_req * 4, cudaMemcpyHostToDevice, ctx->stream));
   if (ctx->profile) { ctx->ev_used = 0; cudaEventRecord(ctx->call_begin, ctx->stream); }
   if (mk_eligible(ctx, ctx->target, T)) {
     MkCall c;
     c.mode = mk::CALL_VALIDATE; c.n_req = n_req; c.draft = draft_dev;
+    c.req_host = req_ids_host; c.k_host = k_host; c.off_host = off.data();
     c.target_tokens = target_tokens_dev; c.accept_len = accept_len_dev; c.commit = commit; c.logits = logits_dev_or_null;
     int rc = launch_forward_mk(ctx, ctx->target, T, 0, T, c);
     if (rc) return rc;
@@ -1061,6 +1097,9 @@ int stairs_validate(stairs_ctx* ctx, int n_req, const int32_t* req_ids_host, con
       for (int i = 0; i < n_req; ++i) ctx->n_seq_ub[req_ids_host[i]] += k_host[i] + 1;
     return STAIRS_OK;
   }
+  CK(cudaMemcpyAsync(ws + L.val_req, req_ids_host, (size_t)n_req * 4, cudaMemcpyHostToDevice, ctx->stream));
+  CK(cudaMemcpyAsync(ws + L.val_k, k_host, (size_t)n_req * 4, cudaMemcpyHostToDevice, ctx->stream));
+  CK(cudaMemcpyAsync(ws + L.val_off, off.data(), (size_t)n_req * 4, cudaMemcpyHostToDevice, ctx->stream));
   ctx->in_validate = true;
   RowParams p = base_rows(ctx);
   p.mode = ROWS_VALIDATE; p.n_req = n_req; p.draft = draft_dev;
@@ -1093,16 +1132,19 @@ int stairs_validate_host(stairs_ctx* ctx, int n_req, const int32_t* req_ids_host
   const Layout& L = ctx->lay;
   const int km = ctx->cfg.k_max;
   int* d_dev = reinterpret_cast<int*>(ws + L.draft_buf);
-  int* tt_dev = reinterpret_cast<int*>(ws + L.tt_buf);
-  int* al_dev = reinterpret_cast<int*>(ws + L.al_buf);
-  if (km > 0 && draft_host)
-    CK(cudaMemcpyAsync(d_dev, draft_host, (size_t)n_req * km * 4, cudaMemcpyHostToDevice, ctx->stream));
-  int rc = stairs_validate(ctx, n_req, req_ids_host, k_host, draft_host ? d_dev : nullptr, tt_dev, al_dev, nullptr, commit);
+  // drafts: staged in pinned memory, one asynchronous copy; results: the pass writes them straight
+  // into pinned host memory, so nothing is copied back
+  if (km > 0 && draft_host) {
+    memcpy(ctx->io_host + ctx->io_draft, draft_host, (size_t)n_req * km * 4);
+    CK(cudaMemcpyAsync(d_dev, ctx->io_host + ctx->io_draft, (size_t)n_req * km * 4, cudaMemcpyHostToDevice, ctx->stream));
+  }
+  int rc = stairs_validate(ctx, n_req, req_ids_host, k_host, draft_host ? d_dev : nullptr, ctx->io_dev + ctx->io_tt,
+                           ctx->io_dev + ctx->io_al, nullptr, commit);
   if (rc) return rc;
-  CK(cudaMemcpyAsync(target_tokens_host, tt_dev, (size_t)n_req * (km + 1) * 4, cudaMemcpyDeviceToHost, ctx->stream));
-  CK(cudaMemcpyAsync(accept_len_host, al_dev, (size_t)n_req * 4, cudaMemcpyDeviceToHost, ctx->stream));
   rc = stairs_sync(ctx);
   if (rc) return rc;
+  memcpy(target_tokens_host, ctx->io_host + ctx->io_tt, (size_t)n_req * (km + 1) * 4);
+  memcpy(accept_len_host, ctx->io_host + ctx->io_al, (size_t)n_req * 4);
   if (commit)  // the host now knows the exact new lengths
     for (int i = 0; i < n_req; ++i) ctx->n_seq_ub[req_ids_host[i]] += accept_len_host[i] - k_host[i];
   return STAIRS_OK;
@@ -1120,37 +1162,44 @@ int stairs_generate(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_
   cudaEvent_t e0, e1, e2, e3;
   CK(cudaEventCreate(&e0)); CK(cudaEventCreate(&e1)); CK(cudaEventCreate(&e2)); CK(cudaEventCreate(&e3));
   auto cleanup = [&]() { cudaEventDestroy(e0); cudaEventDestroy(e1); cudaEventDestroy(e2); cudaEventDestroy(e3); };
-  cudaEventRecord(e0, ctx->stream);
-  rc = stairs_prefill(ctx, req, prompt_host, n_prompt);
-  cudaEventRecord(e1, ctx->stream);
-  if (!rc) rc = stairs_sync(ctx);
-  if (rc) { cleanup(); return rc; }
   float ms = 0.f;
-  cudaEventElapsedTime(&ms, e0, e1);
+  {
+    cudaError_t pe = cudaEventRecord(e0, ctx->stream);
+    rc = pe == cudaSuccess ? stairs_prefill(ctx, req, prompt_host, n_prompt) : fail(ctx, STAIRS_ECUDA, "cudaEventRecord: %s", cudaGetErrorString(pe));
+    if (!rc && (pe = cudaEventRecord(e1, ctx->stream)) != cudaSuccess) rc = fail(ctx, STAIRS_ECUDA, "cudaEventRecord: %s", cudaGetErrorString(pe));
+    if (!rc) rc = stairs_sync(ctx);
+    if (!rc && (pe = cudaEventElapsedTime(&ms, e0, e1)) != cudaSuccess) rc = fail(ctx, STAIRS_ECUDA, "cudaEventElapsedTime: %s", cudaGetErrorString(pe));
+    if (rc) { cleanup(); return rc; }
+  }
   s.prefill_ms = ms;
   const int km = ctx->cfg.k_max;
   int* d_dev = reinterpret_cast<int*>(ctx->ws + ctx->lay.draft_buf);
-  int* tt_dev = reinterpret_cast<int*>(ctx->ws + ctx->lay.tt_buf);
-  int* al_dev = reinterpret_cast<int*>(ctx->ws + ctx->lay.al_buf);
-  std::vector<int> tt(km + 1);
-  std::vector<int> draft_h(std::max(km, 1));
+  // results land in pinned host memory (written by the pass itself); the drafted tokens come back
+  // with one small copy into the same block
+  int* tt_dev = ctx->io_dev + ctx->io_tt;
+  int* al_dev = ctx->io_dev + ctx->io_al;
+  const int* tt = ctx->io_host + ctx->io_tt;
+  const int* al_h = ctx->io_host + ctx->io_al;
+  int* draft_h = ctx->io_host + ctx->io_draft;
+  (void)km;
   int produced = 0;
   bool stop = false;
+  cudaError_t ce = cudaSuccess;
   while (produced < max_new && !stop) {
     const int k_eff = std::min(k, max_new - produced - 1);
-    int al = 0;
-    cudaEventRecord(e1, ctx->stream);
+    if ((ce = cudaEventRecord(e1, ctx->stream)) != cudaSuccess) break;
     if (k_eff > 0 && (rc = stairs_draft(ctx, req, k_eff, d_dev))) break;
-    cudaEventRecord(e2, ctx->stream);
+    if ((ce = cudaEventRecord(e2, ctx->stream)) != cudaSuccess) break;
     if ((rc = stairs_validate(ctx, 1, &req, &k_eff, d_dev, tt_dev, al_dev, nullptr, 1))) break;
-    cudaEventRecord(e3, ctx->stream);
-    if (k_eff > 0) cudaMemcpyAsync(draft_h.data(), d_dev, (size_t)k_eff * 4, cudaMemcpyDeviceToHost, ctx->stream);
-    cudaMemcpyAsync(tt.data(), tt_dev, (size_t)(k_eff + 1) * 4, cudaMemcpyDeviceToHost, ctx->stream);
-    cudaMemcpyAsync(&al, al_dev, 4, cudaMemcpyDeviceToHost, ctx->stream);
+    if ((ce = cudaEventRecord(e3, ctx->stream)) != cudaSuccess) break;
+    if (k_eff > 0 && (ce = cudaMemcpyAsync(draft_h, d_dev, (size_t)k_eff * 4, cudaMemcpyDeviceToHost, ctx->stream)) != cudaSuccess) break;
     if ((rc = stairs_sync(ctx))) break;
+    const int al = al_h[0];
     ctx->n_seq_ub[req] += al - k_eff;
-    cudaEventElapsedTime(&ms, e1, e2); s.draft_ms += ms;
-    cudaEventElapsedTime(&ms, e2, e3); s.validate_ms += ms;
+    if ((ce = cudaEventElapsedTime(&ms, e1, e2)) != cudaSuccess) break;
+    s.draft_ms += ms;
+    if ((ce = cudaEventElapsedTime(&ms, e2, e3)) != cudaSuccess) break;
+    s.validate_ms += ms;
     s.iterations++; s.drafted += k_eff; s.accepted += al;
     for (int r = 0; r <= al && !stop; ++r) {
       const int t = r < al ? draft_h[r] : tt[al];
@@ -1159,10 +1208,11 @@ int stairs_generate(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_
       if (eos >= 0 && t == eos) stop = true;
     }
   }
+  if (!rc && ce != cudaSuccess) rc = fail(ctx, STAIRS_ECUDA, "stairs_generate: %s", cudaGetErrorString(ce));
   if (!rc) {
-    cudaEventRecord(e3, ctx->stream);
-    rc = stairs_sync(ctx);
-    cudaEventElapsedTime(&ms, e0, e3);
+    cudaError_t fe = cudaEventRecord(e3, ctx->stream);
+    rc = fe == cudaSuccess ? stairs_sync(ctx) : fail(ctx, STAIRS_ECUDA, "cudaEventRecord: %s", cudaGetErrorString(fe));
+    if (!rc && (fe = cudaEventElapsedTime(&ms, e0, e3)) != cudaSuccess) rc = fail(ctx, STAIRS_ECUDA, "cudaEventElapsedTime: %s", cudaGetErrorString(fe));
     s.total_ms = ms;
   }
   cleanup();
@@ -1215,7 +1265,9 @@ int stairs_sync(stairs_ctx* ctx) {
     ctx->bar_base = 0;
     // kind: 1 shared-memory barrier (block, thread, parity), 2 grid barrier (block, thread, target),
     // 3 split-tile flags (phase, block, last block of the tile, tile)
-    return fail(ctx, (int)code, "a device-side bounded wait expired (code %u; first: kind %u at %u, %u, %u, %u); results of the last calls are invalid",
+    // 4 attention-scratch guard (unit slot, slots available, request, unit)
+    return fail(ctx, (int)code, "%s (code %u; first: kind %u at %u, %u, %u, %u); results of the last calls are invalid",
+                where[0] == 4u ? "the device-side attention scratch was too small for a call" : "a device-side bounded wait expired",
                 code, where[0], where[1], where[2], where[3], where[4]);
   }
   return STAIRS_OK;
@@ -1285,6 +1337,7 @@ int stairs_destroy(stairs_ctx* ctx) {
   if (ctx->call_begin) cudaEventDestroy(ctx->call_begin);
   if (ctx->call_end) cudaEventDestroy(ctx->call_end);
   if (ctx->status_host) cudaFreeHost(ctx->status_host);
+  if (ctx->io_host) cudaFreeHost(ctx->io_host);
   delete ctx;
   return STAIRS_OK;
 }

@@ -36,6 +36,14 @@
 #include "gemm_tc.cuh"
 #include "kernels_basic.cuh"
 
+// Device-side timestamps for tuning (per-phase stamps written to a scratch area while profiling
+// is on) are compiled in only with -DSTAIRS_TRACE; the shipped kernel carries none of them.
+#ifdef STAIRS_TRACE
+#define MK_TRACE_PTR(expr) (expr)
+#else
+#define MK_TRACE_PTR(expr) (static_cast<unsigned long long*>(nullptr))
+#endif
+
 namespace stairs {
 namespace mk {
 
@@ -77,7 +85,7 @@ struct Params {
   const bf16* tok_emb; const bf16* pos_emb;
   // call
   int mode; int n_req; int slot; int draft_step;
-  const int* val_req; const int* val_k; const int* val_off;
+  int val_req[64]; int val_k[64]; int val_off[64];   // validate: slot, draft length and first row of each request (a call has <= 64 rows)
   const int* draft; int k_max;
   int* seq; int* n_seq; int max_seq_len;
   int* tok; int* pos; int* req;
@@ -807,7 +815,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           if (B.ph <= ready_ph) {
             uint8_t* b_dst = smem + (size_t)b_stage * stage_bytes + A_STAGE_BYTES;
             tma_load_2d(b_dst, P.maps + B.x_map, B.kk * BK, 0, ctl->full + b_stage, pol_x);   // hi and lo rows in one box
-            if (P.trace && cta == 0 && B.ph != traced_ph) { traced_ph = B.ph; P.trace[(size_t)B.ph * 8 + 7] = globaltimer_ns(); }
+            if (MK_TRACE_PTR(P.trace) && cta == 0 && B.ph != traced_ph) { traced_ph = B.ph; MK_TRACE_PTR(P.trace)[(size_t)B.ph * 8 + 7] = globaltimer_ns(); }
             ++b_count;
             if (++b_stage == stages) b_stage = 0;
             advance(B);
@@ -840,7 +848,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         if (remaining <= 0) continue;
         int kk = (int)(kr.begin % kblocks);
         bool seg_first = true;
-        unsigned long long* trm = (P.trace && cta == 0) ? P.trace + (size_t)ph * 8 : nullptr;
+        unsigned long long* trm = (MK_TRACE_PTR(P.trace) && cta == 0) ? MK_TRACE_PTR(P.trace) + (size_t)ph * 8 : nullptr;
         bool first_k = true;
         while (remaining > 0 && ok) {
           const bool seg_last = (remaining == 1) || (kk == kblocks - 1);
@@ -906,8 +914,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       }
 
       bool gemm_worked = false;
-      const bool tracing = P.trace && et == 0 && (cta == 0 || cta == G - 1);
-      unsigned long long* tr = tracing ? P.trace + ((size_t)(cta == 0 ? 0 : 1) * P.n_phases + ph) * 8 : nullptr;
+      const bool tracing = MK_TRACE_PTR(P.trace) && et == 0 && (cta == 0 || cta == G - 1);
+      unsigned long long* tr = tracing ? MK_TRACE_PTR(P.trace) + ((size_t)(cta == 0 ? 0 : 1) * P.n_phases + ph) * 8 : nullptr;
       if (tracing) tr[0] = globaltimer_ns();
       if (p.kind == PH_EMBED) {
         if (cta == 0)
@@ -928,9 +936,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             const int qblk = u % a.n_qblk, rest = u / a.n_qblk;
             const int range = rest % a.n_ranges, kvh = rest / a.n_ranges;
             const int slot = u0 + u;
-            if (slot < P.attn_part_units)
-              attn_unit(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok,
-                        (P.trace && et == 0 && u == first) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr);
+            if (slot >= P.attn_part_units) {
+              // cannot happen while the host's bound holds; never compute part of a call silently
+              if (et == 0) { W.note(4u, (unsigned)slot, (unsigned)P.attn_part_units, (unsigned)i, (unsigned)u); ctl->abort_flag = 1; }
+              ok = group_ok(ctl, et);
+              break;
+            }
+            attn_unit(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok,
+                        (MK_TRACE_PTR(P.trace) && et == 0 && u == first) ? MK_TRACE_PTR(P.trace) + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr);
           }
           u0 += a.units; g0 += P.Hkv * a.n_qblk;
         }
@@ -1211,7 +1224,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
           acc_bits ^= 1u << buf;
           tc_fence_after();
           const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * 2 * P.t_box);
-          unsigned long long* tra = (P.trace && et == 0 && !whole) ? P.trace + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
+          unsigned long long* tra = (MK_TRACE_PTR(P.trace) && et == 0 && !whole) ? MK_TRACE_PTR(P.trace) + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
           if (!finisher) {
             if (tra) tra[4] = globaltimer_ns();
             float* mine = P.partial + (size_t)cta * P.t_box * BM;
@@ -1457,7 +1470,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       if (!ok) break;
       if (tracing) tr[1] = globaltimer_ns();
       // every CTA's completion time of the phase, after the two detailed traces
-      if (P.trace && et == 0) P.trace[(size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8] = globaltimer_ns();
+      if (MK_TRACE_PTR(P.trace) && et == 0) MK_TRACE_PTR(P.trace)[(size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8] = globaltimer_ns();
       // Publish this CTA's part of the phase.  A CTA may arrive for phase ph only once every
       // CTA has arrived for phase ph-1: otherwise CTAs without work in two consecutive GEMM
       // phases would run ahead and their arrivals would be mistaken for the slower CTAs' ones
@@ -1490,7 +1503,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
   if (ctl->abort_flag) {
     if (threadIdx.x == 0) {
       atomicExch(P.bar + 1, 1ull);   // tell the other CTAs
-      *reinterpret_cast<volatile unsigned int*>(P.status + STATUS_ERROR) = 5u;  // STAIRS_ETIMEOUT
+      // STAIRS_ETIMEOUT, or STAIRS_ENOSPC when the first note is the attention-scratch guard's
+      *reinterpret_cast<volatile unsigned int*>(P.status + STATUS_ERROR) =
+          *reinterpret_cast<volatile unsigned int*>(P.status + STATUS_WHERE) == 4u ? 2u : 5u;
       __threadfence_system();
       // let the copies in flight land before the CTA's shared memory is given up (a stage whose
       // activation tile was never issued cannot complete: the loop is bounded, by at least ~1 ms so

@@ -94,9 +94,12 @@ def test_config1_validate_logits_match_oracle():
 @pytest.mark.parametrize("shape", [small_b(8, 2, 64), small_b(4, 4, 80, d=320, f=640), small_b(4, 1, 128, d=512),
                                    small_a()], ids=["gqa_hd64", "mha_hd80", "mqa_hd128", "family_a"])
 @pytest.mark.parametrize("k", [0, 1, 4, 8])
-def test_stair_rows_match_oracle_bf16(shape, k):
+@pytest.mark.parametrize("std", [0.03, 0.05], ids=["std0.03", "std0.05"])
+def test_stair_rows_match_oracle_bf16(shape, k, std):
+    # weight scale 0.03 gives these small models the logit scale of the benchmark configs (about
+    # 0.7); 0.05 is the harder case for the absolute logit bar (logit scale about 2)
     st = _stairs()
-    tsrc, dsrc = sources(shape)
+    tsrc, dsrc = sources(shape, std=std)
     tgt, _ = gu.oracle_pair(tsrc)
     prompt = list(wl.zipf_tokens(37, shape.vocab, 21))          # crosses two 16-token pages, ragged tail
     eng = st.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=96, k_max=8, kv_page_tokens=16, prefill_chunk=16)
