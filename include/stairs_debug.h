@@ -26,6 +26,10 @@ int stairs_profile_read(stairs_ctx *ctx, float *gemm_ms, int32_t *gemm_launches,
  * profiling is on). */
 int stairs_debug_buffer(stairs_ctx *ctx, int which, void **ptr_dev, size_t *bytes);
 
+/* Tuning knob of the persistent kernel, for sweeps.  what 0: 64-element k-blocks per pipeline
+ * stage (0 = chosen per row box, 1 or 2).  Takes effect with the next call. */
+int stairs_debug_tune(stairs_ctx *ctx, int what, long long value);
+
 #ifdef __cplusplus
 }
 #endif

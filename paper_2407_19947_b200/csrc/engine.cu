@@ -41,6 +41,9 @@ constexpr int MK_TBOX_SLOTS = MK_MAX_ROWS / 16;
 struct DevModel {
   float* rope_inv = nullptr;     // device: theta^(-2i/hd), i < hd/2
   float* ln_aux = nullptr;       // device: LayerNorm u/c vectors (see build_program)
+  bf16* w13 = nullptr;           // device: SwiGLU models, per layer [tiles][64 gate rows | 64 up rows][d] (see k_pack_gate_up)
+  size_t w13_layer = 0;          // elements per layer
+  std::vector<const bf16*> w13_ptr;   // per layer: its packed matrix (possibly another model's, for shared layers)
   bool prog_built[MK_TBOX_SLOTS] = {false, false, false, false};
   char* prog_base = nullptr;     // device: per t_box slot, phases followed by tensor maps
   size_t prog_slot_bytes = 0, prog_maps_off = 0;
@@ -58,7 +61,7 @@ struct DevModel {
 
 struct Layout {
   size_t status, seq, n_seq, page_table, tok, pos, req, val_req, val_k, val_off, keys, x, h, qkv, q,
-      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_flags, mk_bar, attn_part, prog_t, prog_d, mk_trace, mk_stats, attn_cnt, rope_t, rope_d, aux_t, aux_d, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
+      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_flags, mk_bar, attn_part, prog_t, prog_d, mk_trace, mk_stats, attn_cnt, rope_t, rope_d, aux_t, aux_d, w13_t, w13_d, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
   int max_rows, logit_rows, max_pages, n_pages, t_box_max, attn_units, stat_tiles, attn_cnt_n;
   size_t prog_slot_t, prog_slot_d, prog_maps_off_t, prog_maps_off_d;
   size_t kv_t_layer, kv_d_layer;
@@ -100,6 +103,7 @@ struct stairs_ctx {
   unsigned long long wait_limit = 0;
   bool use_mk = false;
   unsigned long long bar_base = 0;   // grid-barrier arrivals consumed by earlier launches
+  int kps_force = 0;                 // tuning: k-blocks per pipeline stage (0 = chosen per row box)
 };
 
 namespace {
@@ -245,6 +249,13 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     };
     L->aux_t = take(t.wdtype == 1 ? aux(t) : 0);
     L->aux_d = take((t.wdtype == 1 && has_draft) ? aux(d) : 0);
+    // SwiGLU models: gate and up rows interleaved per 64-row tile, so the persistent kernel streams
+    // them as one matrix (a one-time repack of borrowed weights into the workspace)
+    auto w13 = [&](const stairs_model& m) {
+      return m.act == 1 ? (size_t)((m.d_ff + 63) / 64) * 128 * m.d_model * 2 * m.n_layers : (size_t)0;
+    };
+    L->w13_t = take(t.wdtype == 1 ? w13(t) : 0);
+    L->w13_d = take((t.wdtype == 1 && has_draft) ? w13(d) : 0);
   }
   const size_t pool_tokens = (size_t)L->n_pages * pt;
   L->kv_t_layer = pool_tokens * t.n_kv_heads * t.head_dim * es;
@@ -293,6 +304,19 @@ bool encode_map(stairs_ctx* ctx, CUtensorMap* out, const void* ptr, long long ro
   cuuint32_t box[2] = {(cuuint32_t)tc::BK, (cuuint32_t)box_rows};
   cuuint32_t es[2] = {1, 1};
   CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// 3-D view of the same matrix for the persistent kernel: [K / 64][rows][64], box = 64 k-elements x
+// box_rows rows x kps k-blocks, 128-byte swizzle: one copy brings kps consecutive K-major slabs.
+bool encode_map3(stairs_ctx* ctx, CUtensorMap* out, const void* ptr, long long rows, long long K, int box_rows, int kps) {
+  cuuint64_t dims[3] = {(cuuint64_t)tc::BK, (cuuint64_t)rows, (cuuint64_t)(K / tc::BK)};
+  cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)tc::BK * 2};
+  cuuint32_t box[3] = {(cuuint32_t)tc::BK, (cuuint32_t)box_rows, (cuuint32_t)kps};
+  cuuint32_t es[3] = {1, 1, 1};
+  CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -407,9 +431,43 @@ __global__ void k_ln_aux(const bf16* __restrict__ W, const float* __restrict__ g
   if (lane == 0) { u[n] = su; c[n] = sc; }
 }
 
-// One-time per model: rotary frequency table and, for LayerNorm models, the u/c vectors.
-int setup_mk_model(stairs_ctx* ctx, DevModel& M, size_t rope_off, size_t aux_off) {
+// out[(128 t + j), :] = gate[64 t + j, :] and out[(128 t + 64 + j), :] = up[64 t + j, :] for j < 64
+// (rows past d_ff are zero): every 128-row tile of `out` holds 64 gate rows and the matching 64 up
+// rows, which is the shape the SwiGLU epilogue of the persistent kernel works on.
+__global__ void k_pack_gate_up(const bf16* __restrict__ gate, const bf16* __restrict__ up, bf16* __restrict__ out, int F, int d) {
+  const int row = blockIdx.x;                      // row of `out`
+  const int t = row >> 7, j = row & 127;
+  const int src_row = t * 64 + (j & 63);
+  const bf16* src = (j < 64 ? gate : up) + (size_t)src_row * d;
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+  for (int i = threadIdx.x; i < d / 8; i += blockDim.x)
+    reinterpret_cast<uint4*>(out + (size_t)row * d)[i] = src_row < F ? reinterpret_cast<const uint4*>(src)[i] : zero;
+}
+
+// One-time per model: rotary frequency table, the interleaved gate/up matrices of SwiGLU models
+// and, for LayerNorm models, the u/c vectors.
+int setup_mk_model(stairs_ctx* ctx, DevModel& M, size_t rope_off, size_t aux_off, size_t w13_off, const DevModel* other) {
   const stairs_model& m = M.m;
+  if (m.act == 1) {
+    M.w13 = reinterpret_cast<bf16*>(ctx->ws + w13_off);
+    const int rows = (m.d_ff + 63) / 64 * 128;
+    M.w13_layer = (size_t)rows * m.d_model;
+    M.w13_ptr.assign(m.n_layers, nullptr);
+    for (int l = 0; l < m.n_layers; ++l) {
+      // an early-exit assistant whose layer is one of the other model's layers shares its packed copy
+      const bf16* shared = nullptr;
+      if (other && other->w13)
+        for (int j = 0; j < other->m.n_layers && !shared; ++j)
+          if (other->layers[j].w_gate_or_fc1 == M.layers[l].w_gate_or_fc1 && other->layers[j].w_up == M.layers[l].w_up &&
+              other->m.d_ff == m.d_ff)
+            shared = other->w13_ptr[j];
+      if (shared) { M.w13_ptr[l] = shared; continue; }
+      bf16* dst = M.w13 + (size_t)l * M.w13_layer;
+      k_pack_gate_up<<<rows, 128, 0, ctx->stream>>>((const bf16*)M.layers[l].w_gate_or_fc1, (const bf16*)M.layers[l].w_up, dst, m.d_ff, m.d_model);
+      M.w13_ptr[l] = dst;
+    }
+    CK(cudaGetLastError());
+  }
   M.rope_inv = reinterpret_cast<float*>(ctx->ws + rope_off);
   std::vector<float> inv(std::max(m.head_dim / 2, 1));
   for (int i = 0; i < m.head_dim / 2; ++i)
@@ -441,26 +499,44 @@ int setup_mk_model(stairs_ctx* ctx, DevModel& M, size_t rope_off, size_t aux_off
   return STAIRS_OK;
 }
 
+// Attention with two K/V chunk buffers where they are cheap (small heads) or needed (contexts so long
+// that a unit walks several chunks).
+int mk_att_dbl(const stairs_ctx* ctx, const stairs_model& m) {
+  return (m.head_dim <= 64 || (long long)ctx->cfg.max_seq_len * m.n_kv_heads / mk::ATT_CHUNK > 2ll * ctx->sm_count) ? 1 : 0;
+}
+int mk_kps(const stairs_ctx* ctx, const stairs_model& m, int t_box) {
+  const int dbl = mk_att_dbl(ctx, m);
+  if (ctx->kps_force > 0 && mk::pick_stages(t_box, m.head_dim, dbl, ctx->kps_force) >= 2) return ctx->kps_force;
+  return mk::pick_kps(t_box, m.head_dim, dbl);
+}
+
 int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
   const stairs_model& m = M.m;
   const Layout& L = ctx->lay;
   const int slot = t_box / 16 - 1;
   const int d = m.d_model, nq = m.n_heads * m.head_dim, nkv = m.n_kv_heads * m.head_dim, nqkv = nq + 2 * nkv, F = m.d_ff;
   char* ws = ctx->ws;
+  const int kps = mk_kps(ctx, m, t_box);
   std::vector<CUtensorMap> maps((size_t)7 * m.n_layers + 4);
-  for (int l = 0; l < m.n_layers; ++l) {
-    const LayerMaps& t = M.maps[l];
+  bool ok = true;
+  for (int l = 0; l < m.n_layers && ok; ++l) {
+    const stairs_layer_w& w = M.layers[l];
     CUtensorMap* b = &maps[(size_t)7 * l];
-    b[0] = t.wq; b[1] = t.wk; b[2] = t.wv; b[3] = t.wo; b[4] = t.w1; b[5] = t.w3; b[6] = t.w2;
+    ok = ok && encode_map3(ctx, &b[0], w.wq, nq, d, tc::BM, kps) && encode_map3(ctx, &b[1], w.wk, nkv, d, tc::BM, kps) &&
+         encode_map3(ctx, &b[2], w.wv, nkv, d, tc::BM, kps) && encode_map3(ctx, &b[3], w.wo, d, nq, tc::BM, kps);
+    if (m.act == 1) ok = ok && encode_map3(ctx, &b[4], M.w13_ptr[l], (F + 63) / 64 * 128, d, tc::BM, kps);
+    else ok = ok && encode_map3(ctx, &b[4], w.w_gate_or_fc1, F, d, tc::BM, kps);
+    b[5] = b[4];
+    ok = ok && encode_map3(ctx, &b[6], w.w_down_or_fc2, d, F, tc::BM, kps);
   }
   const int i_head = 7 * m.n_layers, i_h = i_head + 1, i_o = i_head + 2, i_ff = i_head + 3;
-  maps[i_head] = M.head_map;
+  ok = ok && encode_map3(ctx, &maps[i_head], M.w.lm_head, m.vocab, d, tc::BM, kps);
   // activation operands: the lo parts' rows follow the hi parts' t_box rows, so one box of
   // 2 * t_box rows brings both
-  bool ok = encode_map(ctx, &maps[i_h], ws + L.h, 2 * L.max_rows, d, 2 * t_box) &&
-            encode_map(ctx, &maps[i_o], ws + L.o, 2 * L.max_rows, nq, 2 * t_box) &&
-            encode_map(ctx, &maps[i_ff], ws + L.ff, 2 * L.max_rows, F, 2 * t_box);
-  if (!ok) return fail(ctx, STAIRS_ECUDA, "cuTensorMapEncodeTiled failed for an activation buffer");
+  ok = ok && encode_map3(ctx, &maps[i_h], ws + L.h, 2 * L.max_rows, d, 2 * t_box, kps) &&
+       encode_map3(ctx, &maps[i_o], ws + L.o, 2 * L.max_rows, nq, 2 * t_box, kps) &&
+       encode_map3(ctx, &maps[i_ff], ws + L.ff, 2 * L.max_rows, F, 2 * t_box, kps);
+  if (!ok) return fail(ctx, STAIRS_ECUDA, "cuTensorMapEncodeTiled failed for a weight matrix or an activation buffer");
   std::vector<mk::Phase> ph;
   auto gemm = [&](int layer, int w0, int w1, int w2, int n_src, const int* rows, bool dual, int xmap, int K, int epi, void* out, int ldo) -> mk::Phase& {
     mk::Phase p;
@@ -468,7 +544,8 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
     p.kind = mk::PH_GEMM; p.layer = layer;
     p.w_map[0] = w0; p.w_map[1] = w1; p.w_map[2] = w2; p.x_map = xmap;
     p.n_src = n_src; p.dual = dual ? 1 : 0;
-    p.kblocks = (K + tc::BK - 1) / tc::BK;
+    p.kblocks = ((K + tc::BK - 1) / tc::BK + kps - 1) / kps;   // pipeline stages (groups of kps k-blocks) per tile
+    p.upt = ((K + tc::BK - 1) / tc::BK + mk::RANGE_UNIT_KB - 1) / mk::RANGE_UNIT_KB;
     int col = 0, tiles = 0;
     if (dual) { p.N = rows[0]; tiles = (rows[0] + 63) / 64; p.src_tiles[0] = tiles; }
     else {
@@ -483,7 +560,7 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
       // finished from more partial tiles, which the finisher reads four at a time.  Model:
       // stream time at ~44 GB/s per SM plus ~1.6 us per batch of four partials.
       const int grid = std::min(ctx->sm_count, TC_GRID_MAX);
-      const double bytes = (double)tiles * p.kblocks * tc::A_STAGE_BYTES;
+      const double bytes = (double)tiles * ((K + tc::BK - 1) / tc::BK) * tc::A_STAGE_BYTES;   // (must not depend on the row box: see RANGE_UNIT_KB)
       double best = 1e30; int best_ge = grid;
       for (int s2 = 1; s2 <= 64; s2 *= 2) {
         const int ge = std::min(grid, tiles * s2);
@@ -539,7 +616,7 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
     }
     const int rf[1] = {F};
     {
-      mk::Phase& p = (m.act == 1) ? gemm(l, b + 4, b + 5, b + 4, 1, rf, true, i_h, d, tc::TC_SWIGLU, ws + L.ff, F)
+      mk::Phase& p = (m.act == 1) ? gemm(l, b + 4, b + 4, b + 4, 1, rf, true, i_h, d, tc::TC_SWIGLU, ws + L.ff, F)
                                   : gemm(l, b + 4, b + 4, b + 4, 1, rf, false, i_h, d, tc::TC_GELU, ws + L.ff, F);
       p.norm_in = 1; p.u = aux_ptr(l, 2); p.c = aux_ptr(l, 3);
     }
@@ -583,7 +660,7 @@ struct MkCall {
 bool mk_eligible(const stairs_ctx* ctx, const DevModel& M, int T) {
   // (the epilogue's vector stores want every GEMM width but the vocabulary to be a multiple of 4)
   return ctx->use_mk && M.m.n_layers >= 1 && T >= 1 && T <= MK_MAX_ROWS && M.m.head_dim % 16 == 0 && M.m.head_dim <= 128 &&
-         M.m.d_model % 4 == 0 && M.m.d_ff % 4 == 0 && M.m.d_model <= 8192;
+         M.m.d_model % 64 == 0 && M.m.d_ff % 64 == 0 && (M.m.n_heads * M.m.head_dim) % 64 == 0 && M.m.d_model <= 8192;
 }
 
 int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, int n_logit_rows, const MkCall& c) {
@@ -611,9 +688,10 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   const int n_run = c.skip_head ? M.n_phases - 2 : M.n_phases;
   P.phases = reinterpret_cast<const mk::Phase*>(base); P.n_phases = n_run;
   P.maps = reinterpret_cast<const CUtensorMap*>(base + M.prog_maps_off);
-  P.T = T; P.t_box = t_box; // two K/V chunk buffers where they are cheap (small heads) or needed (contexts so long that a unit walks several chunks)
-  P.att_dbl = (m.head_dim <= 64 || (long long)ctx->cfg.max_seq_len * m.n_kv_heads / mk::ATT_CHUNK > ctx->sm_count) ? 1 : 0;
-  P.stages = mk::pick_stages(t_box, m.head_dim, P.att_dbl);
+  P.T = T; P.t_box = t_box;
+  P.att_dbl = mk_att_dbl(ctx, m);
+  P.kps = mk_kps(ctx, m, t_box);
+  P.stages = mk::pick_stages(t_box, m.head_dim, P.att_dbl, P.kps);
   P.logit_first_row = logit_first_row; P.n_logit_rows = n_logit_rows;
   P.d = m.d_model; P.Hq = m.n_heads; P.Hkv = m.n_kv_heads; P.hd = m.head_dim; P.F = m.d_ff; P.vocab = m.vocab;
   P.norm_kind = m.norm; P.rope = m.pos; P.rope_theta = m.rope_theta; P.eps = m.norm_eps;
@@ -642,8 +720,8 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.trace = (ctx->profile && &M == &ctx->target) ? reinterpret_cast<unsigned long long*>(ws + L.mk_trace) : nullptr;
   const int grid = std::min(ctx->sm_count, TC_GRID_MAX);
   void* args[] = {&P};
-  CK(cudaLaunchCooperativeKernel((const void*)mk::k_forward, dim3(grid), dim3(tc::THREADS), args,
-                                 mk::smem_bytes(t_box, P.stages, m.head_dim, P.att_dbl), ctx->stream));
+  CK(cudaLaunchCooperativeKernel((const void*)mk::k_forward, dim3(grid), dim3(mk::MK_THREADS), args,
+                                 mk::smem_bytes(t_box, P.stages, m.head_dim, P.att_dbl, P.kps), ctx->stream));
   ctx->bar_base += (unsigned long long)n_run * grid;
   ctx->launches++;
   return STAIRS_OK;
@@ -916,7 +994,7 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
   // position is always written before it becomes visible)
   e = cudaMemsetAsync(ctx->ws, 0, L.tok, ctx->stream);
   if (e == cudaSuccess && L.kv_t_k > L.gemm_counters)  // split-tile counters start at zero and return to zero
-    e = cudaMemsetAsync(ctx->ws + L.gemm_counters, 0, L.kv_t_k - L.gemm_counters, ctx->stream);
+    e = cudaMemsetAsync(ctx->ws + L.gemm_counters, 0, L.w13_t - L.gemm_counters, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
   if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_begin);
   if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_end);
@@ -979,15 +1057,15 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
       const int hdm = has_draft ? std::max(cfg->target.head_dim, cfg->draft.head_dim) : cfg->target.head_dim;
       const long long worst_chunks = ((long long)cfg->max_seq_len + mk::ATT_CHUNK - 1) / mk::ATT_CHUNK;
       const int hkvm = has_draft ? std::max(cfg->target.n_kv_heads, cfg->draft.n_kv_heads) : cfg->target.n_kv_heads;
-      const bool fits = mk::pick_stages(MK_MAX_ROWS, hdm, 1) >= 3 && worst_chunks * hkvm / 64 <= 2 * std::min(ctx->sm_count, TC_GRID_MAX);
+      const bool fits = mk::pick_stages(MK_MAX_ROWS, hdm, 1, 1) >= 3 && worst_chunks * hkvm / 64 <= 2 * std::min(ctx->sm_count, TC_GRID_MAX);
       if (coop && fits && cfg->gemm_impl == 0) {
         e = cudaFuncSetAttribute(mk::k_forward, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_LIMIT);
         if (e == cudaSuccess) {
           ctx->use_mk = true;
           ctx->target.prog_base = ctx->ws + L.prog_t; ctx->target.prog_slot_bytes = L.prog_slot_t; ctx->target.prog_maps_off = L.prog_maps_off_t;
           ctx->draft.prog_base = ctx->ws + L.prog_d; ctx->draft.prog_slot_bytes = L.prog_slot_d; ctx->draft.prog_maps_off = L.prog_maps_off_d;
-          int rc2 = setup_mk_model(ctx, ctx->target, L.rope_t, L.aux_t);
-          if (!rc2 && has_draft) rc2 = setup_mk_model(ctx, ctx->draft, L.rope_d, L.aux_d);
+          int rc2 = setup_mk_model(ctx, ctx->target, L.rope_t, L.aux_t, L.w13_t, nullptr);
+          if (!rc2 && has_draft) rc2 = setup_mk_model(ctx, ctx->draft, L.rope_d, L.aux_d, L.w13_d, &ctx->target);
           if (rc2) {
             g_init_error = ctx->err;
             stairs_destroy(ctx);
@@ -1315,8 +1393,22 @@ int stairs_debug_buffer(stairs_ctx* ctx, int which, void** ptr_dev, size_t* byte
     case 3: *ptr_dev = ctx->ws + off[4]; *bytes = off[5] - off[4]; break;
     case 4: *ptr_dev = ctx->ws + off[5]; *bytes = off[6] - off[5]; break;
     case 5: *ptr_dev = ctx->ws + L.keys; *bytes = keys_end - L.keys; break;
-    case 6: *ptr_dev = ctx->ws + L.mk_trace; *bytes = L.kv_t_k - L.mk_trace; break;
+    case 6: *ptr_dev = ctx->ws + L.mk_trace; *bytes = L.mk_stats - L.mk_trace; break;
     default: return fail(ctx, STAIRS_EINVAL, "unknown buffer %d", which);
+  }
+  return STAIRS_OK;
+}
+
+int stairs_debug_tune(stairs_ctx* ctx, int what, long long value) {
+  if (!ctx) return STAIRS_EINVAL;
+  switch (what) {
+    case 0:
+      if (value != 0 && value != 1 && value != 2) return fail(ctx, STAIRS_EINVAL, "k-blocks per stage must be 0 (auto), 1 or 2");
+      ctx->kps_force = (int)value;
+      for (bool& b : ctx->target.prog_built) b = false;   // programs carry the tensor maps' box depth
+      for (bool& b : ctx->draft.prog_built) b = false;
+      break;
+    default: return fail(ctx, STAIRS_EINVAL, "unknown tuning knob %d", what);
   }
   return STAIRS_OK;
 }

@@ -56,7 +56,8 @@ struct Phase {
   // PH_GEMM
   int w_map[3], x_map;
   int src_tiles[3], src_col[3];
-  int n_src, dual, n_tiles, kblocks, N, epi, ldo;
+  int n_src, dual, n_tiles, kblocks, N, epi, ldo;   // kblocks counts pipeline stages per tile (groups of Params::kps k-blocks)
+  int upt;                   // range units (RANGE_UNIT_KB k-blocks) per tile
   void* out;                 // fp32 or bf16 output
   // Normalisation folded into the GEMMs.  norm_in: the activation operand is bf16(x * gain) and
   // the epilogue applies y = rstd_t * (acc - mean_t * u[n]) + c[n] with u = W.gain, c = W.bias
@@ -79,6 +80,7 @@ struct Params {
   const Phase* phases; int n_phases;
   const CUtensorMap* maps;
   int T, t_box, stages;
+  int kps;                   // k-blocks (64 k-elements each) per pipeline stage: one TMA box and one commit cover all of them
   int logit_first_row, n_logit_rows;
   // model
   int d, Hq, Hkv, hd, F, vocab, norm_kind, rope; float rope_theta, eps;
@@ -114,6 +116,7 @@ struct Params {
   unsigned long long* trace;   // optional: per phase {start, work done, arrived} ns timestamps of CTA 0 and of the last CTA
 };
 
+constexpr int MK_THREADS = THREADS;
 constexpr int ATT_CHUNK = 64;
 constexpr int ATT_QBLK = 48;
 constexpr int VT_LD = 132;                      // row pitch (floats) of the epilogue's 16 x 128 exchange tile
@@ -186,19 +189,30 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void tma_load_2d_ptr(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar, uint64_t policy) {
-  tma_load_2d(dst, map, c0, c1, bar, policy);
-}
 
-// k-block range of this CTA in a GEMM phase: the phase is cut over min(G, total) CTAs so that no
+// Range of pipeline stages of this CTA in a GEMM phase.  The (tile, k) space is cut in UNITS of
+// RANGE_UNIT_KB k-blocks whatever the stage depth of the launch is, so that a tile's segment
+// boundaries - and with them the order of the fp32 additions - do not depend on the row count of
+// the call (calls with more rows use shallower stages): a request gives bit-identical results
+// alone and inside a larger batch.  The phase is cut over min(G, units) CTAs so that no
 // participating range is empty (the split-tile bookkeeping counts one segment per CTA touching a tile).
+constexpr int RANGE_UNIT_KB = 2;
 struct KRange { long long begin, end; int ge; };
-__device__ __forceinline__ KRange phase_range(long long total, int cta, int G, int ge_max) {
+// first stage of unit u: upt units and spt stages per tile, spu stages per unit (the last unit of a tile may be short)
+__device__ __forceinline__ long long unit_to_stage(long long u, int upt, int spt, int spu) {
+  if (spu == 1) return u;
+  const long long tile = u / upt;
+  const int j = (int)(u % upt);
+  return tile * spt + (j * spu < spt ? j * spu : spt);
+}
+__device__ __forceinline__ KRange phase_range(int n_tiles, int upt, int spt, int spu, int cta, int G, int ge_max) {
   KRange r;
+  const long long total = (long long)n_tiles * upt;
   if (ge_max > 0 && ge_max < G) G = ge_max;
   r.ge = (int)(total < (long long)G ? total : (long long)G);
   if (cta >= r.ge) { r.begin = r.end = 0; return r; }
-  r.begin = range_begin(total, cta, r.ge); r.end = range_begin(total, cta + 1, r.ge);
+  r.begin = unit_to_stage(range_begin(total, cta, r.ge), upt, spt, spu);
+  r.end = unit_to_stage(range_begin(total, cta + 1, r.ge), upt, spt, spu);
   return r;
 }
 
@@ -305,6 +319,61 @@ struct Waiter {
     return true;
   }
 };
+
+// Cursor over one CTA's pipeline stages of all GEMM phases, in program order (the TMA producer keeps
+// two, one for weight tiles and one for activation tiles).  Per-phase fields
+// are hoisted into registers on phase entry; tile and k indices advance incrementally.  Scalar
+// fields only: an array indexed at run time would put the cursor in local memory, and with the L1
+// carved down for shared memory every such access is an L2 round trip.
+struct WCursor {
+  int ph, kk, n_tile, remaining, kblocks, dual, n_src, x_map;
+  int st0, st1, wmap0, wmap1, wmap2;   // tiles of sources 0 and 1; tensor-map indices of the (up to) three sources
+  const CUtensorMap* wm0; int row;
+  bool valid;
+  __device__ __forceinline__ void locate(const Params& P) {   // source map and row coordinate of tile n_tile
+    if (dual) { wm0 = P.maps + wmap0; row = n_tile * BM; }   // gate and up rows interleaved by the host: 64 + 64 per tile
+    else {
+      int local = n_tile, wm = wmap0;
+      if (n_src > 1 && local >= st0) {
+        local -= st0; wm = wmap1;
+        if (n_src > 2 && local >= st1) { local -= st1; wm = wmap2; }
+      }
+      wm0 = P.maps + wm; row = local * BM;
+    }
+  }
+  __device__ __forceinline__ void enter(const Params& P, int cta, int G, int from) {   // first GEMM phase >= from in which this CTA has work
+    for (int p_i = from; p_i < P.n_phases; ++p_i) {
+      const Phase& p = P.phases[p_i];
+      if (p.kind != PH_GEMM) continue;
+      const KRange kr = phase_range(p.n_tiles, p.upt, p.kblocks, RANGE_UNIT_KB / P.kps, cta, G, p.ge_max);
+      if (kr.begin >= kr.end) continue;
+      ph = p_i; kblocks = p.kblocks; dual = p.dual; n_src = p.n_src; x_map = p.x_map;
+      st0 = p.src_tiles[0]; st1 = p.src_tiles[1];
+      wmap0 = p.w_map[0]; wmap1 = p.w_map[1]; wmap2 = p.w_map[2];
+      n_tile = (int)(kr.begin / p.kblocks); kk = (int)(kr.begin % p.kblocks);
+      remaining = (int)(kr.end - kr.begin);
+      locate(P);
+      valid = true;
+      return;
+    }
+    valid = false;
+  }
+  __device__ __forceinline__ void advance(const Params& P, int cta, int G) {
+    if (--remaining == 0) { enter(P, cta, G, ph + 1); return; }
+    if (++kk == kblocks) { kk = 0; ++n_tile; locate(P); }
+  }
+};
+
+// Asks L2 for one weight tile ahead of the shared-memory ring (no shared memory, no barrier involved).
+// Tiled 3-D load global -> shared.  The operand matrices [rows, K] are described to TMA as
+// [K / 64][rows][64]: a box of (64, rows of the tile, kps) lands as kps consecutive K-major slabs
+// with the 128-byte swizzle, i.e. several k-blocks per copy instruction.
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
 
 // ---------------------------------------------------------------------------------------------
 // Row helpers
@@ -701,12 +770,14 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ Params P) {
+__global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant__ Params P) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int stages = P.stages;
-  const int b_stage_bytes = P.t_box * BK * 2;               // one part (hi or lo) of the activation tile
-  const int stage_bytes = A_STAGE_BYTES + 2 * b_stage_bytes;
+  const int kps = P.kps;
+  const int a_stage_bytes = kps * A_STAGE_BYTES;            // kps weight slabs of 128 rows x 128 bytes
+  const int b_kb_bytes = 2 * P.t_box * BK * 2;              // activation slab of one k-block: hi rows then lo rows
+  const int stage_bytes = a_stage_bytes + kps * b_kb_bytes;
   uint8_t* tail = smem + (size_t)stages * stage_bytes;
   float* vt = reinterpret_cast<float*>(tail);   // epilogue exchange tile [16][VT_LD]
   Ctl* ctl = reinterpret_cast<Ctl*>(tail + MK_XCH_BYTES);
@@ -739,50 +810,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
     // ================================================================== TMA producer
     if (lane == 0) {
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
-      // Cursor over this CTA's k-blocks of all GEMM phases, in program order.  Per-phase fields
-      // are hoisted into registers on phase entry; tile and k indices advance incrementally.
-      // (scalar fields only: an array indexed at run time would put the cursor in local memory,
-      // and with the L1 carved down for shared memory every such access is an L2 round trip)
-      struct Cursor {
-        int ph, kk, n_tile, remaining, kblocks, dual, n_src, x_map;
-        int st0, st1, wmap0, wmap1, wmap2;   // tiles of sources 0 and 1; tensor-map indices of the (up to) three sources
-        const CUtensorMap* wm0; const CUtensorMap* wm1; int row;
-        bool valid;
-      };
-      auto locate = [&](Cursor& c) {   // source map and row coordinate of tile c.n_tile
-        if (c.dual) { c.wm0 = P.maps + c.wmap0; c.wm1 = P.maps + c.wmap1; c.row = c.n_tile * 64; }
-        else {
-          int local = c.n_tile, wm = c.wmap0;
-          if (c.n_src > 1 && local >= c.st0) {
-            local -= c.st0; wm = c.wmap1;
-            if (c.n_src > 2 && local >= c.st1) { local -= c.st1; wm = c.wmap2; }
-          }
-          c.wm0 = P.maps + wm; c.row = local * BM;
-        }
-      };
-      auto enter = [&](Cursor& c, int from) {   // first GEMM phase >= from in which this CTA has work
-        for (int ph = from; ph < P.n_phases; ++ph) {
-          const Phase& p = P.phases[ph];
-          if (p.kind != PH_GEMM) continue;
-          const KRange kr = phase_range((long long)p.n_tiles * p.kblocks, cta, G, p.ge_max);
-          if (kr.begin >= kr.end) continue;
-          c.ph = ph; c.kblocks = p.kblocks; c.dual = p.dual; c.n_src = p.n_src; c.x_map = p.x_map;
-          c.st0 = p.src_tiles[0]; c.st1 = p.src_tiles[1];
-          c.wmap0 = p.w_map[0]; c.wmap1 = p.w_map[1]; c.wmap2 = p.w_map[2];
-          c.n_tile = (int)(kr.begin / p.kblocks); c.kk = (int)(kr.begin % p.kblocks);
-          c.remaining = (int)(kr.end - kr.begin);
-          locate(c);
-          c.valid = true;
-          return;
-        }
-        c.valid = false;
-      };
-      auto advance = [&](Cursor& c) {
-        if (--c.remaining == 0) { enter(c, c.ph + 1); return; }
-        if (++c.kk == c.kblocks) { c.kk = 0; ++c.n_tile; locate(c); }
-      };
-      Cursor A, B;
-      enter(A, 0); enter(B, 0);
+      WCursor A, B;
+      A.enter(P, cta, G, 0); B.enter(P, cta, G, 0);
       int a_stage = 0, b_stage = 0;
       uint32_t a_par = 0;
       unsigned int a_count = 0, b_count = 0, idle = 0;
@@ -795,12 +824,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         if (A.valid && mbar_test(ctl->empty + a_stage, a_par ^ 1)) {
           uint8_t* a_dst = smem + (size_t)a_stage * stage_bytes;
           mbar_expect_tx(ctl->full + a_stage, (uint32_t)stage_bytes);
-          tma_load_2d(a_dst, A.wm0, A.kk * BK, A.row, ctl->full + a_stage, pol_w);
-          if (A.dual) tma_load_2d(a_dst + A_STAGE_BYTES / 2, A.wm1, A.kk * BK, A.row, ctl->full + a_stage, pol_w);
+          tma_load_3d(a_dst, A.wm0, 0, A.row, A.kk * kps, ctl->full + a_stage, pol_w);
+#ifdef STAIRS_TRACE
+          if (P.trace && cta == 0) P.trace[(size_t)(2 + G) * P.n_phases * 8 + 4000 + a_count] = (unsigned long long)clock64();
+#endif
           ++issued; ++a_count;
           if (++a_stage == stages) { a_stage = 0; a_par ^= 1; }
           p_stage = a_stage; p_phase = a_par;
-          advance(A);
+          A.advance(P, cta, G);
           progress = true;
         }
         if (b_count != a_count) {
@@ -813,12 +844,15 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             if (B.ph > ready_ph) { poll_val = ld_acquire_u64(bar_count); poll_pending = true; }
           }
           if (B.ph <= ready_ph) {
-            uint8_t* b_dst = smem + (size_t)b_stage * stage_bytes + A_STAGE_BYTES;
-            tma_load_2d(b_dst, P.maps + B.x_map, B.kk * BK, 0, ctl->full + b_stage, pol_x);   // hi and lo rows in one box
+            uint8_t* b_dst = smem + (size_t)b_stage * stage_bytes + a_stage_bytes;
+            tma_load_3d(b_dst, P.maps + B.x_map, 0, 0, B.kk * kps, ctl->full + b_stage, pol_x);   // hi and lo rows in one box
             if (MK_TRACE_PTR(P.trace) && cta == 0 && B.ph != traced_ph) { traced_ph = B.ph; MK_TRACE_PTR(P.trace)[(size_t)B.ph * 8 + 7] = globaltimer_ns(); }
+#ifdef STAIRS_TRACE
+            if (P.trace && cta == 0) P.trace[(size_t)(2 + G) * P.n_phases * 8 + 6000 + b_count] = (unsigned long long)clock64();
+#endif
             ++b_count;
             if (++b_stage == stages) b_stage = 0;
-            advance(B);
+            B.advance(P, cta, G);
             progress = true;
           }
         }
@@ -839,11 +873,15 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       int stage = 0; uint32_t phase = 0;
       int buf = 0; uint32_t acc_bits = 0;   // bit b: parity of accumulator b (no run-time indexed array: see the cursor)
       bool ok = true;
+#ifdef STAIRS_TRACE
+      unsigned long long* klog = P.trace ? P.trace + (size_t)(2 + G) * P.n_phases * 8 : nullptr;   // per k-block cycle stamps of CTA 0
+      int kn = 0;
+#endif
       for (int ph = 0; ph < P.n_phases && ok; ++ph) {
         const Phase& p = P.phases[ph];
         if (p.kind != PH_GEMM) continue;
         const int kblocks = p.kblocks;
-        const KRange kr = phase_range((long long)p.n_tiles * kblocks, cta, G, p.ge_max);
+        const KRange kr = phase_range(p.n_tiles, p.upt, kblocks, RANGE_UNIT_KB / kps, cta, G, p.ge_max);
         int remaining = (int)(kr.end - kr.begin);
         if (remaining <= 0) continue;
         int kk = (int)(kr.begin % kblocks);
@@ -857,19 +895,32 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
             if (!ok) break;
             tc_fence_after();
           }
+#ifdef STAIRS_TRACE
+          if (trm) klog[3 * kn] = (unsigned long long)clock64();
+#endif
           ok = W.wait(ctl->full + stage, phase);
           if (!ok) break;
           if (trm && first_k) { trm[5] = globaltimer_ns(); first_k = false; }
+#ifdef STAIRS_TRACE
+          if (trm) klog[3 * kn + 1] = (unsigned long long)clock64();
+#endif
           tc_fence_after();
           const uint32_t a_addr = smem_u32(smem + (size_t)stage * stage_bytes);
-          const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + A_STAGE_BYTES);
+          const uint64_t a_desc = smem_desc_sw128(a_addr), b_desc = smem_desc_sw128(a_addr + (uint32_t)a_stage_bytes);
           const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 2 * P.t_box);
+          // every k-block of the stage (a k-block past the end of K was zero-filled by the copies)
+          for (int j = 0; j < kps; ++j) {
+            const uint64_t aj = a_desc + (uint64_t)((j * A_STAGE_BYTES) >> 4), bj = b_desc + (uint64_t)((j * b_kb_bytes) >> 4);
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k)
-            umma_bf16(d_tmem, a_desc + (uint64_t)(k * UMMA_K * 2 / 16), b_desc + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
-                      (seg_first && k == 0) ? 0u : 1u);
+            for (int k = 0; k < BK / UMMA_K; ++k)
+              umma_bf16(d_tmem, aj + (uint64_t)(k * UMMA_K * 2 / 16), bj + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
+                        (seg_first && j == 0 && k == 0) ? 0u : 1u);
+          }
           umma_commit(ctl->empty + stage);
           if (seg_last) { umma_commit(ctl->acc_full + buf); acc_bits ^= 1u << buf; buf ^= 1; }
+#ifdef STAIRS_TRACE
+          if (trm) { klog[3 * kn + 2] = (unsigned long long)clock64(); ++kn; }
+#endif
           seg_first = seg_last;
           if (++kk == kblocks) kk = 0;
           --remaining;
@@ -1072,7 +1123,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
       } else {
         // ---------------------------------------------------------------- GEMM epilogue
         const long long total = (long long)p.n_tiles * p.kblocks;
-        const KRange kr = phase_range(total, cta, G, p.ge_max);
+        const KRange kr = phase_range(p.n_tiles, p.upt, p.kblocks, RANGE_UNIT_KB / kps, cta, G, p.ge_max);
         const long long kb_begin = kr.begin, kb_end = kr.end;
         const int Ge = kr.ge;
         gemm_worked = kb_begin < kb_end;
@@ -1143,8 +1194,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
         bool first_seg = true;
         long long kb = kb_begin;
         const unsigned long long seg_tag = P.bar_base + (unsigned long long)ph + 1ull;   // unique per launch and phase
-        const unsigned tot32 = (unsigned)total, ge32 = (unsigned)Ge;
-        auto rb = [&](unsigned c) { return (tot32 * c) / ge32; };   // total * Ge < 2^32, checked on the host
+        const unsigned tot32 = (unsigned)(p.n_tiles * p.upt), ge32 = (unsigned)Ge;
+        // first stage of CTA c's range (units * Ge < 2^32, checked on the host)
+        auto rb = [&](unsigned c) { return (unsigned)unit_to_stage((long long)((tot32 * c) / ge32), p.upt, p.kblocks, RANGE_UNIT_KB / kps); };
         const int er = et >> 3, cg = et & 7;
         while (kb < kb_end && ok) {
           const int tile = (int)(kb / p.kblocks), kk0 = (int)(kb % p.kblocks);
@@ -1525,15 +1577,17 @@ __global__ void __launch_bounds__(THREADS, 1) k_forward(const __grid_constant__ 
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, tmem_cols); }
 }
 
-inline size_t smem_bytes(int t_box, int stages, int hd, int dbl) {
-  return 1024 + (size_t)stages * (A_STAGE_BYTES + (size_t)2 * t_box * BK * 2) + MK_XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127) +
+inline size_t smem_bytes(int t_box, int stages, int hd, int dbl, int kps) {
+  return 1024 + (size_t)stages * kps * (A_STAGE_BYTES + (size_t)2 * t_box * BK * 2) + MK_XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127) +
          AttnSmem::bytes(hd, dbl) + 64;
 }
-inline int pick_stages(int t_box, int hd, int dbl) {
+inline int pick_stages(int t_box, int hd, int dbl, int kps) {
   int s = MAX_STAGES;
-  while (s > 1 && smem_bytes(t_box, s, hd, dbl) > (size_t)SMEM_LIMIT) --s;
+  while (s > 1 && smem_bytes(t_box, s, hd, dbl, kps) > (size_t)SMEM_LIMIT) --s;
   return s;
 }
+// k-blocks per stage: two while at least three stages still fit (small row boxes), else one
+inline int pick_kps(int t_box, int hd, int dbl) { return pick_stages(t_box, hd, dbl, 2) >= 3 ? 2 : 1; }
 
 }  // namespace mk
 }  // namespace stairs

@@ -20,7 +20,7 @@ STATUS = {0: "OK", 1: "EINVAL", 2: "ENOSPC", 3: "ESTATE", 4: "ECUDA", 5: "ETIMEO
 EXPORTS = ["stairs_workspace_bytes", "stairs_init", "stairs_prefill", "stairs_draft", "stairs_validate",
            "stairs_validate_host", "stairs_generate", "stairs_sequence", "stairs_truncate", "stairs_sync",
            "stairs_launch_count", "stairs_profile", "stairs_profile_read", "stairs_reset",
-           "stairs_destroy", "stairs_last_error", "stairs_accept_static", "stairs_debug_buffer"]
+           "stairs_destroy", "stairs_last_error", "stairs_accept_static", "stairs_debug_buffer", "stairs_debug_tune"]
 
 STATIC_MAX_ROWS, STATIC_MAX_REQ = 1024, 64
 
@@ -92,6 +92,7 @@ def load_library(path: Optional[str] = None):
     lib.stairs_profile_read.argtypes = [vp, C.POINTER(C.c_float), i32p, C.POINTER(C.c_float)]
     lib.stairs_reset.argtypes = [vp, C.c_int]
     lib.stairs_debug_buffer.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(C.c_size_t)]
+    lib.stairs_debug_tune.argtypes = [vp, C.c_int, C.c_longlong]
     lib.stairs_destroy.argtypes = [vp]
     lib.stairs_accept_static.argtypes = [vp, C.c_int, C.c_int, C.c_int, i32p, vp, C.c_int, vp, vp, vp]
     lib.stairs_last_error.restype = C.c_char_p
@@ -292,6 +293,10 @@ class Stairs:
         assert count * esz <= nbytes.value
         self.sync()
         return self.workspace[off: off + count * esz].view(dtype).clone()
+
+    def debug_tune(self, what: int, value: int):
+        """Unstable tuning knob (see include/stairs_debug.h)."""
+        self._ck(self.lib.stairs_debug_tune(self.h, what, value))
 
     def reset(self, req: int):
         self._ck(self.lib.stairs_reset(self.h, req))
