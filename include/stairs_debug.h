@@ -26,8 +26,10 @@ int stairs_profile_read(stairs_ctx *ctx, float *gemm_ms, int32_t *gemm_launches,
  * profiling is on). */
 int stairs_debug_buffer(stairs_ctx *ctx, int which, void **ptr_dev, size_t *bytes);
 
-/* Tuning knob of the persistent kernel, for sweeps.  what 0: 64-element k-blocks per pipeline
- * stage (0 = chosen per row box, 1 or 2).  Takes effect with the next call. */
+/* Tuning knobs of the persistent kernel, for sweeps.  what 0: 64-element k-blocks per pipeline
+ * stage (0 = chosen per row box, 1 or 2); what 1: K/V chunk buffers of the attention phases
+ * (0 = chosen from the context length, 1..4); what 2: non-zero stages K/V with 16-byte copies
+ * from the compute warps even where tiled bulk copies apply.  Takes effect with the next call. */
 int stairs_debug_tune(stairs_ctx *ctx, int what, long long value);
 
 #ifdef __cplusplus

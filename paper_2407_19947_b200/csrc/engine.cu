@@ -104,6 +104,8 @@ struct stairs_ctx {
   bool use_mk = false;
   unsigned long long bar_base = 0;   // grid-barrier arrivals consumed by earlier launches
   int kps_force = 0;                 // tuning: k-blocks per pipeline stage (0 = chosen per row box)
+  int att_nbuf_force = 0;            // tuning: K/V chunk buffers of the attention phases (0 = chosen from the context length)
+  int att_tma_off = 0;               // tuning: 1 = stage K/V with 16-byte copies from the compute warps even where bulk copies apply
 };
 
 namespace {
@@ -228,7 +230,7 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     auto prog = [&](const stairs_model& m, size_t* maps_off) {
       const size_t ph = align_up((size_t)(8 * std::max(m.n_layers, 1) + 4) * sizeof(mk::Phase), 128);
       *maps_off = ph;
-      return ph + (size_t)(7 * std::max(m.n_layers, 1) + 4) * sizeof(CUtensorMap);
+      return ph + (size_t)(9 * std::max(m.n_layers, 1) + 4) * sizeof(CUtensorMap);   // 7 weight and 2 K/V pool maps per layer
     };
     L->prog_slot_t = t.wdtype == 1 ? prog(t, &L->prog_maps_off_t) : 0;
     L->prog_slot_d = (t.wdtype == 1 && has_draft) ? prog(d, &L->prog_maps_off_d) : 0;
@@ -317,6 +319,19 @@ bool encode_map3(stairs_ctx* ctx, CUtensorMap* out, const void* ptr, long long r
   cuuint32_t box[3] = {(cuuint32_t)tc::BK, (cuuint32_t)box_rows, (cuuint32_t)kps};
   cuuint32_t es[3] = {1, 1, 1};
   CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// One layer's K or V pool [pool rows, Hkv * hd] fp16: box = 64 columns (one 128-byte swizzle row) x
+// box_rows rows (a page, or 64 rows of a larger page).
+bool encode_kv_map(stairs_ctx* ctx, CUtensorMap* out, const void* ptr, long long pool_rows, int nkv, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)nkv, (cuuint64_t)pool_rows};
+  cuuint64_t strides[1] = {(cuuint64_t)nkv * 2};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+  cuuint32_t es[2] = {1, 1};
+  CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, es,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -499,15 +514,33 @@ int setup_mk_model(stairs_ctx* ctx, DevModel& M, size_t rope_off, size_t aux_off
   return STAIRS_OK;
 }
 
-// Attention with two K/V chunk buffers where they are cheap (small heads) or needed (contexts so long
-// that a unit walks several chunks).
-int mk_att_dbl(const stairs_ctx* ctx, const stairs_model& m) {
-  return (m.head_dim <= 64 || (long long)ctx->cfg.max_seq_len * m.n_kv_heads / mk::ATT_CHUNK > 2ll * ctx->sm_count) ? 1 : 0;
-}
-int mk_kps(const stairs_ctx* ctx, const stairs_model& m, int t_box) {
-  const int dbl = mk_att_dbl(ctx, m);
-  if (ctx->kps_force > 0 && mk::pick_stages(t_box, m.head_dim, dbl, ctx->kps_force) >= 2) return ctx->kps_force;
-  return mk::pick_kps(t_box, m.head_dim, dbl);
+// Shared-memory plan of the persistent kernel for one (model, row box): pipeline depth of the GEMM
+// ring against the K/V chunk buffers of the attention phases.
+struct MkPlan { int kps, stages, att_dbl, att_tma, att_nbuf; };
+
+MkPlan mk_plan(const stairs_ctx* ctx, const stairs_model& m, int t_box) {
+  MkPlan pl{};
+  const int hd = m.head_dim;
+  // copy path: two K/V chunk buffers where they are cheap (small heads) or needed (contexts so long
+  // that a unit walks several chunks)
+  pl.att_dbl = (hd <= 64 || (long long)ctx->cfg.max_seq_len * m.n_kv_heads / mk::ATT_CHUNK > 2ll * ctx->sm_count) ? 1 : 0;
+  pl.att_tma = (ctx->att_tma_off == 0 && (hd == 64 || hd == 128)) ? 1 : 0;
+  if (pl.att_tma) {
+    // chunk buffers: as many as one SM's share of the K/V of a layer fills, at most four; the GEMM
+    // ring keeps at least three stages
+    const long long kv_per_cta = (long long)ctx->cfg.max_requests * ctx->cfg.max_seq_len * m.n_kv_heads * hd * 4 / std::max(ctx->sm_count, 1);
+    const long long chunk = (long long)mk::AttnSmem::kv_buf_bytes(hd);
+    int want = (int)std::min<long long>(mk::MAX_KV_BUF, std::max<long long>(1, (kv_per_cta + chunk - 1) / chunk));
+    if (ctx->att_nbuf_force > 0) want = std::min(ctx->att_nbuf_force, (int)mk::MAX_KV_BUF);
+    pl.att_nbuf = want;
+    while (pl.att_nbuf > 1 && mk::pick_stages(t_box, hd, 0, 1, 1, pl.att_nbuf) < 3) --pl.att_nbuf;
+  }
+  auto stages_for = [&](int kps) { return mk::pick_stages(t_box, hd, pl.att_dbl, kps, pl.att_tma, pl.att_nbuf); };
+  pl.kps = 1;
+  if (ctx->kps_force > 0) { if (stages_for(ctx->kps_force) >= 2) pl.kps = ctx->kps_force; }
+  else if (stages_for(2) >= 3) pl.kps = 2;
+  pl.stages = stages_for(pl.kps);
+  return pl;
 }
 
 int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
@@ -516,8 +549,8 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
   const int slot = t_box / 16 - 1;
   const int d = m.d_model, nq = m.n_heads * m.head_dim, nkv = m.n_kv_heads * m.head_dim, nqkv = nq + 2 * nkv, F = m.d_ff;
   char* ws = ctx->ws;
-  const int kps = mk_kps(ctx, m, t_box);
-  std::vector<CUtensorMap> maps((size_t)7 * m.n_layers + 4);
+  const int kps = mk_plan(ctx, m, t_box).kps;
+  std::vector<CUtensorMap> maps((size_t)9 * m.n_layers + 4);
   bool ok = true;
   for (int l = 0; l < m.n_layers && ok; ++l) {
     const stairs_layer_w& w = M.layers[l];
@@ -536,7 +569,15 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
   ok = ok && encode_map3(ctx, &maps[i_h], ws + L.h, 2 * L.max_rows, d, 2 * t_box, kps) &&
        encode_map3(ctx, &maps[i_o], ws + L.o, 2 * L.max_rows, nq, 2 * t_box, kps) &&
        encode_map3(ctx, &maps[i_ff], ws + L.ff, 2 * L.max_rows, F, 2 * t_box, kps);
-  if (!ok) return fail(ctx, STAIRS_ECUDA, "cuTensorMapEncodeTiled failed for a weight matrix or an activation buffer");
+  // K/V pools of every layer, for the attention phases' bulk copies
+  const int i_kv = i_head + 4;
+  const int kv_box_rows = std::min(ctx->cfg.kv_page_tokens, mk::ATT_CHUNK);
+  const long long pool_rows = (long long)L.n_pages * ctx->cfg.kv_page_tokens;
+  if (m.head_dim % 64 == 0)
+    for (int l = 0; l < m.n_layers && ok; ++l)
+      ok = ok && encode_kv_map(ctx, &maps[i_kv + 2 * l], M.kpool + (size_t)l * M.kv_layer_bytes, pool_rows, nkv, kv_box_rows) &&
+           encode_kv_map(ctx, &maps[i_kv + 2 * l + 1], M.vpool + (size_t)l * M.kv_layer_bytes, pool_rows, nkv, kv_box_rows);
+  if (!ok) return fail(ctx, STAIRS_ECUDA, "cuTensorMapEncodeTiled failed for a weight matrix, an activation buffer or a K/V pool");
   std::vector<mk::Phase> ph;
   auto gemm = [&](int layer, int w0, int w1, int w2, int n_src, const int* rows, bool dual, int xmap, int K, int epi, void* out, int ldo) -> mk::Phase& {
     mk::Phase p;
@@ -608,6 +649,7 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
     }
     if (!in_epilogue) simple(mk::PH_PREP, l, nullptr, M.kpool + (size_t)l * M.kv_layer_bytes, M.vpool + (size_t)l * M.kv_layer_bytes);
     simple(mk::PH_ATTN, l, nullptr, M.kpool + (size_t)l * M.kv_layer_bytes, M.vpool + (size_t)l * M.kv_layer_bytes);
+    ph.back().w_map[0] = i_kv + 2 * l; ph.back().w_map[1] = i_kv + 2 * l + 1;   // the layer's K and V pool maps
     simple(mk::PH_COMBINE, l, nullptr, nullptr, nullptr);
     const int rd[1] = {d};
     {
@@ -689,9 +731,11 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.phases = reinterpret_cast<const mk::Phase*>(base); P.n_phases = n_run;
   P.maps = reinterpret_cast<const CUtensorMap*>(base + M.prog_maps_off);
   P.T = T; P.t_box = t_box;
-  P.att_dbl = mk_att_dbl(ctx, m);
-  P.kps = mk_kps(ctx, m, t_box);
-  P.stages = mk::pick_stages(t_box, m.head_dim, P.att_dbl, P.kps);
+  const MkPlan pl = mk_plan(ctx, m, t_box);
+  P.att_dbl = pl.att_dbl; P.att_tma = pl.att_tma; P.att_nbuf = pl.att_nbuf;
+  P.kv_box_rows = std::min(ctx->cfg.kv_page_tokens, mk::ATT_CHUNK);
+  P.kps = pl.kps;
+  P.stages = pl.stages;
   P.logit_first_row = logit_first_row; P.n_logit_rows = n_logit_rows;
   P.d = m.d_model; P.Hq = m.n_heads; P.Hkv = m.n_kv_heads; P.hd = m.head_dim; P.F = m.d_ff; P.vocab = m.vocab;
   P.norm_kind = m.norm; P.rope = m.pos; P.rope_theta = m.rope_theta; P.eps = m.norm_eps;
@@ -721,7 +765,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   const int grid = std::min(ctx->sm_count, TC_GRID_MAX);
   void* args[] = {&P};
   CK(cudaLaunchCooperativeKernel((const void*)mk::k_forward, dim3(grid), dim3(mk::MK_THREADS), args,
-                                 mk::smem_bytes(t_box, P.stages, m.head_dim, P.att_dbl, P.kps), ctx->stream));
+                                 mk::smem_bytes(t_box, P.stages, m.head_dim, P.att_dbl, P.kps, P.att_tma, P.att_nbuf), ctx->stream));
   ctx->bar_base += (unsigned long long)n_run * grid;
   ctx->launches++;
   return STAIRS_OK;
@@ -990,9 +1034,11 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
   ctx->n_seq_ub.assign(cfg->max_requests, 0);
   ctx->active.assign(cfg->max_requests, 0);
   for (int p = L.n_pages - 1; p >= 0; --p) ctx->free_pages.push_back(p);
-  // clear status words, sequences, lengths and page tables (KV pages need no clearing: a
-  // position is always written before it becomes visible)
+  // clear status words, sequences, lengths and page tables; and the K/V pools: a position is always
+  // written before it becomes visible, but the attention phases fetch whole page slices, whose
+  // rows past a request's end are masked yet multiplied (by zero weights), so they must be finite
   e = cudaMemsetAsync(ctx->ws, 0, L.tok, ctx->stream);
+  if (e == cudaSuccess && L.total > L.kv_t_k) e = cudaMemsetAsync(ctx->ws + L.kv_t_k, 0, L.total - L.kv_t_k, ctx->stream);
   if (e == cudaSuccess && L.kv_t_k > L.gemm_counters)  // split-tile counters start at zero and return to zero
     e = cudaMemsetAsync(ctx->ws + L.gemm_counters, 0, L.w13_t - L.gemm_counters, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
@@ -1405,11 +1451,17 @@ int stairs_debug_tune(stairs_ctx* ctx, int what, long long value) {
     case 0:
       if (value != 0 && value != 1 && value != 2) return fail(ctx, STAIRS_EINVAL, "k-blocks per stage must be 0 (auto), 1 or 2");
       ctx->kps_force = (int)value;
-      for (bool& b : ctx->target.prog_built) b = false;   // programs carry the tensor maps' box depth
-      for (bool& b : ctx->draft.prog_built) b = false;
       break;
+    case 1:
+      if (value < 0 || value > mk::MAX_KV_BUF) return fail(ctx, STAIRS_EINVAL, "K/V chunk buffers must be 0 (auto) .. %d", mk::MAX_KV_BUF);
+      ctx->att_nbuf_force = (int)value;
+      break;
+    case 2: ctx->att_tma_off = value ? 1 : 0; break;
     default: return fail(ctx, STAIRS_EINVAL, "unknown tuning knob %d", what);
   }
+  // programs carry the tensor maps' box depth, which follows from the shared-memory plan
+  for (bool& b : ctx->target.prog_built) b = false;
+  for (bool& b : ctx->draft.prog_built) b = false;
   return STAIRS_OK;
 }
 

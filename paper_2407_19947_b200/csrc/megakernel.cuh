@@ -98,7 +98,10 @@ struct Params {
   float4* stats;            // [64 rows][stat_tiles] (mean, M2, count, -) per 128-column tile of x
   int stat_tiles;
   const float* rope_inv;
-  int att_dbl;               // attention: two K/V chunk buffers, the next chunk's copies fly under the current chunk's MMAs
+  int att_dbl;               // attention, copy path: two K/V chunk buffers, the next chunk's copies fly under the current chunk's MMAs
+  int att_tma;               // attention, TMA path (head sizes 64 and 128): a loader warp streams K/V chunks through att_nbuf buffers
+  int att_nbuf;
+  int kv_box_rows;           // rows of one K/V box: min(page_tokens, chunk)
   __half* q16;               // [row][Hq*hd] queries, rotated and scaled by 1/sqrt(hd), written by the QKV epilogue
   float* rope_cs; float* rope_sn;   // [row][hd/2] cos and sin of the call's row positions, written by the embedding phase
      // [hd/2] theta^(-2i/hd)
@@ -116,7 +119,8 @@ struct Params {
   unsigned long long* trace;   // optional: per phase {start, work done, arrived} ns timestamps of CTA 0 and of the last CTA
 };
 
-constexpr int MK_THREADS = THREADS;
+constexpr int MK_THREADS = THREADS + 32;   // the GEMM kernel's six warps plus the K/V loader of the attention phases
+constexpr int MAX_KV_BUF = 4;
 constexpr int ATT_CHUNK = 64;
 constexpr int ATT_QBLK = 48;
 constexpr int VT_LD = 132;                      // row pitch (floats) of the epilogue's 16 x 128 exchange tile
@@ -127,7 +131,12 @@ struct AttnSmem {   // carved after the GEMM ring: Q block (bf16), K and V chunk
   static __host__ __device__ size_t q_bytes(int hd) { return (size_t)ATT_QBLK * k_pitch(hd); }
   static __host__ __device__ size_t kv_bytes(int hd) { return (size_t)ATT_CHUNK * k_pitch(hd); }
   static __host__ __device__ size_t merge_bytes(int hd) { return (size_t)16 * (hd + 4) * 4 + 64; }
-  static __host__ __device__ size_t bytes(int hd, int dbl) { return q_bytes(hd) + (dbl ? 4 : 2) * kv_bytes(hd) + 64; }   // dbl: two K/V chunk buffers
+  // TMA path: a chunk buffer holds K then V, each as hd / 64 column halves of [CHUNK rows][128 bytes] with the 128-byte swizzle
+  static __host__ __device__ size_t kv_buf_bytes(int hd) { return (size_t)2 * ATT_CHUNK * hd * 2; }
+  // copy path: Q block, then one or two padded K/V buffers; TMA path: nbuf chunk buffers (1024-byte aligned), then the Q block
+  static __host__ __device__ size_t bytes(int hd, int dbl, int tma, int nbuf) {
+    return tma ? 1024 + (size_t)nbuf * kv_buf_bytes(hd) + q_bytes(hd) + 64 : q_bytes(hd) + (dbl ? 4 : 2) * kv_bytes(hd) + 64;
+  }
 };
 
 // 16-byte asynchronous copy global -> shared; `on` false writes zeros and reads nothing
@@ -153,6 +162,13 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t* r, const void* p) {
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, const void* p) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(p)));
+}
+// 2^x by the hardware approximation (relative error about 2^-22; the softmax weights are rounded
+// to fp16 afterwards).  Scores are kept in the base-2 domain: the queries carry log2(e) / sqrt(hd).
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
   __half2 v = __floats2half2_rn(lo, hi);
@@ -255,6 +271,8 @@ struct AttnReq { int slot, base, R, off, n_chunks, cpu, n_ranges, n_qblk, units;
 // Shared per-CTA control block.
 struct Ctl {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
+  uint64_t kv_full[MAX_KV_BUF], kv_empty[MAX_KV_BUF];   // attention K/V chunk buffers (TMA path)
+  volatile int areq_ready;                              // the requests' attention geometry below is filled in
   uint32_t tmem_slot;
   volatile int abort_flag;
   volatile int bcast;
@@ -365,6 +383,11 @@ struct WCursor {
 };
 
 // Asks L2 for one weight tile ahead of the shared-memory ring (no shared memory, no barrier involved).
+__device__ __forceinline__ void tma_load_2d_nohint(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar)) : "memory");
+}
 // Tiled 3-D load global -> shared.  The operand matrices [rows, K] are described to TMA as
 // [K / 64][rows][64]: a box of (64, rows of the tile, kps) lands as kps consecutive K-major slabs
 // with the 128-byte swizzle, i.e. several k-blocks per copy instruction.
@@ -497,25 +520,38 @@ __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
 }
 
 
+// Consumer side of the K/V chunk ring of the TMA path: buffer and parity of the next chunk.
+struct KvCons { int buf; uint32_t par; };
+
 // One attention unit, executed by the 128 compute threads (4 warps), on the legacy tensor path
-// (mma.sync m16n8k16; the tiles are far too small for tcgen05).  The unit's queries are cut into
-// blocks of 16 (one MMA M tile); each 64-position chunk is staged once in shared memory and warp
-// w takes positions 16w..16w+15 of it for every block: S = Q.K^T (2 n-tiles x hd/16 k-steps),
-// online softmax per row with quad shuffles, O += P.V with P reused from the accumulator
-// registers and V fetched with ldmatrix.trans.  The four warps' (max, sum, O) states are merged
-// in warp order through a small shared buffer - a fixed order - and the block's result is either
-// final (the unit saw every visible position) or parked for the combine phase.
+// (mma.sync m16n8k16).  The unit's queries are cut into blocks of 16 (one MMA M tile), one warp
+// per block: S = Q.K^T, online softmax per row with quad shuffles, O += P.V with P reused from
+// the accumulator registers and V fetched with ldmatrix.trans; softmax state and output
+// accumulators never leave the warp's registers.  With one or two blocks the warps also split
+// each chunk's positions in two and merge once per unit.  The block's result is either final
+// (the unit saw every visible position) or parked for the combine phase.
+//
+// K/V chunks of 64 positions reach shared memory in one of two ways.  TMA path (head sizes 64 and
+// 128): the loader warp streams them through a ring of buffers with tiled bulk copies (one box per
+// page slice and 64-column half, 128-byte swizzle) and this function only waits on the ring's
+// barriers - chunks of already cached positions are in flight before the phase even starts.
+// Copy path (other head sizes): the compute threads stage padded tiles with 16-byte asynchronous
+// copies, cache rows looked up once per chunk.
+template <bool TMA>
 __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot,
-                          uint8_t* att_smem, Ctl* ctl, int et, bool& ok,
+                          uint8_t* att_smem, Ctl* ctl, int et, bool& ok, KvCons& kvc, const Waiter& W,
                           unsigned long long* tra) {
   const int hd = P.hd, G = P.Hq / P.Hkv, nkv = P.Hkv * hd, nq = P.Hq * hd;
   const int lane = et & 31, w = et >> 5, g = lane >> 2, t4 = lane & 3;
   const int Q = a.R * G;
   const int q0 = qblk * ATT_QBLK, nQ = min(ATT_QBLK, Q - q0);
-  const size_t pitch = AttnSmem::k_pitch(hd);
-  uint8_t* qs = att_smem;                                   // [QBLK][pitch] bf16, rotated and pre-scaled
-  uint8_t* kv0 = qs + AttnSmem::q_bytes(hd);                // chunk buffer b: K [CHUNK][pitch] then V, at kv0 + b * 2 * kv_bytes
+  const size_t pitch = AttnSmem::k_pitch(hd);               // padded row pitch (queries; K/V of the copy path)
   const size_t kvb = AttnSmem::kv_bytes(hd);
+  const size_t kvbuf = AttnSmem::kv_buf_bytes(hd);
+  // TMA path: ring of chunk buffers (1024-byte aligned) then the Q block; copy path: Q block then padded buffers
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem) + 1023) & ~(uintptr_t)1023);
+  uint8_t* qs = TMA ? ring + (size_t)P.att_nbuf * kvbuf : att_smem;   // [QBLK][pitch] fp16, rotated and pre-scaled
+  uint8_t* kv0 = qs + AttnSmem::q_bytes(hd);                // copy path, buffer b: K [CHUNK][pitch] then V, at kv0 + b * 2 * kvb
   uint8_t* ks = kv0;                                        // the buffer being computed on
   uint8_t* vs = ks + kvb;
   __half* kc = reinterpret_cast<__half*>(ph.kc);
@@ -525,14 +561,25 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
 
   const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
   const int n_mt = (nQ + 15) / 16;
-
-  // Stages chunk c (and, with the unit's first chunk, its queries) with 16-byte asynchronous
-  // copies issued by all 128 threads (no registers held, so all of a thread's copies are in
-  // flight together; rows past the end are zero-filled by the copy itself).  One bulk copy per
-  // row was tried first: ~180 small copies per chunk queue up in the copy engine for
-  // microseconds.  The rows of this call's new positions are in the cache already: the QKV
-  // epilogue put them there, as it put the rotated and scaled queries into the query buffer.
   const int pieces = hd * 2 / 16;   // 16-byte pieces per row
+
+  // the unit's queries: query index q -> row r = q / G, head = kvh * G + q % G; rows past the unit's queries are zero
+  auto stage_q = [&]() {
+    const int dj = 128 / pieces, dp = 128 % pieces;
+    int ql = et / pieces, pc = et % pieces;
+    while (ql < ATT_QBLK) {
+      const bool on = ql < nQ;
+      const int q = on ? q0 + ql : q0;
+      cp_async16(qs + (size_t)ql * pitch + pc * 16,
+                 reinterpret_cast<const uint4*>(P.q16 + (size_t)(a.off + q / G) * nq + (size_t)(kvh * G + q % G) * hd) + pc, on);
+      ql += dj; pc += dp;
+      if (pc >= pieces) { pc -= pieces; ++ql; }
+    }
+  };
+  // Copy path: stages chunk c (and, with the unit's first chunk, its queries) with 16-byte
+  // asynchronous copies issued by all 128 threads (no registers held, so all of a thread's copies
+  // are in flight together; rows past the end are zero-filled by the copy itself).  The rows of
+  // this call's new positions are in the cache already: the QKV epilogue put them there.
   auto stage_issue = [&](int c, int b, bool with_q) {
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
@@ -560,24 +607,13 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
         if (pc >= pieces) { pc -= pieces; ++jr; }
       }
     }
-    if (with_q) {
-      // query index q -> row r = q / G, head = kvh * G + q % G; rows past the unit's queries are zero
-      const int dj = 128 / pieces, dp = 128 % pieces;
-      int ql = et / pieces, pc = et % pieces;
-      while (ql < ATT_QBLK) {
-        const bool on = ql < nQ;
-        const int q = on ? q0 + ql : q0;
-        cp_async16(qs + (size_t)ql * pitch + pc * 16,
-                   reinterpret_cast<const uint4*>(P.q16 + (size_t)(a.off + q / G) * nq + (size_t)(kvh * G + q % G) * hd) + pc, on);
-        ql += dj; pc += dp;
-        if (pc >= pieces) { pc -= pieces; ++ql; }
-      }
-    }
+    if (with_q) stage_q();
     cp_async_commit();
   };
 
   if (tra) tra[1] = globaltimer_ns();
-  stage_issue(c_begin, 0, true);
+  if (TMA) { stage_q(); cp_async_commit(); }
+  else stage_issue(c_begin, 0, true);
   if (tra) tra[2] = globaltimer_ns();
 
   // Warp w owns query block (MMA M tile) w of the unit and walks the chunk's four 16-position
@@ -597,16 +633,33 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   for (int nd = 0; nd < 16; ++nd) { o[nd][0] = o[nd][1] = o[nd][2] = o[nd][3] = 0.f; }
 
   int cur = 0;
+  int hold_buf = -1;   // TMA path: the last chunk's buffer is kept (it serves the merge) and released at the end
   for (int c = c_begin; c < c_end && ok; ++c) {
-    // with two chunk buffers the next chunk's copies are issued before this chunk is waited for
-    const bool ahead = P.att_dbl && c + 1 < c_end;
-    if (ahead) { stage_issue(c + 1, cur ^ 1, false); cp_async_wait_but_one(); }
-    else cp_async_wait_all();
-    epi_bar_sync();
-    ks = kv0 + (size_t)cur * 2 * kvb; vs = ks + kvb;
+    if (TMA) {
+      if (c == c_begin) { cp_async_wait_all(); epi_bar_sync(); }   // the queries
+      cur = kvc.buf;
+      if (!W.wait(ctl->kv_full + cur, kvc.par)) { ok = false; break; }   // (the verdict is made uniform after the loop)
+      __syncwarp();
+      ks = ring + (size_t)cur * kvbuf; vs = ks + kvbuf / 2;
+      if (++kvc.buf == P.att_nbuf) { kvc.buf = 0; kvc.par ^= 1u; }
+    } else {
+      // with two chunk buffers the next chunk's copies are issued before this chunk is waited for
+      const bool ahead = P.att_dbl && c + 1 < c_end;
+      if (ahead) { stage_issue(c + 1, cur ^ 1, false); cp_async_wait_but_one(); }
+      else cp_async_wait_all();
+      epi_bar_sync();
+      ks = kv0 + (size_t)cur * 2 * kvb; vs = ks + kvb;
+    }
     if (tra && c == c_begin) tra[4] = globaltimer_ns();
     const int p0 = c * ATT_CHUNK;
     const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
+    const bool all_visible = p0 + ATT_CHUNK - 1 <= a.base;   // (then n_pos is a whole chunk too)
+    // address of the 16-byte piece `piece` of row j of a K or V tile: padded rows (copy path) or
+    // 64-column halves of 128-byte rows with the 128-byte swizzle (TMA path)
+    auto kv_addr = [&](const uint8_t* base, int j, int piece) -> const uint8_t* {
+      if (TMA) return base + (size_t)(piece >> 3) * (ATT_CHUNK * 128) + (size_t)j * 128 + (size_t)(((piece & 7) ^ (j & 7)) << 4);
+      return base + (size_t)j * pitch + (size_t)piece * 16;
+    };
     if (active) {
       // 32 positions (two MMA k-steps of P.V, four n-tiles of S) per round: four independent
       // accumulator chains hide the MMA latency, and the softmax bookkeeping is done once per 32
@@ -619,14 +672,14 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
         // n-tiles (positions x the two halves).  Lane l supplies the address of matrix l / 8,
         // row l % 8.
         const uint8_t* q_lane = qs + (size_t)(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * pitch + (lane >> 4) * 16;
-        const uint8_t* k_lane = ks + (size_t)(sl0 + (lane & 7) + (lane >> 4) * 8) * pitch + ((lane >> 3) & 1) * 16;
+        const int k_row = sl0 + (lane & 7) + (lane >> 4) * 8, k_pc = (lane >> 3) & 1;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           if (kk < ksteps) {
             uint32_t af[4], kf0[4], kf1[4];
             ldmatrix_x4(af, q_lane + kk * 32);
-            ldmatrix_x4(kf0, k_lane + kk * 32);
-            ldmatrix_x4(kf1, k_lane + 16 * pitch + kk * 32);
+            ldmatrix_x4(kf0, kv_addr(ks, k_row, kk * 2 + k_pc));
+            ldmatrix_x4(kf1, kv_addr(ks, k_row + 16, kk * 2 + k_pc));
             mma_16816(sc[0], af, kf0[0], kf0[1]);
             mma_16816(sc[1], af, kf0[2], kf0[3]);
             mma_16816(sc[2], af, kf1[0], kf1[1]);
@@ -634,30 +687,39 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
           }
         }
         // staircase mask (rows past the chunk's last position hold stale data: assigned, never
-        // computed with), row maxima
+        // computed with), row maxima.  A chunk of positions cached before this call is visible to
+        // every query as a whole and needs no mask.
         float mx_a = -INFINITY, mx_b = -INFINITY;
+        if (all_visible) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+          for (int j = 0; j < 4; ++j) {
+            mx_a = fmaxf(mx_a, fmaxf(sc[j][0], sc[j][1])); mx_b = fmaxf(mx_b, fmaxf(sc[j][2], sc[j][3]));
+          }
+          // (rows past the unit's queries hold zero queries: they run along harmlessly and are never written)
+        } else {
 #pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int jl = sl0 + 8 * j + t4 * 2 + e, pj = p0 + jl;
-            const bool in = jl < n_pos;
-            if (!(in && pj <= last_a)) sc[j][e] = -INFINITY;
-            if (!(in && pj <= last_b)) sc[j][2 + e] = -INFINITY;
-            mx_a = fmaxf(mx_a, sc[j][e]); mx_b = fmaxf(mx_b, sc[j][2 + e]);
+          for (int j = 0; j < 4; ++j) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int jl = sl0 + 8 * j + t4 * 2 + e, pj = p0 + jl;
+              const bool in = jl < n_pos;
+              if (!(in && pj <= last_a)) sc[j][e] = -INFINITY;
+              if (!(in && pj <= last_b)) sc[j][2 + e] = -INFINITY;
+              mx_a = fmaxf(mx_a, sc[j][e]); mx_b = fmaxf(mx_b, sc[j][2 + e]);
+            }
           }
         }
         mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1)); mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
         mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1)); mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
         const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
         const float off_a = mn_a == -INFINITY ? 0.f : mn_a, off_b = mn_b == -INFINITY ? 0.f : mn_b;
-        const float corr_a = expf(m_a - off_a), corr_b = expf(m_b - off_b);   // exp(-inf) = 0
+        const float corr_a = fast_exp2(m_a - off_a), corr_b = fast_exp2(m_b - off_b);   // 2^(-inf) = 0
         float sum_a = 0.f, sum_b = 0.f;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
-            sc[j][e] = expf(sc[j][e] - off_a); sc[j][2 + e] = expf(sc[j][2 + e] - off_b);
+            sc[j][e] = fast_exp2(sc[j][e] - off_a); sc[j][2 + e] = fast_exp2(sc[j][2 + e] - off_b);
             sum_a += sc[j][e]; sum_b += sc[j][2 + e];
           }
         }
@@ -672,59 +734,81 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
           pf[h][2] = pack_f16x2(sc[2 * h + 1][0], sc[2 * h + 1][1]); pf[h][3] = pack_f16x2(sc[2 * h + 1][2], sc[2 * h + 1][3]);
         }
         // V fragments: lane supplies the address of row (lane & 15) of a 16-position slice, column block (lane >> 4)
-        const uint8_t* vrow = vs + (size_t)(sl0 + (lane & 15)) * pitch + (lane >> 4) * 16;
-        const bool second = sl0 + 16 < ATT_CHUNK;   // (always true for 64-position chunks walked in steps of 32)
+        const int v_row = sl0 + (lane & 15), v_pc = lane >> 4;
+        // the running maxima often stay put: then the accumulators need no rescaling (one vote per warp)
+        const bool rescale = !__all_sync(0xffffffffu, corr_a == 1.0f && corr_b == 1.0f);
 #pragma unroll
         for (int nd = 0; nd < 16; nd += 2) {
           if (nd < ntiles) {
-            o[nd][0] *= corr_a; o[nd][1] *= corr_a; o[nd][2] *= corr_b; o[nd][3] *= corr_b;
-            o[nd + 1][0] *= corr_a; o[nd + 1][1] *= corr_a; o[nd + 1][2] *= corr_b; o[nd + 1][3] *= corr_b;
+            if (rescale) {
+              o[nd][0] *= corr_a; o[nd][1] *= corr_a; o[nd][2] *= corr_b; o[nd][3] *= corr_b;
+              o[nd + 1][0] *= corr_a; o[nd + 1][1] *= corr_a; o[nd + 1][2] *= corr_b; o[nd + 1][3] *= corr_b;
+            }
             uint32_t vf[4], vg[4];
-            ldmatrix_x4_trans(vf, vrow + nd * 16);
-            if (second) ldmatrix_x4_trans(vg, vrow + 16 * pitch + nd * 16);
+            ldmatrix_x4_trans(vf, kv_addr(vs, v_row, nd + v_pc));
+            ldmatrix_x4_trans(vg, kv_addr(vs, v_row + 16, nd + v_pc));
             mma_16816(o[nd], pf[0], vf[0], vf[1]);
             mma_16816(o[nd + 1], pf[0], vf[2], vf[3]);
-            if (second) {
-              mma_16816(o[nd], pf[1], vg[0], vg[1]);
-              mma_16816(o[nd + 1], pf[1], vg[2], vg[3]);
-            }
+            mma_16816(o[nd], pf[1], vg[0], vg[1]);
+            mma_16816(o[nd + 1], pf[1], vg[2], vg[3]);
           }
         }
       }
     }
-    epi_bar_sync();   // tile may be overwritten by the next chunk or unit
     if (tra && c == c_begin) tra[5] = globaltimer_ns();
-    if (P.att_dbl) cur ^= 1;
-    else if (c + 1 < c_end) stage_issue(c + 1, 0, false);
+    if (TMA) {
+      // this warp is done with the buffer: hand it back to the loader (the unit's last one is kept for the merge)
+      __syncwarp();
+      if (c + 1 < c_end) { if (lane == 0) mbar_arrive(ctl->kv_empty + cur); }
+      else hold_buf = cur;
+    } else {
+      epi_bar_sync();   // tile may be overwritten by the next chunk or unit
+      if (P.att_dbl) cur ^= 1;
+      else if (c + 1 < c_end) stage_issue(c + 1, 0, false);
+    }
   }
-  ks = kv0; vs = ks + kvb;   // (buffer 0 serves the merge below)
-  if (!ok) return;
+  if (TMA) {
+    // one verdict for all 128 threads (a wait may have run out in some of them only)
+    if (!ok) ctl->abort_flag = 1;
+    ok = group_ok(ctl, et);
+    if (!ok) return;
+    ks = ring + (size_t)hold_buf * kvbuf;   // every warp has finished reading it (the barriers above)
+  } else {
+    ks = kv0;   // (buffer 0 serves the merge below)
+    if (!ok) return;
+  }
   if (ps == 2) {
     // second half's state -> shared memory (the K/V tiles are free now) -> merged into the first's
     float4* mb = reinterpret_cast<float4*>(ks);
+    const int ms = ntiles + 1;   // vectors per block: the output n-tiles, then (max, sum)
     if (active && part == 1) {
 #pragma unroll
       for (int nd = 0; nd < 16; ++nd)
-        if (nd < ntiles) mb[(mt * 17 + nd) * 32 + lane] = make_float4(o[nd][0], o[nd][1], o[nd][2], o[nd][3]);
-      mb[(mt * 17 + 16) * 32 + lane] = make_float4(m_a, m_b, l_a, l_b);
+        if (nd < ntiles) mb[(mt * ms + nd) * 32 + lane] = make_float4(o[nd][0], o[nd][1], o[nd][2], o[nd][3]);
+      mb[(mt * ms + ntiles) * 32 + lane] = make_float4(m_a, m_b, l_a, l_b);
     }
     epi_bar_sync();
     if (active && part == 0) {
-      const float4 st = mb[(mt * 17 + 16) * 32 + lane];
+      const float4 st = mb[(mt * ms + ntiles) * 32 + lane];
       const float M_a = fmaxf(m_a, st.x), M_b = fmaxf(m_b, st.y);
       const float off_a = M_a == -INFINITY ? 0.f : M_a, off_b = M_b == -INFINITY ? 0.f : M_b;
-      const float wa = expf(m_a - off_a), wa2 = expf(st.x - off_a), wb = expf(m_b - off_b), wb2 = expf(st.y - off_b);
+      const float wa = fast_exp2(m_a - off_a), wa2 = fast_exp2(st.x - off_a), wb = fast_exp2(m_b - off_b), wb2 = fast_exp2(st.y - off_b);
       l_a = l_a * wa + st.z * wa2; l_b = l_b * wb + st.w * wb2;
       m_a = M_a; m_b = M_b;
 #pragma unroll
       for (int nd = 0; nd < 16; ++nd)
         if (nd < ntiles) {
-          const float4 v = mb[(mt * 17 + nd) * 32 + lane];
+          const float4 v = mb[(mt * ms + nd) * 32 + lane];
           o[nd][0] = o[nd][0] * wa + v.x * wa2; o[nd][1] = o[nd][1] * wa + v.y * wa2;
           o[nd][2] = o[nd][2] * wb + v.z * wb2; o[nd][3] = o[nd][3] * wb + v.w * wb2;
         }
     }
-    // (the next unit's staging starts with a barrier of its own before it overwrites the tiles)
+    // (copy path: the next unit's staging starts with a barrier of its own before it overwrites the tiles)
+  }
+  if (TMA) {
+    // the merge buffer (the last chunk's tiles) goes back to the loader: one arrival per warp
+    __syncwarp();
+    if (lane == 0) mbar_arrive(ctl->kv_empty + hold_buf);
   }
   if (!active || part != 0) return;
 
@@ -792,7 +876,8 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
     for (int s = 0; s < stages; ++s) { mbar_init(ctl->full + s, 1); mbar_init(ctl->empty + s, 1); }
     mbar_init(ctl->acc_full + 0, 1); mbar_init(ctl->acc_full + 1, 1);
     mbar_init(ctl->acc_empty + 0, 4); mbar_init(ctl->acc_empty + 1, 4);
-    ctl->abort_flag = 0; ctl->bcast = 0;
+    for (int b = 0; b < MAX_KV_BUF; ++b) { mbar_init(ctl->kv_full + b, 1); mbar_init(ctl->kv_empty + b, 4); }
+    ctl->abort_flag = 0; ctl->bcast = 0; ctl->areq_ready = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) tmem_alloc(&ctl->tmem_slot, tmem_cols);
@@ -929,6 +1014,90 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
         if (trm) trm[6] = globaltimer_ns();
       }
     }
+  } else if (warp == 6) {
+    // ================================================================== K/V loader of the attention phases (TMA path)
+    // Walks this CTA's attention units of every attention phase in the compute group's order and
+    // streams their K/V chunks through the ring of chunk buffers: per chunk one box per (K or V,
+    // 64-column half, page slice), each issued by its own lane.  Chunks that hold only positions
+    // cached by earlier calls are fetched as soon as a buffer is free - also ahead of the phase;
+    // a chunk with positions of this call waits for the grid barrier that publishes them.
+    if (P.att_tma) {
+      bool ok = true;
+      {
+        bool seen = false;
+        if (lane == 0) {
+          const long long t0 = clock64();
+          while (!(seen = ctl->areq_ready != 0)) { if (W.poll_abort(t0)) break; }
+        }
+        ok = __shfl_sync(0xffffffffu, seen ? 1 : 0, 0) != 0;
+        __syncwarp();
+      }
+      const int hd = P.hd, halves = hd / 64, box_rows = P.kv_box_rows, slots = ATT_CHUNK / box_rows;
+      const int n_boxes = 2 * halves * slots;
+      const size_t kvbuf = AttnSmem::kv_buf_bytes(hd);
+      uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem) + 1023) & ~(uintptr_t)1023);
+      // this lane's box: which tensor (K, V), which 64-column half, which page slice of the chunk
+      const int b_which = lane / (halves * slots), b_half = (lane % (halves * slots)) / slots, b_slot = lane % slots;
+      int buf = 0; uint32_t par = 0;
+      uint32_t used = 0, last_par = 0;   // per buffer: ever filled, and the parity of its latest fill
+      const int n_req = P.mode == CALL_VALIDATE ? P.n_req : 1;
+      for (int ph = 0; ph < P.n_phases && ok; ++ph) {
+        const Phase& p = P.phases[ph];
+        if (p.kind != PH_ATTN) continue;
+        const CUtensorMap* kmap = P.maps + p.w_map[0];
+        const CUtensorMap* vmap = P.maps + p.w_map[1];
+        bool published = false;   // the grid barrier before this phase has completed
+        int u0 = 0;
+        for (int i = 0; i < n_req && ok; ++i) {
+          const AttnReq a = ctl->areq[i];
+          const int* pt = P.page_table + (size_t)a.slot * P.max_pages;
+          const int first = (cta - u0 % G + G) % G;
+          for (int u = first; u < a.units && ok; u += G) {
+            const int rest = u / a.n_qblk;
+            const int range = rest % a.n_ranges, kvh = rest / a.n_ranges;
+            const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
+            for (int c = c_begin; c < c_end && ok; ++c) {
+              const int p0 = c * ATT_CHUNK;
+              bool go = true;
+              if (lane == 0) {
+                if (p0 + ATT_CHUNK > a.base && !published) go = W.wait_grid(bar_count, P.bar_base + (unsigned long long)ph * G);
+                if (go) go = W.wait(ctl->kv_empty + buf, par ^ 1u);
+              }
+              ok = __shfl_sync(0xffffffffu, go ? 1 : 0, 0) != 0;
+              if (!ok) break;
+              if (p0 + ATT_CHUNK > a.base && !published) { published = true; fence_proxy_async(); }
+              // page slices of the chunk inside the request's page table (the rest keeps its old, finite contents)
+              const int valid_slots = min(slots, (P.max_pages * P.page_tokens - p0) / box_rows);
+              if (lane == 0) mbar_expect_tx(ctl->kv_full + buf, (uint32_t)(2 * halves * valid_slots * box_rows * 128));
+              __syncwarp();
+              if (lane < n_boxes && b_slot < valid_slots) {
+                const int pz = p0 + b_slot * box_rows;
+                const int row = pt[pz / P.page_tokens] * P.page_tokens + pz % P.page_tokens;
+                uint8_t* dst = ring + (size_t)buf * kvbuf + (size_t)b_which * (kvbuf / 2) + (size_t)b_half * (ATT_CHUNK * 128) + (size_t)b_slot * box_rows * 128;
+                tma_load_2d_nohint(dst, b_which ? vmap : kmap, kvh * hd + b_half * 64, row, ctl->kv_full + buf);
+              }
+              __syncwarp();
+              used |= 1u << buf;
+              last_par = (last_par & ~(1u << buf)) | (par << buf);
+              if (++buf == P.att_nbuf) { buf = 0; par ^= 1u; }
+            }
+          }
+          u0 += a.units;
+        }
+      }
+      // After an abort copies may still be in flight: they must land before the CTA's shared memory
+      // is given up (bounded, like the producer's drain below; after a healthy pass every fill
+      // was consumed, so these tests succeed at once).
+      if (lane == 0) {
+        const long long t0 = clock64();
+        const unsigned long long drain_limit = P.wait_limit > 2000000ull ? P.wait_limit : 2000000ull;
+        for (int b = 0; b < P.att_nbuf; ++b)
+          if (used & (1u << b))
+            while (!mbar_try(ctl->kv_full + b, (last_par >> b) & 1u)) {
+              if ((unsigned long long)(clock64() - t0) > drain_limit) break;
+            }
+      }
+    }
   } else {
     // ================================================================== compute group (warps 2..5)
     const int quad = warp & 3;
@@ -946,8 +1115,17 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
       if (et < PH_WORDS) ctl->phc[0][et] = __ldcg(reinterpret_cast<const uint32_t*>(P.phases) + et);
       const int n_req0 = P.mode == CALL_VALIDATE ? P.n_req : 1;
       if (et < n_req0 && et < 64) ctl->areq[et] = attn_req(P, et, G);
+      if (P.att_tma) {
+        // the chunk buffers start out finite: a box that is never fetched (past the page table) must not feed NaNs to P.V
+        uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem) + 1023) & ~(uintptr_t)1023);
+        const int n16 = (int)((size_t)P.att_nbuf * AttnSmem::kv_buf_bytes(P.hd) / 16);
+        for (int i = et; i < n16; i += 128) reinterpret_cast<uint4*>(ring)[i] = make_uint4(0u, 0u, 0u, 0u);
+        fence_proxy_async();   // later bulk copies (async proxy) into these buffers
+      }
       epi_bar_sync();
+      if (et == 0) { __threadfence_block(); ctl->areq_ready = 1; }
     }
+    KvCons kvc{0, 0u};
     for (int ph = 0; ph < P.n_phases && ok; ++ph) {
       const Phase& p = *reinterpret_cast<const Phase*>(ctl->phc[ph & 1]);
       // the next phase's descriptor: fetched now, parked in shared memory at the end of this phase
@@ -993,8 +1171,9 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
               ok = group_ok(ctl, et);
               break;
             }
-            attn_unit(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok,
-                        (MK_TRACE_PTR(P.trace) && et == 0 && u == first) ? MK_TRACE_PTR(P.trace) + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr);
+            unsigned long long* tra_u = (MK_TRACE_PTR(P.trace) && et == 0 && u == first) ? MK_TRACE_PTR(P.trace) + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
+            if (P.att_tma) attn_unit<true>(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok, kvc, W, tra_u);
+            else attn_unit<false>(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok, kvc, W, tra_u);
           }
           u0 += a.units; g0 += P.Hkv * a.n_qblk;
         }
@@ -1038,7 +1217,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
                   mu = -INFINITY; lu = 0.f;
                   if (r < nr) { mu = __ldcg(base + r * stride + hd); lu = __ldcg(base + r * stride + hd + 1); }
                 }
-                const float wgt = mu == -INFINITY ? 0.f : expf(mu - M);   // 0 for lanes past the last range
+                const float wgt = mu == -INFINITY ? 0.f : fast_exp2(mu - M);   // 0 for lanes past the last range (maxima are base-2 exponents)
                 L += lu * wgt;
                 const int nb = min(32, nr - rb);
                 for (int g0 = 0; g0 < nb; g0 += 16) {
@@ -1075,7 +1254,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
         // phase rotates, converts and files q, k and v.  One item = one pair of one head of one row.
         const int hd = P.hd, half = hd / 2, nq = P.Hq * hd, nkv = P.Hkv * hd, nqkv = nq + 2 * nkv, heads = P.Hq + 2 * P.Hkv;
         const int items = P.T * heads * half;
-        const float qscale = 1.0f / sqrtf((float)hd);
+        const float qscale = 1.4426950408889634f / sqrtf((float)hd);   // log2(e) / sqrt(hd): the softmax works in base 2
         for (int it = cta * 128 + et; it < items; it += G * 128) {
           const int i = it % half, hs = (it / half) % heads, t = it / (half * heads);
           const float* row = P.qkv + (size_t)t * nqkv + (size_t)hs * hd;   // q heads, then k heads, then v heads
@@ -1486,7 +1665,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
                     if (P.hd == 128) { rot(a[0], a[2], rca, rsa); rot(a[1], a[3], rcb, rsb); }
                     else { rot(a[0], a[1], rca, rsa); rot(a[2], a[3], rcb, rsb); }
                   }
-                  const float qscale = src_s == 0 ? 1.0f / sqrtf((float)P.hd) : 1.0f;
+                  const float qscale = src_s == 0 ? 1.4426950408889634f / sqrtf((float)P.hd) : 1.0f;   // log2(e) / sqrt(hd): the softmax works in base 2
                   const int nq_all = P.Hq * P.hd, nkv_all = P.Hkv * P.hd;
                   __half* dst = src_s == 0 ? P.q16 + (size_t)t * nq_all
                                            : reinterpret_cast<__half*>(src_s == 1 ? p.kc : p.vc) + (size_t)kv_row * nkv_all;
@@ -1577,13 +1756,13 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, tmem_cols); }
 }
 
-inline size_t smem_bytes(int t_box, int stages, int hd, int dbl, int kps) {
+inline size_t smem_bytes(int t_box, int stages, int hd, int dbl, int kps, int tma = 0, int nbuf = 0) {
   return 1024 + (size_t)stages * kps * (A_STAGE_BYTES + (size_t)2 * t_box * BK * 2) + MK_XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127) +
-         AttnSmem::bytes(hd, dbl) + 64;
+         AttnSmem::bytes(hd, dbl, tma, nbuf) + 64;
 }
-inline int pick_stages(int t_box, int hd, int dbl, int kps) {
+inline int pick_stages(int t_box, int hd, int dbl, int kps, int tma = 0, int nbuf = 0) {
   int s = MAX_STAGES;
-  while (s > 1 && smem_bytes(t_box, s, hd, dbl, kps) > (size_t)SMEM_LIMIT) --s;
+  while (s > 1 && smem_bytes(t_box, s, hd, dbl, kps, tma, nbuf) > (size_t)SMEM_LIMIT) --s;
   return s;
 }
 // k-blocks per stage: two while at least three stages still fit (small row boxes), else one
