@@ -171,6 +171,130 @@ def time_validate(eng, torch, k, drafts_dev, steps, warmup):
     return e0.elapsed_time(e1) * 1e3 / steps
 
 
+def workload_label(w, prefix, k, n_req):
+    """One string for both arms, so the two lines name the same workload."""
+    return f"{w.name}: prefix {prefix}, k {k}, {n_req * (k + 1)} stair rows, {n_req} request{'s' if n_req > 1 else ''} per call, commit=0"
+
+
+def prefill_flops(shape, n_tokens: int) -> float:
+    """Useful floating-point operations of one model's prefill of n_tokens positions: every layer
+    matrix once per token (2 flops per weight) plus causal attention (scores and weighted values)."""
+    es = 2 if shape.wdtype == wl.WDTYPE_BF16 else 4
+    layer_params = (shape.weight_bytes_per_call() // es - shape.vocab * shape.d_model)     # without the LM head
+    gemm = 2.0 * layer_params * n_tokens
+    attn = 4.0 * shape.n_layers * shape.n_heads * shape.head_dim * (n_tokens * (n_tokens + 1) / 2.0)
+    return gemm + attn
+
+
+def timed_prefill(eng, torch, req, prompt):
+    """ms of stairs_prefill (both models) with CUDA events on the engine's stream."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(eng.stream)
+    eng.prefill(req, prompt)
+    e1.record(eng.stream)
+    eng.sync()
+    return e0.elapsed_time(e1)
+
+
+def forced_acceptance_sweep(eng, torch, w, prompt, cont, kf, n_gen, seed):
+    """Tokens/s of the validate loop alone (no draft model) with drafts taken from the known greedy
+    continuation `cont`, each drafted token corrupted with probability 1 - alpha."""
+    out = {}
+    rng = np.random.default_rng(seed)
+    vocab = w.target.vocab
+    for alpha in (0.0, 0.5, 0.8, 1.0):
+        eng.prefill(0, prompt)
+        produced, calls = 0, 0
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        while produced < n_gen:
+            want = np.array(list(cont[produced:produced + kf]) + [0] * kf, dtype=np.int32)[:kf]
+            bad = rng.random(kf) >= alpha
+            want = np.where(bad, (want + 1) % vocab, want).astype(np.int32)
+            _, acc = eng.validate_host([0], [kf], want[None], commit=True)
+            produced += int(acc[0]) + 1
+            calls += 1
+        dt = time.perf_counter() - t0
+        out[f"alpha_{alpha}"] = {"tokens_per_s": produced / dt, "validate_calls": calls, "tokens_per_call": produced / calls}
+    return out
+
+
+def generation_point(eng, prompt, k, n_new):
+    out, st = eng.generate(0, prompt, k, n_new)
+    decode_ms = st["total_ms"] - st["prefill_ms"]
+    return out, {"tokens_per_s": n_new / (decode_ms * 1e-3), "acceptance": st["accepted"] / max(st["drafted"], 1),
+                 "iterations": st["iterations"], "draft_ms": st["draft_ms"], "validate_ms": st["validate_ms"],
+                 "prefill_ms": st["prefill_ms"]}
+
+
+def extra_workload(idx, torch, stairs, local_rank, peak, tflops_peak):
+    """Validate latency, prefill and generation of one of the larger configs, on a fresh context."""
+    w, prefix, k, n_req = pick_workload(f"cfg{idx}")
+    shape = w.target
+    tsrc, dsrc = wl.make_sources(w, backend="torch-cuda")
+    n_new = w.max_new
+    eng = stairs.Stairs(tsrc, dsrc, max_requests=n_req, max_seq_len=prefix + n_new + 16, k_max=8 if idx != 3 else 4,
+                        kv_page_tokens=64, device_index=local_rank)
+    res = {"workload": workload_label(w, prefix, k, n_req)}
+    try:
+        reqs = list(range(n_req))
+        prompts = [wl.prompt_tokens(w, request=r, n=prefix + 1) for r in reqs]
+        pre_ms = [timed_prefill(eng, torch, r, prompts[r]) for r in reqs]
+        fl = sum(prefill_flops(shape, prefix) + prefill_flops(w.draft, prefix) for _ in reqs)
+        res["prefill"] = {"ms_per_request": float(np.mean(pre_ms)), "tokens_per_s": prefix / (float(np.mean(pre_ms)) * 1e-3),
+                          "useful_tflops": fl / (sum(pre_ms) * 1e-3) / 1e12,
+                          "frac_of_bf16_sustained_peak": fl / (sum(pre_ms) * 1e-3) / 1e12 / tflops_peak if tflops_peak else None,
+                          "note": "target and assistant, 64 positions per pass of the persistent kernel (weights re-streamed every pass; "
+                                  "operands are bf16 hi+lo pairs, so the tensor pipe does twice the useful work)"}
+        # validate latency per k (uniform random drafts: the time does not depend on the accept length)
+        rng = np.random.default_rng(6)
+        per_k = {}
+        for kk in ((0, 1, 2, 4, 8) if idx == 4 else (k,)):
+            dd = torch.from_numpy(rng.integers(0, shape.vocab, size=(n_req, eng.k_max)).astype(np.int32)).to(eng.device)
+            tt = torch.zeros((n_req, eng.k_max + 1), dtype=torch.int32, device=eng.device)
+            al = torch.zeros((n_req,), dtype=torch.int32, device=eng.device)
+            n_it = 30 if idx != 5 else 15
+            for _ in range(3):
+                eng.validate(reqs, [kk] * n_req, dd, commit=False, out=(tt, al))
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(eng.stream)
+            for _ in range(n_it):
+                eng.validate(reqs, [kk] * n_req, dd, commit=False, out=(tt, al))
+            e1.record(eng.stream)
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / n_it
+            ab = algorithmic_bytes(shape, prefix, kk, n_req)
+            per_k[f"k{kk}"] = {"us_per_call": us, "hbm_gbs": ab / (us * 1e-6) / 1e9, "frac_of_measured_peak": ab / (us * 1e-6) / 1e9 / peak,
+                               "frac_of_nominal_8TBs": ab / (us * 1e-6) / 1e9 / NOMINAL_HBM_GBS}
+        res["validate"] = per_k
+        # every logit of one call finite (a guard against silently skipped work)
+        dd = torch.from_numpy(rng.integers(0, shape.vocab, size=(n_req, eng.k_max)).astype(np.int32)).to(eng.device)
+        _, _, lg = eng.validate(reqs, [k] * n_req, dd, want_logits=True)
+        eng.sync()
+        res["logits_finite"] = bool(torch.isfinite(lg).all())
+        del lg
+        if idx in (3, 4):
+            gen_prompt = prompts[0][:prefix]
+            out0, g0 = generation_point(eng, gen_prompt, 0, n_new)
+            res["prefill"]["generate_prefill_ms"] = g0["prefill_ms"]
+            gen = {"k0": g0}
+            for kk in ((1, 2, 3, 4, 5, 6, 7, 8) if idx == 4 else (k,)):
+                outk, gk = generation_point(eng, gen_prompt, kk, n_new)
+                gk["identical_to_k0"] = outk == out0
+                gk["speedup_vs_k0"] = gk["tokens_per_s"] / g0["tokens_per_s"]
+                gen[f"k{kk}"] = gk
+            res["generation"] = {"prompt": len(gen_prompt), "new_tokens": n_new, "per_k": gen}
+            res["forced_acceptance_k4"] = forced_acceptance_sweep(eng, torch, w, gen_prompt, out0, 4, min(n_new, 96), 7)
+    finally:
+        eng.close()
+        del eng
+        tsrc.drop_cache(); dsrc.drop_cache()
+        torch.cuda.empty_cache()
+    return res
+
+
 def run_reference(args, rank, world):
     """The oracle timed on the host cores.  Each step is one stair row (an independent no-cache
     fp32 forward) at a prefix shortened so that the whole run stays within a few minutes; the
@@ -205,7 +329,7 @@ def run_reference(args, rank, world):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(np.mean(times)) * 1e3,
             "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"{w.name}: prefix {prefix}, k {k}, {n_req * (k + 1)} stair rows, {n_req} request{'s' if n_req > 1 else ''}"},
+            "config": {"workload": workload_label(w, prefix, k, n_req)},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -334,7 +458,7 @@ def run_ours(args, rank, local_rank, world):
         "metric": METRIC, "value": us_per_call, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{w.name}: prefix {prefix}, k {k}, {n_req * (k + 1)} stair rows, {n_req} request{'s' if n_req > 1 else ''} per GPU, commit=0",
+        "config": {"workload": workload_label(w, prefix, k, n_req),
                    "l2": "inputs larger than L2 (weights %.2f GB per call)" % (wbytes / 1e9),
                    "replicas": world},
         "clocks": clocks,
@@ -386,63 +510,19 @@ def run_ours(args, rank, local_rank, world):
                 line["validate_grid"] = grid
         except Exception as ex:
             line["validate_grid"] = {"error": str(ex)}
-        try:
-            if args.workload == "cfg2" and args.layers == 0:
-                eng.close()
-                eng = None
-                del d_dev
-                tsrc.drop_cache()
-                torch.cuda.empty_cache()
-                w7, p7, k7, _ = pick_workload("cfg4")
-                t7, d7 = wl.make_sources(w7, backend="torch-cuda")
-                e7 = stairs.Stairs(t7, d7, max_requests=1, max_seq_len=p7 + 256, k_max=k7, kv_page_tokens=64,
-                                   device_index=local_rank)
-                e7.prefill(0, wl.prompt_tokens(w7, n=p7 + 1))
-                rng = np.random.default_rng(6)
-                per_k = {}
-                for kk in (0, 1, 2, 4, 8):
-                    dd = torch.from_numpy(rng.integers(0, w7.target.vocab, size=(16, k7)).astype(np.int32)).to(e7.device)
-                    us = time_validate(e7, torch, kk, dd, 30, 3)
-                    ab = algorithmic_bytes(w7.target, p7, kk)
-                    per_k[f"k{kk}"] = {"us_per_call": us, "hbm_gbs": ab / (us * 1e-6) / 1e9,
-                                       "frac_of_measured_peak": ab / (us * 1e-6) / 1e9 / peak,
-                                       "frac_of_nominal_8TBs": ab / (us * 1e-6) / 1e9 / NOMINAL_HBM_GBS}
-                g0, s0 = e7.generate(0, wl.prompt_tokens(w7, n=p7), 0, 96)
-                g4, s4 = e7.generate(0, wl.prompt_tokens(w7, n=p7), 4, 96)
-                # forced-acceptance sweep: drafts come from the known greedy continuation, each token
-                # corrupted with probability 1 - alpha; tokens/s of the validate loop alone (no draft
-                # model), against its own alpha = 0 and against k = 0 greedy
-                sweep = {}
-                kf, n_gen = 4, 64
-                base_prompt = wl.prompt_tokens(w7, n=p7)
-                rngf = np.random.default_rng(7)
-                for alpha in (0.0, 0.5, 0.8, 1.0):
-                    e7.prefill(0, base_prompt)
-                    produced, calls = 0, 0
-                    torch.cuda.synchronize()
-                    t0 = time.perf_counter()
-                    while produced < n_gen:
-                        want = np.array(g0[produced:produced + kf] + [0] * kf, dtype=np.int32)[:kf]
-                        bad = rngf.random(kf) >= alpha
-                        want = np.where(bad, (want + 1) % w7.target.vocab, want).astype(np.int32)
-                        _, acc = e7.validate_host([0], [kf], want[None], commit=True)
-                        produced += int(acc[0]) + 1
-                        calls += 1
-                    dt = time.perf_counter() - t0
-                    sweep[f"alpha_{alpha}"] = {"tokens_per_s": produced / dt, "validate_calls": calls,
-                                               "tokens_per_call": produced / calls}
-                line["target_7b"] = {"workload": f"{w7.name}: prefix {p7}", "validate": per_k,
-                                     "forced_acceptance_k4": sweep,
-                                     "greedy_tokens_per_s": 96 / ((s0["total_ms"] - s0["prefill_ms"]) * 1e-3),
-                                     "stairs_k4_tokens_per_s": 96 / ((s4["total_ms"] - s4["prefill_ms"]) * 1e-3),
-                                     "acceptance_k4": s4["accepted"] / max(s4["drafted"], 1),
-                                     "identical_output": g0 == g4}
-                e7.close()
-                e7 = None
-                t7.drop_cache(); d7.drop_cache()
-                torch.cuda.empty_cache()
-        except Exception as ex:
-            line["target_7b"] = {"error": str(ex)}
+        # the larger configs, each on a fresh context: validate latency, prefill, generation
+        if args.workload == "cfg2" and args.layers == 0:
+            eng.close()
+            eng = None
+            del d_dev
+            tsrc.drop_cache()
+            torch.cuda.empty_cache()
+            tfl = peaks.get("bf16_tflops_sustained")
+            for idx in (3, 4, 5):
+                try:
+                    line[f"cfg{idx}"] = extra_workload(idx, torch, stairs, local_rank, peak, float(tfl) if tfl else None)
+                except Exception as ex:  # reported, never hidden
+                    line[f"cfg{idx}"] = {"error": f"{type(ex).__name__}: {ex}"}
     # the oracle beside it, on this host's cores, on a bounded sample
     if world == 1 and not args.no_cpu_baseline and not args.timed_only:
         cb_prefix = min(prefix, args.cpu_prefix)

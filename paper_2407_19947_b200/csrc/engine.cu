@@ -526,14 +526,16 @@ MkPlan mk_plan(const stairs_ctx* ctx, const stairs_model& m, int t_box) {
   pl.att_dbl = (hd <= 64 || (long long)ctx->cfg.max_seq_len * m.n_kv_heads / mk::ATT_CHUNK > 2ll * ctx->sm_count) ? 1 : 0;
   pl.att_tma = (ctx->att_tma_off == 0 && (hd == 64 || hd == 128)) ? 1 : 0;
   if (pl.att_tma) {
-    // chunk buffers: as many as one SM's share of the K/V of a layer fills, at most four; the GEMM
-    // ring keeps at least three stages
+    // chunk buffers: as many whole chunks as one SM's share of a layer's K/V holds, at most four,
+    // and only while the GEMM ring keeps four single-k-block stages (measured: the ring matters more)
     const long long kv_per_cta = (long long)ctx->cfg.max_requests * ctx->cfg.max_seq_len * m.n_kv_heads * hd * 4 / std::max(ctx->sm_count, 1);
     const long long chunk = (long long)mk::AttnSmem::kv_buf_bytes(hd);
-    int want = (int)std::min<long long>(mk::MAX_KV_BUF, std::max<long long>(1, (kv_per_cta + chunk - 1) / chunk));
-    if (ctx->att_nbuf_force > 0) want = std::min(ctx->att_nbuf_force, (int)mk::MAX_KV_BUF);
-    pl.att_nbuf = want;
-    while (pl.att_nbuf > 1 && mk::pick_stages(t_box, hd, 0, 1, 1, pl.att_nbuf) < 3) --pl.att_nbuf;
+    pl.att_nbuf = (int)std::min<long long>(mk::MAX_KV_BUF, std::max<long long>(1, kv_per_cta / chunk));
+    while (pl.att_nbuf > 1 && mk::pick_stages(t_box, hd, 0, 1, 1, pl.att_nbuf) < 4) --pl.att_nbuf;
+    if (ctx->att_nbuf_force > 0) {
+      pl.att_nbuf = std::min(ctx->att_nbuf_force, (int)mk::MAX_KV_BUF);
+      while (pl.att_nbuf > 1 && mk::pick_stages(t_box, hd, 0, 1, 1, pl.att_nbuf) < 2) --pl.att_nbuf;
+    }
   }
   auto stages_for = [&](int kps) { return mk::pick_stages(t_box, hd, pl.att_dbl, kps, pl.att_tma, pl.att_nbuf); };
   pl.kps = 1;
