@@ -169,6 +169,17 @@ int stairs_generate(stairs_ctx *ctx, int req, const int32_t *prompt_host, int n_
                     int k, int max_new, int32_t eos, int32_t *out_host, int32_t *n_out,
                     stairs_stats *stats_or_null);
 
+/* The same generation with a draft length that follows the acceptance, the schedule of the
+ * sequential assisted generation the paper compares stairs with (Section 3.2; Section 4.1: that
+ * method sets the length dynamically): the first iteration drafts k_first (>= 1) tokens; after an
+ * iteration that kept every drafted token the next one drafts two more (at most k_max), after
+ * any other iteration one fewer (at least one).  Checking the drafts left to right in one causal
+ * pass is what the deduplicated stairs pass does anyway, so the two methods differ only in this
+ * schedule here; the output is still the main model's own greedy output.  Errors: as above. */
+int stairs_generate_adaptive(stairs_ctx *ctx, int req, const int32_t *prompt_host, int n_prompt,
+                             int k_first, int max_new, int32_t eos, int32_t *out_host,
+                             int32_t *n_out, stairs_stats *stats_or_null);
+
 /* Copies the request's committed sequence length (and, if seq_host != NULL, up to
  * capacity tokens of the sequence) to the host.  Waits. */
 int stairs_sequence(stairs_ctx *ctx, int req, int32_t *seq_host, int capacity, int32_t *n_seq);

@@ -23,6 +23,9 @@ What it follows (paper section / figure):
   ground truth; the walk ends at the first failure or the end of the batch and
   returns the ground truth (`stairs_validate_walk`).
 * Section 3.2 ("such a cycle repeats"): the outer loop (`stairs_generate`).
+* Section 3.2 and 4.1: the sequential assisted generation the paper compares with, one
+  causal pass over context + draft and a dynamically set draft length
+  (`assisted_generate`).
 
 Precision: fp32 throughout (weights of bf16 models are the bf16 bit patterns
 widened exactly to fp32).  Every stair row is an independent full causal
@@ -37,7 +40,10 @@ first-mismatch search on exhaustive small cases; stairs output == stand-alone
 greedy output for any draft and any k; k = 0 == greedy; family-A forward against
 torch.nn.TransformerEncoderLayer; family-B forward against the HuggingFace Llama
 implementation; closed-form special cases (uniform attention, position-shift
-invariance of RoPE, causality).  Acceptance-rate values are an empirical
+invariance of RoPE, causality); `assisted_generate` output == stand-alone greedy output
+for any draft, and its draft-length schedule against closed forms (a perfect assistant: +2
+per iteration up to the cap; an always-wrong one: down to 1, one token per iteration).
+Acceptance-rate values are an empirical
 property of random weights: parity unpinned, reported only.
 """
 from __future__ import annotations
@@ -300,4 +306,43 @@ def stairs_generate(target_model: OracleModel, draft_model, prompt, k: int, max_
         stats["iterations"] += 1
         stats["drafted"] += k_eff
         stats["accepted"] += res["accept_len"]
+    return out[:max_new], stats
+
+
+# ----------------------------------------------------------------------------
+# sequential assisted generation with a dynamic draft length (Section 3.2, Section 4.1)
+# ----------------------------------------------------------------------------
+def assisted_generate(target_model: OracleModel, draft_model, prompt, k_first: int, k_max: int,
+                      max_new: int, draft_fn=None):
+    """The comparison method of the paper (Section 3.2): the assistant drafts, the main model
+    processes the context plus the whole draft in ONE causal forward pass and its predictions
+    are compared with the drafted tokens from left to right; the first main-model token that
+    differs replaces the draft from there on.  The draft length is set dynamically
+    (Section 4.1); the schedule taken here is the one of the library the paper uses: two more
+    tokens after an iteration that kept every draft, one fewer (at least one) otherwise, never
+    more than k_max.  Returns (new_tokens, stats); stats["k_schedule"] lists the draft lengths."""
+    ctx = [int(t) for t in prompt]
+    out = []
+    stats = {"iterations": 0, "drafted": 0, "accepted": 0, "k_schedule": []}
+    k_cur = int(k_first)
+    while len(out) < max_new:
+        k_eff = min(k_cur, max_new - len(out) - 1)
+        if draft_fn is not None:
+            d = [int(t) for t in draft_fn(ctx, k_eff)]
+        else:
+            d = draft_tokens(draft_model, ctx, k_eff)
+        lg = forward_logits(target_model, ctx + d, all_positions=True)[len(ctx) - 1:]
+        pred = [argmax_lowest(row) for row in lg]           # main model's token after ctx + d[:r], r = 0..k
+        a = 0
+        while a < k_eff and d[a] == pred[a]:
+            a += 1
+        emitted = d[:a] + [pred[a]]
+        out.extend(emitted)
+        ctx.extend(emitted)
+        stats["iterations"] += 1
+        stats["drafted"] += k_eff
+        stats["accepted"] += a
+        stats["k_schedule"].append(k_eff)
+        if k_eff > 0:
+            k_cur = min(k_cur + 2, k_max) if a == k_eff else max(1, k_cur - 1)
     return out[:max_new], stats

@@ -102,6 +102,7 @@ struct stairs_ctx {
   size_t io_draft = 0, io_tt = 0, io_al = 0;   // offsets in ints
   unsigned long long wait_limit = 0;
   bool use_mk = false;
+  bool draft_shares_kv = false;      // early-exit assistant on the persistent kernel: it uses the main model's K/V pools
   unsigned long long bar_base = 0;   // grid-barrier arrivals consumed by earlier launches
   int kps_force = 0;                 // tuning: k-blocks per pipeline stage (0 = chosen per row box)
   int att_nbuf_force = 0;            // tuning: K/V chunk buffers of the attention phases (0 = chosen from the context length)
@@ -743,6 +744,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.norm_kind = m.norm; P.rope = m.pos; P.rope_theta = m.rope_theta; P.eps = m.norm_eps;
   P.tok_emb = (const bf16*)M.w.tok_emb; P.pos_emb = (const bf16*)M.w.pos_emb;
   P.mode = c.mode; P.n_req = c.n_req; P.slot = c.slot; P.draft_step = c.draft_step;
+  P.draft_first_rows = ctx->draft_shares_kv ? 1 : 2;
   if (c.mode == mk::CALL_VALIDATE)
     for (int i = 0; i < c.n_req; ++i) { P.val_req[i] = c.req_host[i]; P.val_k[i] = c.k_host[i]; P.val_off[i] = c.off_host[i]; }
   P.draft = c.draft; P.k_max = ctx->cfg.k_max;
@@ -1119,6 +1121,24 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
             stairs_destroy(ctx);
             return rc2;
           }
+          // Early-exit assistant (its layers are the main model's first layers, same tensors): the K/V
+          // it would compute for a position are bit for bit those the main model computes for the
+          // same token (results do not depend on a call's row count), so it works on the main
+          // model's pools: no second prefill, no second cache.  Every position it writes is one the
+          // next validation pass writes again before reading it.
+          if (has_draft && mk_eligible(ctx, ctx->draft, 1) && mk_eligible(ctx, ctx->target, 1) &&
+              cfg->draft.n_layers <= cfg->target.n_layers && cfg->draft.n_heads == cfg->target.n_heads &&
+              cfg->draft.n_kv_heads == cfg->target.n_kv_heads && cfg->draft.head_dim == cfg->target.head_dim &&
+              cfg->draft.d_ff == cfg->target.d_ff) {
+            bool same = true;
+            for (int l = 0; l < cfg->draft.n_layers && same; ++l)
+              same = memcmp(&ctx->draft.layers[l], &ctx->target.layers[l], sizeof(stairs_layer_w)) == 0;
+            if (same) {
+              ctx->draft_shares_kv = true;
+              ctx->draft.kpool = ctx->target.kpool; ctx->draft.vpool = ctx->target.vpool;
+              ctx->draft.kv_layer_bytes = ctx->target.kv_layer_bytes;
+            }
+          }
         }
       }
     }
@@ -1147,7 +1167,8 @@ int stairs_prefill(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_p
   ctx->n_seq_ub[req] = n_prompt;
   rc = prefill_model(ctx, ctx->target, req, n_prompt - 1);
   if (rc) return rc;
-  if (ctx->draft.present) rc = prefill_model(ctx, ctx->draft, req, n_prompt - 1);
+  // (an assistant that shares the main model's cache finds the prompt's K/V of its layers there already)
+  if (ctx->draft.present && !ctx->draft_shares_kv) rc = prefill_model(ctx, ctx->draft, req, n_prompt - 1);
   return rc;
 }
 
@@ -1166,7 +1187,7 @@ int stairs_draft(stairs_ctx* ctx, int req, int k, int32_t* draft_dev) {
     RowParams p = base_rows(ctx);
     p.slot = req; p.draft = draft_dev; p.first = j;
     p.mode = j == 0 ? ROWS_DRAFT_FIRST : ROWS_DRAFT_NEXT;
-    const int T = j == 0 ? 2 : 1;
+    const int T = (j == 0 && !ctx->draft_shares_kv) ? 2 : 1;
     if (mk_eligible(ctx, ctx->draft, T)) {
       MkCall c;
       c.mode = j == 0 ? mk::CALL_DRAFT_FIRST : mk::CALL_DRAFT_NEXT;
@@ -1276,8 +1297,15 @@ int stairs_validate_host(stairs_ctx* ctx, int n_req, const int32_t* req_ids_host
   return STAIRS_OK;
 }
 
-int stairs_generate(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_prompt, int k, int max_new,
-                    int32_t eos, int32_t* out_host, int32_t* n_out, stairs_stats* stats) {
+}  // extern "C"
+
+namespace {
+
+// The generation loop behind stairs_generate and stairs_generate_adaptive.  adaptive: the draft
+// length follows the acceptance (all drafts kept: two more next time, otherwise one fewer, never
+// below one), the schedule of the sequential assisted generation the paper compares with.
+int generate_loop(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_prompt, int k, int max_new,
+                  int32_t eos, int32_t* out_host, int32_t* n_out, stairs_stats* stats, bool adaptive) {
   int rc = check_slot(ctx, req, false);
   if (rc) return rc;
   if (!out_host || !n_out || max_new < 0) return fail(ctx, STAIRS_EINVAL, "bad generate arguments");
@@ -1311,8 +1339,9 @@ int stairs_generate(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_
   int produced = 0;
   bool stop = false;
   cudaError_t ce = cudaSuccess;
+  int k_cur = k;
   while (produced < max_new && !stop) {
-    const int k_eff = std::min(k, max_new - produced - 1);
+    const int k_eff = std::min(k_cur, max_new - produced - 1);
     if ((ce = cudaEventRecord(e1, ctx->stream)) != cudaSuccess) break;
     if (k_eff > 0 && (rc = stairs_draft(ctx, req, k_eff, d_dev))) break;
     if ((ce = cudaEventRecord(e2, ctx->stream)) != cudaSuccess) break;
@@ -1327,6 +1356,7 @@ int stairs_generate(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_
     if ((ce = cudaEventElapsedTime(&ms, e2, e3)) != cudaSuccess) break;
     s.validate_ms += ms;
     s.iterations++; s.drafted += k_eff; s.accepted += al;
+    if (adaptive && k_eff > 0) k_cur = al == k_eff ? std::min(k_cur + 2, ctx->cfg.k_max) : std::max(1, k_cur - 1);
     for (int r = 0; r <= al && !stop; ++r) {
       const int t = r < al ? draft_h[r] : tt[al];
       if (produced < max_new) out_host[produced] = t;
@@ -1346,6 +1376,21 @@ int stairs_generate(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_
   *n_out = std::min(produced, max_new);
   if (stats) *stats = s;
   return STAIRS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int stairs_generate(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_prompt, int k, int max_new,
+                    int32_t eos, int32_t* out_host, int32_t* n_out, stairs_stats* stats) {
+  return generate_loop(ctx, req, prompt_host, n_prompt, k, max_new, eos, out_host, n_out, stats, false);
+}
+
+int stairs_generate_adaptive(stairs_ctx* ctx, int req, const int32_t* prompt_host, int n_prompt, int k_first, int max_new,
+                             int32_t eos, int32_t* out_host, int32_t* n_out, stairs_stats* stats) {
+  if (ctx && k_first < 1) return fail(ctx, STAIRS_EINVAL, "k_first=%d: the adaptive schedule starts from at least one drafted token", k_first);
+  return generate_loop(ctx, req, prompt_host, n_prompt, k_first, max_new, eos, out_host, n_out, stats, true);
 }
 
 int stairs_sequence(stairs_ctx* ctx, int req, int32_t* seq_host, int capacity, int32_t* n_seq) {

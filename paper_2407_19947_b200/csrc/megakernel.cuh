@@ -87,6 +87,7 @@ struct Params {
   const bf16* tok_emb; const bf16* pos_emb;
   // call
   int mode; int n_req; int slot; int draft_step;
+  int draft_first_rows;      // rows of the assistant's first step: 2 (it re-reads the last two committed tokens), or 1 when it shares the main model's cache
   int val_req[64]; int val_k[64]; int val_off[64];   // validate: slot, draft length and first row of each request (a call has <= 64 rows)
   const int* draft; int k_max;
   int* seq; int* n_seq; int max_seq_len;
@@ -422,7 +423,7 @@ __device__ __forceinline__ RowInfo row_info(const Params& P, int t) {
   } else if (P.mode == CALL_DRAFT_FIRST) {
     r.slot = P.slot;
     const int n = P.n_seq[P.slot];
-    r.pos = n - 2 + t;
+    r.pos = n - P.draft_first_rows + t;
     r.tok = clampv(P.seq[(size_t)P.slot * P.max_seq_len + r.pos]);
   } else {
     r.slot = P.slot;
@@ -440,7 +441,7 @@ __device__ __forceinline__ int cache_row_of(const Params& P, int t) {
     while (i + 1 < P.n_req && P.val_off[i + 1] <= t) ++i;
     slot = P.val_req[i]; pos = P.n_seq[slot] - 1 + (t - P.val_off[i]);
   } else if (P.mode == CALL_PREFILL) { slot = P.slot; pos = P.draft_step + t; }
-  else if (P.mode == CALL_DRAFT_FIRST) { slot = P.slot; pos = P.n_seq[slot] - 2 + t; }
+  else if (P.mode == CALL_DRAFT_FIRST) { slot = P.slot; pos = P.n_seq[slot] - P.draft_first_rows + t; }
   else { slot = P.slot; pos = P.n_seq[slot] - 1 + P.draft_step; }
   return P.page_table[(size_t)slot * P.max_pages + pos / P.page_tokens] * P.page_tokens + pos % P.page_tokens;
 }
@@ -503,7 +504,7 @@ __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
   } else if (P.mode == CALL_PREFILL) {
     a.slot = P.slot; a.R = P.T; a.off = 0; a.base = P.draft_step;
   } else if (P.mode == CALL_DRAFT_FIRST) {
-    a.slot = P.slot; a.R = 2; a.off = 0; a.base = P.n_seq[P.slot] - 2;
+    a.slot = P.slot; a.R = P.draft_first_rows; a.off = 0; a.base = P.n_seq[P.slot] - P.draft_first_rows;
   } else {
     a.slot = P.slot; a.R = 1; a.off = 0; a.base = P.n_seq[P.slot] - 1 + P.draft_step;
   }

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libstairs_b200.so")
 STATUS = {0: "OK", 1: "EINVAL", 2: "ENOSPC", 3: "ESTATE", 4: "ECUDA", 5: "ETIMEOUT", 6: "EUNSUPPORTED"}
 
 EXPORTS = ["stairs_workspace_bytes", "stairs_init", "stairs_prefill", "stairs_draft", "stairs_validate",
-           "stairs_validate_host", "stairs_generate", "stairs_sequence", "stairs_truncate", "stairs_sync",
+           "stairs_validate_host", "stairs_generate", "stairs_generate_adaptive", "stairs_sequence", "stairs_truncate", "stairs_sync",
            "stairs_launch_count", "stairs_profile", "stairs_profile_read", "stairs_reset",
            "stairs_destroy", "stairs_last_error", "stairs_accept_static", "stairs_debug_buffer", "stairs_debug_tune"]
 
@@ -83,6 +83,7 @@ def load_library(path: Optional[str] = None):
     lib.stairs_validate_host.argtypes = [vp, C.c_int, i32p, i32p, i32p, i32p, i32p, C.c_int]
     lib.stairs_generate.argtypes = [vp, C.c_int, i32p, C.c_int, C.c_int, C.c_int, C.c_int32, i32p, i32p,
                                     C.POINTER(CStats)]
+    lib.stairs_generate_adaptive.argtypes = lib.stairs_generate.argtypes
     lib.stairs_sequence.argtypes = [vp, C.c_int, i32p, C.c_int, i32p]
     lib.stairs_truncate.argtypes = [vp, C.c_int, C.c_int]
     lib.stairs_sync.argtypes = [vp]
@@ -247,14 +248,14 @@ class Stairs:
                                                _ptr(tt), _ptr(al), int(commit)))
         return tt, al
 
-    def generate(self, req: int, prompt: Sequence[int], k: int, max_new: int, eos: int = -1):
-        """Returns (new_tokens list, stats dict)."""
+    def generate(self, req: int, prompt: Sequence[int], k: int, max_new: int, eos: int = -1, adaptive: bool = False):
+        """Returns (new_tokens list, stats dict).  adaptive: stairs_generate_adaptive, k is the first draft length."""
         p = _i32(prompt)
         out = np.zeros(max(max_new, 1), np.int32)
         n_out = C.c_int32(0)
         st = CStats()
-        self._ck(self.lib.stairs_generate(self.h, req, _ptr(p), len(p), k, max_new, eos, _ptr(out),
-                                          C.byref(n_out), C.byref(st)))
+        fn = self.lib.stairs_generate_adaptive if adaptive else self.lib.stairs_generate
+        self._ck(fn(self.h, req, _ptr(p), len(p), k, max_new, eos, _ptr(out), C.byref(n_out), C.byref(st)))
         stats = {n: getattr(st, n) for n, _ in CStats._fields_}
         return [int(x) for x in out[: n_out.value]], stats
 

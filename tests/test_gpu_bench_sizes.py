@@ -197,7 +197,10 @@ def test_drafted_tokens_match_the_oracle_assistant(early_exit):
     drf = so.OracleModel(dshape, dsrc)
     prompt = list(wl.zipf_tokens(45, shape.vocab, 12))
     eng = st.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=128, k_max=6, kv_page_tokens=16)
+    launches = eng.launch_count()
     eng.prefill(0, prompt)
+    # an early-exit assistant works on the main model's cache: the 44 prompt positions take one pass, not one per model
+    assert eng.launch_count() - launches == (1 if early_exit else 2)
     decisive = 0
     for k in (1, 3, 6):
         d_dev = eng.draft(0, k)

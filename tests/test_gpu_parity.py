@@ -323,3 +323,31 @@ def test_long_prefix_positions_split_over_several_units(shape):
     eng2.sync()
     assert float((logits2 - logits).abs().max()) < 0.03
     eng.close(); eng2.close()
+
+
+def test_adaptive_draft_length_generation_matches_the_oracle_schedule():
+    # sequential assisted generation with a dynamic draft length (Sections 3.2 and 4.1): on the tiny
+    # fp32 config the tokens are exact, so the library must walk the very schedule the oracle walks
+    st = _stairs()
+    w = wl.workload(1)
+    tsrc, dsrc = wl.make_sources(w)
+    prompt = wl.prompt_tokens(w)
+    tgt, drf = gu.oracle_pair(tsrc, dsrc)
+    eng = st.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=128, k_max=6, kv_page_tokens=16)
+    out, stats = eng.generate(0, prompt, 2, 24, adaptive=True)
+    ref, ref_stats = so.assisted_generate(tgt, drf, prompt, 2, 6, 24)
+    assert out == ref == so.greedy_generate(tgt, prompt, 24)
+    assert (stats["iterations"], stats["drafted"], stats["accepted"]) == (ref_stats["iterations"], ref_stats["drafted"], ref_stats["accepted"])
+    with pytest.raises(st.StairsError) as e:
+        eng.generate(0, prompt, 0, 8, adaptive=True)
+    assert e.value.code == 1
+    eng.close()
+    # and on a bf16 model through the persistent kernel: same output as plain greedy on the same kernels
+    shape = small_b(8, 2, 64, layers=4)
+    tsrc, dsrc = sources(shape, draft_layers=2)
+    eng = st.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=160, k_max=6, kv_page_tokens=16)
+    p2 = list(wl.zipf_tokens(50, shape.vocab, 8))
+    g0, _ = eng.generate(0, p2, 0, 48)
+    ga, sa = eng.generate(0, p2, 3, 48, adaptive=True)
+    assert ga == g0 and sa["emitted"] >= 48 and sa["accepted"] <= sa["drafted"]
+    eng.close()

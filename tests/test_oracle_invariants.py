@@ -99,3 +99,45 @@ def test_config1_matches_committed_golden_tokens():
     out, stats = so.stairs_generate(tgt, drf, prompt, w.k, w.max_new)
     assert out == golden
     assert so.greedy_generate(tgt, prompt, 8) == golden[:8]
+
+
+@pytest.mark.parametrize("family", ["a", "b"])
+def test_early_exit_assistant_hidden_states_are_the_main_models_first_layers(family):
+    # An assistant made of the main model's first n layers sees, at every position, exactly the main
+    # model's residual stream after n layers; by causality (pinned in test_oracle_forward) a
+    # position's stream does not depend on later tokens either.  This is what lets such an assistant
+    # work on the main model's K/V cache instead of keeping its own.
+    tgt, drf = small_pair(family)
+    seq = wl.uniform_tokens(13, tgt.shape.vocab, 5)
+    n = drf.shape.n_layers
+    np.testing.assert_array_equal(so.forward_hidden(drf, seq), so.forward_hidden(tgt, seq, n_layers=n))
+    # (a shorter sequence takes other BLAS blocking: equal up to fp32 rounding, not bit for bit)
+    np.testing.assert_allclose(so.forward_hidden(tgt, seq, n_layers=n)[:9], so.forward_hidden(tgt, seq[:9], n_layers=n),
+                               rtol=1e-4, atol=1e-5)
+
+
+@pytest.mark.parametrize("family", ["a", "b"])
+def test_assisted_generation_equals_greedy_and_follows_its_schedule(family):
+    # Section 3.2 / 4.1: one causal pass over context + draft, draft length set dynamically
+    tgt, drf = small_pair(family)
+    prompt = wl.uniform_tokens(8, tgt.shape.vocab, 2)
+    ref = so.greedy_generate(tgt, prompt, 20)
+    out, stats = so.assisted_generate(tgt, drf, prompt, 2, 6, 20)
+    assert out == ref
+    assert stats["drafted"] == sum(stats["k_schedule"]) and stats["accepted"] <= stats["drafted"]
+    # a perfect assistant (the main model itself): every draft kept, so 2, 4, 6, ... tokens drafted
+    # and k + 1 tokens emitted per iteration
+    out_p, st_p = so.assisted_generate(tgt, tgt, prompt, 2, 6, 20)
+    assert out_p == ref and st_p["accepted"] == st_p["drafted"]
+    assert st_p["k_schedule"][:3] == [2, 4, 6] and st_p["iterations"] == 4     # 3 + 5 + 7 + the last 5 of 20
+    # an assistant that is always wrong: the length decays to 1 and every iteration emits one token
+    wrong = lambda ctx, k: [(ref[len(ctx) - len(prompt) + i] + 1) % tgt.shape.vocab for i in range(k)]
+    out_w, st_w = so.assisted_generate(tgt, None, prompt, 3, 6, 20, draft_fn=wrong)
+    assert out_w == ref and st_w["accepted"] == 0 and st_w["iterations"] == 20
+    assert st_w["k_schedule"][:4] == [3, 2, 1, 1]
+    # the causal pass gives the same predictions as the stairs rows computed one by one
+    d = so.draft_tokens(drf, list(prompt), 4)
+    rows = so.stairs_rows(prompt, d)
+    one_by_one = so.stairs_target_tokens(tgt, rows)
+    lg = so.forward_logits(tgt, list(prompt) + d, all_positions=True)[len(prompt) - 1:]
+    assert [so.argmax_lowest(r) for r in lg] == one_by_one
