@@ -29,7 +29,9 @@ int stairs_debug_buffer(stairs_ctx *ctx, int which, void **ptr_dev, size_t *byte
 /* Tuning knobs of the persistent kernel, for sweeps.  what 0: 64-element k-blocks per pipeline
  * stage (0 = chosen per row box, 1 or 2); what 1: K/V chunk buffers of the attention phases
  * (0 = chosen from the context length, 1..4); what 2: non-zero stages K/V with 16-byte copies
- * from the compute warps even where tiled bulk copies apply.  Takes effect with the next call. */
+ * from the compute warps even where tiled bulk copies apply; what 3: 1 keeps the attention
+ * contractions on mma.sync even where the tcgen05 path applies, 2 uses the tcgen05 path for every
+ * call it can serve (0: chosen per call).  Takes effect with the next call. */
 int stairs_debug_tune(stairs_ctx *ctx, int what, long long value);
 
 #ifdef __cplusplus

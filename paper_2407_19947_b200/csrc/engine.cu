@@ -37,6 +37,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 constexpr int MK_MAX_ROWS = 64;          // rows per call the persistent kernel handles
 constexpr int MK_TBOX_SLOTS = MK_MAX_ROWS / 16;
+constexpr int MK_PROG_SLOTS = MK_TBOX_SLOTS * 2;   // one program per (row box, k-blocks per stage)
 
 struct DevModel {
   float* rope_inv = nullptr;     // device: theta^(-2i/hd), i < hd/2
@@ -44,7 +45,7 @@ struct DevModel {
   bf16* w13 = nullptr;           // device: SwiGLU models, per layer [tiles][64 gate rows | 64 up rows][d] (see k_pack_gate_up)
   size_t w13_layer = 0;          // elements per layer
   std::vector<const bf16*> w13_ptr;   // per layer: its packed matrix (possibly another model's, for shared layers)
-  bool prog_built[MK_TBOX_SLOTS] = {false, false, false, false};
+  bool prog_built[MK_PROG_SLOTS] = {};
   char* prog_base = nullptr;     // device: per t_box slot, phases followed by tensor maps
   size_t prog_slot_bytes = 0, prog_maps_off = 0;
   int n_phases = 0;
@@ -65,6 +66,7 @@ struct Layout {
   int max_rows, logit_rows, max_pages, n_pages, t_box_max, attn_units, stat_tiles, attn_cnt_n;
   size_t prog_slot_t, prog_slot_d, prog_maps_off_t, prog_maps_off_d;
   size_t kv_t_layer, kv_d_layer;
+  size_t attn_part_bytes;
 };
 
 }  // namespace
@@ -106,6 +108,8 @@ struct stairs_ctx {
   unsigned long long bar_base = 0;   // grid-barrier arrivals consumed by earlier launches
   int kps_force = 0;                 // tuning: k-blocks per pipeline stage (0 = chosen per row box)
   int att_nbuf_force = 0;            // tuning: K/V chunk buffers of the attention phases (0 = chosen from the context length)
+  int att_tc_force = 0;              // tuning: 1 = tcgen05 attention for every call it can serve
+  int att_tc_off = 0;                // tuning: 1 = attention contractions on mma.sync even where the tcgen05 path applies
   int att_tma_off = 0;               // tuning: 1 = stage K/V with 16-byte copies from the compute warps even where bulk copies apply
 };
 
@@ -149,8 +153,8 @@ const char* check_model(const stairs_model& m) {
 // kernel picks chunks per unit so that kv heads x position ranges fit the grid (or, for contexts
 // too long for that, at most twice the grid: stairs_init checks this); the rows of the call can
 // add one more range per kv head.
-int attn_unit_bound(int hkv, int gq, int rows) {
-  const int n_qblk = (rows * gq + mk::ATT_QBLK - 1) / mk::ATT_QBLK;
+int attn_unit_bound(int hkv, int gq, int rows, int qblk = mk::ATT_QBLK) {
+  const int n_qblk = (rows * gq + qblk - 1) / qblk;
   return (2 * TC_GRID_MAX + 2 * hkv) * std::max(n_qblk, 1);
 }
 
@@ -227,7 +231,10 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     const int rows_req = std::min(c.k_max + 1, MK_MAX_ROWS);
     const int n_qblk = (rows_req * gq + mk::ATT_QBLK - 1) / mk::ATT_QBLK;
     L->attn_units = std::max(c.max_requests * attn_unit_bound(hkv, gq, rows_req), attn_unit_bound(hkv, gq, MK_MAX_ROWS));
-    L->attn_part = take(t.wdtype == 1 ? (size_t)L->attn_units * mk::ATT_QBLK * (hdm + 4) * 4 : 0);
+    // (the tcgen05 attention path has fewer units of 128 query rows each: sized for whichever is larger)
+    const int units_tc = std::max(c.max_requests * attn_unit_bound(hkv, gq, rows_req, mk::ATT_QBLK_TC), attn_unit_bound(hkv, gq, MK_MAX_ROWS, mk::ATT_QBLK_TC));
+    L->attn_part_bytes = std::max((size_t)L->attn_units * mk::ATT_QBLK, (size_t)units_tc * mk::ATT_QBLK_TC) * (hdm + 4) * 4;
+    L->attn_part = take(t.wdtype == 1 ? L->attn_part_bytes : 0);
     auto prog = [&](const stairs_model& m, size_t* maps_off) {
       const size_t ph = align_up((size_t)(8 * std::max(m.n_layers, 1) + 4) * sizeof(mk::Phase), 128);
       *maps_off = ph;
@@ -235,8 +242,8 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     };
     L->prog_slot_t = t.wdtype == 1 ? prog(t, &L->prog_maps_off_t) : 0;
     L->prog_slot_d = (t.wdtype == 1 && has_draft) ? prog(d, &L->prog_maps_off_d) : 0;
-    L->prog_t = take(L->prog_slot_t * MK_TBOX_SLOTS);
-    L->prog_d = take(L->prog_slot_d * MK_TBOX_SLOTS);
+    L->prog_t = take(L->prog_slot_t * MK_PROG_SLOTS);
+    L->prog_d = take(L->prog_slot_d * MK_PROG_SLOTS);
     L->mk_trace = take(t.wdtype == 1 ? (size_t)(2 * 8 + 8 * TC_GRID_MAX) * (8 * std::max(t.n_layers, 1) + 4) * 8 : 0);
     L->stat_tiles = (t.d_model + tc::BM - 1) / tc::BM;
     L->mk_stats = take(t.wdtype == 1 ? (size_t)MK_MAX_ROWS * L->stat_tiles * 16 : 0);
@@ -517,42 +524,55 @@ int setup_mk_model(stairs_ctx* ctx, DevModel& M, size_t rope_off, size_t aux_off
 
 // Shared-memory plan of the persistent kernel for one (model, row box): pipeline depth of the GEMM
 // ring against the K/V chunk buffers of the attention phases.
-struct MkPlan { int kps, stages, att_dbl, att_tma, att_nbuf; };
+struct MkPlan { int kps, stages, att_dbl, att_tma, att_nbuf, att_tc, att_qblk, att_q_rows; };
 
-MkPlan mk_plan(const stairs_ctx* ctx, const stairs_model& m, int t_box) {
+// q_rows_call: query rows (rows x grouped heads of the largest request, at most 128) of this call; 0 = the
+// largest a call of this row box can have (the stage depth kps, which the programs' tensor maps carry,
+// is decided for that case, so that it is the same for every call of the row box)
+MkPlan mk_plan(const stairs_ctx* ctx, const stairs_model& m, int t_box, int q_rows_call = 0, int tc_call = -1) {
   MkPlan pl{};
   const int hd = m.head_dim;
+  const int gq = m.n_heads / m.n_kv_heads;
+  auto round8 = [](int v) { return (v + 7) / 8 * 8; };
+  const int q_rows_max = std::min(mk::ATT_QBLK_TC, round8(t_box * gq));
   // copy path: two K/V chunk buffers where they are cheap (small heads) or needed (contexts so long
   // that a unit walks several chunks)
   pl.att_dbl = (hd <= 64 || (long long)ctx->cfg.max_seq_len * m.n_kv_heads / mk::ATT_CHUNK > 2ll * ctx->sm_count) ? 1 : 0;
   pl.att_tma = (ctx->att_tma_off == 0 && (hd == 64 || hd == 128)) ? 1 : 0;
+  // tcgen05 attention: possible where the bulk-copy path is; used by the calls it pays for (tc_call, see
+  // launch_forward_mk); tc_call < 0 plans for the mode that needs more shared memory
+  const bool tc_possible = pl.att_tma && ctx->att_tc_off == 0;
+  pl.att_tc = (tc_possible && tc_call != 0) ? 1 : 0;
+  pl.att_qblk = pl.att_tc ? mk::ATT_QBLK_TC : mk::ATT_QBLK;
+  pl.att_q_rows = pl.att_tc ? (q_rows_call > 0 ? std::min(q_rows_max, round8(q_rows_call)) : q_rows_max) : 0;
+  // K/V chunk buffers wanted (bulk-copy paths): as many whole chunks as one SM's share of a layer's K/V
+  // holds, at most four; the tcgen05 path wants two at least, so that a chunk loads while the previous
+  // one is multiplied.  Measured: the GEMM ring matters more than chunk buffers, so a buffer beyond
+  // the minimum is only added while the ring keeps three two-k-block stages (or four single ones).
+  int want = 0, least = 0;
   if (pl.att_tma) {
-    // chunk buffers: as many whole chunks as one SM's share of a layer's K/V holds, at most four,
-    // and only while the GEMM ring keeps four single-k-block stages (measured: the ring matters more)
     const long long kv_per_cta = (long long)ctx->cfg.max_requests * ctx->cfg.max_seq_len * m.n_kv_heads * hd * 4 / std::max(ctx->sm_count, 1);
     const long long chunk = (long long)mk::AttnSmem::kv_buf_bytes(hd);
-    pl.att_nbuf = (int)std::min<long long>(mk::MAX_KV_BUF, std::max<long long>(1, kv_per_cta / chunk));
-    while (pl.att_nbuf > 1 && mk::pick_stages(t_box, hd, 0, 1, 1, pl.att_nbuf) < 4) --pl.att_nbuf;
-    if (ctx->att_nbuf_force > 0) {
-      pl.att_nbuf = std::min(ctx->att_nbuf_force, (int)mk::MAX_KV_BUF);
-      while (pl.att_nbuf > 1 && mk::pick_stages(t_box, hd, 0, 1, 1, pl.att_nbuf) < 2) --pl.att_nbuf;
-    }
+    least = pl.att_tc ? 2 : 1;
+    want = (int)std::min<long long>(mk::MAX_KV_BUF, std::max<long long>(least, kv_per_cta / chunk));
+    if (ctx->att_nbuf_force > 0) want = least = std::min(ctx->att_nbuf_force, (int)mk::MAX_KV_BUF);
   }
-  auto stages_for = [&](int kps) { return mk::pick_stages(t_box, hd, pl.att_dbl, kps, pl.att_tma, pl.att_nbuf); };
-  pl.kps = 1;
-  if (ctx->kps_force > 0) { if (stages_for(ctx->kps_force) >= 2) pl.kps = ctx->kps_force; }
-  else if (stages_for(2) >= 3) pl.kps = 2;
-  pl.stages = stages_for(pl.kps);
+  auto stages_for = [&](int kps, int nbuf) { return mk::pick_stages(t_box, hd, pl.att_dbl, kps, pl.att_tma, nbuf, pl.att_q_rows); };
+  pl.kps = (ctx->kps_force > 0) ? ctx->kps_force : (stages_for(2, least) >= 3 ? 2 : 1);
+  if (stages_for(pl.kps, least) < 2) pl.kps = 1;
+  pl.att_nbuf = least;
+  while (pl.att_nbuf < want && stages_for(pl.kps, pl.att_nbuf + 1) >= (pl.kps == 2 ? 3 : 4)) ++pl.att_nbuf;
+  pl.stages = stages_for(pl.kps, pl.att_nbuf);
   return pl;
 }
 
-int build_program(stairs_ctx* ctx, DevModel& M, int t_box) {
+
+int build_program(stairs_ctx* ctx, DevModel& M, int t_box, int kps) {
   const stairs_model& m = M.m;
   const Layout& L = ctx->lay;
-  const int slot = t_box / 16 - 1;
+  const int slot = (t_box / 16 - 1) * 2 + (kps - 1);
   const int d = m.d_model, nq = m.n_heads * m.head_dim, nkv = m.n_kv_heads * m.head_dim, nqkv = nq + 2 * nkv, F = m.d_ff;
   char* ws = ctx->ws;
-  const int kps = mk_plan(ctx, m, t_box).kps;
   std::vector<CUtensorMap> maps((size_t)9 * m.n_layers + 4);
   bool ok = true;
   for (int l = 0; l < m.n_layers && ok; ++l) {
@@ -713,19 +733,34 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   const Layout& L = ctx->lay;
   char* ws = ctx->ws;
   const int t_box = (T + 15) / 16 * 16;
-  const int slot = t_box / 16 - 1;
-  if (!M.prog_built[slot]) {
-    int rc = build_program(ctx, M, t_box);
-    if (rc) return rc;
-  }
+  int q_rows_call = 0, tc_call = 0;
+  long long units_avail = 0;
   {
     // attention scratch: refuse a call whose units might not fit rather than compute part of it
     const int hkv = m.n_kv_heads, gq = m.n_heads / m.n_kv_heads;
     long long need = 0;
-    if (c.mode == mk::CALL_VALIDATE) for (int i = 0; i < c.n_req; ++i) need += attn_unit_bound(hkv, gq, c.k_host[i] + 1);
-    else need = attn_unit_bound(hkv, gq, T);
-    if (need > L.attn_units)
-      return fail(ctx, STAIRS_ENOSPC, "attention scratch holds %d units, this call may need %lld", L.attn_units, need);
+    // The tcgen05 attention path pays where a unit walks many chunks (long contexts) or a request has
+    // many query rows (prefill passes: 128 queries share a chunk instead of 48); short units are
+    // quicker on the register path, whose per-unit set-up is smaller.
+    int r_max0 = 0; long long len_max = 0;
+    if (c.mode == mk::CALL_VALIDATE) for (int i = 0; i < c.n_req; ++i) { r_max0 = std::max(r_max0, c.k_host[i] + 1); len_max = std::max<long long>(len_max, ctx->n_seq_ub[c.req_host[i]]); }
+    else { r_max0 = T; len_max = ctx->n_seq_ub[c.slot]; }
+    const long long chunks_per_unit = (len_max / mk::ATT_CHUNK + 1) * hkv / std::max(ctx->sm_count, 1);
+    tc_call = (ctx->att_tc_force > 0 || chunks_per_unit >= 6 || r_max0 * gq >= 96) ? 1 : 0;
+    const MkPlan pl0 = mk_plan(ctx, m, t_box, 0, tc_call);
+    int r_max = 0;
+    if (c.mode == mk::CALL_VALIDATE) for (int i = 0; i < c.n_req; ++i) { need += attn_unit_bound(hkv, gq, c.k_host[i] + 1, pl0.att_qblk); r_max = std::max(r_max, c.k_host[i] + 1); }
+    else { need = attn_unit_bound(hkv, gq, T, pl0.att_qblk); r_max = T; }
+    q_rows_call = std::min(r_max * gq, (int)mk::ATT_QBLK_TC);
+    units_avail = (long long)(L.attn_part_bytes / ((size_t)pl0.att_qblk * (m.head_dim + 4) * 4));
+    if (need > units_avail)
+      return fail(ctx, STAIRS_ENOSPC, "attention scratch holds %lld units, this call may need %lld", units_avail, need);
+  }
+  const MkPlan pl = mk_plan(ctx, m, t_box, q_rows_call, tc_call);
+  const int slot = (t_box / 16 - 1) * 2 + (pl.kps - 1);
+  if (!M.prog_built[slot]) {
+    int rc = build_program(ctx, M, t_box, pl.kps);
+    if (rc) return rc;
   }
   mk::Params P;
   memset(&P, 0, sizeof P);
@@ -734,8 +769,8 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.phases = reinterpret_cast<const mk::Phase*>(base); P.n_phases = n_run;
   P.maps = reinterpret_cast<const CUtensorMap*>(base + M.prog_maps_off);
   P.T = T; P.t_box = t_box;
-  const MkPlan pl = mk_plan(ctx, m, t_box);
   P.att_dbl = pl.att_dbl; P.att_tma = pl.att_tma; P.att_nbuf = pl.att_nbuf;
+  P.att_tc = pl.att_tc; P.att_qblk = pl.att_qblk; P.att_q_rows = pl.att_q_rows;
   P.kv_box_rows = std::min(ctx->cfg.kv_page_tokens, mk::ATT_CHUNK);
   P.kps = pl.kps;
   P.stages = pl.stages;
@@ -760,7 +795,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.target_tokens = c.target_tokens; P.accept_len = c.accept_len; P.commit = c.commit; P.draft_out = c.draft_out;
   P.partial = reinterpret_cast<float*>(ws + L.gemm_partial); P.counters = reinterpret_cast<int*>(ws + L.gemm_counters);
   P.seg_flags = reinterpret_cast<unsigned long long*>(ws + L.mk_flags);
-  P.attn_part = reinterpret_cast<float*>(ws + L.attn_part); P.attn_part_units = L.attn_units;
+  P.attn_part = reinterpret_cast<float*>(ws + L.attn_part); P.attn_part_units = (int)units_avail;
   P.stats = reinterpret_cast<float4*>(ws + L.mk_stats); P.stat_tiles = L.stat_tiles;
   P.rope_inv = M.rope_inv; P.rope_cs = M.rope_inv + m.head_dim / 2; P.rope_sn = P.rope_cs + 64 * (m.head_dim / 2); P.attn_cnt = reinterpret_cast<int*>(ws + L.attn_cnt);
   P.bar = reinterpret_cast<unsigned long long*>(ws + L.mk_bar); P.bar_base = ctx->bar_base;
@@ -769,7 +804,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   const int grid = std::min(ctx->sm_count, TC_GRID_MAX);
   void* args[] = {&P};
   CK(cudaLaunchCooperativeKernel((const void*)mk::k_forward, dim3(grid), dim3(mk::MK_THREADS), args,
-                                 mk::smem_bytes(t_box, P.stages, m.head_dim, P.att_dbl, P.kps, P.att_tma, P.att_nbuf), ctx->stream));
+                                 mk::smem_bytes(t_box, P.stages, m.head_dim, P.att_dbl, P.kps, P.att_tma, P.att_nbuf, P.att_q_rows), ctx->stream));
   ctx->bar_base += (unsigned long long)n_run * grid;
   ctx->launches++;
   return STAIRS_OK;
@@ -1504,6 +1539,7 @@ int stairs_debug_tune(stairs_ctx* ctx, int what, long long value) {
       ctx->att_nbuf_force = (int)value;
       break;
     case 2: ctx->att_tma_off = value ? 1 : 0; break;
+    case 3: ctx->att_tc_off = value == 1 ? 1 : 0; ctx->att_tc_force = value == 2 ? 1 : 0; break;
     default: return fail(ctx, STAIRS_EINVAL, "unknown tuning knob %d", what);
   }
   // programs carry the tensor maps' box depth, which follows from the shared-memory plan

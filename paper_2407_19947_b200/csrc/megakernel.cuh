@@ -103,6 +103,9 @@ struct Params {
   int att_tma;               // attention, TMA path (head sizes 64 and 128): a loader warp streams K/V chunks through att_nbuf buffers
   int att_nbuf;
   int kv_box_rows;           // rows of one K/V box: min(page_tokens, chunk)
+  int att_tc;                // attention on tcgen05 (with att_tma): S = Q.K^T and O += P.V as M = 128 MMAs, accumulators in TMEM
+  int att_qblk;              // queries per attention unit: 48 (mma.sync path), 128 (tcgen05 path)
+  int att_q_rows;            // tcgen05 path: rows of the Q and P tiles kept in shared memory (queries of a unit, rounded up to 8)
   __half* q16;               // [row][Hq*hd] queries, rotated and scaled by 1/sqrt(hd), written by the QKV epilogue
   float* rope_cs; float* rope_sn;   // [row][hd/2] cos and sin of the call's row positions, written by the embedding phase
      // [hd/2] theta^(-2i/hd)
@@ -123,7 +126,8 @@ struct Params {
 constexpr int MK_THREADS = THREADS + 32;   // the GEMM kernel's six warps plus the K/V loader of the attention phases
 constexpr int MAX_KV_BUF = 4;
 constexpr int ATT_CHUNK = 64;
-constexpr int ATT_QBLK = 48;
+constexpr int ATT_QBLK = 48;                    // queries per unit on the mma.sync path
+constexpr int ATT_QBLK_TC = 128;                // ... on the tcgen05 path (the MMA's M)
 constexpr int VT_LD = 132;                      // row pitch (floats) of the epilogue's 16 x 128 exchange tile
 constexpr int MK_XCH_BYTES = 16 * VT_LD * 4;     // the tile itself
 
@@ -135,7 +139,12 @@ struct AttnSmem {   // carved after the GEMM ring: Q block (bf16), K and V chunk
   // TMA path: a chunk buffer holds K then V, each as hd / 64 column halves of [CHUNK rows][128 bytes] with the 128-byte swizzle
   static __host__ __device__ size_t kv_buf_bytes(int hd) { return (size_t)2 * ATT_CHUNK * hd * 2; }
   // copy path: Q block, then one or two padded K/V buffers; TMA path: nbuf chunk buffers (1024-byte aligned), then the Q block
-  static __host__ __device__ size_t bytes(int hd, int dbl, int tma, int nbuf) {
+  // tcgen05 path (tc_q_rows > 0): Q tile (hd / 64 halves of [q_rows][128 bytes]) and P tile ([q_rows][128 bytes]),
+  // both swizzled, then the chunk buffers; an M = 128 MMA reads 128 rows from a tile's start, so at
+  // least 16 KB of this region must follow the P tile: the first chunk buffer does
+  static __host__ __device__ size_t tc_head_bytes(int hd, int q_rows) { return (size_t)(hd / 64 + 2) * q_rows * 128; }   // Q halves, two P tiles
+  static __host__ __device__ size_t bytes(int hd, int dbl, int tma, int nbuf, int tc_q_rows = 0) {
+    if (tc_q_rows > 0) return 1024 + tc_head_bytes(hd, tc_q_rows) + (size_t)nbuf * kv_buf_bytes(hd) + 64;
     return tma ? 1024 + (size_t)nbuf * kv_buf_bytes(hd) + q_bytes(hd) + 64 : q_bytes(hd) + (dbl ? 4 : 2) * kv_bytes(hd) + 64;
   }
 };
@@ -197,6 +206,8 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
   return t;
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// the same for this CTA's shared memory only (tiles written with plain stores, read by the tensor core)
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -273,6 +284,9 @@ struct AttnReq { int slot, base, R, off, n_chunks, cpu, n_ranges, n_qblk, units;
 struct Ctl {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
   uint64_t kv_full[MAX_KV_BUF], kv_empty[MAX_KV_BUF];   // attention K/V chunk buffers (TMA path)
+  // tcgen05 attention: S of a chunk is in TMEM (two S buffers) / the chunk's P tile is written and O rescaled
+  // (two P tiles; one arrival per compute warp) / the unit's Q tile is staged / a P.V has completed
+  uint64_t s_full[2], p_full[2], q_full, o_done;
   volatile int areq_ready;                              // the requests' attention geometry below is filled in
   uint32_t tmem_slot;
   volatile int abort_flag;
@@ -515,14 +529,21 @@ __device__ __forceinline__ AttnReq attn_req(const Params& P, int i, int G) {
   while (cpu < 64 && P.Hkv * ((c0 + cpu - 1) / cpu) > G) cpu <<= 1;   // one unit per CTA where possible: a unit's fixed cost exceeds a chunk's
   a.cpu = cpu;
   a.n_ranges = (a.n_chunks + cpu - 1) / cpu;
-  a.n_qblk = (a.R * (P.Hq / P.Hkv) + ATT_QBLK - 1) / ATT_QBLK;
+  a.n_qblk = (a.R * (P.Hq / P.Hkv) + P.att_qblk - 1) / P.att_qblk;
   a.units = P.Hkv * a.n_ranges * a.n_qblk;
   return a;
 }
 
 
-// Consumer side of the K/V chunk ring of the TMA path: buffer and parity of the next chunk.
-struct KvCons { int buf; uint32_t par; };
+// Consumer side of the K/V chunk ring of the TMA path: buffer and parity of the next chunk; parity of
+// the tcgen05 path's MMA-completion barrier.
+struct KvCons { int buf; uint32_t par; uint32_t sc; uint32_t o_par; };   // sc: chunks of the tcgen05 path so far (S / P buffer = sc & 1)
+
+// First chunk buffer of the TMA paths (1024-byte aligned; the tcgen05 path keeps its Q and P tiles in front of it).
+__device__ __forceinline__ uint8_t* att_ring_base(const Params& P, uint8_t* att_smem) {
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem) + 1023) & ~(uintptr_t)1023);
+  return P.att_tc ? base + AttnSmem::tc_head_bytes(P.hd, P.att_q_rows) : base;
+}
 
 // One attention unit, executed by the 128 compute threads (4 warps), on the legacy tensor path
 // (mma.sync m16n8k16).  The unit's queries are cut into blocks of 16 (one MMA M tile), one warp
@@ -550,7 +571,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   const size_t kvb = AttnSmem::kv_bytes(hd);
   const size_t kvbuf = AttnSmem::kv_buf_bytes(hd);
   // TMA path: ring of chunk buffers (1024-byte aligned) then the Q block; copy path: Q block then padded buffers
-  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem) + 1023) & ~(uintptr_t)1023);
+  uint8_t* ring = att_ring_base(P, att_smem);
   uint8_t* qs = TMA ? ring + (size_t)P.att_nbuf * kvbuf : att_smem;   // [QBLK][pitch] fp16, rotated and pre-scaled
   uint8_t* kv0 = qs + AttnSmem::q_bytes(hd);                // copy path, buffer b: K [CHUNK][pitch] then V, at kv0 + b * 2 * kvb
   uint8_t* ks = kv0;                                        // the buffer being computed on
@@ -841,7 +862,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     for (int half_row = 0; half_row < 2; ++half_row) {
       const int ql = half_row ? ql_b : ql_a;
       if (ql < nQ) {
-        float* dst = P.attn_part + ((size_t)part_slot * ATT_QBLK + ql) * (hd + 4);
+        float* dst = P.attn_part + ((size_t)part_slot * P.att_qblk + ql) * (hd + 4);
 #pragma unroll
         for (int nd = 0; nd < 16; ++nd)
           if (nd < ntiles)
@@ -850,6 +871,281 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
       }
     }
   }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Attention unit on the 5th-generation tensor cores
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t smem_desc_sw128_ex(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3ffff) >> 4);
+  d |= (uint64_t)(lbo >> 4) << 16;               // MN-major operands: distance between 64-element column blocks
+  d |= (uint64_t)(sbo >> 4) << 32;               // distance between 8-row groups
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;                        // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: fp32 accumulator, fp16 A and B, A K-major, B K-major or MN-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc_f16(int n, int b_mn_major) {
+  return (1u << 4) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane, written.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+        "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+        "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15]))
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
+// One attention unit with both contractions on tcgen05 (head sizes 64 and 128, K/V chunks from the
+// loader warp's ring).  The unit's up to 128 queries are the M rows: thread (TMEM lane) q owns query q.
+// Per 64-position chunk:
+//   S[q, j] = sum_d Q[q, d] K[j, d]   A = Q tile (K-major, swizzled, staged once per unit), B = the K chunk
+//                                     as the bulk copies left it (K-major), accumulator S in TMEM;
+//   every thread reads its row of S, applies the staircase mask, updates its running maximum and sum
+//   (base 2) and writes its row of P = 2^(S - max) as fp16 into a swizzled P tile;
+//   O[q, :] += sum_j P[q, j] V[j, :]  A = P tile, B = the V chunk as copied ([position][head dim]: MN-major
+//                                     for the MMA, column blocks 8 KB apart, 8-row groups 1 KB apart),
+//                                     accumulator O in TMEM across the unit's chunks.
+// The MMAs are issued by the MMA warp's thread (attn_issue_tc below), which runs one chunk ahead: S of
+// chunk c + 1 is computed while these threads work on chunk c (two S buffers in TMEM, two P tiles).
+// When a running maximum moves, the warp rescales its rows of O in TMEM (load, multiply, store) after
+// the previous P.V has completed and before it releases the P tile.  Rows past the unit's queries run
+// along on zero queries.  This function is the compute group's side.
+__device__ __noinline__ void attn_unit_tc(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot,
+                                          uint8_t* att_smem, Ctl* ctl, int et, bool& ok, KvCons& kvc, const Waiter& W,
+                                          uint32_t tmem_s, uint32_t tmem_o) {
+  const int hd = P.hd, G = P.Hq / P.Hkv, nq = P.Hq * hd, halves = hd / 64;
+  const int lane = et & 31, quad = ((et >> 5) + 2) & 3;       // compute warps are warps 2..5: TMEM lane quadrant = warp & 3
+  const int ql = quad * 32 + lane;                             // this thread's query row (TMEM lane)
+  const int Q = a.R * G;
+  const int q0 = qblk * P.att_qblk, nQ = min(P.att_qblk, Q - q0);
+  const int q_rows = P.att_q_rows;
+  uint8_t* qs = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem) + 1023) & ~(uintptr_t)1023);   // halves x [q_rows][128 B]
+  uint8_t* psm = qs + (size_t)halves * q_rows * 128;           // two P tiles of [q_rows][128 B]
+  const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
+  const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
+
+  // the unit's queries, swizzled: query index q -> row r = q / G, head = kvh * G + q % G; rows past nQ are zero.
+  // (Every S MMA of the previous unit has completed: its chunks were all waited for.)
+  {
+    const int pieces = hd / 8;                                 // 16-byte pieces per query
+    for (int it = et; it < q_rows * pieces; it += 128) {
+      const int r = it / pieces, c = it % pieces;
+      const bool on = r < nQ;
+      const int q = on ? q0 + r : q0;
+      cp_async16(qs + (size_t)(c >> 3) * q_rows * 128 + (size_t)r * 128 + (size_t)(((c & 7) ^ (r & 7)) << 4),
+                 reinterpret_cast<const uint4*>(P.q16 + (size_t)(a.off + q / G) * nq + (size_t)(kvh * G + q % G) * hd) + c, on);
+    }
+    cp_async_commit();
+    cp_async_wait_all();
+    fence_proxy_async_smem();                                  // the tensor core reads these tiles through the async proxy
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&ctl->q_full);
+  }
+  const bool mine = ql < nQ;
+  const int last = mine ? a.base + (q0 + ql) / G : -1;         // last visible position of this thread's query
+  float m_run = -INFINITY, l_run = 0.f;
+
+  for (int c = c_begin; c < c_end && ok; ++c) {
+    const uint32_t sb = kvc.sc & 1u, s_par = (kvc.sc >> 1) & 1u;
+#ifdef STAIRS_TRACE
+    unsigned long long* tl = (P.trace && blockIdx.x == 0 && et == 64 && kvc.sc < 300u) ? P.trace + (size_t)(2 + gridDim.x) * P.n_phases * 8 + 8000 + kvc.sc * 6 : nullptr;
+    if (tl) tl[0] = (unsigned long long)clock64();
+#endif
+    ++kvc.sc;
+    if (!W.wait(ctl->s_full + sb, s_par)) { ok = false; break; }   // S of chunk c is in TMEM
+#ifdef STAIRS_TRACE
+    if (tl) tl[1] = (unsigned long long)clock64();
+#endif
+    __syncwarp();
+    tc_fence_after();
+    const int p0 = c * ATT_CHUNK;
+    const int n_pos = min(ATT_CHUNK, a.base + a.R - p0);
+    const bool all_visible = p0 + ATT_CHUNK - 1 <= a.base;
+    float sv[ATT_CHUNK];
+#pragma unroll
+    for (int j0 = 0; j0 < ATT_CHUNK; j0 += 16) tmem_ld16(tmem_s + sb * ATT_CHUNK + lane_sel + (uint32_t)j0, sv + j0);
+#ifdef STAIRS_TRACE
+    if (tl) tl[2] = (unsigned long long)clock64();
+#endif
+    if (!all_visible) {
+#pragma unroll
+      for (int j = 0; j < ATT_CHUNK; ++j)
+        if (!(j < n_pos && p0 + j <= last)) sv[j] = -INFINITY;
+    }
+    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
+#pragma unroll
+    for (int j = 0; j < ATT_CHUNK; j += 4) {
+      mx4[0] = fmaxf(mx4[0], sv[j]); mx4[1] = fmaxf(mx4[1], sv[j + 1]); mx4[2] = fmaxf(mx4[2], sv[j + 2]); mx4[3] = fmaxf(mx4[3], sv[j + 3]);
+    }
+    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+    // The reference exponent m_run only follows the running maximum when that has moved by more than
+    // 2^8: until then P = 2^(S - m_run) may exceed 1 (at most 256: fine in fp16, and the sums are fp32),
+    // and O needs no rescaling - the same reference scales O and the sum, so the quotient is unchanged.
+    const float m_seen = fmaxf(m_run, mx);
+    const float m_new = (m_seen > m_run + 8.0f || m_run == -INFINITY) ? m_seen : m_run;
+    const float off = m_new == -INFINITY ? 0.f : m_new;
+    const float corr = fast_exp2(m_run - off);                 // 1 when the reference stays; 2^(-inf) = 0
+    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+    uint32_t pk[ATT_CHUNK / 2];
+#pragma unroll
+    for (int j = 0; j < ATT_CHUNK; j += 2) {
+      const float e0 = fast_exp2(sv[j] - off), e1 = fast_exp2(sv[j + 1] - off);
+      sum4[(j >> 1) & 3] += e0 + e1;
+      pk[j / 2] = pack_f16x2(e0, e1);
+    }
+    l_run = l_run * corr + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+    m_run = m_new;
+    // the row of P: eight 16-byte pieces, swizzled like every K-major tile (the P.V that read this tile two
+    // chunks ago has completed: the wait below covered it one chunk ago)
+    if (ql < q_rows) {
+      uint8_t* prow_s = psm + (size_t)sb * q_rows * 128 + (size_t)ql * 128;
+#pragma unroll
+      for (int cpc = 0; cpc < 8; ++cpc)
+        *reinterpret_cast<uint4*>(prow_s + (size_t)((cpc ^ (ql & 7)) << 4)) = make_uint4(pk[4 * cpc], pk[4 * cpc + 1], pk[4 * cpc + 2], pk[4 * cpc + 3]);
+    }
+#ifdef STAIRS_TRACE
+    if (tl) tl[3] = (unsigned long long)clock64();
+#endif
+    if (c > c_begin) {
+      // the previous chunk's P.V has completed; O is rescaled where a maximum moved
+      if (!W.wait(&ctl->o_done, kvc.o_par)) { ok = false; break; }
+      kvc.o_par ^= 1u;
+      __syncwarp();
+      tc_fence_after();
+      if (__any_sync(0xffffffffu, corr != 1.0f)) {
+        for (int d0 = 0; d0 < hd; d0 += 16) {
+          float ov[16];
+          tmem_ld16(tmem_o + lane_sel + (uint32_t)d0, ov);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) ov[j] *= corr;
+          tmem_st16(tmem_o + lane_sel + (uint32_t)d0, ov);
+        }
+      }
+    }
+#ifdef STAIRS_TRACE
+    if (tl) tl[4] = (unsigned long long)clock64();
+#endif
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(ctl->p_full + sb);              // this warp's rows of P (and of O) are ready for the chunk's P.V
+#ifdef STAIRS_TRACE
+    if (tl) tl[5] = (unsigned long long)clock64();
+#endif
+  }
+  // the unit's last P.V has completed
+  if (ok) {
+    if (!W.wait(&ctl->o_done, kvc.o_par)) ok = false;
+    kvc.o_par ^= 1u;
+  }
+  __syncwarp();
+  if (!ok) ctl->abort_flag = 1;
+  ok = group_ok(ctl, et);                                      // one verdict for all 128 threads
+  if (!ok) return;
+  tc_fence_after();
+  // this thread's row: the final output when the unit saw every visible position, else the state
+  // (O, max, sum) for the combine phase.  (All lanes take part in the TMEM loads.)
+  const int q = q0 + (mine ? ql : 0);
+  const float inv = a.n_ranges == 1 ? (l_run > 0.f ? 1.0f / l_run : 0.f) : 1.0f;
+  bf16* orow = P.o + (size_t)(a.off + q / G) * P.Hq * hd + (size_t)(kvh * G + q % G) * hd;
+  float* prow = P.attn_part + ((size_t)part_slot * P.att_qblk + (mine ? ql : 0)) * (hd + 4);
+  for (int d0 = 0; d0 < hd; d0 += 16) {
+    float ov[16];
+    tmem_ld16(tmem_o + lane_sel + (uint32_t)d0, ov);
+    if (mine) {
+      if (a.n_ranges == 1) {
+#pragma unroll
+        for (int j = 0; j < 16; j += 4)
+          store_split4(orow, (size_t)(d0 + j), (size_t)P.lo_row * P.Hq * hd, make_float4(ov[j] * inv, ov[j + 1] * inv, ov[j + 2] * inv, ov[j + 3] * inv));
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(prow + d0 + j) = make_float4(ov[j], ov[j + 1], ov[j + 2], ov[j + 3]);
+      }
+    }
+  }
+  if (mine && a.n_ranges != 1) { prow[hd] = m_run; prow[hd + 1] = l_run; }
+  tc_fence_before();
+  // (the next unit's first P.V overwrites O only after these threads have released that unit's first P tile)
+}
+
+// The MMA warp's side of the tcgen05 attention: walks this CTA's units of one attention phase in the
+// compute group's order and issues, per chunk, S = Q.K^T (as soon as the chunk's tiles have landed) and,
+// one chunk behind, O += P.V (once the compute warps have released the P tile); a commit after each S
+// signals the compute group, commits after each P.V hand the chunk buffer back to the loader and
+// publish the completion.  mc: this thread's running state across phases.
+struct AttIssue { int buf; uint32_t par; uint32_t sc; uint32_t q_par; };
+__device__ __noinline__ bool attn_issue_tc(const Params& P, Ctl* ctl, uint8_t* att_smem, int cta, int G, const Waiter& W,
+                                           uint32_t tmem_s, uint32_t tmem_o, AttIssue& mc) {
+  const int hd = P.hd, halves = hd / 64, q_rows = P.att_q_rows;
+  uint8_t* qs = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem) + 1023) & ~(uintptr_t)1023);
+  uint8_t* psm = qs + (size_t)halves * q_rows * 128;
+  uint8_t* ring = psm + (size_t)2 * q_rows * 128;
+  const size_t kvbuf = AttnSmem::kv_buf_bytes(hd);
+  const uint32_t idesc_s = instr_desc_f16(ATT_CHUNK, 0), idesc_o = instr_desc_f16(hd, 1);
+  const int n_req = P.mode == CALL_VALIDATE ? P.n_req : 1;
+  int u0 = 0;
+  for (int i = 0; i < n_req; ++i) {
+    const AttnReq a = ctl->areq[i];
+    const int first = (cta - u0 % G + G) % G;
+    for (int u = first; u < a.units; u += G) {
+      const int rest = u / a.n_qblk;
+      const int range = rest % a.n_ranges;
+      const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
+      if (!W.wait(&ctl->q_full, mc.q_par)) return false;      // the unit's Q tile is staged
+      mc.q_par ^= 1u;
+      // Two streams of work, each issued as soon as its input is there: S of the next chunk (its tiles
+      // have landed; at most one chunk ahead of the P.V stream, because there are two S buffers) and
+      // P.V of the oldest chunk whose P tile the compute warps have released.  Taking whichever is
+      // ready keeps a late chunk from holding up the P.V that frees a buffer for the loader.
+      int s_next = c_begin, pv_next = c_begin;
+      int pv_buf = mc.buf; uint32_t pv_n = mc.sc;              // buffer and running chunk number of the next P.V
+      long long t_idle = 0; bool idle = false;
+      while (pv_next < c_end) {
+        bool progress = false;
+        if (s_next < c_end && s_next - pv_next <= 1 && mbar_test(ctl->kv_full + mc.buf, mc.par)) {
+          tc_fence_after();
+          const uint32_t sb = mc.sc & 1u;
+          const uint32_t kb = smem_u32(ring + (size_t)mc.buf * kvbuf);
+          for (int h = 0; h < halves; ++h)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma_bf16(tmem_s + sb * ATT_CHUNK, smem_desc_sw128_ex(smem_u32(qs) + (uint32_t)(h * q_rows * 128 + k * 32), 16, 1024),
+                        smem_desc_sw128_ex(kb + (uint32_t)(h * ATT_CHUNK * 128 + k * 32), 16, 1024), idesc_s, (h | k) ? 1u : 0u);
+          umma_commit(ctl->s_full + sb);
+          ++mc.sc; ++s_next;
+          if (++mc.buf == P.att_nbuf) { mc.buf = 0; mc.par ^= 1u; }
+          progress = true;
+        }
+        if (pv_next < s_next && mbar_test(ctl->p_full + (pv_n & 1u), (pv_n >> 1) & 1u)) {
+          tc_fence_after();
+          const uint32_t vb = smem_u32(ring + (size_t)pv_buf * kvbuf + kvbuf / 2);
+          const uint32_t pb = smem_u32(psm + (size_t)(pv_n & 1u) * q_rows * 128);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            umma_bf16(tmem_o, smem_desc_sw128_ex(pb + (uint32_t)(k * 32), 16, 1024),
+                      smem_desc_sw128_ex(vb + (uint32_t)(k * 2048), (uint32_t)(ATT_CHUNK * 128), 1024), idesc_o, (pv_next > c_begin || k > 0) ? 1u : 0u);
+          umma_commit(ctl->kv_empty + pv_buf);
+          umma_commit(&ctl->o_done);
+          ++pv_n; ++pv_next;
+          if (++pv_buf == P.att_nbuf) pv_buf = 0;
+          progress = true;
+        }
+        if (progress) idle = false;
+        else {
+          if (!idle) { idle = true; t_idle = clock64(); }
+          if (W.poll_abort(t_idle)) { W.note(5u, (unsigned)cta, (unsigned)s_next, (unsigned)pv_next, (unsigned)mc.sc); return false; }
+        }
+      }
+    }
+    u0 += a.units;
+  }
+  return true;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -871,13 +1167,19 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = gridDim.x, cta = blockIdx.x;
   uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < 4 * P.t_box) tmem_cols <<= 1;   // two accumulators, each with hi-part and lo-part columns
+  // two GEMM accumulators, each with hi-part and lo-part columns; tcgen05 attention adds S (one chunk) and O (head size)
+  const uint32_t tmem_att = (uint32_t)(4 * P.t_box);
+  while ((int)tmem_cols < 4 * P.t_box + (P.att_tc ? 2 * ATT_CHUNK + P.hd : 0)) tmem_cols <<= 1;   // two S buffers, O
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) { mbar_init(ctl->full + s, 1); mbar_init(ctl->empty + s, 1); }
     mbar_init(ctl->acc_full + 0, 1); mbar_init(ctl->acc_full + 1, 1);
     mbar_init(ctl->acc_empty + 0, 4); mbar_init(ctl->acc_empty + 1, 4);
-    for (int b = 0; b < MAX_KV_BUF; ++b) { mbar_init(ctl->kv_full + b, 1); mbar_init(ctl->kv_empty + b, 4); }
+    // a chunk buffer is handed back by the four compute warps (mma.sync path) or by one tcgen05.commit
+    for (int b = 0; b < MAX_KV_BUF; ++b) { mbar_init(ctl->kv_full + b, 1); mbar_init(ctl->kv_empty + b, P.att_tc ? 1 : 4); }
+    mbar_init(ctl->s_full + 0, 1); mbar_init(ctl->s_full + 1, 1);
+    mbar_init(ctl->p_full + 0, 4); mbar_init(ctl->p_full + 1, 4);
+    mbar_init(&ctl->q_full, 4); mbar_init(&ctl->o_done, 1);
     ctl->abort_flag = 0; ctl->bcast = 0; ctl->areq_ready = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -963,8 +1265,20 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
       unsigned long long* klog = P.trace ? P.trace + (size_t)(2 + G) * P.n_phases * 8 : nullptr;   // per k-block cycle stamps of CTA 0
       int kn = 0;
 #endif
+      AttIssue att_mc{0, 0u, 0u, 0u};
+      bool areq_seen = false;
       for (int ph = 0; ph < P.n_phases && ok; ++ph) {
         const Phase& p = P.phases[ph];
+        if (p.kind == PH_ATTN && P.att_tc) {
+          // attention contractions of this CTA's units (the compute group does the softmax in between)
+          if (!areq_seen) {
+            const long long t0 = clock64();
+            while (!(areq_seen = ctl->areq_ready != 0)) { if (W.poll_abort(t0)) break; }
+            if (!areq_seen) { ok = false; break; }
+          }
+          ok = attn_issue_tc(P, ctl, att_smem, cta, G, W, tmem_base + tmem_att, tmem_base + tmem_att + 2 * ATT_CHUNK, att_mc);
+          continue;
+        }
         if (p.kind != PH_GEMM) continue;
         const int kblocks = p.kblocks;
         const KRange kr = phase_range(p.n_tiles, p.upt, kblocks, RANGE_UNIT_KB / kps, cta, G, p.ge_max);
@@ -1036,7 +1350,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
       const int hd = P.hd, halves = hd / 64, box_rows = P.kv_box_rows, slots = ATT_CHUNK / box_rows;
       const int n_boxes = 2 * halves * slots;
       const size_t kvbuf = AttnSmem::kv_buf_bytes(hd);
-      uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem) + 1023) & ~(uintptr_t)1023);
+      uint8_t* ring = att_ring_base(P, att_smem);
       // this lane's box: which tensor (K, V), which 64-column half, which page slice of the chunk
       const int b_which = lane / (halves * slots), b_half = (lane % (halves * slots)) / slots, b_slot = lane % slots;
       int buf = 0; uint32_t par = 0;
@@ -1059,6 +1373,12 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
             const int c_begin = range * a.cpu, c_end = min(a.n_chunks, c_begin + a.cpu);
             for (int c = c_begin; c < c_end && ok; ++c) {
               const int p0 = c * ATT_CHUNK;
+              // page slices of the chunk inside the request's page table (the rest keeps its old, finite contents);
+              // this lane's cache row is looked up before the wait for a free buffer, under which its latency hides
+              const int valid_slots = min(slots, (P.max_pages * P.page_tokens - p0) / box_rows);
+              const bool my_box = lane < n_boxes && b_slot < valid_slots;
+              const int pz = p0 + b_slot * box_rows;
+              const int row = my_box ? __ldcg(pt + pz / P.page_tokens) * P.page_tokens + pz % P.page_tokens : 0;
               bool go = true;
               if (lane == 0) {
                 if (p0 + ATT_CHUNK > a.base && !published) go = W.wait_grid(bar_count, P.bar_base + (unsigned long long)ph * G);
@@ -1067,13 +1387,9 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
               ok = __shfl_sync(0xffffffffu, go ? 1 : 0, 0) != 0;
               if (!ok) break;
               if (p0 + ATT_CHUNK > a.base && !published) { published = true; fence_proxy_async(); }
-              // page slices of the chunk inside the request's page table (the rest keeps its old, finite contents)
-              const int valid_slots = min(slots, (P.max_pages * P.page_tokens - p0) / box_rows);
               if (lane == 0) mbar_expect_tx(ctl->kv_full + buf, (uint32_t)(2 * halves * valid_slots * box_rows * 128));
               __syncwarp();
-              if (lane < n_boxes && b_slot < valid_slots) {
-                const int pz = p0 + b_slot * box_rows;
-                const int row = pt[pz / P.page_tokens] * P.page_tokens + pz % P.page_tokens;
+              if (my_box) {
                 uint8_t* dst = ring + (size_t)buf * kvbuf + (size_t)b_which * (kvbuf / 2) + (size_t)b_half * (ATT_CHUNK * 128) + (size_t)b_slot * box_rows * 128;
                 tma_load_2d_nohint(dst, b_which ? vmap : kmap, kvh * hd + b_half * 64, row, ctl->kv_full + buf);
               }
@@ -1118,15 +1434,16 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
       if (et < n_req0 && et < 64) ctl->areq[et] = attn_req(P, et, G);
       if (P.att_tma) {
         // the chunk buffers start out finite: a box that is never fetched (past the page table) must not feed NaNs to P.V
-        uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem) + 1023) & ~(uintptr_t)1023);
-        const int n16 = (int)((size_t)P.att_nbuf * AttnSmem::kv_buf_bytes(P.hd) / 16);
-        for (int i = et; i < n16; i += 128) reinterpret_cast<uint4*>(ring)[i] = make_uint4(0u, 0u, 0u, 0u);
+        uint8_t* ring = att_ring_base(P, att_smem);
+        uint8_t* first = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem) + 1023) & ~(uintptr_t)1023);   // (the Q and P tiles too)
+        const int n16 = (int)((size_t)(ring - first) + (size_t)P.att_nbuf * AttnSmem::kv_buf_bytes(P.hd)) / 16;
+        for (int i = et; i < n16; i += 128) reinterpret_cast<uint4*>(first)[i] = make_uint4(0u, 0u, 0u, 0u);
         fence_proxy_async();   // later bulk copies (async proxy) into these buffers
       }
       epi_bar_sync();
       if (et == 0) { __threadfence_block(); ctl->areq_ready = 1; }
     }
-    KvCons kvc{0, 0u};
+    KvCons kvc{0, 0u, 0u, 0u};
     for (int ph = 0; ph < P.n_phases && ok; ++ph) {
       const Phase& p = *reinterpret_cast<const Phase*>(ctl->phc[ph & 1]);
       // the next phase's descriptor: fetched now, parked in shared memory at the end of this phase
@@ -1173,7 +1490,8 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
               break;
             }
             unsigned long long* tra_u = (MK_TRACE_PTR(P.trace) && et == 0 && u == first) ? MK_TRACE_PTR(P.trace) + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
-            if (P.att_tma) attn_unit<true>(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok, kvc, W, tra_u);
+            if (P.att_tc) attn_unit_tc(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok, kvc, W, tmem_base + tmem_att, tmem_base + tmem_att + 2 * ATT_CHUNK);
+            else if (P.att_tma) attn_unit<true>(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok, kvc, W, tra_u);
             else attn_unit<false>(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok, kvc, W, tra_u);
           }
           u0 += a.units; g0 += P.Hkv * a.n_qblk;
@@ -1192,10 +1510,10 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
             int it = ((cta * 4 + quad) - item0) % (G * 4);
             if (it < 0) it += G * 4;
             for (; it < items; it += G * 4) {
-              const int kvh = it / Q, q = it % Q, qblk = q / ATT_QBLK, ql = q % ATT_QBLK;
+              const int kvh = it / Q, q = it % Q, qblk = q / P.att_qblk, ql = q % P.att_qblk;
               const int first_slot = u0 + (kvh * a.n_ranges) * a.n_qblk + qblk;
-              const size_t stride = (size_t)a.n_qblk * ATT_QBLK * (hd + 4);
-              const float* base = P.attn_part + ((size_t)first_slot * ATT_QBLK + ql) * (hd + 4);
+              const size_t stride = (size_t)a.n_qblk * P.att_qblk * (hd + 4);
+              const float* base = P.attn_part + ((size_t)first_slot * P.att_qblk + ql) * (hd + 4);
               // (max, sum) of range lane, lane + 32, ...: one load round for up to 32 ranges, then
               // the ranges' output vectors sixteen loads at a time; weights travel by shuffle and
               // the accumulation stays in range order
@@ -1757,13 +2075,13 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, tmem_cols); }
 }
 
-inline size_t smem_bytes(int t_box, int stages, int hd, int dbl, int kps, int tma = 0, int nbuf = 0) {
+inline size_t smem_bytes(int t_box, int stages, int hd, int dbl, int kps, int tma = 0, int nbuf = 0, int tc_q_rows = 0) {
   return 1024 + (size_t)stages * kps * (A_STAGE_BYTES + (size_t)2 * t_box * BK * 2) + MK_XCH_BYTES + ((sizeof(Ctl) + 127) & ~(size_t)127) +
-         AttnSmem::bytes(hd, dbl, tma, nbuf) + 64;
+         AttnSmem::bytes(hd, dbl, tma, nbuf, tc_q_rows) + 64;
 }
-inline int pick_stages(int t_box, int hd, int dbl, int kps, int tma = 0, int nbuf = 0) {
+inline int pick_stages(int t_box, int hd, int dbl, int kps, int tma = 0, int nbuf = 0, int tc_q_rows = 0) {
   int s = MAX_STAGES;
-  while (s > 1 && smem_bytes(t_box, s, hd, dbl, kps, tma, nbuf) > (size_t)SMEM_LIMIT) --s;
+  while (s > 1 && smem_bytes(t_box, s, hd, dbl, kps, tma, nbuf, tc_q_rows) > (size_t)SMEM_LIMIT) --s;
   return s;
 }
 // k-blocks per stage: two while at least three stages still fit (small row boxes), else one
