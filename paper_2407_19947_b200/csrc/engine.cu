@@ -62,8 +62,8 @@ struct DevModel {
 
 struct Layout {
   size_t status, seq, n_seq, page_table, tok, pos, req, val_req, val_k, val_off, keys, x, h, qkv, q,
-      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_flags, mk_bar, attn_part, prog_t, prog_d, mk_trace, mk_stats, attn_cnt, rope_t, rope_d, aux_t, aux_d, w13_t, w13_d, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
-  int max_rows, logit_rows, max_pages, n_pages, t_box_max, attn_units, stat_tiles, attn_cnt_n;
+      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_flags, mk_bar, attn_part, prog_t, prog_d, mk_trace, mk_stats, rope_t, rope_d, aux_t, aux_d, w13_t, w13_d, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
+  int max_rows, logit_rows, max_pages, n_pages, t_box_max, attn_units, stat_tiles;
   size_t prog_slot_t, prog_slot_d, prog_maps_off_t, prog_maps_off_d;
   size_t kv_t_layer, kv_d_layer;
   size_t attn_part_bytes;
@@ -247,8 +247,6 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     L->mk_trace = take(t.wdtype == 1 ? (size_t)(2 * 8 + 8 * TC_GRID_MAX) * (8 * std::max(t.n_layers, 1) + 4) * 8 : 0);
     L->stat_tiles = (t.d_model + tc::BM - 1) / tc::BM;
     L->mk_stats = take(t.wdtype == 1 ? (size_t)MK_MAX_ROWS * L->stat_tiles * 16 : 0);
-    L->attn_cnt_n = c.max_requests * hkv * std::max(n_qblk, 1);
-    L->attn_cnt = take(t.wdtype == 1 ? (size_t)L->attn_cnt_n * 4 : 0);
     L->rope_t = take(t.wdtype == 1 ? (size_t)t.head_dim * 2 * (1 + 2 * 64) : 0);   // inverse frequencies, then cos and sin of 64 rows
     L->rope_d = take((t.wdtype == 1 && has_draft) ? (size_t)d.head_dim * 2 * (1 + 2 * 64) : 0);
     // LayerNorm models: u = W.gain and c = W.bias per normalised GEMM (fp32)
@@ -561,7 +559,8 @@ MkPlan mk_plan(const stairs_ctx* ctx, const stairs_model& m, int t_box, int q_ro
   pl.kps = (ctx->kps_force > 0) ? ctx->kps_force : (stages_for(2, least) >= 3 ? 2 : 1);
   if (stages_for(pl.kps, least) < 2) pl.kps = 1;
   pl.att_nbuf = least;
-  while (pl.att_nbuf < want && stages_for(pl.kps, pl.att_nbuf + 1) >= (pl.kps == 2 ? 3 : 4)) ++pl.att_nbuf;
+  // (the tcgen05 path is used where attention dominates the call: there a third buffer is worth a fourth stage)
+  while (pl.att_nbuf < want && stages_for(pl.kps, pl.att_nbuf + 1) >= ((pl.kps == 2 || (pl.att_tc && pl.att_nbuf < 3)) ? 3 : 4)) ++pl.att_nbuf;
   pl.stages = stages_for(pl.kps, pl.att_nbuf);
   return pl;
 }
@@ -797,7 +796,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.seg_flags = reinterpret_cast<unsigned long long*>(ws + L.mk_flags);
   P.attn_part = reinterpret_cast<float*>(ws + L.attn_part); P.attn_part_units = (int)units_avail;
   P.stats = reinterpret_cast<float4*>(ws + L.mk_stats); P.stat_tiles = L.stat_tiles;
-  P.rope_inv = M.rope_inv; P.rope_cs = M.rope_inv + m.head_dim / 2; P.rope_sn = P.rope_cs + 64 * (m.head_dim / 2); P.attn_cnt = reinterpret_cast<int*>(ws + L.attn_cnt);
+  P.rope_inv = M.rope_inv; P.rope_cs = M.rope_inv + m.head_dim / 2; P.rope_sn = P.rope_cs + 64 * (m.head_dim / 2);
   P.bar = reinterpret_cast<unsigned long long*>(ws + L.mk_bar); P.bar_base = ctx->bar_base;
   P.status = ctx->status_dev; P.wait_limit = ctx->wait_limit;
   P.trace = (ctx->profile && &M == &ctx->target) ? reinterpret_cast<unsigned long long*>(ws + L.mk_trace) : nullptr;
@@ -1466,7 +1465,6 @@ int stairs_sync(stairs_ctx* ctx) {
     cudaMemsetAsync(ctx->ws + ctx->lay.mk_bar, 0, 64, ctx->stream);   // barrier count and abort word
     cudaMemsetAsync(ctx->ws + ctx->lay.gemm_counters, 0, (size_t)TC_COUNTERS * 4, ctx->stream);
     cudaMemsetAsync(ctx->ws + ctx->lay.mk_flags, 0, (size_t)TC_GRID_MAX * 8, ctx->stream);   // tags restart with the barrier count
-    cudaMemsetAsync(ctx->ws + ctx->lay.attn_cnt, 0, (size_t)ctx->lay.attn_cnt_n * 4, ctx->stream);
     cudaStreamSynchronize(ctx->stream);
     ctx->bar_base = 0;
     // kind: 1 shared-memory barrier (block, thread, parity), 2 grid barrier (block, thread, target),

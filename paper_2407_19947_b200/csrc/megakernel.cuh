@@ -109,7 +109,6 @@ struct Params {
   __half* q16;               // [row][Hq*hd] queries, rotated and scaled by 1/sqrt(hd), written by the QKV epilogue
   float* rope_cs; float* rope_sn;   // [row][hd/2] cos and sin of the call's row positions, written by the embedding phase
      // [hd/2] theta^(-2i/hd)
-  int* attn_cnt;            // (reserved; the combine phase needs no counters)
   float* logits;            // optional dump
   int* target_tokens; int* accept_len; int commit; int* draft_out;
   // scratch

@@ -351,3 +351,43 @@ def test_adaptive_draft_length_generation_matches_the_oracle_schedule():
     ga, sa = eng.generate(0, p2, 3, 48, adaptive=True)
     assert ga == g0 and sa["emitted"] >= 48 and sa["accepted"] <= sa["drafted"]
     eng.close()
+
+
+@pytest.mark.parametrize("hq,hkv,hd", [(8, 2, 64), (4, 1, 128), (4, 4, 64)], ids=["gqa4_hd64", "mqa4_hd128", "mha_hd64"])
+def test_tcgen05_attention_path_matches_oracle(hq, hkv, hd):
+    # The attention contractions on the 5th-generation tensor cores are chosen per call for long
+    # contexts and prefill passes; here they are switched on for every call, so that small models
+    # reach them too: prefill passes of 64 rows (up to 256 queries per kv head: two query blocks),
+    # contexts split over several units (partial states merged by the combine phase) and not, two
+    # requests in one call, several draft lengths.  Same bars as everywhere.
+    st = _stairs()
+    shape = wl.family_b(2, hq * hd if hq * hd <= 512 else 512, hq, hkv, hd, 512, 2048, 1024)
+    tsrc, dsrc = sources(shape, std=0.05)
+    tgt, _ = gu.oracle_pair(tsrc)
+    eng = st.Stairs(tsrc, dsrc, max_requests=2, max_seq_len=700, k_max=8, kv_page_tokens=32)
+    eng.debug_tune(3, 2)
+    prompts = [list(wl.zipf_tokens(n, shape.vocab, 40 + i)) for i, n in enumerate((611, 75))]
+    for i, p in enumerate(prompts):
+        eng.prefill(i, p)
+    for ks in ([8, 3], [0, 8], [1, 1]):
+        drafts = np.zeros((2, 8), np.int32)
+        for i in range(2):
+            cont = so.greedy_generate(tgt, prompts[i], ks[i] + 1)
+            drafts[i, :ks[i]] = wl.forced_draft(np.array(cont), ks[i] // 2, shape.vocab, 5 + i)
+        tt, al, logits = eng.validate([0, 1], ks, torch.from_numpy(drafts).cuda(), commit=False, want_logits=True)
+        eng.sync()
+        logits = logits.cpu().numpy()
+        row = 0
+        for i in range(2):
+            ref, _ = gu.oracle_stair_logits(tgt, prompts[i], drafts[i, :ks[i]])
+            gpu_tok = tt.cpu().numpy()[i]
+            gu.check_rows_against_oracle(logits[row:row + ks[i] + 1], gpu_tok, ref, gu.LOGIT_TOL_BF16)
+            assert int(al.cpu()[i]) == gu.first_mismatch(drafts[i, :ks[i]], gpu_tok)
+            row += ks[i] + 1
+    # the same calls on the register path agree closely (different summation order only)
+    _, _, lg_tc = eng.validate([0, 1], [8, 3], torch.from_numpy(drafts).cuda(), want_logits=True)
+    eng.debug_tune(3, 1)
+    _, _, lg_mma = eng.validate([0, 1], [8, 3], torch.from_numpy(drafts).cuda(), want_logits=True)
+    eng.sync()
+    assert float((lg_tc - lg_mma).abs().max()) < 5e-3
+    eng.close()
