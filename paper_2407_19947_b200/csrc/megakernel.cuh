@@ -10,20 +10,29 @@
 // barrier that publishes it has completed.  HBM therefore keeps streaming through barriers,
 // norms and attention.
 //
-// Roles per CTA (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner,
-// warps 2-5 = "compute group": GEMM epilogues and every non-GEMM phase (rows+embedding,
-// attention, combine, accept).  GEMM work is cut into contiguous k-block ranges per CTA; a tile
-// cut over several CTAs is finished by the CTA that owns its first k-block, which adds the other
-// CTAs' parked partial tiles in k order once their flags are up.  Normalisation is folded into
-// the GEMMs (operand x * gain, epilogue rescales by the row's 1/std from per-tile statistics).
+// Roles per CTA (224 threads): warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner (GEMM phases, and
+// the attention phases' contractions on the tcgen05 path), warps 2-5 = "compute group": GEMM epilogues
+// and every non-GEMM phase (rows+embedding, attention softmax, combine, accept), warp 6 = K/V loader of
+// the attention phases.  A GEMM pipeline stage holds one or two 64-element k-blocks, fetched by ONE
+// 3-D bulk tensor copy per operand and freed by ONE commit (issue costs, not bandwidth, bound the
+// single-thread roles).  GEMM work is cut into contiguous ranges per CTA, in units of two k-blocks
+// whatever the stage depth, so results do not depend on the call's row count; a tile cut over
+// several CTAs is finished by the CTA that owns its first k-block, which adds the other CTAs' parked
+// partial tiles in k order once their flags are up.  Normalisation is folded into the GEMMs (operand
+// x * gain, epilogue rescales by the row's 1/std from per-tile statistics).
 //
-// Attention (staircase mask over the paged cache): a unit is (request, kv head, range of
-// 64-position chunks, block of <= 48 queries); all rows x grouped heads of the request share the
-// K/V chunk, staged in shared memory by 16-byte asynchronous copies (cache rows looked up once
-// per chunk, so pages need not be contiguous).  Queries (rotated, scaled, fp16) and the new
-// positions' K/V are filed by the QKV projection's epilogue.  Scores and P.V run on fp16
-// mma.sync tiles, one warp per 16-query block, online softmax in registers.  Unit boundaries
-// depend only on the request's own committed length, never on the other requests in the call.
+// Attention (staircase mask over the paged cache): a unit is (request, kv head, range of 64-position
+// chunks, block of queries); all rows x grouped heads of the request share the K/V chunk.  Queries
+// (rotated, scaled by log2(e)/sqrt(hd), fp16) and the new positions' K/V are filed by the QKV
+// projection's epilogue.  Three ways through a unit, chosen by the host per model and call:
+//  - head sizes 64/128, long contexts or many query rows: chunks streamed by the loader warp with
+//    tiled bulk copies (128-byte swizzle) through a ring of buffers; S = Q.K^T and O += P.V as
+//    tcgen05 MMAs (M = 128 queries, accumulators in TMEM) issued by the MMA warp one chunk ahead of
+//    the compute group's base-2 online softmax;
+//  - head sizes 64/128 otherwise: the same ring, contractions on fp16 mma.sync tiles, one warp per
+//    16-query block, softmax state in registers;
+//  - other head sizes: padded tiles staged by 16-byte asynchronous copies from the compute warps.
+// Unit boundaries depend only on the request's own committed length, never on the other requests.
 //
 // With 227 KB of shared memory the L1 is nearly gone: every global or local access is an L2 round
 // trip.  Phase descriptors and request geometry are therefore kept in shared memory, cursors in
