@@ -743,9 +743,10 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
     // quicker on the register path, whose per-unit set-up is smaller.
     int r_max0 = 0; long long len_max = 0;
     if (c.mode == mk::CALL_VALIDATE) for (int i = 0; i < c.n_req; ++i) { r_max0 = std::max(r_max0, c.k_host[i] + 1); len_max = std::max<long long>(len_max, ctx->n_seq_ub[c.req_host[i]]); }
-    else { r_max0 = T; len_max = ctx->n_seq_ub[c.slot]; }
+    else { r_max0 = T; len_max = c.mode == mk::CALL_PREFILL ? c.draft_step + T : ctx->n_seq_ub[c.slot]; }
     const long long chunks_per_unit = (len_max / mk::ATT_CHUNK + 1) * hkv / std::max(ctx->sm_count, 1);
-    tc_call = (ctx->att_tc_force > 0 || chunks_per_unit >= 6 || r_max0 * gq >= 96) ? 1 : 0;
+    // (with many query rows its tiles take shared memory from the GEMM ring: only past a few thousand positions)
+    tc_call = (ctx->att_tc_force > 0 || chunks_per_unit >= 6 || (r_max0 * gq >= 96 && len_max >= 4096)) ? 1 : 0;
     const MkPlan pl0 = mk_plan(ctx, m, t_box, 0, tc_call);
     int r_max = 0;
     if (c.mode == mk::CALL_VALIDATE) for (int i = 0; i < c.n_req; ++i) { need += attn_unit_bound(hkv, gq, c.k_host[i] + 1, pl0.att_qblk); r_max = std::max(r_max, c.k_host[i] + 1); }
