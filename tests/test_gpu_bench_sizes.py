@@ -119,18 +119,33 @@ def test_config4_shape_long_prompt_single_request_slot():
 
 
 def test_config4_full_depth_at_the_benchmarked_prompt():
-    # all k+1 rows of one call at the full 32 layers and the 1024-token prompt
+    # all k+1 rows of three consecutive stairs iterations at the full 32 layers and the 1024-token
+    # prompt: each call's drafts are forced from the library's own continuation (a different accept
+    # length every time), the call commits, and the oracle recomputes the rows from the committed context
     st = _stairs()
     w = wl.workload(4)
     tsrc, dsrc = wl.make_sources(w, backend="torch-cuda")
     prompt = list(wl.prompt_tokens(w, n=1025))
     eng = st.Stairs(tsrc, dsrc, max_requests=1, max_seq_len=1025 + 64, k_max=8, kv_page_tokens=64)
     eng.prefill(0, prompt)
-    cont = _own_continuation(eng, prompt, 9)
-    draft = wl.forced_draft(np.array(cont), 4, w.target.vocab, 11)
     tgt = so.OracleModel(w.target, tsrc, keep=False)     # one layer widened at a time
-    err, exact, ref, gpu_tok = _validate_and_compare(eng, tgt, prompt, draft, 8, check_row0=False)
-    print(f"config 4, 32 layers, prompt 1025: logit max-abs err {err:.4f}, decisive rows {exact}/9")
+    ctx = list(prompt)
+    for it, (k, a) in enumerate(((8, 4), (5, 5), (8, 0))):
+        cont = _own_continuation(eng, ctx, k + 1)
+        draft = wl.forced_draft(np.array(cont), a, w.target.vocab, 11 + it)
+        d_dev = torch.zeros(8, dtype=torch.int32, device="cuda")
+        d_dev[:k] = torch.from_numpy(draft)
+        tt, al, logits = eng.validate([0], [k], d_dev, commit=True, want_logits=True)
+        eng.sync()
+        ref = _oracle_rows(tgt, ctx, draft, check_row0=False)
+        gpu_tok = tt.cpu().numpy()[0]
+        err, exact = gu.check_rows_against_oracle(logits.cpu().numpy(), gpu_tok, ref, gu.LOGIT_TOL_BF16)
+        acc = int(al.cpu()[0])
+        assert acc == gu.first_mismatch(draft, gpu_tok) == a
+        print(f"config 4, 32 layers, context {len(ctx)}, k {k}: logit max-abs err {err:.4f}, decisive rows {exact}/{k + 1}, accepted {acc}")
+        new_ctx = eng.sequence(0)
+        assert new_ctx == ctx + [int(t) for t in draft[:acc]] + [int(gpu_tok[acc])]
+        ctx = new_ctx
     eng.close()
     tsrc.drop_cache(); dsrc.drop_cache()
 
