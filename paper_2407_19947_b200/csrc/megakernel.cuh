@@ -233,22 +233,22 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
 // alone and inside a larger batch.  The phase is cut over min(G, units) CTAs so that no
 // participating range is empty (the split-tile bookkeeping counts one segment per CTA touching a tile).
 constexpr int RANGE_UNIT_KB = 2;
-struct KRange { long long begin, end; int ge; };
+struct KRange { int begin, end; int ge; };   // 32-bit throughout: units * CTAs < 2^32 is checked on the host, and 64-bit divisions are long code
 // first stage of unit u: upt units and spt stages per tile, spu stages per unit (the last unit of a tile may be short)
-__device__ __forceinline__ long long unit_to_stage(long long u, int upt, int spt, int spu) {
-  if (spu == 1) return u;
-  const long long tile = u / upt;
-  const int j = (int)(u % upt);
-  return tile * spt + (j * spu < spt ? j * spu : spt);
+__device__ __forceinline__ int unit_to_stage(unsigned u, int upt, int spt, int spu) {
+  if (spu == 1) return (int)u;
+  const unsigned tile = u / (unsigned)upt;
+  const int j = (int)(u - tile * (unsigned)upt);
+  return (int)tile * spt + (j * spu < spt ? j * spu : spt);
 }
 __device__ __forceinline__ KRange phase_range(int n_tiles, int upt, int spt, int spu, int cta, int G, int ge_max) {
   KRange r;
-  const long long total = (long long)n_tiles * upt;
+  const unsigned total = (unsigned)n_tiles * (unsigned)upt;
   if (ge_max > 0 && ge_max < G) G = ge_max;
-  r.ge = (int)(total < (long long)G ? total : (long long)G);
+  r.ge = (int)(total < (unsigned)G ? total : (unsigned)G);
   if (cta >= r.ge) { r.begin = r.end = 0; return r; }
-  r.begin = unit_to_stage(range_begin(total, cta, r.ge), upt, spt, spu);
-  r.end = unit_to_stage(range_begin(total, cta + 1, r.ge), upt, spt, spu);
+  r.begin = unit_to_stage((total * (unsigned)cta) / (unsigned)r.ge, upt, spt, spu);
+  r.end = unit_to_stage((total * (unsigned)(cta + 1)) / (unsigned)r.ge, upt, spt, spu);
   return r;
 }
 
@@ -332,9 +332,11 @@ struct Waiter {
     if ((unsigned long long)(clock64() - t0) > limit) { *abort_flag = 1; return true; }
     return false;
   }
-  // mbarrier wait (bounded)
-  __device__ __forceinline__ bool wait(uint64_t* bar, uint32_t parity) const {
-    if (mbar_try(bar, parity)) return true;
+  // mbarrier wait (bounded).  The polling loops are kept out of line: they are inlined nowhere, so the
+  // many wait sites cost a test and a call each instead of a copy of the loop (the kernel's code has
+  // to stay inside the instruction cache: every phase runs its code once, and code that misses runs
+  // at a fraction of the warm issue rate).
+  __device__ __noinline__ bool wait_slow(uint64_t* bar, uint32_t parity) const {
     const long long t0 = clock64();
     int spins = 0;
     while (true) {
@@ -346,8 +348,12 @@ struct Waiter {
       if ((++spins & 255) == 0 && ld_acquire_u64(gabort)) { *abort_flag = 1; return false; }
     }
   }
+  __device__ __forceinline__ bool wait(uint64_t* bar, uint32_t parity) const {
+    if (mbar_try(bar, parity)) return true;
+    return wait_slow(bar, parity);
+  }
   // grid barrier wait: arrivals >= target
-  __device__ __forceinline__ bool wait_grid(const unsigned long long* counter, unsigned long long target) const {
+  __device__ __noinline__ bool wait_grid(const unsigned long long* counter, unsigned long long target) const {
     const long long t0 = clock64();
     int spins = 0;
     while (ld_acquire_u64(counter) < target) {
@@ -391,8 +397,8 @@ struct WCursor {
       ph = p_i; kblocks = p.kblocks; dual = p.dual; n_src = p.n_src; x_map = p.x_map;
       st0 = p.src_tiles[0]; st1 = p.src_tiles[1];
       wmap0 = p.w_map[0]; wmap1 = p.w_map[1]; wmap2 = p.w_map[2];
-      n_tile = (int)(kr.begin / p.kblocks); kk = (int)(kr.begin % p.kblocks);
-      remaining = (int)(kr.end - kr.begin);
+      n_tile = kr.begin / p.kblocks; kk = kr.begin - n_tile * p.kblocks;
+      remaining = kr.end - kr.begin;
       locate(P);
       valid = true;
       return;
@@ -485,24 +491,22 @@ __device__ void embed_row(const Params& P, int t, const RowInfo& r, const float*
   bf16* hr = P.h + (size_t)t * d;
   const bf16* e = P.tok_emb + (size_t)r.tok * d;
   const bf16* pe = P.pos_emb ? P.pos_emb + (size_t)r.pos * d : nullptr;
-  float xv[64];   // d <= 8192
+  // (rolled loops: this runs once per row and call, and code that is executed once costs its
+  // instruction fetch - the second pass re-reads this thread's own stores instead of keeping
+  // the row in registers)
   float s1 = 0.f;
-#pragma unroll
-  for (int i = 0; i < 64; ++i) {
-    const int col = et + 128 * i;
-    float v = 0.f;
-    if (col < d) {
-      v = __bfloat162float(e[col]);
-      if (pe) v += __bfloat162float(pe[col]);
-      xr[col] = v;
-      store_split(hr, col, (size_t)P.lo_row * d, v * g[col]);
-    }
-    xv[i] = v; s1 += v;
+#pragma unroll 4
+  for (int col = et; col < d; col += 128) {
+    float v = __bfloat162float(e[col]);
+    if (pe) v += __bfloat162float(pe[col]);
+    xr[col] = v;
+    store_split(hr, col, (size_t)P.lo_row * d, v * g[col]);
+    s1 += v;
   }
   const float mean = group_sum(s1, red, et) / (float)d;
   float s2 = 0.f;
-#pragma unroll
-  for (int i = 0; i < 64; ++i) { const int col = et + 128 * i; if (col < d) { const float c = xv[i] - mean; s2 += c * c; } }
+#pragma unroll 4
+  for (int col = et; col < d; col += 128) { const float c = xr[col] - mean; s2 += c * c; }
   const float m2 = group_sum(s2, red, et);
   for (int tile = et; tile < P.stat_tiles; tile += 128)
     P.stats[(size_t)t * P.stat_tiles + tile] = tile == 0 ? make_float4(mean, m2, (float)d, 0.f) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1290,9 +1294,9 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
         if (p.kind != PH_GEMM) continue;
         const int kblocks = p.kblocks;
         const KRange kr = phase_range(p.n_tiles, p.upt, kblocks, RANGE_UNIT_KB / kps, cta, G, p.ge_max);
-        int remaining = (int)(kr.end - kr.begin);
+        int remaining = kr.end - kr.begin;
         if (remaining <= 0) continue;
-        int kk = (int)(kr.begin % kblocks);
+        int kk = kr.begin % kblocks;
         bool seg_first = true;
         unsigned long long* trm = (MK_TRACE_PTR(P.trace) && cta == 0) ? MK_TRACE_PTR(P.trace) + (size_t)ph * 8 : nullptr;
         bool first_k = true;
@@ -1523,7 +1527,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
               const size_t stride = (size_t)a.n_qblk * P.att_qblk * (hd + 4);
               const float* base = P.attn_part + ((size_t)first_slot * P.att_qblk + ql) * (hd + 4);
               // (max, sum) of range lane, lane + 32, ...: one load round for up to 32 ranges, then
-              // the ranges' output vectors sixteen loads at a time; weights travel by shuffle and
+              // the ranges' output vectors eight loads at a time; weights travel by shuffle and
               // the accumulation stays in range order
               const int nr = a.n_ranges, dd = lane * 4;
               float M = -INFINITY, m0 = -INFINITY, l0 = 0.f;
@@ -1547,14 +1551,14 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
                 const float wgt = mu == -INFINITY ? 0.f : fast_exp2(mu - M);   // 0 for lanes past the last range (maxima are base-2 exponents)
                 L += lu * wgt;
                 const int nb = min(32, nr - rb);
-                for (int g0 = 0; g0 < nb; g0 += 16) {
-                  float4 v[16];
+                for (int g0 = 0; g0 < nb; g0 += 8) {
+                  float4 v[8];
 #pragma unroll
-                  for (int u = 0; u < 16; ++u)
+                  for (int u = 0; u < 8; ++u)
                     v[u] = (g0 + u < nb && dd < hd) ? __ldcg(reinterpret_cast<const float4*>(base + (size_t)(rb + g0 + u) * stride + dd))
                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                  for (int u = 0; u < 16; ++u) {
+                  for (int u = 0; u < 8; ++u) {
                     const float wu = __shfl_sync(0xffffffffu, wgt, (g0 + u) & 31);
                     acc.x += v[u].x * wu; acc.y += v[u].y * wu; acc.z += v[u].z * wu; acc.w += v[u].w * wu;
                   }
@@ -1628,9 +1632,8 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
         }
       } else {
         // ---------------------------------------------------------------- GEMM epilogue
-        const long long total = (long long)p.n_tiles * p.kblocks;
         const KRange kr = phase_range(p.n_tiles, p.upt, p.kblocks, RANGE_UNIT_KB / kps, cta, G, p.ge_max);
-        const long long kb_begin = kr.begin, kb_end = kr.end;
+        const int kb_begin = kr.begin, kb_end = kr.end;
         const int Ge = kr.ge;
         gemm_worked = kb_begin < kb_end;
         const int Tvalid = P.T;
@@ -1698,16 +1701,16 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
         }
         if (tracing) tr[3] = globaltimer_ns();
         bool first_seg = true;
-        long long kb = kb_begin;
+        int kb = kb_begin;
         const unsigned long long seg_tag = P.bar_base + (unsigned long long)ph + 1ull;   // unique per launch and phase
         const unsigned tot32 = (unsigned)(p.n_tiles * p.upt), ge32 = (unsigned)Ge;
         // first stage of CTA c's range (units * Ge < 2^32, checked on the host)
-        auto rb = [&](unsigned c) { return (unsigned)unit_to_stage((long long)((tot32 * c) / ge32), p.upt, p.kblocks, RANGE_UNIT_KB / kps); };
+        auto rb = [&](unsigned c) { return (unsigned)unit_to_stage((tot32 * c) / ge32, p.upt, p.kblocks, RANGE_UNIT_KB / kps); };
         const int er = et >> 3, cg = et & 7;
         while (kb < kb_end && ok) {
-          const int tile = (int)(kb / p.kblocks), kk0 = (int)(kb % p.kblocks);
-          const long long tile_first = (long long)tile * p.kblocks, tile_end = tile_first + p.kblocks;
-          const long long seg_end = tile_end < kb_end ? tile_end : kb_end;
+          const int tile = kb / p.kblocks, kk0 = kb - tile * p.kblocks;
+          const int tile_first = tile * p.kblocks, tile_end = tile_first + p.kblocks;
+          const int seg_end = tile_end < kb_end ? tile_end : kb_end;
           // The CTA that owns a tile's first k-block finishes the tile; a CTA whose segment starts
           // inside a tile (always the first segment of its range, so at most one per phase) parks
           // the partial sums in its slot and raises its flag.  The finisher's segment is the
@@ -1850,102 +1853,116 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
                 epi_bar_sync();
               }
               if (ok) {
+                // Each phase runs this code once per tile, so its instruction fetch is what it costs:
+                // the loads that must be in flight together are unrolled, everything per column group
+                // is a rolled loop over the four groups of the thread (the sums wait in the exchange tile).
                 const int t = c0 + er;
                 const bool row_on = t < Tvalid;
-                const float* vrow = vt + er * VT_LD;
-                float4 a[4];
-                bool on[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  const int col = (cg + 8 * q) * 4;
-                  on[q] = row_on && (p.dual ? (col & 63) < ncols : col < ncols);
-                  a[q] = on[q] ? *reinterpret_cast<const float4*>(vrow + col) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-                if (!whole) {
-                  // the other segments' partial sums: six segments' loads in flight together, the
-                  // additions in k order
-                  for (unsigned c = (unsigned)cta + 1; c <= last_c; c += 6) {
-                    float4 tmp[6][4];
-#pragma unroll
-                    for (int u = 0; u < 6; ++u) {
-                      const float* part = P.partial + ((size_t)min(c + u, last_c) * P.t_box + (row_on ? t : 0)) * BM;
-#pragma unroll
-                      for (int q = 0; q < 4; ++q)
-                        tmp[u][q] = (on[q] && c + u <= last_c) ? __ldcg(reinterpret_cast<const float4*>(part + (cg + 8 * q) * 4))
-                                                               : make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-#pragma unroll
-                    for (int u = 0; u < 6; ++u) {
-#pragma unroll
-                      for (int q = 0; q < 4; ++q) { a[q].x += tmp[u][q].x; a[q].y += tmp[u][q].y; a[q].z += tmp[u][q].z; a[q].w += tmp[u][q].w; }
-                    }
-                  }
-                }
-                if (tra) {
-                  asm volatile("" ::"f"(a[0].x), "f"(a[0].w), "f"(a[1].x), "f"(a[1].w), "f"(a[2].x), "f"(a[2].w), "f"(a[3].x), "f"(a[3].w));
-                  tra[6] = globaltimer_ns();
-                }
-                if (p.norm_in && row_on) {
-                  // fold the normalisation in: y = rstd_t * (acc - mean_t * u[n]) + c[n]
-                  const float rs = ctl->rstd[t], mu = ctl->mu[t];
+                float* vrow = vt + er * VT_LD;
+                const bool add_res = p.epi == TC_ADD_F32;
+                if (!whole || add_res) {
+                  float4 a[4];
+                  bool on[4];
 #pragma unroll
                   for (int q = 0; q < 4; ++q) {
-                    const float4 u4 = *reinterpret_cast<const float4*>(ctl->utile + (cg + 8 * q) * 4);
-                    const float4 c4 = *reinterpret_cast<const float4*>(ctl->ctile + (cg + 8 * q) * 4);
-                    a[q].x = rs * (a[q].x - mu * u4.x) + c4.x; a[q].y = rs * (a[q].y - mu * u4.y) + c4.y;
-                    a[q].z = rs * (a[q].z - mu * u4.z) + c4.z; a[q].w = rs * (a[q].w - mu * u4.w) + c4.w;
+                    const int col = (cg + 8 * q) * 4;
+                    on[q] = row_on && (p.dual ? (col & 63) < ncols : col < ncols);
+                    a[q] = on[q] ? *reinterpret_cast<const float4*>(vrow + col) : make_float4(0.f, 0.f, 0.f, 0.f);
                   }
-                }
-                if (p.epi == TC_ADD_F32) {
-                  // residual update; with a following normalised GEMM also its operand bf16(x * gain)
-                  // and this tile's row statistics (count, mean, centred sum of squares)
-                  float cnt = 0.f, sum = 0.f;
+                  if (!whole) {
+                    // the other segments' partial sums: six segments' loads in flight together, the
+                    // additions in k order
+                    for (unsigned c = (unsigned)cta + 1; c <= last_c; c += 6) {
+                      float4 tmp[6][4];
 #pragma unroll
-                  for (int q = 0; q < 4; ++q) {
-                    if (on[q]) {
-                      const int col = (cg + 8 * q) * 4;
-                      const size_t o = (size_t)t * p.ldo + n0 + col;
-                      const float4 x4 = c0 == 0 ? xq[q] : __ldcg(reinterpret_cast<const float4*>(out_f32 + o));
-                      a[q] = make_float4(x4.x + a[q].x, x4.y + a[q].y, x4.z + a[q].z, x4.w + a[q].w);
-                      *reinterpret_cast<float4*>(out_f32 + o) = a[q];
-                      if (p.next_g) {
-                        const float4 g4 = *reinterpret_cast<const float4*>(ctl->gtile + col);
-                        store_split4(P.h, o, (size_t)P.lo_row * p.ldo, make_float4(a[q].x * g4.x, a[q].y * g4.y, a[q].z * g4.z, a[q].w * g4.w));
+                      for (int u = 0; u < 6; ++u) {
+                        const float* part = P.partial + ((size_t)min(c + u, last_c) * P.t_box + (row_on ? t : 0)) * BM;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                          tmp[u][q] = (on[q] && c + u <= last_c) ? __ldcg(reinterpret_cast<const float4*>(part + (cg + 8 * q) * 4))
+                                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
                       }
-                      cnt += 4.f; sum += (a[q].x + a[q].y) + (a[q].z + a[q].w);
+#pragma unroll
+                      for (int u = 0; u < 6; ++u) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) { a[q].x += tmp[u][q].x; a[q].y += tmp[u][q].y; a[q].z += tmp[u][q].z; a[q].w += tmp[u][q].w; }
+                      }
                     }
                   }
-                  if (tra) { asm volatile("" ::"f"(sum), "f"(cnt)); tra[7] = globaltimer_ns(); }
-                  if (p.next_g) {
-                    float mean = cnt > 0.f ? sum / cnt : 0.f, m2 = 0.f;
+                  if (tra) {
+                    asm volatile("" ::"f"(a[0].x), "f"(a[0].w), "f"(a[1].x), "f"(a[1].w), "f"(a[2].x), "f"(a[2].w), "f"(a[3].x), "f"(a[3].w));
+                    tra[6] = globaltimer_ns();
+                  }
+                  if (add_res) {
+                    // residual update (a residual GEMM has no folded normalisation)
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                       if (on[q]) {
-                        const float d0 = a[q].x - mean, d1 = a[q].y - mean, d2 = a[q].z - mean, d3 = a[q].w - mean;
+                        const size_t o = (size_t)t * p.ldo + n0 + (cg + 8 * q) * 4;
+                        const float4 x4 = c0 == 0 ? xq[q] : __ldcg(reinterpret_cast<const float4*>(out_f32 + o));
+                        a[q] = make_float4(x4.x + a[q].x, x4.y + a[q].y, x4.z + a[q].z, x4.w + a[q].w);
+                        *reinterpret_cast<float4*>(out_f32 + o) = a[q];
+                      }
+                    }
+                  }
+#pragma unroll
+                  for (int q = 0; q < 4; ++q)
+                    if (on[q]) *reinterpret_cast<float4*>(vrow + (cg + 8 * q) * 4) = a[q];   // (this thread's own slots)
+                }
+                // column group `col` of this thread's row, with the folded normalisation
+                // y = rstd_t * (acc - mean_t * u[n]) + c[n] where the GEMM has one
+                const float rs = (p.norm_in && row_on) ? ctl->rstd[t] : 1.0f, mu = (p.norm_in && row_on) ? ctl->mu[t] : 0.f;
+                auto group = [&](int col) -> float4 {
+                  float4 v = *reinterpret_cast<const float4*>(vrow + col);
+                  if (p.norm_in) {
+                    const float4 u4 = *reinterpret_cast<const float4*>(ctl->utile + col);
+                    const float4 c4 = *reinterpret_cast<const float4*>(ctl->ctile + col);
+                    v.x = rs * (v.x - mu * u4.x) + c4.x; v.y = rs * (v.y - mu * u4.y) + c4.y;
+                    v.z = rs * (v.z - mu * u4.z) + c4.z; v.w = rs * (v.w - mu * u4.w) + c4.w;
+                  }
+                  return v;
+                };
+                if (add_res) {
+                  // with a following normalised GEMM: its operand bf16(x * gain) and this tile's row
+                  // statistics (count, mean, centred sum of squares; two passes over the row's 128 values)
+                  if (p.next_g) {
+                    float cnt = 0.f, sum = 0.f;
+#pragma unroll 1
+                    for (int q = 0; q < 4; ++q) {
+                      const int col = (cg + 8 * q) * 4;
+                      if (row_on && col < ncols) {
+                        const float4 x4 = *reinterpret_cast<const float4*>(vrow + col);
+                        const float4 g4 = *reinterpret_cast<const float4*>(ctl->gtile + col);
+                        store_split4(P.h, (size_t)t * p.ldo + n0 + col, (size_t)P.lo_row * p.ldo, make_float4(x4.x * g4.x, x4.y * g4.y, x4.z * g4.z, x4.w * g4.w));
+                        cnt += 4.f; sum += (x4.x + x4.y) + (x4.z + x4.w);
+                      }
+                    }
+                    if (tra) { asm volatile("" ::"f"(sum), "f"(cnt)); tra[7] = globaltimer_ns(); }
+#pragma unroll
+                    for (int o = 1; o < 8; o <<= 1) { cnt += __shfl_xor_sync(0xffffffffu, cnt, o); sum += __shfl_xor_sync(0xffffffffu, sum, o); }
+                    const float mean = cnt > 0.f ? sum / cnt : 0.f;
+                    float m2 = 0.f;
+#pragma unroll 1
+                    for (int q = 0; q < 4; ++q) {
+                      const int col = (cg + 8 * q) * 4;
+                      if (row_on && col < ncols) {
+                        const float4 x4 = *reinterpret_cast<const float4*>(vrow + col);
+                        const float d0 = x4.x - mean, d1 = x4.y - mean, d2 = x4.z - mean, d3 = x4.w - mean;
                         m2 += (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
                       }
                     }
-                    // merge the eight threads of the row, pairwise and symmetrically
 #pragma unroll
-                    for (int o = 1; o < 8; o <<= 1) {
-                      const float c2 = __shfl_xor_sync(0xffffffffu, cnt, o), mean2 = __shfl_xor_sync(0xffffffffu, mean, o),
-                                  m22 = __shfl_xor_sync(0xffffffffu, m2, o);
-                      const float tot = cnt + c2;
-                      if (tot > 0.f) {
-                        const float delta = mean2 - mean;
-                        const float mm = (cnt * mean + c2 * mean2) / tot;
-                        m2 = m2 + m22 + delta * delta * cnt * c2 / tot;
-                        mean = mm; cnt = tot;
-                      }
-                    }
+                    for (int o = 1; o < 8; o <<= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
                     if (cg == 0 && row_on) P.stats[(size_t)t * P.stat_tiles + tile] = make_float4(mean, m2, cnt, 0.f);
                   }
                 } else if (p.epi == TC_SWIGLU) {
-#pragma unroll
+                  // gate columns (cg + 8 q) * 4 of the tile's first half, the matching up columns 64 further
+#pragma unroll 1
                   for (int q = 0; q < 2; ++q) {
-                    if (on[q]) {
-                      const float4 g4 = a[q], u4 = a[q + 2];
-                      store_split4(out_act, (size_t)t * p.ldo + n0 + (cg + 8 * q) * 4, (size_t)P.lo_row * p.ldo,
+                    const int col = (cg + 8 * q) * 4;
+                    if (row_on && col < ncols) {
+                      const float4 g4 = group(col), u4 = group(col + 64);
+                      store_split4(out_act, (size_t)t * p.ldo + n0 + col, (size_t)P.lo_row * p.ldo,
                                    make_float4(silu_f(g4.x) * u4.x, silu_f(g4.y) * u4.y, silu_f(g4.z) * u4.z, silu_f(g4.w) * u4.w));
                     }
                   }
@@ -1953,10 +1970,11 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
                   // logits (optional) and the row's running argmax; the vocabulary need not be a
                   // multiple of 4, so validity and stores are per element
                   unsigned long long key = 0ull;
-#pragma unroll
+#pragma unroll 1
                   for (int q = 0; q < 4; ++q) {
                     const int col = (cg + 8 * q) * 4;
-                    const float e4[4] = {a[q].x, a[q].y, a[q].z, a[q].w};
+                    const float4 v4 = group(col);
+                    const float e4[4] = {v4.x, v4.y, v4.z, v4.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                       if (row_on && col + e < ncols) {
@@ -1975,42 +1993,42 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
                 } else if (p.qkv_prep) {
                   // q: rotate, scale by 1/sqrt(hd), fp16, to the query buffer; k: rotate, fp16, to
                   // its row of the cache; v: fp16 to the cache.  The rotation pairs column i with
-                  // i + hd/2 of a head; with hd = 128 (a tile is one head) or 64 (two heads) both
-                  // columns of a pair belong to the same thread.
+                  // i + hd/2 of a head; with hd = 128 (a tile is one head: groups 0 and 2, 1 and 3) or
+                  // 64 (two heads: groups 0 and 1, 2 and 3) both columns of a pair belong to the same thread.
                   int kv_row = kv_row0;
                   float4 rca = rc0a, rcb = rc0b, rsa = rs0a, rsb = rs0b;
                   if (c0 != 0 && row_on) {
                     if (src_s >= 1) kv_row = kv_row_of(t);
                     if (P.rope && src_s < 2) rope_of(t, rca, rsa, rcb, rsb);
                   }
-                  if (P.rope && src_s < 2) {
-                    auto rot = [](float4& lo, float4& hi, const float4& cs, const float4& sn) {
+                  const float qscale = src_s == 0 ? 1.4426950408889634f / sqrtf((float)P.hd) : 1.0f;   // log2(e) / sqrt(hd): the softmax works in base 2
+                  const int nq_all = P.Hq * P.hd, nkv_all = P.Hkv * P.hd;
+                  __half* dst = (src_s == 0 ? P.q16 + (size_t)t * nq_all
+                                            : reinterpret_cast<__half*>(src_s == 1 ? p.kc : p.vc) + (size_t)kv_row * nkv_all) + (n0 - src_col0);
+#pragma unroll 1
+                  for (int pi = 0; pi < 2; ++pi) {
+                    const int col_lo = (P.hd == 128 ? cg + 8 * pi : cg + 16 * pi) * 4, col_hi = col_lo + (P.hd == 128 ? 64 : 32);
+                    float4 lo = group(col_lo), hi = group(col_hi);
+                    if (P.rope && src_s < 2) {
+                      const float4 cs = pi ? rcb : rca, sn = pi ? rsb : rsa;
                       const float4 l = lo, h = hi;
                       lo = make_float4(l.x * cs.x - h.x * sn.x, l.y * cs.y - h.y * sn.y, l.z * cs.z - h.z * sn.z, l.w * cs.w - h.w * sn.w);
                       hi = make_float4(h.x * cs.x + l.x * sn.x, h.y * cs.y + l.y * sn.y, h.z * cs.z + l.z * sn.z, h.w * cs.w + l.w * sn.w);
-                    };
-                    if (P.hd == 128) { rot(a[0], a[2], rca, rsa); rot(a[1], a[3], rcb, rsb); }
-                    else { rot(a[0], a[1], rca, rsa); rot(a[2], a[3], rcb, rsb); }
-                  }
-                  const float qscale = src_s == 0 ? 1.4426950408889634f / sqrtf((float)P.hd) : 1.0f;   // log2(e) / sqrt(hd): the softmax works in base 2
-                  const int nq_all = P.Hq * P.hd, nkv_all = P.Hkv * P.hd;
-                  __half* dst = src_s == 0 ? P.q16 + (size_t)t * nq_all
-                                           : reinterpret_cast<__half*>(src_s == 1 ? p.kc : p.vc) + (size_t)kv_row * nkv_all;
-                  const int colsrc0 = n0 - src_col0;
-#pragma unroll
-                  for (int q = 0; q < 4; ++q) {
-                    if (on[q])
-                      *reinterpret_cast<uint2*>(dst + colsrc0 + (cg + 8 * q) * 4) =
-                          make_uint2(pack_f16x2(a[q].x * qscale, a[q].y * qscale), pack_f16x2(a[q].z * qscale, a[q].w * qscale));
+                    }
+                    if (row_on && col_lo < ncols)
+                      *reinterpret_cast<uint2*>(dst + col_lo) = make_uint2(pack_f16x2(lo.x * qscale, lo.y * qscale), pack_f16x2(lo.z * qscale, lo.w * qscale));
+                    if (row_on && col_hi < ncols)
+                      *reinterpret_cast<uint2*>(dst + col_hi) = make_uint2(pack_f16x2(hi.x * qscale, hi.y * qscale), pack_f16x2(hi.z * qscale, hi.w * qscale));
                   }
                 } else {
-#pragma unroll
+#pragma unroll 1
                   for (int q = 0; q < 4; ++q) {
-                    if (on[q]) {
-                      const size_t o = (size_t)t * p.ldo + n0 + (cg + 8 * q) * 4;
-                      if (p.epi == TC_STORE_F32) *reinterpret_cast<float4*>(out_f32 + o) = a[q];
-                      else store_split4(out_act, o, (size_t)P.lo_row * p.ldo,
-                                        make_float4(gelu_erf(a[q].x), gelu_erf(a[q].y), gelu_erf(a[q].z), gelu_erf(a[q].w)));
+                    const int col = (cg + 8 * q) * 4;
+                    if (row_on && col < ncols) {
+                      const float4 v4 = group(col);
+                      const size_t o = (size_t)t * p.ldo + n0 + col;
+                      if (p.epi == TC_STORE_F32) *reinterpret_cast<float4*>(out_f32 + o) = v4;
+                      else store_split4(out_act, o, (size_t)P.lo_row * p.ldo, make_float4(gelu_erf(v4.x), gelu_erf(v4.y), gelu_erf(v4.z), gelu_erf(v4.w)));
                     }
                   }
                 }
