@@ -62,7 +62,7 @@ struct DevModel {
 
 struct Layout {
   size_t status, seq, n_seq, page_table, tok, pos, req, val_req, val_k, val_off, keys, x, h, qkv, q,
-      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_flags, mk_bar, attn_part, prog_t, prog_d, mk_trace, mk_stats, rope_t, rope_d, aux_t, aux_d, w13_t, w13_d, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
+      o, ff, logits, draft_buf, tt_buf, al_buf, gemm_partial, gemm_counters, mk_partial, mk_partial_bytes, mk_bar, attn_part, prog_t, prog_d, mk_trace, mk_stats, rope_t, rope_d, aux_t, aux_d, w13_t, w13_d, kv_t_k, kv_t_v, kv_d_k, kv_d_v, total;
   int max_rows, logit_rows, max_pages, n_pages, t_box_max, attn_units, stat_tiles;
   size_t prog_slot_t, prog_slot_d, prog_maps_off_t, prog_maps_off_d;
   size_t kv_t_layer, kv_d_layer;
@@ -220,7 +220,10 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
   L->al_buf = take((size_t)c.max_requests * 4);
   L->gemm_partial = take(t.wdtype == 1 ? (size_t)TC_GRID_MAX * 2 * L->t_box_max * tc::BM * 4 : 0);
   L->gemm_counters = take(t.wdtype == 1 ? (size_t)TC_COUNTERS * 4 : 0);
-  L->mk_flags = take(t.wdtype == 1 ? (size_t)TC_GRID_MAX * 8 : 0);   // split-tile flags of the persistent kernel
+  // split-tile partial sums of the persistent kernel: two sets (alternate GEMM phases) of one slot per CTA;
+  // every element holds the "empty" pattern between uses
+  L->mk_partial_bytes = t.wdtype == 1 ? (size_t)2 * TC_GRID_MAX * L->t_box_max * tc::BM * 4 : 0;
+  L->mk_partial = take(L->mk_partial_bytes);
   {
     // persistent-kernel scratch: attention unit states and the per-(model, row box) programs
     const int hkv = mx(t.n_kv_heads, d.n_kv_heads), hdm = mx(t.head_dim, d.head_dim);
@@ -793,8 +796,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.keys = reinterpret_cast<unsigned long long*>(ws + L.keys); P.n_keys = L.max_rows;
   P.logits = c.logits;
   P.target_tokens = c.target_tokens; P.accept_len = c.accept_len; P.commit = c.commit; P.draft_out = c.draft_out;
-  P.partial = reinterpret_cast<float*>(ws + L.gemm_partial); P.counters = reinterpret_cast<int*>(ws + L.gemm_counters);
-  P.seg_flags = reinterpret_cast<unsigned long long*>(ws + L.mk_flags);
+  P.partial = reinterpret_cast<float*>(ws + L.mk_partial); P.counters = reinterpret_cast<int*>(ws + L.gemm_counters);
   P.attn_part = reinterpret_cast<float*>(ws + L.attn_part); P.attn_part_units = (int)units_avail;
   P.stats = reinterpret_cast<float4*>(ws + L.mk_stats); P.stat_tiles = L.stat_tiles;
   P.rope_inv = M.rope_inv; P.rope_cs = M.rope_inv + m.head_dim / 2; P.rope_sn = P.rope_cs + 64 * (m.head_dim / 2);
@@ -1080,6 +1082,7 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
   if (e == cudaSuccess && L.total > L.kv_t_k) e = cudaMemsetAsync(ctx->ws + L.kv_t_k, 0, L.total - L.kv_t_k, ctx->stream);
   if (e == cudaSuccess && L.kv_t_k > L.gemm_counters)  // split-tile counters start at zero and return to zero
     e = cudaMemsetAsync(ctx->ws + L.gemm_counters, 0, L.w13_t - L.gemm_counters, ctx->stream);
+  if (e == cudaSuccess && L.mk_partial_bytes) e = cudaMemsetAsync(ctx->ws + L.mk_partial, 0xff, L.mk_partial_bytes, ctx->stream);   // all slots empty
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
   if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_begin);
   if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_end);
@@ -1465,11 +1468,11 @@ int stairs_sync(stairs_ctx* ctx) {
     for (int i = 1; i <= 5; ++i) ctx->status_host[i] = 0;
     cudaMemsetAsync(ctx->ws + ctx->lay.mk_bar, 0, 64, ctx->stream);   // barrier count and abort word
     cudaMemsetAsync(ctx->ws + ctx->lay.gemm_counters, 0, (size_t)TC_COUNTERS * 4, ctx->stream);
-    cudaMemsetAsync(ctx->ws + ctx->lay.mk_flags, 0, (size_t)TC_GRID_MAX * 8, ctx->stream);   // tags restart with the barrier count
+    if (ctx->lay.mk_partial_bytes) cudaMemsetAsync(ctx->ws + ctx->lay.mk_partial, 0xff, ctx->lay.mk_partial_bytes, ctx->stream);   // all partial-sum slots empty again
     cudaStreamSynchronize(ctx->stream);
     ctx->bar_base = 0;
     // kind: 1 shared-memory barrier (block, thread, parity), 2 grid barrier (block, thread, target),
-    // 3 split-tile flags (phase, block, last block of the tile, tile)
+    // 3 split-tile partial sums (phase, block, last block of the tile, tile)
     // 4 attention-scratch guard (unit slot, slots available, request, unit)
     return fail(ctx, (int)code, "%s (code %u; first: kind %u at %u, %u, %u, %u); results of the last calls are invalid",
                 where[0] == 4u ? "the device-side attention scratch was too small for a call" : "a device-side bounded wait expired",

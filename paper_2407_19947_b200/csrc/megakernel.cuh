@@ -121,7 +121,6 @@ struct Params {
   float* logits;            // optional dump
   int* target_tokens; int* accept_len; int commit; int* draft_out;
   // scratch
-  unsigned long long* seg_flags;   // one flag per CTA: the tag of the phase whose partial its slot holds
   float* partial; int* counters;
   float* attn_part;         // [units][QBLK][hd + 4]: O, running max, running sum, pad
   int attn_part_units;
@@ -204,6 +203,21 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 }
 __device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+// Split-tile partial sums travel without a flag: a slot element holds PARTIAL_EMPTY (a NaN pattern that
+// arithmetic never produces - the hardware's NaN is 0x7fffffff) until its producer stores the sum, the
+// consumer polls the elements it needs and puts the pattern back.  Element-wise relaxed accesses at GPU scope.
+constexpr uint32_t PARTIAL_EMPTY = 0xffffffffu;
+__device__ __forceinline__ void st_relaxed_f32(float* p, float v) {
+  asm volatile("st.relaxed.gpu.global.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
+}
+__device__ __forceinline__ uint4 ld_relaxed_u4(const float* p) {
+  uint4 v;
+  asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_relaxed_u4(float* p, uint4 v) {
+  asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 __device__ __forceinline__ void red_release_add_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
@@ -1456,6 +1470,23 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
       if (et == 0) { __threadfence_block(); ctl->areq_ready = 1; }
     }
     KvCons kvc{0, 0u, 0u, 0u};
+    // Split-tile partial sums: two sets of slots, used by alternate GEMM phases; the slots a finisher
+    // has read are emptied again one GEMM phase later (or at the end of the kernel), while it waits
+    // for that phase's accumulator - off the chain that ends a phase, and before the set's next use.
+    int gph = 0;                               // GEMM phases so far
+    unsigned pend_first = 1u, pend_last = 0u;  // slots (CTAs) read and not yet emptied
+    int pend_set = 0;
+    auto slot_of = [&](int set, unsigned c) { return P.partial + ((size_t)set * G + c) * P.t_box * BM; };
+    auto empty_pending = [&]() {
+      const int er_ = et >> 3, cg_ = et & 7;
+      for (unsigned c = pend_first; c <= pend_last; ++c)
+        for (int t = er_; t < P.T; t += 16) {
+          float* row = slot_of(pend_set, c) + (size_t)t * BM;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) st_relaxed_u4(row + (cg_ + 8 * q) * 4, make_uint4(PARTIAL_EMPTY, PARTIAL_EMPTY, PARTIAL_EMPTY, PARTIAL_EMPTY));
+        }
+      pend_first = 1u; pend_last = 0u;
+    };
     for (int ph = 0; ph < P.n_phases && ok; ++ph) {
       const Phase& p = *reinterpret_cast<const Phase*>(ctl->phc[ph & 1]);
       // the next phase's descriptor: fetched now, parked in shared memory at the end of this phase
@@ -1632,6 +1663,8 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
         }
       } else {
         // ---------------------------------------------------------------- GEMM epilogue
+        empty_pending();
+        const int pset = gph & 1;
         const KRange kr = phase_range(p.n_tiles, p.upt, p.kblocks, RANGE_UNIT_KB / kps, cta, G, p.ge_max);
         const int kb_begin = kr.begin, kb_end = kr.end;
         const int Ge = kr.ge;
@@ -1702,7 +1735,6 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
         if (tracing) tr[3] = globaltimer_ns();
         bool first_seg = true;
         int kb = kb_begin;
-        const unsigned long long seg_tag = P.bar_base + (unsigned long long)ph + 1ull;   // unique per launch and phase
         const unsigned tot32 = (unsigned)(p.n_tiles * p.upt), ge32 = (unsigned)Ge;
         // first stage of CTA c's range (units * Ge < 2^32, checked on the host)
         auto rb = [&](unsigned c) { return (unsigned)unit_to_stage((tot32 * c) / ge32, p.upt, p.kblocks, RANGE_UNIT_KB / kps); };
@@ -1788,7 +1820,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
           unsigned long long* tra = (MK_TRACE_PTR(P.trace) && et == 0 && !whole) ? MK_TRACE_PTR(P.trace) + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
           if (!finisher) {
             if (tra) tra[4] = globaltimer_ns();
-            float* mine = P.partial + (size_t)cta * P.t_box * BM;
+            float* mine = slot_of(pset, (unsigned)cta);
             for (int c0 = 0; c0 < Tvalid; c0 += 16) {   // only rows that exist
               float v[16];
               tmem_ld16(taddr + (uint32_t)c0, v);
@@ -1800,17 +1832,16 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
               }
               const int jn = min(16, Tvalid - c0);
 #pragma unroll
-              for (int j = 0; j < 16; ++j) if (j < jn) mine[(size_t)(c0 + j) * BM + m] = v[j];
+              for (int j = 0; j < 16; ++j) if (j < jn) st_relaxed_f32(mine + (size_t)(c0 + j) * BM + m, v[j]);
             }
+            // (no flag and no fence: the finisher polls the values themselves)
             tc_fence_before();
             if (lane == 0) mbar_arrive(ctl->acc_empty + buf);
-            epi_bar_sync();
-            // release: cumulative over the group's stores, which the barrier ordered before it
-            if (et == 0) st_release_u64(P.seg_flags + cta, seg_tag);
             if (tra) tra[5] = globaltimer_ns();
           } else {
             unsigned last_c = (unsigned)cta;   // CTAs cta + 1 .. last_c hold the tile's other segments
             if (!whole) while (last_c + 1 < ge32 && rb(last_c + 1) < (unsigned)tile_end) ++last_c;
+            if (!whole) { pend_first = (unsigned)cta + 1u; pend_last = last_c; pend_set = pset; }   // (at most one split tile is finished per phase)
             for (int c0 = 0; c0 < Tvalid; c0 += 16) {
               {
                 float v[16];
@@ -1828,31 +1859,9 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 16; ++j) vt[j * VT_LD + m] = v[j];
               }
-              if (!whole && c0 == 0) {
-                if (tra) tra[1] = globaltimer_ns();
-                if (et < 32) {
-                  // one lane per other segment: wait (bounded) until its flag carries this phase's tag
-                  const long long t0 = clock64();
-                  bool all_set;
-                  do {
-                    bool mine_set = true;
-                    for (unsigned cc = (unsigned)cta + 1 + (unsigned)lane; cc <= last_c; cc += 32)
-                      if (ld_acquire_u64(P.seg_flags + cc) != seg_tag) mine_set = false;
-                    all_set = __all_sync(0xffffffffu, mine_set);
-                    if (!all_set) {
-                      bool give_up = false;
-                      if (lane == 0) give_up = W.poll_abort(t0);
-                      if (__shfl_sync(0xffffffffu, give_up ? 1 : 0, 0)) break;
-                    }
-                  } while (!all_set);
-                  if (lane == 0 && !all_set) { ctl->abort_flag = 1; W.note(3u, (unsigned)ph, (unsigned)cta, last_c, (unsigned)tile); }
-                }
-                ok = group_ok(ctl, et);   // also orders the other threads' partial reads after the acquires
-                if (tra) tra[2] = globaltimer_ns();
-              } else {
-                epi_bar_sync();
-              }
-              if (ok) {
+              epi_bar_sync();   // the exchange tile is complete
+              if (tra && !whole && c0 == 0) tra[1] = globaltimer_ns();
+              {
                 // Each phase runs this code once per tile, so its instruction fetch is what it costs:
                 // the loads that must be in flight together are unrolled, everything per column group
                 // is a rolled loop over the four groups of the thread (the sums wait in the exchange tile).
@@ -1870,24 +1879,43 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
                     a[q] = on[q] ? *reinterpret_cast<const float4*>(vrow + col) : make_float4(0.f, 0.f, 0.f, 0.f);
                   }
                   if (!whole) {
-                    // the other segments' partial sums: six segments' loads in flight together, the
-                    // additions in k order
+                    // The other segments' partial sums, six segments' loads in flight together, added in k
+                    // order.  A slot element reads PARTIAL_EMPTY until its producer has stored the sum: when
+                    // one does, the thread waits on a single element (little traffic while others still
+                    // stream weights) and then looks at all of them again.  All waits are bounded.
                     for (unsigned c = (unsigned)cta + 1; c <= last_c; c += 6) {
-                      float4 tmp[6][4];
+                      uint4 tmp[6][4];
+                      const float* probe = slot_of(pset, min(c + 5, last_c)) + (size_t)(row_on ? t : 0) * BM + cg * 4;
+                      long long t0 = 0;
+                      bool timing = false, give_up = false;
+                      while (true) {
+                        uint32_t mx = 0u;
 #pragma unroll
-                      for (int u = 0; u < 6; ++u) {
-                        const float* part = P.partial + ((size_t)min(c + u, last_c) * P.t_box + (row_on ? t : 0)) * BM;
+                        for (int u = 0; u < 6; ++u) {
+                          const float* part = slot_of(pset, min(c + u, last_c)) + (size_t)(row_on ? t : 0) * BM;
 #pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                          tmp[u][q] = (on[q] && c + u <= last_c) ? __ldcg(reinterpret_cast<const float4*>(part + (cg + 8 * q) * 4))
-                                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+                          for (int q = 0; q < 4; ++q) {
+                            tmp[u][q] = (on[q] && c + u <= last_c) ? ld_relaxed_u4(part + (cg + 8 * q) * 4) : make_uint4(0u, 0u, 0u, 0u);
+                            mx = max(max(mx, max(tmp[u][q].x, tmp[u][q].y)), max(tmp[u][q].z, tmp[u][q].w));
+                          }
+                        }
+                        if (mx != PARTIAL_EMPTY || give_up) break;
+                        do {
+                          if (!timing) { t0 = clock64(); timing = true; }
+                          if (W.poll_abort(t0)) { W.note(3u, (unsigned)ph, (unsigned)cta, last_c, (unsigned)tile); give_up = true; break; }   // (the verdict follows the chunk's last barrier)
+                          __nanosleep(32);
+                        } while (ld_relaxed_u4(probe).x == PARTIAL_EMPTY);
                       }
 #pragma unroll
                       for (int u = 0; u < 6; ++u) {
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) { a[q].x += tmp[u][q].x; a[q].y += tmp[u][q].y; a[q].z += tmp[u][q].z; a[q].w += tmp[u][q].w; }
+                        for (int q = 0; q < 4; ++q) {
+                          a[q].x += __uint_as_float(tmp[u][q].x); a[q].y += __uint_as_float(tmp[u][q].y);
+                          a[q].z += __uint_as_float(tmp[u][q].z); a[q].w += __uint_as_float(tmp[u][q].w);
+                        }
                       }
                     }
+                    if (tra && c0 == 0) tra[2] = globaltimer_ns();
                   }
                   if (tra) {
                     asm volatile("" ::"f"(a[0].x), "f"(a[0].w), "f"(a[1].x), "f"(a[1].w), "f"(a[2].x), "f"(a[2].w), "f"(a[3].x), "f"(a[3].w));
@@ -2033,7 +2061,11 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
                   }
                 }
               }
-              epi_bar_sync();   // the exchange tile is reused by the next chunk
+              // one verdict for the 128 threads (a poll above may have run out in some of them; one that
+              // thread 0 misses here is seen at the next verdict or at the end of the kernel)
+              if (et == 0) ctl->bcast = ctl->abort_flag ? 0 : 1;
+              epi_bar_sync();   // (the exchange tile is reused by the next chunk)
+              ok = ctl->bcast != 0;
               if (!ok) break;
             }
             if (tra) tra[3] = globaltimer_ns();
@@ -2070,7 +2102,9 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
       if (et == 0) red_release_add_u64(P.bar, 1ull);
       if (tracing) tr[2] = globaltimer_ns();
       waited = false;
+      if (p.kind == PH_GEMM) ++gph;
     }
+    if (ok) empty_pending();   // (after an abort the host empties every slot)
   }
 
   // ================================================================== teardown
