@@ -237,7 +237,7 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     // (the tcgen05 attention path has fewer units of 128 query rows each: sized for whichever is larger)
     const int units_tc = std::max(c.max_requests * attn_unit_bound(hkv, gq, rows_req, mk::ATT_QBLK_TC), attn_unit_bound(hkv, gq, MK_MAX_ROWS, mk::ATT_QBLK_TC));
     L->attn_part_bytes = std::max((size_t)L->attn_units * mk::ATT_QBLK, (size_t)units_tc * mk::ATT_QBLK_TC) * (hdm + 4) * 4;
-    L->attn_part = take(t.wdtype == 1 ? L->attn_part_bytes : 0);
+    L->attn_part = take(t.wdtype == 1 ? 2 * L->attn_part_bytes : 0);   // two sets (alternate attention phases), every word "empty" between uses
     auto prog = [&](const stairs_model& m, size_t* maps_off) {
       const size_t ph = align_up((size_t)(8 * std::max(m.n_layers, 1) + 4) * sizeof(mk::Phase), 128);
       *maps_off = ph;
@@ -675,7 +675,6 @@ int build_program(stairs_ctx* ctx, DevModel& M, int t_box, int kps) {
     if (!in_epilogue) simple(mk::PH_PREP, l, nullptr, M.kpool + (size_t)l * M.kv_layer_bytes, M.vpool + (size_t)l * M.kv_layer_bytes);
     simple(mk::PH_ATTN, l, nullptr, M.kpool + (size_t)l * M.kv_layer_bytes, M.vpool + (size_t)l * M.kv_layer_bytes);
     ph.back().w_map[0] = i_kv + 2 * l; ph.back().w_map[1] = i_kv + 2 * l + 1;   // the layer's K and V pool maps
-    simple(mk::PH_COMBINE, l, nullptr, nullptr, nullptr);
     const int rd[1] = {d};
     {
       mk::Phase& p = gemm(l, b + 3, b + 3, b + 3, 1, rd, false, i_o, nq, tc::TC_ADD_F32, ws + L.x, d);
@@ -798,6 +797,7 @@ int launch_forward_mk(stairs_ctx* ctx, DevModel& M, int T, int logit_first_row, 
   P.target_tokens = c.target_tokens; P.accept_len = c.accept_len; P.commit = c.commit; P.draft_out = c.draft_out;
   P.partial = reinterpret_cast<float*>(ws + L.mk_partial); P.counters = reinterpret_cast<int*>(ws + L.gemm_counters);
   P.attn_part = reinterpret_cast<float*>(ws + L.attn_part); P.attn_part_units = (int)units_avail;
+  P.attn_set_stride = L.attn_part_bytes / 4;
   P.stats = reinterpret_cast<float4*>(ws + L.mk_stats); P.stat_tiles = L.stat_tiles;
   P.rope_inv = M.rope_inv; P.rope_cs = M.rope_inv + m.head_dim / 2; P.rope_sn = P.rope_cs + 64 * (m.head_dim / 2);
   P.bar = reinterpret_cast<unsigned long long*>(ws + L.mk_bar); P.bar_base = ctx->bar_base;
@@ -1083,6 +1083,7 @@ int stairs_init(const stairs_config* cfg, const stairs_weights* target, const st
   if (e == cudaSuccess && L.kv_t_k > L.gemm_counters)  // split-tile counters start at zero and return to zero
     e = cudaMemsetAsync(ctx->ws + L.gemm_counters, 0, L.w13_t - L.gemm_counters, ctx->stream);
   if (e == cudaSuccess && L.mk_partial_bytes) e = cudaMemsetAsync(ctx->ws + L.mk_partial, 0xff, L.mk_partial_bytes, ctx->stream);   // all slots empty
+  if (e == cudaSuccess && L.mk_partial_bytes) e = cudaMemsetAsync(ctx->ws + L.attn_part, 0xff, 2 * L.attn_part_bytes, ctx->stream);   // and all parked attention states
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
   if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_begin);
   if (e == cudaSuccess) e = cudaEventCreate(&ctx->call_end);
@@ -1469,11 +1470,12 @@ int stairs_sync(stairs_ctx* ctx) {
     cudaMemsetAsync(ctx->ws + ctx->lay.mk_bar, 0, 64, ctx->stream);   // barrier count and abort word
     cudaMemsetAsync(ctx->ws + ctx->lay.gemm_counters, 0, (size_t)TC_COUNTERS * 4, ctx->stream);
     if (ctx->lay.mk_partial_bytes) cudaMemsetAsync(ctx->ws + ctx->lay.mk_partial, 0xff, ctx->lay.mk_partial_bytes, ctx->stream);   // all partial-sum slots empty again
+    if (ctx->lay.mk_partial_bytes) cudaMemsetAsync(ctx->ws + ctx->lay.attn_part, 0xff, 2 * ctx->lay.attn_part_bytes, ctx->stream);
     cudaStreamSynchronize(ctx->stream);
     ctx->bar_base = 0;
     // kind: 1 shared-memory barrier (block, thread, parity), 2 grid barrier (block, thread, target),
     // 3 split-tile partial sums (phase, block, last block of the tile, tile)
-    // 4 attention-scratch guard (unit slot, slots available, request, unit)
+    // 4 attention-scratch guard (unit slot, slots available, request, unit), 5 parked attention states (phase, block)
     return fail(ctx, (int)code, "%s (code %u; first: kind %u at %u, %u, %u, %u); results of the last calls are invalid",
                 where[0] == 4u ? "the device-side attention scratch was too small for a call" : "a device-side bounded wait expired",
                 code, where[0], where[1], where[2], where[3], where[4]);

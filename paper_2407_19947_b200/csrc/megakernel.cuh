@@ -58,7 +58,7 @@ namespace mk {
 
 using namespace tc;
 
-enum PhaseKind { PH_EMBED = 0, PH_GEMM = 2, PH_ATTN = 3, PH_COMBINE = 4, PH_PREP = 5, PH_ACCEPT = 6 };
+enum PhaseKind { PH_EMBED = 0, PH_GEMM = 2, PH_ATTN = 3, PH_PREP = 5, PH_ACCEPT = 6 };
 
 struct Phase {
   int kind, layer;
@@ -122,8 +122,9 @@ struct Params {
   int* target_tokens; int* accept_len; int commit; int* draft_out;
   // scratch
   float* partial; int* counters;
-  float* attn_part;         // [units][QBLK][hd + 4]: O, running max, running sum, pad
+  float* attn_part;         // two sets of [units][QBLK][hd + 4]: O, running max, running sum, pad; every word PARTIAL_EMPTY between uses
   int attn_part_units;
+  size_t attn_set_stride;   // floats between the two sets of parked states (alternate attention phases)
   unsigned long long* bar;  // [0] arrivals (monotonic), [1] abort word
   unsigned long long bar_base;
   unsigned int* status; unsigned long long wait_limit;
@@ -214,6 +215,11 @@ __device__ __forceinline__ void st_relaxed_f32(float* p, float v) {
 __device__ __forceinline__ uint4 ld_relaxed_u4(const float* p) {
   uint4 v;
   asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint2 ld_relaxed_u2(const float* p) {
+  uint2 v;
+  asm volatile("ld.relaxed.gpu.global.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
   return v;
 }
 __device__ __forceinline__ void st_relaxed_u4(float* p, uint4 v) {
@@ -577,7 +583,7 @@ __device__ __forceinline__ uint8_t* att_ring_base(const Params& P, uint8_t* att_
 // the accumulator registers and V fetched with ldmatrix.trans; softmax state and output
 // accumulators never leave the warp's registers.  With one or two blocks the warps also split
 // each chunk's positions in two and merge once per unit.  The block's result is either final
-// (the unit saw every visible position) or parked for the combine phase.
+// (the unit saw every visible position) or parked for the merge at the end of the attention phase.
 //
 // K/V chunks of 64 positions reach shared memory in one of two ways.  TMA path (head sizes 64 and
 // 128): the loader warp streams them through a ring of buffers with tiled bulk copies (one box per
@@ -586,7 +592,7 @@ __device__ __forceinline__ uint8_t* att_ring_base(const Params& P, uint8_t* att_
 // Copy path (other head sizes): the compute threads stage padded tiles with 16-byte asynchronous
 // copies, cache rows looked up once per chunk.
 template <bool TMA>
-__device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot,
+__device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot, int part_set,
                           uint8_t* att_smem, Ctl* ctl, int et, bool& ok, KvCons& kvc, const Waiter& W,
                           unsigned long long* tra) {
   const int hd = P.hd, G = P.Hq / P.Hkv, nkv = P.Hkv * hd, nq = P.Hq * hd;
@@ -861,7 +867,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
   if (!active || part != 0) return;
 
   // write this warp's 16 rows straight from the accumulator fragments: the final output when the
-  // unit saw every visible position, else the state (O, max, sum) for the combine phase
+  // unit saw every visible position, else the state (O, max, sum) for the merge that ends the phase
   if (a.n_ranges == 1) {
     const float ia = l_a > 0.f ? 1.0f / l_a : 0.f, ib = l_b > 0.f ? 1.0f / l_b : 0.f;
 #pragma unroll
@@ -888,7 +894,7 @@ __device__ void attn_unit(const Params& P, const Phase& ph, const AttnReq& a, in
     for (int half_row = 0; half_row < 2; ++half_row) {
       const int ql = half_row ? ql_b : ql_a;
       if (ql < nQ) {
-        float* dst = P.attn_part + ((size_t)part_slot * P.att_qblk + ql) * (hd + 4);
+        float* dst = P.attn_part + (size_t)part_set * P.attn_set_stride + ((size_t)part_slot * P.att_qblk + ql) * (hd + 4);
 #pragma unroll
         for (int nd = 0; nd < 16; ++nd)
           if (nd < ntiles)
@@ -942,7 +948,7 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float* v) {
 // When a running maximum moves, the warp rescales its rows of O in TMEM (load, multiply, store) after
 // the previous P.V has completed and before it releases the P tile.  Rows past the unit's queries run
 // along on zero queries.  This function is the compute group's side.
-__device__ __noinline__ void attn_unit_tc(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot,
+__device__ __noinline__ void attn_unit_tc(const Params& P, const Phase& ph, const AttnReq& a, int kvh, int range, int qblk, int part_slot, int part_set,
                                           uint8_t* att_smem, Ctl* ctl, int et, bool& ok, KvCons& kvc, const Waiter& W,
                                           uint32_t tmem_s, uint32_t tmem_o) {
   const int hd = P.hd, G = P.Hq / P.Hkv, nq = P.Hq * hd, halves = hd / 64;
@@ -1076,11 +1082,11 @@ __device__ __noinline__ void attn_unit_tc(const Params& P, const Phase& ph, cons
   if (!ok) return;
   tc_fence_after();
   // this thread's row: the final output when the unit saw every visible position, else the state
-  // (O, max, sum) for the combine phase.  (All lanes take part in the TMEM loads.)
+  // (O, max, sum) for the merge that ends the phase.  (All lanes take part in the TMEM loads.)
   const int q = q0 + (mine ? ql : 0);
   const float inv = a.n_ranges == 1 ? (l_run > 0.f ? 1.0f / l_run : 0.f) : 1.0f;
   bf16* orow = P.o + (size_t)(a.off + q / G) * P.Hq * hd + (size_t)(kvh * G + q % G) * hd;
-  float* prow = P.attn_part + ((size_t)part_slot * P.att_qblk + (mine ? ql : 0)) * (hd + 4);
+  float* prow = P.attn_part + (size_t)part_set * P.attn_set_stride + ((size_t)part_slot * P.att_qblk + (mine ? ql : 0)) * (hd + 4);
   for (int d0 = 0; d0 < hd; d0 += 16) {
     float ov[16];
     tmem_ld16(tmem_o + lane_sel + (uint32_t)d0, ov);
@@ -1487,8 +1493,34 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
         }
       pend_first = 1u; pend_last = 0u;
     };
+    // Parked attention states: two sets, used by alternate attention phases.  The states are merged
+    // inside the attention phase itself (each warp polls the words it needs: no grid barrier in
+    // between); a CTA empties the slots of its own units one attention phase later, while it waits
+    // for that phase's inputs, and those of the last phase at the end of the kernel.
+    int aph = 0;   // attention phases so far
+    auto empty_own_states = [&](int set) {
+      const int n_req_ = P.mode == CALL_VALIDATE ? P.n_req : 1;
+      const int Gq_ = P.Hq / P.Hkv, row_words = P.hd + 4;
+      int u0_ = 0;
+      for (int i = 0; i < n_req_; ++i) {
+        const AttnReq a = ctl->areq[i];
+        if (a.n_ranges > 1) {
+          const int first = (cta - u0_ % G + G) % G;
+          for (int u = first; u < a.units; u += G) {
+            const int qblk = u % a.n_qblk;
+            const int nQ = min(P.att_qblk, a.R * Gq_ - qblk * P.att_qblk);
+            if (u0_ + u >= P.attn_part_units) break;
+            float* st = P.attn_part + (size_t)set * P.attn_set_stride + (size_t)(u0_ + u) * P.att_qblk * row_words;
+            for (int w4 = et; w4 < nQ * row_words / 4; w4 += 128)
+              st_relaxed_u4(st + w4 * 4, make_uint4(PARTIAL_EMPTY, PARTIAL_EMPTY, PARTIAL_EMPTY, PARTIAL_EMPTY));
+          }
+        }
+        u0_ += a.units;
+      }
+    };
     for (int ph = 0; ph < P.n_phases && ok; ++ph) {
       const Phase& p = *reinterpret_cast<const Phase*>(ctl->phc[ph & 1]);
+      if (p.kind == PH_ATTN && aph > 0) empty_own_states((aph & 1) ^ 1);   // (read by the previous attention phase, which every CTA has left)
       // the next phase's descriptor: fetched now, parked in shared memory at the end of this phase
       const uint32_t next_word = (et < PH_WORDS && ph + 1 < P.n_phases) ? __ldcg(reinterpret_cast<const uint32_t*>(P.phases + ph + 1) + et) : 0u;
       if (p.kind != PH_GEMM && !waited) {
@@ -1533,83 +1565,113 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
               break;
             }
             unsigned long long* tra_u = (MK_TRACE_PTR(P.trace) && et == 0 && u == first) ? MK_TRACE_PTR(P.trace) + (size_t)2 * P.n_phases * 8 + ((size_t)cta * P.n_phases + ph) * 8 : nullptr;
-            if (P.att_tc) attn_unit_tc(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok, kvc, W, tmem_base + tmem_att, tmem_base + tmem_att + 2 * ATT_CHUNK);
-            else if (P.att_tma) attn_unit<true>(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok, kvc, W, tra_u);
-            else attn_unit<false>(P, p, a, kvh, range, qblk, slot, att_smem, ctl, et, ok, kvc, W, tra_u);
+            if (P.att_tc) attn_unit_tc(P, p, a, kvh, range, qblk, slot, aph & 1, att_smem, ctl, et, ok, kvc, W, tmem_base + tmem_att, tmem_base + tmem_att + 2 * ATT_CHUNK);
+            else if (P.att_tma) attn_unit<true>(P, p, a, kvh, range, qblk, slot, aph & 1, att_smem, ctl, et, ok, kvc, W, tra_u);
+            else attn_unit<false>(P, p, a, kvh, range, qblk, slot, aph & 1, att_smem, ctl, et, ok, kvc, W, tra_u);
           }
           u0 += a.units; g0 += P.Hkv * a.n_qblk;
         }
-      } else if (p.kind == PH_COMBINE) {
         // Requests whose positions were split over several units: merge the parked states of every
         // (kv head, query) in position order.  One warp per item; each lane owns 4 consecutive
-        // elements of head_dim, so every partial is one 16-byte load per lane.
-        const int n_req = P.mode == CALL_VALIDATE ? P.n_req : 1;
-        const int hd = P.hd, Gq = P.Hq / P.Hkv;
-        int u0 = 0, item0 = 0;
-        for (int i = 0; i < n_req; ++i) {
-          const AttnReq a = ctl->areq[i];
-          if (a.n_ranges > 1) {
-            const int Q = a.R * Gq, items = P.Hkv * Q;
-            int it = ((cta * 4 + quad) - item0) % (G * 4);
-            if (it < 0) it += G * 4;
-            for (; it < items; it += G * 4) {
-              const int kvh = it / Q, q = it % Q, qblk = q / P.att_qblk, ql = q % P.att_qblk;
-              const int first_slot = u0 + (kvh * a.n_ranges) * a.n_qblk + qblk;
-              const size_t stride = (size_t)a.n_qblk * P.att_qblk * (hd + 4);
-              const float* base = P.attn_part + ((size_t)first_slot * P.att_qblk + ql) * (hd + 4);
-              // (max, sum) of range lane, lane + 32, ...: one load round for up to 32 ranges, then
-              // the ranges' output vectors eight loads at a time; weights travel by shuffle and
-              // the accumulation stays in range order
-              const int nr = a.n_ranges, dd = lane * 4;
-              float M = -INFINITY, m0 = -INFINITY, l0 = 0.f;
-              for (int rb = 0; rb < nr; rb += 32) {
-                const int r = rb + lane;
-                float mu = -INFINITY, lu = 0.f;
-                if (r < nr) { mu = __ldcg(base + r * stride + hd); lu = __ldcg(base + r * stride + hd + 1); }
-                if (rb == 0) { m0 = mu; l0 = lu; }
-                M = fmaxf(M, mu);
-              }
-              M = warp_max(M);
-              float L = 0.f;
-              float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-              for (int rb = 0; rb < nr; rb += 32) {
-                const int r = rb + lane;
-                float mu = m0, lu = l0;
-                if (rb != 0) {
+        // elements of head_dim, so every partial is one 16-byte load per lane.  The states come
+        // from other CTAs' units of this same phase: a word reads PARTIAL_EMPTY until it has been
+        // stored, and the warp repeats its loads (bounded) until none does.
+        if (ok) {
+          const int hd = P.hd, Gq = P.Hq / P.Hkv;
+          const float* set_base = P.attn_part + (size_t)(aph & 1) * P.attn_set_stride;
+          int u0c = 0, item0 = 0;
+          bool gave_up = false;
+          auto backoff = [&](long long& t0, bool& timing) {   // warp-uniform: true when the wait has run out
+            if (!timing) { t0 = clock64(); timing = true; }
+            bool quit = false;
+            if (lane == 0) quit = W.poll_abort(t0);
+            quit = __shfl_sync(0xffffffffu, quit ? 1 : 0, 0) != 0;
+            if (quit && lane == 0) W.note(5u, (unsigned)ph, (unsigned)cta, 0u, 0u);
+            if (!quit) __nanosleep(64);
+            return quit;
+          };
+          for (int i = 0; i < n_req; ++i) {
+            const AttnReq a = ctl->areq[i];
+            if (a.n_ranges > 1) {
+              const int Q = a.R * Gq, items = P.Hkv * Q;
+              int it = ((cta * 4 + quad) - item0) % (G * 4);
+              if (it < 0) it += G * 4;
+              for (; it < items && !gave_up; it += G * 4) {
+                const int kvh = it / Q, q = it % Q, qblk = q / P.att_qblk, ql = q % P.att_qblk;
+                const int first_slot = u0c + (kvh * a.n_ranges) * a.n_qblk + qblk;
+                const size_t stride = (size_t)a.n_qblk * P.att_qblk * (hd + 4);
+                const float* base = set_base + ((size_t)first_slot * P.att_qblk + ql) * (hd + 4);
+                // (max, sum) of range lane, lane + 32, ...: one load round for up to 32 ranges, then
+                // the ranges' output vectors eight loads at a time; weights travel by shuffle and
+                // the accumulation stays in range order
+                const int nr = a.n_ranges, dd = lane * 4;
+                long long t0 = 0;
+                bool timing = false;
+                auto state_of = [&](int r, float& mu, float& lu) {   // all lanes call it together
                   mu = -INFINITY; lu = 0.f;
-                  if (r < nr) { mu = __ldcg(base + r * stride + hd); lu = __ldcg(base + r * stride + hd + 1); }
+                  while (true) {
+                    uint2 v = make_uint2(0u, 0u);
+                    if (r < nr) v = ld_relaxed_u2(base + r * stride + hd);
+                    if (!__any_sync(0xffffffffu, v.x == PARTIAL_EMPTY || v.y == PARTIAL_EMPTY)) {
+                      if (r < nr) { mu = __uint_as_float(v.x); lu = __uint_as_float(v.y); }
+                      return;
+                    }
+                    if (backoff(t0, timing)) { gave_up = true; return; }
+                  }
+                };
+                float M = -INFINITY, m0 = -INFINITY, l0 = 0.f;
+                for (int rb = 0; rb < nr && !gave_up; rb += 32) {
+                  float mu, lu;
+                  state_of(rb + lane, mu, lu);
+                  if (rb == 0) { m0 = mu; l0 = lu; }
+                  M = fmaxf(M, mu);
                 }
-                const float wgt = mu == -INFINITY ? 0.f : fast_exp2(mu - M);   // 0 for lanes past the last range (maxima are base-2 exponents)
-                L += lu * wgt;
-                const int nb = min(32, nr - rb);
-                for (int g0 = 0; g0 < nb; g0 += 8) {
-                  float4 v[8];
+                M = warp_max(M);
+                float L = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int rb = 0; rb < nr && !gave_up; rb += 32) {
+                  float mu = m0, lu = l0;
+                  if (rb != 0) state_of(rb + lane, mu, lu);
+                  const float wgt = mu == -INFINITY ? 0.f : fast_exp2(mu - M);   // 0 for lanes past the last range (maxima are base-2 exponents)
+                  L += lu * wgt;
+                  const int nb = min(32, nr - rb);
+                  for (int g0 = 0; g0 < nb && !gave_up; g0 += 8) {
+                    uint4 v[8];
+                    while (true) {
+                      uint32_t mx = 0u;
 #pragma unroll
-                  for (int u = 0; u < 8; ++u)
-                    v[u] = (g0 + u < nb && dd < hd) ? __ldcg(reinterpret_cast<const float4*>(base + (size_t)(rb + g0 + u) * stride + dd))
-                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+                      for (int u = 0; u < 8; ++u) {
+                        v[u] = (g0 + u < nb && dd < hd) ? ld_relaxed_u4(base + (size_t)(rb + g0 + u) * stride + dd) : make_uint4(0u, 0u, 0u, 0u);
+                        mx = max(max(mx, max(v[u].x, v[u].y)), max(v[u].z, v[u].w));
+                      }
+                      if (!__any_sync(0xffffffffu, mx == PARTIAL_EMPTY)) break;
+                      if (backoff(t0, timing)) { gave_up = true; break; }
+                    }
 #pragma unroll
-                  for (int u = 0; u < 8; ++u) {
-                    const float wu = __shfl_sync(0xffffffffu, wgt, (g0 + u) & 31);
-                    acc.x += v[u].x * wu; acc.y += v[u].y * wu; acc.z += v[u].z * wu; acc.w += v[u].w * wu;
+                    for (int u = 0; u < 8; ++u) {
+                      const float wu = __shfl_sync(0xffffffffu, wgt, (g0 + u) & 31);
+                      acc.x += __uint_as_float(v[u].x) * wu; acc.y += __uint_as_float(v[u].y) * wu;
+                      acc.z += __uint_as_float(v[u].z) * wu; acc.w += __uint_as_float(v[u].w) * wu;
+                    }
                   }
                 }
+                L = warp_sum(L);
+                if (dd < hd) {
+                  bf16* orow = P.o + (size_t)(a.off + q / Gq) * P.Hq * hd + (size_t)(kvh * Gq + q % Gq) * hd + dd;
+                  const float inv = 1.0f / L;
+                  const __nv_bfloat162 h01 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), h23 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+                  *reinterpret_cast<uint2*>(orow) = make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
+                  *reinterpret_cast<uint2*>(orow + (size_t)P.lo_row * P.Hq * hd) =
+                      make_uint2(pack_bf16x2(acc.x * inv - __low2float(h01), acc.y * inv - __high2float(h01)),
+                                 pack_bf16x2(acc.z * inv - __low2float(h23), acc.w * inv - __high2float(h23)));
+                }
               }
-              L = warp_sum(L);
-              if (dd < hd) {
-                bf16* orow = P.o + (size_t)(a.off + q / Gq) * P.Hq * hd + (size_t)(kvh * Gq + q % Gq) * hd + dd;
-                const float inv = 1.0f / L;
-                const __nv_bfloat162 h01 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), h23 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-                *reinterpret_cast<uint2*>(orow) = make_uint2(*reinterpret_cast<const uint32_t*>(&h01), *reinterpret_cast<const uint32_t*>(&h23));
-                *reinterpret_cast<uint2*>(orow + (size_t)P.lo_row * P.Hq * hd) =
-                    make_uint2(pack_bf16x2(acc.x * inv - __low2float(h01), acc.y * inv - __high2float(h01)),
-                               pack_bf16x2(acc.z * inv - __low2float(h23), acc.w * inv - __high2float(h23)));
-              }
+              item0 += items;
             }
-            item0 += items;
+            u0c += a.units;
           }
-          u0 += a.units;
         }
+        ++aph;
       } else if (p.kind == PH_PREP) {
         // Models whose head size is neither 64 nor 128: a rotation pair (i, i + hd/2) need not sit in
         // one thread (or one tile) of the QKV epilogue, so that epilogue stores fp32 and this extra
@@ -2104,7 +2166,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
       waited = false;
       if (p.kind == PH_GEMM) ++gph;
     }
-    if (ok) empty_pending();   // (after an abort the host empties every slot)
+    if (ok) { empty_pending(); if (aph > 0) empty_own_states((aph - 1) & 1); }   // (after an abort the host empties every slot)
   }
 
   // ================================================================== teardown

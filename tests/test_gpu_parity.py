@@ -358,7 +358,7 @@ def test_tcgen05_attention_path_matches_oracle(hq, hkv, hd):
     # The attention contractions on the 5th-generation tensor cores are chosen per call for long
     # contexts and prefill passes; here they are switched on for every call, so that small models
     # reach them too: prefill passes of 64 rows (up to 256 queries per kv head: two query blocks),
-    # contexts split over several units (partial states merged by the combine phase) and not, two
+    # contexts split over several units (partial states merged by the merge at the end of the attention phase) and not, two
     # requests in one call, several draft lengths.  Same bars as everywhere.
     st = _stairs()
     shape = wl.family_b(2, hq * hd if hq * hd <= 512 else 512, hq, hkv, hd, 512, 2048, 1024)
