@@ -233,7 +233,7 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.global;" ::: "memory"); }   // (global memory is all these fences are about)
 // the same for this CTA's shared memory only (tiles written with plain stores, read by the tensor core)
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
@@ -1348,8 +1348,9 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
               umma_bf16(d_tmem, aj + (uint64_t)(k * UMMA_K * 2 / 16), bj + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
                         (seg_first && j == 0 && k == 0) ? 0u : 1u);
           }
-          umma_commit(ctl->empty + stage);
+          // (a commit costs about 240 cycles of issue time: the one the epilogue waits for goes first)
           if (seg_last) { umma_commit(ctl->acc_full + buf); acc_bits ^= 1u << buf; buf ^= 1; }
+          umma_commit(ctl->empty + stage);
 #ifdef STAIRS_TRACE
           if (trm) { klog[3 * kn + 2] = (unsigned long long)clock64(); ++kn; }
 #endif
@@ -1470,7 +1471,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
         uint8_t* first = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem) + 1023) & ~(uintptr_t)1023);   // (the Q and P tiles too)
         const int n16 = (int)((size_t)(ring - first) + (size_t)P.att_nbuf * AttnSmem::kv_buf_bytes(P.hd)) / 16;
         for (int i = et; i < n16; i += 128) reinterpret_cast<uint4*>(first)[i] = make_uint4(0u, 0u, 0u, 0u);
-        fence_proxy_async();   // later bulk copies (async proxy) into these buffers
+        fence_proxy_async_smem();   // later bulk copies (async proxy) into these buffers
       }
       epi_bar_sync();
       if (et == 0) { __threadfence_block(); ctl->areq_ready = 1; }
@@ -2150,7 +2151,13 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
       // barrier orders before it.  A CTA that had GEMM work in this phase already knows that
       // barrier ph-1 completed (its activation tiles were loaded after that), so only idle CTAs
       // look at the counter.
+#ifdef STAIRS_TRACE
+      if (tracing && cta != 0) tr[5] = globaltimer_ns();
+#endif
       fence_proxy_async();   // later TMA (async proxy) reads of these generic-proxy writes
+#ifdef STAIRS_TRACE
+      if (tracing && cta != 0) tr[6] = globaltimer_ns();
+#endif
       if (et < PH_WORDS) ctl->phc[(ph + 1) & 1][et] = next_word;   // (the barriers below publish it)
       if (ph > 0 && p.kind == PH_GEMM && !gemm_worked) {
         if (et == 0) ctl->bcast = W.wait_grid(bar_count, P.bar_base + (unsigned long long)ph * G) ? 1 : 0;
@@ -2161,6 +2168,9 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
       } else {
         epi_bar_sync();
       }
+#ifdef STAIRS_TRACE
+      if (tracing && cta != 0) tr[7] = globaltimer_ns();
+#endif
       if (et == 0) red_release_add_u64(P.bar, 1ull);
       if (tracing) tr[2] = globaltimer_ns();
       waited = false;
