@@ -1990,7 +1990,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
                     for (int q = 0; q < 4; ++q) {
                       if (on[q]) {
                         const size_t o = (size_t)t * p.ldo + n0 + (cg + 8 * q) * 4;
-                        const float4 x4 = c0 == 0 ? xq[q] : __ldcg(reinterpret_cast<const float4*>(out_f32 + o));
+                        const float4 x4 = xq[q];   // (requested before the accumulator was waited for, or during the previous chunk)
                         a[q] = make_float4(x4.x + a[q].x, x4.y + a[q].y, x4.z + a[q].z, x4.w + a[q].w);
                         *reinterpret_cast<float4*>(out_f32 + o) = a[q];
                       }
@@ -1999,6 +1999,16 @@ __global__ void __launch_bounds__(MK_THREADS, 1) k_forward(const __grid_constant
 #pragma unroll
                   for (int q = 0; q < 4; ++q)
                     if (on[q]) *reinterpret_cast<float4*>(vrow + (cg + 8 * q) * 4) = a[q];   // (this thread's own slots)
+                  if (add_res && c0 + 16 < Tvalid) {
+                    // calls of more than 16 rows: the next chunk's old residual values are requested now,
+                    // so that they do not add an L2 round trip to that chunk
+                    const int tn = t + 16;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                      const int col = (cg + 8 * q) * 4;
+                      xq[q] = (tn < Tvalid && col < ncols) ? __ldcg(reinterpret_cast<const float4*>(out_f32 + (size_t)tn * p.ldo + n0 + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                  }
                 }
                 // column group `col` of this thread's row, with the folded normalisation
                 // y = rstd_t * (acc - mean_t * u[n]) + c[n] where the GEMM has one
