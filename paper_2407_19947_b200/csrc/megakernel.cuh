@@ -12,13 +12,14 @@
 //
 // Roles per CTA (224 threads): warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner (GEMM phases, and
 // the attention phases' contractions on the tcgen05 path), warps 2-5 = "compute group": GEMM epilogues
-// and every non-GEMM phase (rows+embedding, attention softmax, combine, accept), warp 6 = K/V loader of
+// and every non-GEMM phase (rows+embedding, attention softmax and state merge, accept), warp 6 = K/V loader of
 // the attention phases.  A GEMM pipeline stage holds one or two 64-element k-blocks, fetched by ONE
 // 3-D bulk tensor copy per operand and freed by ONE commit (issue costs, not bandwidth, bound the
 // single-thread roles).  GEMM work is cut into contiguous ranges per CTA, in units of two k-blocks
 // whatever the stage depth, so results do not depend on the call's row count; a tile cut over
 // several CTAs is finished by the CTA that owns its first k-block, which adds the other CTAs' parked
-// partial tiles in k order once their flags are up.  Normalisation is folded into the GEMMs (operand
+// partial tiles in k order; no flags: a parked word reads as an "empty" pattern until it has been
+// stored, and the finisher polls the words it needs.  Normalisation is folded into the GEMMs (operand
 // x * gain, epilogue rescales by the row's 1/std from per-tile statistics).
 //
 // Attention (staircase mask over the paged cache): a unit is (request, kv head, range of 64-position
@@ -38,7 +39,7 @@
 // trip.  Phase descriptors and request geometry are therefore kept in shared memory, cursors in
 // scalar registers, and loads that feed a dependent chain are issued together.
 //
-// All waits (mbarriers, grid barrier, split-tile flags) are clock-bounded: on expiry the CTA
+// All waits (mbarriers, grid barrier, polls of parked sums and states) are clock-bounded: on expiry the CTA
 // raises an abort flag (shared memory) and a global abort word that every other CTA's waits poll,
 // so the whole grid drains, frees TMEM and exits with STAIRS_ETIMEOUT in the status word.
 #pragma once
