@@ -23,7 +23,8 @@ int stairs_profile_read(stairs_ctx *ctx, float *gemm_ms, int32_t *gemm_launches,
  * workspace after a pass (which: 0 residual x fp32 [rows, d], 1 normed h, 2 qkv fp32,
  * 3 attention output o, 4 MLP activation ff, 5 argmax keys u64, 6 per-phase timestamps of the
  * persistent kernel, u64 ns [2 CTAs][phases][8 stamps: start, work done, arrived, prologue done, first tile ready, first MMA, last MMA, first activation load], written while
- * profiling is on). */
+ * profiling is on; 7 the persistent kernel's split-tile partial-sum slots and 8 its parked attention
+ * states, both u32 words that all read 0xffffffff ("empty") between calls). */
 int stairs_debug_buffer(stairs_ctx *ctx, int which, void **ptr_dev, size_t *bytes);
 
 /* Tuning knobs of the persistent kernel, for sweeps.  what 0: 64-element k-blocks per pipeline

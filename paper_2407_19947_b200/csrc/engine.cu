@@ -1526,6 +1526,8 @@ int stairs_debug_buffer(stairs_ctx* ctx, int which, void** ptr_dev, size_t* byte
     case 4: *ptr_dev = ctx->ws + off[5]; *bytes = off[6] - off[5]; break;
     case 5: *ptr_dev = ctx->ws + L.keys; *bytes = keys_end - L.keys; break;
     case 6: *ptr_dev = ctx->ws + L.mk_trace; *bytes = L.mk_stats - L.mk_trace; break;
+    case 7: *ptr_dev = ctx->ws + L.mk_partial; *bytes = L.mk_partial_bytes; break;
+    case 8: *ptr_dev = ctx->ws + L.attn_part; *bytes = L.mk_partial_bytes ? 2 * L.attn_part_bytes : 0; break;
     default: return fail(ctx, STAIRS_EINVAL, "unknown buffer %d", which);
   }
   return STAIRS_OK;

@@ -1,4 +1,6 @@
 """Helpers shared by the GPU parity tests (oracle on the host, library on the device)."""
+import ctypes as C
+
 import numpy as np
 
 from oracle import stairs_oracle as so
@@ -43,3 +45,17 @@ def check_rows_against_oracle(gpu_logits, gpu_tokens, oracle_logits, tol):
         else:  # near-tie: the GPU's token must be within the margin of the oracle's best
             assert lg[int(gpu_tokens[r])] >= lg[best] - MARGIN
     return err, exact
+
+
+def assert_polled_scratch_empty(eng, tag):
+    """The persistent kernel's flagless hand-over buffers (split-tile sums, parked attention states):
+    every word must read 0xffffffff ("empty") between calls."""
+    import torch
+    eng.sync()
+    for which in (7, 8):
+        ptr, nbytes = C.c_void_p(), C.c_size_t()
+        eng._ck(eng.lib.stairs_debug_buffer(eng.h, which, C.byref(ptr), C.byref(nbytes)))
+        assert nbytes.value > 0
+        words = eng.debug_buffer(which, torch.int32, nbytes.value // 4)
+        bad = int((words != -1).sum())
+        assert bad == 0, f"{bad} words of scratch {which} are not empty after {tag}"

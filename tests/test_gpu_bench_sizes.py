@@ -74,6 +74,7 @@ def test_config2_full_depth_at_the_benchmarked_prefix():
     draft = wl.forced_draft(np.array(cont), 6, w.target.vocab, 3)
     err, exact, ref, gpu_tok = _validate_and_compare(eng, tgt, prompt, draft, 8)
     print(f"config 2, prefix 2048: logit max-abs err {err:.4f}, decisive rows {exact}/9")
+    gu.assert_polled_scratch_empty(eng, "the calls of this test")
     eng.close()
     tsrc.drop_cache(); dsrc.drop_cache()
 
@@ -92,6 +93,7 @@ def test_config3_shape_matches_oracle(layers, n_prompt, k):
     draft = d_dev.cpu().numpy()[:k]
     err, exact, _, _ = _validate_and_compare(eng, tgt, prompt, draft, k, check_row0=layers <= 4)
     print(f"config 3 shape, {layers} layers, prompt {n_prompt}: logit max-abs err {err:.4f}, decisive rows {exact}/{k + 1}")
+    gu.assert_polled_scratch_empty(eng, "the calls of this test")
     eng.close()
     tsrc.drop_cache(); dsrc.drop_cache()
 
@@ -114,6 +116,7 @@ def test_config4_shape_long_prompt_single_request_slot():
     g0, _ = eng.generate(0, prompt, 0, 12)
     g8, s8 = eng.generate(0, prompt, 8, 12)
     assert g0 == g8
+    gu.assert_polled_scratch_empty(eng, "the calls of this test")
     eng.close()
     tsrc.drop_cache(); dsrc.drop_cache()
 
@@ -146,6 +149,7 @@ def test_config4_full_depth_at_the_benchmarked_prompt():
         new_ctx = eng.sequence(0)
         assert new_ctx == ctx + [int(t) for t in draft[:acc]] + [int(gpu_tok[acc])]
         ctx = new_ctx
+    gu.assert_polled_scratch_empty(eng, "the calls of this test")
     eng.close()
     tsrc.drop_cache(); dsrc.drop_cache()
 
@@ -162,6 +166,7 @@ def test_config5_one_request_at_the_full_prefix_two_layers():
     draft = wl.uniform_tokens(8, w.target.vocab, 5)
     err, exact, _, _ = _validate_and_compare(eng, tgt, prompt, draft, 8, check_row0=False)
     print(f"config 5 shape, 2 layers, prefix 16384: logit max-abs err {err:.4f}, decisive rows {exact}/9")
+    gu.assert_polled_scratch_empty(eng, "the calls of this test")
     eng.close()
     tsrc.drop_cache()
 
@@ -180,6 +185,7 @@ def test_units_that_walk_several_chunks(n_prompt):
     cont = _own_continuation(eng, prompt, 9)
     draft = wl.forced_draft(np.array(cont), 5, shape.vocab, 9)
     _validate_and_compare(eng, tgt, prompt, draft, 8)
+    gu.assert_polled_scratch_empty(eng, "the calls of this test")
     eng.close()
 
 
@@ -230,6 +236,7 @@ def test_drafted_tokens_match_the_oracle_assistant(early_exit):
         eng.sync()
         decisive += _check_drafted_tokens(drf, ctx, d_dev.cpu().numpy()[:3])
     assert decisive >= 2     # random-init models are often undecided; the checks above hold either way
+    gu.assert_polled_scratch_empty(eng, "the calls of this test")
     eng.close()
 
 
@@ -244,5 +251,6 @@ def test_drafted_tokens_config4_shape_two_layer_draft():
     d_dev = eng.draft(0, 4)
     eng.sync()
     _check_drafted_tokens(drf, prompt, d_dev.cpu().numpy()[:4])
+    gu.assert_polled_scratch_empty(eng, "the calls of this test")
     eng.close()
     tsrc.drop_cache(); dsrc.drop_cache()

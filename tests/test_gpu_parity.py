@@ -325,6 +325,39 @@ def test_long_prefix_positions_split_over_several_units(shape):
     eng.close(); eng2.close()
 
 
+def test_polled_scratch_is_empty_again_after_every_kind_of_call():
+    # The persistent kernel hands split-tile sums and parked attention states over without flags:
+    # a word reads 0xffffffff until it has been stored, and whoever read it puts the pattern back.
+    # Whatever a call looked like (prefill passes of 64 rows, single draft rows, batched validate
+    # calls with split contexts, a context switch to other shapes), every word must read "empty"
+    # once the call is over - a leftover would be taken for a finished sum by a later call.
+    st = _stairs()
+    shape = small_b(8, 2, 64).replace(max_pos=512)
+    tsrc, dsrc = sources(shape)
+    eng = st.Stairs(tsrc, dsrc, max_requests=3, max_seq_len=400, k_max=8, kv_page_tokens=32)
+
+    def all_empty(tag):
+        gu.assert_polled_scratch_empty(eng, tag)
+
+    all_empty("init")
+    prompts = [list(wl.zipf_tokens(n, shape.vocab, 50 + i)) for i, n in enumerate((334, 70, 9))]
+    for i, p in enumerate(prompts):
+        eng.prefill(i, p)
+        all_empty(f"prefill of {len(p)} tokens")
+    d_dev = torch.from_numpy(np.random.default_rng(5).integers(0, shape.vocab, size=(3, 8)).astype(np.int32)).cuda()
+    for ks in ([8, 3, 0], [0, 0, 0], [5, 8, 8]):
+        eng.validate([0, 1, 2], ks, d_dev, commit=False)
+        all_empty(f"validate {ks}")
+    eng.validate([1], [4], d_dev[1:2].contiguous(), commit=True)
+    all_empty("committing validate")
+    eng.draft(0, 6)
+    all_empty("draft")
+    out, _ = eng.generate(2, prompts[2], 4, 12)
+    all_empty("generate")
+    assert len(out) == 12
+    eng.close()
+
+
 def test_adaptive_draft_length_generation_matches_the_oracle_schedule():
     # sequential assisted generation with a dynamic draft length (Sections 3.2 and 4.1): on the tiny
     # fp32 config the tokens are exact, so the library must walk the very schedule the oracle walks
@@ -390,4 +423,5 @@ def test_tcgen05_attention_path_matches_oracle(hq, hkv, hd):
     _, _, lg_mma = eng.validate([0, 1], [8, 3], torch.from_numpy(drafts).cuda(), want_logits=True)
     eng.sync()
     assert float((lg_tc - lg_mma).abs().max()) < 5e-3
+    gu.assert_polled_scratch_empty(eng, "tcgen05 attention calls")
     eng.close()
