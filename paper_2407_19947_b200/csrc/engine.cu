@@ -232,7 +232,6 @@ bool compute_layout(const stairs_config& c, Layout* L, const char** why) {
     // attn_unit_bound).  A validate call holds up to max_requests requests of k_max + 1 rows; a
     // prefill pass of the persistent kernel is one request of MK_MAX_ROWS rows.
     const int rows_req = std::min(c.k_max + 1, MK_MAX_ROWS);
-    const int n_qblk = (rows_req * gq + mk::ATT_QBLK - 1) / mk::ATT_QBLK;
     L->attn_units = std::max(c.max_requests * attn_unit_bound(hkv, gq, rows_req), attn_unit_bound(hkv, gq, MK_MAX_ROWS));
     // (the tcgen05 attention path has fewer units of 128 query rows each: sized for whichever is larger)
     const int units_tc = std::max(c.max_requests * attn_unit_bound(hkv, gq, rows_req, mk::ATT_QBLK_TC), attn_unit_bound(hkv, gq, MK_MAX_ROWS, mk::ATT_QBLK_TC));
